@@ -1,0 +1,170 @@
+/*
+ * fdkv -- FreqDepthKV hot path on one B200 (sm_100a): prefill-time compression of adjacent-layer
+ * K/V pairs, the routing probe, and decode attention over the compressed cache.
+ *
+ * C ABI.  Plain pointers and sizes only.  Unless a parameter says HOST, pointers are DEVICE pointers.
+ *
+ * Conventions
+ *  - Every call returns an fdkv_status.  Argument errors are detected on the host before anything is
+ *    enqueued.  No call throws, aborts or traps the device.
+ *  - The library never allocates device memory.  The caller owns two device buffers for the lifetime
+ *    of the context: an ARENA (packed caches of all sequences, generated-token tails, lookup tables)
+ *    and a WORKSPACE (staging of one sequence's compression, histograms, split-K partials).  Sizes come
+ *    from fdkv_sizes().  Both must be 256-byte aligned.
+ *  - Work is enqueued on the stream the caller passes (a cudaStream_t, given as void*; NULL = the legacy
+ *    default stream) and the call returns without waiting, except where stated (fdkv_commit, fdkv_get_*,
+ *    the *_host variants).
+ *  - Tensors are dense row-major in the storage dtype of the context (float32 or bf16) unless strides
+ *    are given.  Device pointers to tensors must be 16-byte aligned; strides are in elements and must be
+ *    multiples of 8.
+ *  - A "unit" is (sequence, layer pair p = layers 2p and 2p+1, KV head h).  Query head i reads KV head
+ *    i / (n_q_heads / n_kv_heads).
+ *  - A context is not thread-safe.
+ *
+ * Notation follows the paper's Method section: T context length, d head dimension, Z0 / Z1 the low /
+ * high frequency depth coefficients of Eq. 1 with the 2x2 orthonormal DCT-II, c = 1/sqrt(2).
+ */
+#ifndef FDKV_H
+#define FDKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FDKV_OK = 0,
+    FDKV_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, bad shape, stride, range or order          */
+    FDKV_ERR_UNSUPPORTED = 2, /* shape or dtype this build has no kernel for                           */
+    FDKV_ERR_ARENA_FULL = 3,  /* the arena cannot hold what fdkv_commit needs; nothing was changed     */
+    FDKV_ERR_WORKSPACE = 4,   /* workspace smaller than fdkv_sizes() says                              */
+    FDKV_ERR_STATE = 5,       /* call order (probe before compress, decode before commit, tail full)   */
+    FDKV_ERR_CUDA = 6,        /* a CUDA runtime call failed; see fdkv_last_cuda_error()                */
+    FDKV_ERR_TIMEOUT = 7,     /* a bounded device-side wait gave up (reported by fdkv_device_status)   */
+    FDKV_ERR_DEVICE = 8       /* a device-side consistency check failed (fdkv_device_status)           */
+} fdkv_status;
+
+typedef enum { FDKV_F32 = 0, FDKV_BF16 = 1 } fdkv_dtype;
+typedef enum { FDKV_MODE_SHARED = 0, FDKV_MODE_RESIDUAL = 1, FDKV_MODE_EXACT = 2 } fdkv_mode;
+
+typedef struct {
+    int32_t n_layers;    /* even; pair p = layers 2p, 2p+1 (block size B = 2 of Eq. 1)                 */
+    int32_t n_q_heads;   /* multiple of n_kv_heads; group size n_q_heads / n_kv_heads <= 8             */
+    int32_t n_kv_heads;
+    int32_t head_dim;    /* 64 or 128                                                                  */
+    int32_t max_batch;   /* number of sequence slots                                                   */
+    int32_t max_prefill; /* largest T; max_prefill * head_dim < 2^31 (int32 flat indices)              */
+    int32_t max_tail;    /* generated tokens kept uncompressed per layer and sequence                  */
+    int32_t dtype;       /* fdkv_dtype: storage type of K, V, Q and of the stored coefficients         */
+    int32_t keep_num;    /* residual keep fraction: k = floor(T * head_dim * keep_num / keep_den)      */
+    int32_t keep_den;    /*   entries per (unit, K or V); 0 <= keep_num <= keep_den                    */
+} fdkv_config;
+
+typedef struct fdkv_ctx fdkv_ctx;
+
+/* Bytes the caller must provide.  arena_bytes is the worst case (every unit in exact mode). */
+fdkv_status fdkv_sizes(const fdkv_config* cfg /*HOST*/, size_t* arena_bytes /*HOST*/,
+                       size_t* workspace_bytes /*HOST*/);
+
+/* Creates the host-side context over caller-owned device memory and zero-initialises the tail counters
+ * and the device status word (synchronously, on the legacy default stream).  The context keeps the pointers;
+ * the caller frees the buffers only after fdkv_destroy.                                                   */
+fdkv_status fdkv_create(const fdkv_config* cfg /*HOST*/, void* arena, size_t arena_bytes, void* workspace,
+                        size_t workspace_bytes, fdkv_ctx** out /*HOST*/);
+void fdkv_destroy(fdkv_ctx* ctx);
+/* Forgets every committed sequence and empties the arena and all tails (synchronous). */
+fdkv_status fdkv_reset(fdkv_ctx* ctx);
+
+/*
+ * Prefill compression (Method, Eq. 1 and Eq. 3; residual set in entry-magnitude form).
+ * For every pair p in [pair_begin, pair_end), every KV head h and for K and V separately:
+ *   z0 = rs((x0 + x1) * c32), z1 = rs((x0 - x1) * c32)   one float32 add, one float32 multiply by the
+ *        float32 nearest 1/sqrt(2), rs = rounding to the storage dtype (nearest even);
+ *   the k entries of z1 with the largest magnitude are kept (ties: lowest flat index t*d + ch) and
+ *   emitted in ascending flat index as (int32 index, stored value).
+ * k_layers / v_layers: HOST arrays of n_layers DEVICE pointers (only the layers of the pair range are
+ *   read); element (t, h, ch) of layer l is at ptr[l] + t*stride_t + h*stride_h + ch.
+ * Results are staged in the workspace for sequence slot `seq` (one sequence is staged at a time; a call
+ * for another slot discards the previous staging).  The caller keeps K/V alive until fdkv_commit returns.
+ */
+fdkv_status fdkv_compress_prefill(fdkv_ctx* ctx, int32_t seq, int32_t pair_begin, int32_t pair_end, int32_t T,
+                                  const void* const* k_layers /*HOST*/, const void* const* v_layers /*HOST*/,
+                                  int64_t stride_t, int64_t stride_h, void* stream);
+
+/*
+ * Routing probe (Method, Eq. 2 and the argmin of Eq. 3) for the staged sequence.
+ * For every unit of the pair range and mode m in {shared, residual}:
+ *   E(m) = mean over (layer of the pair, group query head g, probe query q) of
+ *          sum_{j <= probe_pos[q]} ( Q[l][q][h*G+g] . (c * R^(m)[j,:]) / sqrt(d) )^2,
+ *   R^(shared) = Z1 of K, R^(residual) = Z1 of K with the kept entries removed; E(exact) = 0.
+ *   L(m) = E(m) + lambda * Omega(m), Omega = bytes(m) / bytes(exact) (K and V, int32 indices counted);
+ *   mode = argmin, ties to the lowest id.  The same mode applies to K and V.
+ * q_layers: HOST array of n_layers DEVICE pointers to [W][n_q_heads][head_dim].
+ * probe_pos: HOST int32[W], strictly ascending, each in [0, T).  1 <= W <= 128.
+ * modes (may be NULL): DEVICE int32[pair_end-pair_begin][n_kv_heads].
+ * scores (may be NULL): DEVICE float[pair_end-pair_begin][n_kv_heads][2] = {E(shared), E(residual)}.
+ */
+fdkv_status fdkv_probe(fdkv_ctx* ctx, int32_t seq, int32_t pair_begin, int32_t pair_end,
+                       const void* const* q_layers /*HOST*/, const int32_t* probe_pos /*HOST*/, int32_t W,
+                       double lambda, int32_t* modes, float* scores, void* stream);
+
+/* Overrides the modes of the staged sequence (forced-mode tests, ablations, benchmark mode mix).
+ * modes_host: HOST int32[n_layers/2][n_kv_heads], each 0, 1 or 2.                                        */
+fdkv_status fdkv_set_modes(fdkv_ctx* ctx, int32_t seq, const int32_t* modes_host /*HOST*/);
+
+/* Packs the staged sequence into the arena, keeping per unit only what its mode reads at decode time
+ * (shared: Z0 of K and V; residual: Z0 plus the two lists; exact: the original rows of both layers).
+ * Waits for the stream (it needs the modes on the host), then enqueues the copies and waits again.
+ * Every pair of the sequence must have been compressed, and probed or given a mode.                      */
+fdkv_status fdkv_commit(fdkv_ctx* ctx, int32_t seq, void* stream);
+
+/*
+ * Decode attention for one layer (Method, the paragraph after Eq. 3), split-K over the sequence.
+ * For sequence b < batch and query head i (KV head h = i / G), over rows 0..T-1 reconstructed by the
+ * unit's mode (shared: c*z0; residual: c*(z0 + s*z1 on kept entries), s = +1 for layer 2p, -1 for 2p+1;
+ * exact: the original row) followed by the layer's uncompressed tail rows:
+ *   logit = khat . q / sqrt(d);  out = softmax(logit) . vhat      (float32 accumulation)
+ * q: [batch][n_q_heads][d].  k_new / v_new: [batch][n_kv_heads][d], appended to the layer's tail before
+ * attending, or both NULL (no append).  out: [batch][n_q_heads][d] in out_dtype.
+ * Sequence slots 0..batch-1 must be committed.
+ */
+fdkv_status fdkv_decode_attn(fdkv_ctx* ctx, int32_t layer, int32_t batch, const void* q, const void* k_new,
+                             const void* v_new, void* out, int32_t out_dtype, void* stream);
+
+/* Same call with HOST buffers: copies q (and k_new, v_new) to the device, runs the layer, copies out back and
+ * waits for the stream.  Buffers should be pinned for the copies to overlap.                              */
+fdkv_status fdkv_decode_attn_host(fdkv_ctx* ctx, int32_t layer, int32_t batch, const void* q /*HOST*/,
+                                  const void* k_new /*HOST*/, const void* v_new /*HOST*/, void* out /*HOST*/,
+                                  int32_t out_dtype, void* stream);
+
+/* Sets the tail length of every layer of a sequence (0 empties the tails; n <= current length). */
+fdkv_status fdkv_set_tail_len(fdkv_ctx* ctx, int32_t seq, int32_t n, void* stream);
+
+/* Introspection of the STAGED sequence (valid from fdkv_compress_prefill until the next one).  Synchronous. */
+fdkv_status fdkv_get_shared(fdkv_ctx* ctx, int32_t seq, int32_t pair, int32_t kv_head, int32_t is_v,
+                            void* z0_out /*DEVICE [T][d] storage dtype*/, void* stream);
+fdkv_status fdkv_get_residual(fdkv_ctx* ctx, int32_t seq, int32_t pair, int32_t kv_head, int32_t is_v,
+                              int32_t* idx_out /*DEVICE [k]*/, void* val_out /*DEVICE [k] storage dtype*/,
+                              int32_t* count_host /*HOST*/, void* stream);
+/* Modes of a committed (or mode-overridden) sequence: HOST int32[n_layers/2][n_kv_heads]. */
+fdkv_status fdkv_get_modes(fdkv_ctx* ctx, int32_t seq, int32_t* modes_host /*HOST*/);
+/* Bytes a committed sequence holds in the arena per mode, and what the uncompressed cache would take. */
+fdkv_status fdkv_footprint(fdkv_ctx* ctx, int32_t seq, size_t* bytes_by_mode_host /*HOST [3]*/,
+                           size_t* exact_equiv_bytes_host /*HOST*/);
+/* Bytes the decode kernels read from the packed cache for one call of `layer` over `batch` sequences
+ * (coefficient or exact rows, residual lists and their tile offsets, tails): the roofline numerator.      */
+fdkv_status fdkv_decode_bytes(fdkv_ctx* ctx, int32_t layer, int32_t batch, size_t* bytes_host /*HOST*/);
+
+/* Reads the device status word (synchronises the device): FDKV_OK, FDKV_ERR_TIMEOUT or FDKV_ERR_DEVICE.  */
+fdkv_status fdkv_device_status(fdkv_ctx* ctx);
+int32_t fdkv_last_cuda_error(void);
+const char* fdkv_status_str(fdkv_status s);
+/* Kernels launched by this library since it was loaded (all contexts). */
+int64_t fdkv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDKV_H */

@@ -1,0 +1,246 @@
+"""Thin ctypes binding over libfdkv.so: argument marshalling only, every step runs in the CUDA kernels.
+
+torch is used for device memory and streams.  Importing this module loads the shared library and raises if
+it is missing; there is no CPU or eager fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfdkv.so")
+
+F32, BF16 = 0, 1
+SHARED, RESIDUAL, EXACT = 0, 1, 2
+_STATUS = ["ok", "invalid argument", "unsupported", "arena full", "workspace too small", "state", "cuda error",
+           "device timeout", "device check failed"]
+
+
+class FdkvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        name = _STATUS[code] if 0 <= code < len(_STATUS) else str(code)
+        super().__init__(f"{where}: fdkv status {code} ({name})")
+
+
+class _Config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "max_batch", "max_prefill",
+                                         "max_tail", "dtype", "keep_num", "keep_den")]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_06519_b200.build` "
+                          "(nvcc, sm_100a); this package has no fallback path")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    P = C.POINTER
+    sig = {
+        "fdkv_sizes": [P(_Config), P(sz), P(sz)],
+        "fdkv_create": [P(_Config), vp, sz, vp, sz, P(vp)],
+        "fdkv_reset": [vp],
+        "fdkv_compress_prefill": [vp, i32, i32, i32, i32, P(vp), P(vp), i64, i64, vp],
+        "fdkv_probe": [vp, i32, i32, i32, P(vp), P(i32), i32, C.c_double, vp, vp, vp],
+        "fdkv_set_modes": [vp, i32, P(i32)],
+        "fdkv_commit": [vp, i32, vp],
+        "fdkv_decode_attn": [vp, i32, i32, vp, vp, vp, vp, i32, vp],
+        "fdkv_decode_attn_host": [vp, i32, i32, vp, vp, vp, vp, i32, vp],
+        "fdkv_set_tail_len": [vp, i32, i32, vp],
+        "fdkv_get_shared": [vp, i32, i32, i32, i32, vp, vp],
+        "fdkv_get_residual": [vp, i32, i32, i32, i32, vp, vp, P(i32), vp],
+        "fdkv_get_modes": [vp, i32, P(i32)],
+        "fdkv_footprint": [vp, i32, P(sz), P(sz)],
+        "fdkv_decode_bytes": [vp, i32, i32, P(sz)],
+        "fdkv_device_status": [vp],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = C.c_int
+    lib.fdkv_destroy.argtypes = [vp]
+    lib.fdkv_destroy.restype = None
+    lib.fdkv_last_cuda_error.restype = C.c_int32
+    lib.fdkv_status_str.argtypes = [C.c_int]
+    lib.fdkv_status_str.restype = C.c_char_p
+    lib.fdkv_launch_count.restype = C.c_int64
+    return lib
+
+
+_lib = _load()
+
+
+def launch_count() -> int:
+    return int(_lib.fdkv_launch_count())
+
+
+def last_cuda_error() -> int:
+    return int(_lib.fdkv_last_cuda_error())
+
+
+@dataclass
+class Config:
+    n_layers: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    max_batch: int
+    max_prefill: int
+    max_tail: int
+    dtype: int
+    keep_num: int
+    keep_den: int
+
+    def c(self) -> _Config:
+        return _Config(*(int(getattr(self, f[0])) for f in _Config._fields_))
+
+
+def sizes(cfg: Config):
+    a, w = C.c_size_t(0), C.c_size_t(0)
+    st = _lib.fdkv_sizes(C.byref(cfg.c()), C.byref(a), C.byref(w))
+    if st:
+        raise FdkvError(st, "fdkv_sizes")
+    return a.value, w.value
+
+
+def _check(st: int, where: str):
+    if st:
+        raise FdkvError(st, where)
+
+
+def _stream(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+class Context:
+    """One fdkv context over torch-owned device memory."""
+
+    def __init__(self, cfg: Config, device="cuda:0", arena_bytes: int | None = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("fdkv needs a CUDA device; there is no CPU path")
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.tdtype = torch.bfloat16 if cfg.dtype == BF16 else torch.float32
+        worst, work = sizes(cfg)
+        self.arena_bytes = int(arena_bytes if arena_bytes is not None else worst)
+        with torch.cuda.device(self.device):
+            self.arena = torch.empty(self.arena_bytes, dtype=torch.uint8, device=self.device)
+            self.work = torch.empty(work, dtype=torch.uint8, device=self.device)
+            h = C.c_void_p()
+            torch.cuda.synchronize()
+            _check(_lib.fdkv_create(C.byref(cfg.c()), self.arena.data_ptr(), self.arena_bytes, self.work.data_ptr(), work,
+                                    C.byref(h)), "fdkv_create")
+        self.h = h
+        self.n_pairs = cfg.n_layers // 2
+
+    def close(self):
+        if getattr(self, "h", None):
+            _lib.fdkv_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self):
+        _check(_lib.fdkv_reset(self.h), "fdkv_reset")
+
+    def compress_prefill(self, seq, pair_begin, pair_end, T, k_layers, v_layers, stream=None):
+        """k_layers / v_layers: per-layer tensors [T, n_kv_heads, head_dim] (None outside the pair range)."""
+        L = self.cfg.n_layers
+        ref = k_layers[2 * pair_begin]
+        kp = (C.c_void_p * L)(*[None if t is None else t.data_ptr() for t in k_layers])
+        vp = (C.c_void_p * L)(*[None if t is None else t.data_ptr() for t in v_layers])
+        for t in list(k_layers) + list(v_layers):
+            if t is not None and (t.stride() != ref.stride() or t.dtype != self.tdtype or t.stride(2) != 1):
+                raise ValueError("all K/V layers must share one [T, Hkv, d] strided layout and the context dtype")
+        _check(_lib.fdkv_compress_prefill(self.h, seq, pair_begin, pair_end, T, kp, vp, ref.stride(0), ref.stride(1),
+                                          _stream(stream)), "fdkv_compress_prefill")
+
+    def probe(self, seq, pair_begin, pair_end, q_layers, probe_pos, lam, stream=None):
+        """q_layers: per-layer contiguous [W, n_q_heads, head_dim]; returns (modes int32 [pairs, Hkv], scores f32 [pairs, Hkv, 2])."""
+        L = self.cfg.n_layers
+        W = len(probe_pos)
+        qp = (C.c_void_p * L)(*[None if t is None else t.data_ptr() for t in q_layers])
+        pos = (C.c_int32 * W)(*[int(p) for p in probe_pos])
+        n = (pair_end - pair_begin) * self.cfg.n_kv_heads
+        modes = torch.empty(n, dtype=torch.int32, device=self.device)
+        scores = torch.empty(n * 2, dtype=torch.float32, device=self.device)
+        _check(_lib.fdkv_probe(self.h, seq, pair_begin, pair_end, qp, pos, W, float(lam), _ptr(modes), _ptr(scores),
+                               _stream(stream)), "fdkv_probe")
+        return modes.view(pair_end - pair_begin, -1), scores.view(pair_end - pair_begin, -1, 2)
+
+    def set_modes(self, seq, modes):
+        flat = [int(m) for m in torch.as_tensor(modes).reshape(-1).tolist()]
+        arr = (C.c_int32 * len(flat))(*flat)
+        if len(flat) != self.n_pairs * self.cfg.n_kv_heads:
+            raise ValueError("modes must have n_pairs * n_kv_heads entries")
+        _check(_lib.fdkv_set_modes(self.h, seq, arr), "fdkv_set_modes")
+
+    def commit(self, seq, stream=None):
+        _check(_lib.fdkv_commit(self.h, seq, _stream(stream)), "fdkv_commit")
+
+    def decode_attn(self, layer, q, k_new=None, v_new=None, out=None, out_dtype=None, stream=None):
+        """q: [batch, n_q_heads, d]; returns out [batch, n_q_heads, d]."""
+        batch = q.shape[0]
+        od = self.cfg.dtype if out_dtype is None else out_dtype
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.bfloat16 if od == BF16 else torch.float32, device=self.device)
+        _check(_lib.fdkv_decode_attn(self.h, layer, batch, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), od,
+                                     _stream(stream)), "fdkv_decode_attn")
+        return out
+
+    def decode_attn_host(self, layer, q, k_new, v_new, out, out_dtype, stream=None):
+        """Same with host (ideally pinned) tensors; synchronous."""
+        _check(_lib.fdkv_decode_attn_host(self.h, layer, q.shape[0], _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
+                                          out_dtype, _stream(stream)), "fdkv_decode_attn_host")
+        return out
+
+    def set_tail_len(self, seq, n, stream=None):
+        _check(_lib.fdkv_set_tail_len(self.h, seq, n, _stream(stream)), "fdkv_set_tail_len")
+
+    def get_shared(self, seq, pair, kv_head, is_v, T, stream=None):
+        out = torch.empty((T, self.cfg.head_dim), dtype=self.tdtype, device=self.device)
+        _check(_lib.fdkv_get_shared(self.h, seq, pair, kv_head, int(is_v), _ptr(out), _stream(stream)), "fdkv_get_shared")
+        return out
+
+    def get_residual(self, seq, pair, kv_head, is_v, stream=None):
+        cnt = C.c_int32(0)
+        _check(_lib.fdkv_get_residual(self.h, seq, pair, kv_head, int(is_v), None, None, C.byref(cnt), _stream(stream)),
+               "fdkv_get_residual")
+        k = cnt.value
+        idx = torch.empty(k, dtype=torch.int32, device=self.device)
+        val = torch.empty(k, dtype=self.tdtype, device=self.device)
+        _check(_lib.fdkv_get_residual(self.h, seq, pair, kv_head, int(is_v), _ptr(idx), _ptr(val), C.byref(cnt),
+                                      _stream(stream)), "fdkv_get_residual")
+        return idx, val
+
+    def get_modes(self, seq):
+        n = self.n_pairs * self.cfg.n_kv_heads
+        arr = (C.c_int32 * n)()
+        _check(_lib.fdkv_get_modes(self.h, seq, arr), "fdkv_get_modes")
+        return torch.tensor(list(arr), dtype=torch.int32).view(self.n_pairs, -1)
+
+    def footprint(self, seq):
+        by = (C.c_size_t * 3)()
+        ex = C.c_size_t(0)
+        _check(_lib.fdkv_footprint(self.h, seq, by, C.byref(ex)), "fdkv_footprint")
+        return list(by), ex.value
+
+    def decode_bytes(self, layer, batch):
+        b = C.c_size_t(0)
+        _check(_lib.fdkv_decode_bytes(self.h, layer, batch, C.byref(b)), "fdkv_decode_bytes")
+        return b.value
+
+    def device_status(self):
+        return int(_lib.fdkv_device_status(self.h))

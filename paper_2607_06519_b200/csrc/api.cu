@@ -1,0 +1,526 @@
+// Host side of the C ABI: argument checks, workspace / arena bookkeeping, launch sequencing.
+#include <atomic>
+#include <cstring>
+#include <new>
+
+#include "fdkv_internal.h"
+
+using namespace fdkv;
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+std::atomic<int32_t> g_last_cuda{0};
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+fdkv_status cuda_fail(cudaError_t e) {
+    g_last_cuda.store((int32_t)e);
+    return FDKV_ERR_CUDA;
+}
+#define CU(x)                                         \
+    do {                                              \
+        cudaError_t e__ = (x);                        \
+        if (e__ != cudaSuccess) return cuda_fail(e__); \
+    } while (0)
+
+bool make_shape(const fdkv_config& c, Shape& s) {
+    if (c.n_layers <= 0 || (c.n_layers & 1) || c.n_layers > 1024) return false;
+    if (c.n_kv_heads <= 0 || c.n_q_heads <= 0 || c.n_q_heads % c.n_kv_heads) return false;
+    const int G = c.n_q_heads / c.n_kv_heads;
+    if (!(G == 1 || G == 2 || G == 4 || G == 8)) return false;
+    if (c.head_dim != 64 && c.head_dim != 128) return false;
+    if (c.max_batch <= 0 || c.max_prefill <= 0 || c.max_tail < 0) return false;
+    if ((int64_t)c.max_prefill * c.head_dim >= (int64_t)1 << 31) return false;
+    if (c.dtype != FDKV_F32 && c.dtype != FDKV_BF16) return false;
+    if (c.keep_den <= 0 || c.keep_num < 0 || c.keep_num > c.keep_den) return false;
+    s.L = c.n_layers; s.P = c.n_layers / 2; s.Hq = c.n_q_heads; s.Hkv = c.n_kv_heads; s.G = G; s.d = c.head_dim;
+    s.max_batch = c.max_batch; s.Tmax = c.max_prefill; s.max_tail = c.max_tail;
+    s.dtype = c.dtype; s.esize = c.dtype == FDKV_BF16 ? 2 : 4;
+    s.keep_num = c.keep_num; s.keep_den = c.keep_den;
+    s.kmax = (int64_t)s.Tmax * s.d * s.keep_num / s.keep_den;
+    s.kcap = (int64_t)align_up((size_t)(s.kmax + kListPad), 64);
+    s.ntiles_max = (s.Tmax + kResTile - 1) / kResTile;
+    s.nptiles_max = (s.Tmax + kProbeTile - 1) / kProbeTile;
+    s.NU = s.P * s.Hkv;
+    s.NT = 2 * s.NU;
+    return true;
+}
+
+void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
+    const size_t unit_elems = (size_t)s.Tmax * s.d;
+    w.status = take(256);
+    w.z0 = take((size_t)s.NT * unit_elems * s.esize);
+    w.z1 = take((size_t)s.NT * unit_elems * s.esize);
+    w.hist = take((size_t)s.NT * kHistBins * 4);
+    w.sel = take((size_t)s.NT * sizeof(SelState));
+    w.tile_cnt = take((size_t)s.NT * s.ntiles_max * 8);
+    w.tile_eq = take((size_t)s.NT * s.ntiles_max * 4);
+    w.tile_off = take((size_t)s.NT * (s.ntiles_max + 1) * 4);
+    w.idx = take((size_t)s.NT * s.kcap * 4);
+    w.val = take((size_t)s.NT * s.kcap * s.esize);
+    w.probe_part = take((size_t)s.NU * s.nptiles_max * 16);
+    w.probe_pos = take((size_t)kMaxW * 4 + (size_t)s.L * 8);
+    w.scores = take((size_t)s.NU * 16);
+    w.modes = take((size_t)s.NU * 4);
+    w.partials = take((size_t)s.max_batch * s.Hq * kMaxSplits * (s.d + 2) * 4);
+    w.io_q = take((size_t)s.max_batch * s.Hq * s.d * 4);
+    w.io_k = take((size_t)s.max_batch * s.Hkv * s.d * 4);
+    w.io_v = take((size_t)s.max_batch * s.Hkv * s.d * 4);
+    w.io_out = take((size_t)s.max_batch * s.Hq * s.d * 4);
+    w.total = o;
+
+    o = 0;
+    a.tail_len = take((size_t)s.L * s.max_batch * 4);
+    a.desc = take((size_t)s.max_batch * s.L * s.Hkv * sizeof(UnitDesc));
+    const size_t tail = (size_t)s.L * s.max_batch * s.Hkv * s.max_tail * s.d * s.esize;
+    a.tail_k = take(tail);
+    a.tail_v = take(tail);
+    a.bump = o;
+    const size_t exact_unit = 4 * align_up(unit_elems * s.esize);
+    const size_t resid_unit = 2 * align_up(unit_elems * s.esize) + 2 * align_up((size_t)s.kcap * 4) +
+                              2 * align_up((size_t)s.kcap * s.esize) + 2 * align_up((size_t)(s.ntiles_max + 1) * 4);
+    a.worst_total = a.bump + (size_t)s.max_batch * s.NU * (exact_unit > resid_unit ? exact_unit : resid_unit);
+}
+
+inline cudaStream_t S(void* p) { return reinterpret_cast<cudaStream_t>(p); }
+template <typename T>
+inline T* wsp(fdkv_ctx* c, size_t off) { return reinterpret_cast<T*>(c->work + off); }
+template <typename T>
+inline T* arp(fdkv_ctx* c, size_t off) { return reinterpret_cast<T*>(c->arena + off); }
+
+bool seq_ok(fdkv_ctx* c, int seq) { return c && seq >= 0 && seq < c->s.max_batch; }
+
+}  // namespace
+
+namespace fdkv {
+void count_launch(int n) { g_launches.fetch_add(n); }
+cudaError_t launch_set_tail_len(int32_t* tail_len, int L, int max_batch, int seq, int n, cudaStream_t st);
+}  // namespace fdkv
+
+extern "C" {
+
+fdkv_status fdkv_sizes(const fdkv_config* cfg, size_t* arena_bytes, size_t* workspace_bytes) {
+    Shape s;
+    if (!cfg || !make_shape(*cfg, s)) return cfg ? FDKV_ERR_UNSUPPORTED : FDKV_ERR_INVALID_ARG;
+    WsLayout w;
+    ArenaLayout a;
+    make_layouts(s, w, a);
+    if (arena_bytes) *arena_bytes = a.worst_total;
+    if (workspace_bytes) *workspace_bytes = w.total;
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes, void* workspace,
+                        size_t workspace_bytes, fdkv_ctx** out) {
+    if (!cfg || !arena || !workspace || !out) return FDKV_ERR_INVALID_ARG;
+    if (!aligned(arena, 256) || !aligned(workspace, 256)) return FDKV_ERR_INVALID_ARG;
+    Shape s;
+    if (!make_shape(*cfg, s)) return FDKV_ERR_UNSUPPORTED;
+    fdkv_ctx* c = new (std::nothrow) fdkv_ctx();
+    if (!c) return FDKV_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->s = s;
+    make_layouts(s, c->ws, c->ar);
+    if (workspace_bytes < c->ws.total) { delete c; return FDKV_ERR_WORKSPACE; }
+    if (arena_bytes < c->ar.bump) { delete c; return FDKV_ERR_ARENA_FULL; }
+    c->arena = (char*)arena;
+    c->arena_bytes = arena_bytes;
+    c->work = (char*)workspace;
+    c->work_bytes = workspace_bytes;
+    c->bump = c->ar.bump;
+    c->pair_compressed.assign(s.P, 0);
+    c->pair_probed.assign(s.P, 0);
+    c->k_layers.assign(s.L, nullptr);
+    c->v_layers.assign(s.L, nullptr);
+    c->seqs.resize(s.max_batch);
+    for (auto& q : c->seqs) { q.modes.assign(s.NU, -1); q.tail_len.assign(s.L, 0); }
+    c->desc_host.resize((size_t)s.max_batch * s.L * s.Hkv);
+    cudaError_t e = cudaMemset(c->arena + c->ar.tail_len, 0, (size_t)s.L * s.max_batch * 4);
+    if (e == cudaSuccess) e = cudaMemset(c->work + c->ws.status, 0, 256);
+    if (e == cudaSuccess) e = cudaMemset(c->arena + c->ar.desc, 0, c->desc_host.size() * sizeof(UnitDesc));
+    if (e != cudaSuccess) { delete c; return cuda_fail(e); }
+    *out = c;
+    return FDKV_OK;
+}
+
+void fdkv_destroy(fdkv_ctx* ctx) { delete ctx; }
+
+fdkv_status fdkv_reset(fdkv_ctx* c) {
+    if (!c) return FDKV_ERR_INVALID_ARG;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemset(c->arena + c->ar.tail_len, 0, (size_t)c->s.L * c->s.max_batch * 4));
+    CU(cudaMemset(c->work + c->ws.status, 0, 256));
+    c->bump = c->ar.bump;
+    c->staged_seq = -1;
+    for (auto& q : c->seqs) {
+        q.committed = false;
+        q.T = 0;
+        q.modes.assign(c->s.NU, -1);
+        q.tail_len.assign(c->s.L, 0);
+        q.bytes_by_mode[0] = q.bytes_by_mode[1] = q.bytes_by_mode[2] = 0;
+    }
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, int32_t T,
+                                  const void* const* k_layers, const void* const* v_layers, int64_t stride_t,
+                                  int64_t stride_h, void* stream) {
+    if (!seq_ok(c, seq) || !k_layers || !v_layers) return FDKV_ERR_INVALID_ARG;
+    const Shape& s = c->s;
+    if (pb < 0 || pe > s.P || pb >= pe) return FDKV_ERR_INVALID_ARG;
+    if (T < 1 || T > s.Tmax) return FDKV_ERR_INVALID_ARG;
+    if (stride_h < s.d || stride_t < s.d || (stride_t % 8) || (stride_h % 8)) return FDKV_ERR_INVALID_ARG;
+    for (int l = 2 * pb; l < 2 * pe; ++l)
+        if (!k_layers[l] || !v_layers[l] || !aligned(k_layers[l], 16) || !aligned(v_layers[l], 16))
+            return FDKV_ERR_INVALID_ARG;
+    if (c->seqs[seq].committed) return FDKV_ERR_STATE;
+    if (c->staged_seq != seq || c->staged_T != T) {
+        c->staged_seq = seq;
+        c->staged_T = T;
+        std::fill(c->pair_compressed.begin(), c->pair_compressed.end(), 0);
+        std::fill(c->pair_probed.begin(), c->pair_probed.end(), 0);
+        c->modes_overridden = false;
+        c->seqs[seq].modes.assign(s.NU, -1);
+        c->stride_t = stride_t;
+        c->stride_h = stride_h;
+    } else if (c->stride_t != stride_t || c->stride_h != stride_h) {
+        return FDKV_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = S(stream);
+    const int ut_begin = pb * s.Hkv * 2, ut_count = (pe - pb) * s.Hkv * 2;
+    CU(cudaMemsetAsync(wsp<uint32_t>(c, c->ws.hist) + (size_t)ut_begin * kHistBins, 0, (size_t)ut_count * kHistBins * 4, st));
+    for (int p = pb; p < pe; ++p) {
+        CompressArgs a;
+        a.k0 = k_layers[2 * p]; a.k1 = k_layers[2 * p + 1];
+        a.v0 = v_layers[2 * p]; a.v1 = v_layers[2 * p + 1];
+        a.stride_t = stride_t; a.stride_h = stride_h;
+        a.T = T; a.d = s.d; a.Hkv = s.Hkv;
+        a.ut_base = p * s.Hkv * 2;
+        a.unit_stride = (int64_t)s.Tmax * s.d;
+        a.z0 = c->work + c->ws.z0; a.z1 = c->work + c->ws.z1;
+        a.hist = wsp<uint32_t>(c, c->ws.hist);
+        CU(launch_split_hist(a, s.dtype, st));
+        c->k_layers[2 * p] = a.k0; c->k_layers[2 * p + 1] = a.k1;
+        c->v_layers[2 * p] = a.v0; c->v_layers[2 * p + 1] = a.v1;
+    }
+    SelectArgs sa;
+    sa.ut_begin = ut_begin; sa.ut_count = ut_count;
+    sa.T = T; sa.d = s.d;
+    sa.k = (int64_t)T * s.d * s.keep_num / s.keep_den;
+    sa.unit_stride = (int64_t)s.Tmax * s.d; sa.kcap = s.kcap; sa.ntiles_max = s.ntiles_max;
+    sa.z1 = c->work + c->ws.z1;
+    sa.hist = wsp<uint32_t>(c, c->ws.hist);
+    sa.sel = wsp<SelState>(c, c->ws.sel);
+    sa.tile_cnt = wsp<uint32_t>(c, c->ws.tile_cnt);
+    sa.tile_eq = wsp<uint32_t>(c, c->ws.tile_eq);
+    sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
+    sa.idx = wsp<int32_t>(c, c->ws.idx);
+    sa.val = c->work + c->ws.val;
+    sa.status = wsp<int32_t>(c, c->ws.status);
+    CU(launch_select_and_compact(sa, s.dtype, st));
+    for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; }
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const void* const* q_layers,
+                       const int32_t* probe_pos, int32_t W, double lambda, int32_t* modes, float* scores,
+                       void* stream) {
+    if (!seq_ok(c, seq) || !q_layers || !probe_pos) return FDKV_ERR_INVALID_ARG;
+    const Shape& s = c->s;
+    if (pb < 0 || pe > s.P || pb >= pe || W < 1 || W > kMaxW) return FDKV_ERR_INVALID_ARG;
+    if (!(lambda >= 0.0)) return FDKV_ERR_INVALID_ARG;
+    if (c->staged_seq != seq) return FDKV_ERR_STATE;
+    for (int p = pb; p < pe; ++p)
+        if (!c->pair_compressed[p]) return FDKV_ERR_STATE;
+    const int T = c->staged_T;
+    for (int i = 0; i < W; ++i)
+        if (probe_pos[i] < 0 || probe_pos[i] >= T || (i && probe_pos[i] <= probe_pos[i - 1])) return FDKV_ERR_INVALID_ARG;
+    for (int l = 2 * pb; l < 2 * pe; ++l)
+        if (!q_layers[l] || !aligned(q_layers[l], 16)) return FDKV_ERR_INVALID_ARG;
+    cudaStream_t st = S(stream);
+    int32_t* pos_dev = wsp<int32_t>(c, c->ws.probe_pos);
+    const void** qptr_dev = reinterpret_cast<const void**>(c->work + c->ws.probe_pos + kMaxW * 4);
+    CU(cudaMemcpyAsync(pos_dev, probe_pos, (size_t)W * 4, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(qptr_dev + 2 * pb, q_layers + 2 * pb, (size_t)(pe - pb) * 2 * sizeof(void*), cudaMemcpyHostToDevice, st));
+    ProbeArgs a;
+    a.unit_begin = pb * s.Hkv; a.unit_count = (pe - pb) * s.Hkv;
+    a.T = T; a.d = s.d; a.Hq = s.Hq; a.Hkv = s.Hkv; a.G = s.G; a.W = W;
+    a.unit_stride = (int64_t)s.Tmax * s.d; a.kcap = s.kcap;
+    a.ntiles_max = s.ntiles_max; a.nptiles_max = s.nptiles_max;
+    a.z1 = c->work + c->ws.z1;
+    a.idx = wsp<int32_t>(c, c->ws.idx);
+    a.tile_off = wsp<int32_t>(c, c->ws.tile_off);
+    a.q_layers_dev = qptr_dev;
+    a.pos = pos_dev;
+    a.part = wsp<double>(c, c->ws.probe_part);
+    a.scores = wsp<double>(c, c->ws.scores);
+    a.modes = wsp<int32_t>(c, c->ws.modes);
+    a.lambda = lambda;
+    const double e = s.esize, Td = (double)T * s.d;
+    const double k = (double)((int64_t)T * s.d * s.keep_num / s.keep_den);
+    const double b_sh = 2.0 * Td * e, b_rs = b_sh + 2.0 * k * (e + 4.0), b_ex = 4.0 * Td * e;
+    a.omega[0] = b_sh / b_ex; a.omega[1] = b_rs / b_ex; a.omega[2] = 1.0;
+    a.modes_out = modes; a.scores_out = scores;
+    CU(launch_probe(a, s.dtype, st));
+    for (int p = pb; p < pe; ++p) c->pair_probed[p] = 1;
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_set_modes(fdkv_ctx* c, int32_t seq, const int32_t* modes_host) {
+    if (!seq_ok(c, seq) || !modes_host) return FDKV_ERR_INVALID_ARG;
+    if (c->staged_seq != seq) return FDKV_ERR_STATE;
+    for (int i = 0; i < c->s.NU; ++i)
+        if (modes_host[i] < 0 || modes_host[i] > 2) return FDKV_ERR_INVALID_ARG;
+    c->seqs[seq].modes.assign(modes_host, modes_host + c->s.NU);
+    c->modes_overridden = true;
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
+    if (!seq_ok(c, seq)) return FDKV_ERR_INVALID_ARG;
+    if (c->staged_seq != seq || c->seqs[seq].committed) return FDKV_ERR_STATE;
+    const Shape& s = c->s;
+    for (int p = 0; p < s.P; ++p)
+        if (!c->pair_compressed[p] || (!c->modes_overridden && !c->pair_probed[p])) return FDKV_ERR_STATE;
+    cudaStream_t st = S(stream);
+    SeqState& q = c->seqs[seq];
+    CU(cudaStreamSynchronize(st));
+    if (!c->modes_overridden)
+        CU(cudaMemcpy(q.modes.data(), c->work + c->ws.modes, (size_t)s.NU * 4, cudaMemcpyDeviceToHost));
+    const int T = c->staged_T;
+    const size_t rows = (size_t)T * s.d * s.esize;
+    const int64_t k = (int64_t)T * s.d * s.keep_num / s.keep_den;
+    const int ntiles = (T + kResTile - 1) / kResTile;
+    // list copies include the slack so that aligned over-reads of the last tile stay inside the allocation
+    const size_t idx_b = (size_t)(k + kListPad) * 4, val_b = (size_t)(k + kListPad) * s.esize, off_b = (size_t)(ntiles + 1) * 4;
+    size_t need = 0;
+    for (int u = 0; u < s.NU; ++u) {
+        const int m = q.modes[u];
+        if (m < 0 || m > 2) return FDKV_ERR_STATE;
+        if (m == FDKV_MODE_EXACT) need += 4 * align_up(rows);
+        else need += 2 * align_up(rows) + (m == FDKV_MODE_RESIDUAL ? 2 * (align_up(idx_b) + align_up(val_b) + align_up(off_b)) : 0);
+    }
+    if (c->bump + need > c->arena_bytes) return FDKV_ERR_ARENA_FULL;
+    size_t o = c->bump;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return c->arena + r; };
+    size_t by_mode[3] = {0, 0, 0};
+    const size_t unit_stride_b = (size_t)s.Tmax * s.d * s.esize;
+    for (int u = 0; u < s.NU; ++u) {
+        const int m = q.modes[u], p = u / s.Hkv, h = u % s.Hkv;
+        UnitDesc* d0 = &c->desc_host[((size_t)seq * s.L + 2 * p) * s.Hkv + h];
+        UnitDesc* d1 = &c->desc_host[((size_t)seq * s.L + 2 * p + 1) * s.Hkv + h];
+        std::memset(d0, 0, sizeof(UnitDesc));
+        std::memset(d1, 0, sizeof(UnitDesc));
+        d0->mode = d1->mode = m;
+        d0->T = d1->T = T;
+        d0->sign = 1.f;
+        d1->sign = -1.f;
+        if (m == FDKV_MODE_EXACT) {
+            const void* src[4] = {c->k_layers[2 * p], c->k_layers[2 * p + 1], c->v_layers[2 * p], c->v_layers[2 * p + 1]};
+            char* dst[4];
+            for (int i = 0; i < 4; ++i) {
+                dst[i] = take(rows);
+                const char* sp = (const char*)src[i] + (size_t)h * c->stride_h * s.esize;
+                CU(launch_strided_copy(sp, c->stride_t, dst[i], T, s.d, s.esize, st));
+            }
+            d0->k_rows = dst[0]; d1->k_rows = dst[1];
+            d0->v_rows = dst[2]; d1->v_rows = dst[3];
+            by_mode[2] += 4 * rows;
+        } else {
+            for (int is_v = 0; is_v < 2; ++is_v) {
+                const size_t ut = (size_t)u * 2 + is_v;
+                char* z0 = take(rows);
+                CU(cudaMemcpyAsync(z0, c->work + c->ws.z0 + ut * unit_stride_b, rows, cudaMemcpyDeviceToDevice, st));
+                (is_v ? d0->v_rows : d0->k_rows) = z0;
+                (is_v ? d1->v_rows : d1->k_rows) = z0;
+                by_mode[m] += rows;
+                if (m == FDKV_MODE_RESIDUAL) {
+                    char* pi = take(idx_b);
+                    char* pv = take(val_b);
+                    char* po = take(off_b);
+                    CU(cudaMemcpyAsync(pi, c->work + c->ws.idx + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
+                    CU(cudaMemcpyAsync(pv, c->work + c->ws.val + ut * s.kcap * s.esize, val_b, cudaMemcpyDeviceToDevice, st));
+                    CU(cudaMemcpyAsync(po, c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, off_b, cudaMemcpyDeviceToDevice, st));
+                    for (UnitDesc* d : {d0, d1}) {
+                        (is_v ? d->v_idx : d->k_idx) = (const int32_t*)pi;
+                        (is_v ? d->v_val : d->k_val) = pv;
+                        (is_v ? d->v_off : d->k_off) = (const int32_t*)po;
+                    }
+                    by_mode[1] += (size_t)k * (4 + s.esize);
+                }
+            }
+        }
+    }
+    const size_t seq_desc = (size_t)s.L * s.Hkv;
+    CU(cudaMemcpyAsync(c->arena + c->ar.desc + (size_t)seq * seq_desc * sizeof(UnitDesc), &c->desc_host[(size_t)seq * seq_desc],
+                       seq_desc * sizeof(UnitDesc), cudaMemcpyHostToDevice, st));
+    CU(cudaStreamSynchronize(st));
+    c->bump = o;
+    q.committed = true;
+    q.T = T;
+    for (int i = 0; i < 3; ++i) q.bytes_by_mode[i] = by_mode[i];
+    return FDKV_OK;
+}
+
+static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const void* q, const void* k_new,
+                               const void* v_new, void* out, int32_t out_dtype, cudaStream_t st) {
+    const Shape& s = c->s;
+    int Tmax = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (!c->seqs[b].committed) return FDKV_ERR_STATE;
+        Tmax = c->seqs[b].T > Tmax ? c->seqs[b].T : Tmax;
+    }
+    if (k_new) {
+        for (int b = 0; b < batch; ++b)
+            if (c->seqs[b].tail_len[layer] >= s.max_tail) return FDKV_ERR_STATE;
+        for (int b = 0; b < batch; ++b) c->seqs[b].tail_len[layer]++;
+    }
+    DecodeArgs a;
+    a.desc = arp<UnitDesc>(c, c->ar.desc);
+    a.L = s.L; a.layer = layer; a.batch = batch; a.Hq = s.Hq; a.Hkv = s.Hkv; a.G = s.G; a.d = s.d;
+    a.max_tail = s.max_tail; a.max_batch = s.max_batch; a.Tmax_batch = Tmax;
+    a.q = q; a.k_new = k_new; a.v_new = v_new; a.out = out; a.out_dtype = out_dtype;
+    a.tail_k = c->arena + c->ar.tail_k; a.tail_v = c->arena + c->ar.tail_v;
+    a.tail_len = arp<int32_t>(c, c->ar.tail_len);
+    a.partials = wsp<float>(c, c->ws.partials);
+    a.status = wsp<int32_t>(c, c->ws.status);
+    CU(launch_decode(a, s.dtype, st));
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_decode_attn(fdkv_ctx* c, int32_t layer, int32_t batch, const void* q, const void* k_new,
+                             const void* v_new, void* out, int32_t out_dtype, void* stream) {
+    if (!c || !q || !out) return FDKV_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->s.L || batch < 1 || batch > c->s.max_batch) return FDKV_ERR_INVALID_ARG;
+    if ((k_new == nullptr) != (v_new == nullptr)) return FDKV_ERR_INVALID_ARG;
+    if (out_dtype != FDKV_F32 && out_dtype != FDKV_BF16) return FDKV_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(out, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return FDKV_ERR_INVALID_ARG;
+    return decode_impl(c, layer, batch, q, k_new, v_new, out, out_dtype, S(stream));
+}
+
+fdkv_status fdkv_decode_attn_host(fdkv_ctx* c, int32_t layer, int32_t batch, const void* q, const void* k_new,
+                                  const void* v_new, void* out, int32_t out_dtype, void* stream) {
+    if (!c || !q || !out) return FDKV_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->s.L || batch < 1 || batch > c->s.max_batch) return FDKV_ERR_INVALID_ARG;
+    if ((k_new == nullptr) != (v_new == nullptr)) return FDKV_ERR_INVALID_ARG;
+    if (out_dtype != FDKV_F32 && out_dtype != FDKV_BF16) return FDKV_ERR_INVALID_ARG;
+    const Shape& s = c->s;
+    cudaStream_t st = S(stream);
+    const size_t qb = (size_t)batch * s.Hq * s.d * s.esize, kb = (size_t)batch * s.Hkv * s.d * s.esize;
+    const size_t ob = (size_t)batch * s.Hq * s.d * (out_dtype == FDKV_BF16 ? 2 : 4);
+    CU(cudaMemcpyAsync(c->work + c->ws.io_q, q, qb, cudaMemcpyHostToDevice, st));
+    if (k_new) {
+        CU(cudaMemcpyAsync(c->work + c->ws.io_k, k_new, kb, cudaMemcpyHostToDevice, st));
+        CU(cudaMemcpyAsync(c->work + c->ws.io_v, v_new, kb, cudaMemcpyHostToDevice, st));
+    }
+    fdkv_status r = decode_impl(c, layer, batch, c->work + c->ws.io_q, k_new ? c->work + c->ws.io_k : nullptr,
+                                k_new ? c->work + c->ws.io_v : nullptr, c->work + c->ws.io_out, out_dtype, st);
+    if (r != FDKV_OK) return r;
+    CU(cudaMemcpyAsync(out, c->work + c->ws.io_out, ob, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_set_tail_len(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
+    if (!seq_ok(c, seq) || n < 0) return FDKV_ERR_INVALID_ARG;
+    for (int l = 0; l < c->s.L; ++l)
+        if (n > c->seqs[seq].tail_len[l]) return FDKV_ERR_INVALID_ARG;
+    CU(launch_set_tail_len(arp<int32_t>(c, c->ar.tail_len), c->s.L, c->s.max_batch, seq, n, S(stream)));
+    c->seqs[seq].tail_len.assign(c->s.L, n);
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_get_shared(fdkv_ctx* c, int32_t seq, int32_t pair, int32_t h, int32_t is_v, void* z0_out, void* stream) {
+    if (!seq_ok(c, seq) || !z0_out || pair < 0 || pair >= c->s.P || h < 0 || h >= c->s.Hkv) return FDKV_ERR_INVALID_ARG;
+    if (c->staged_seq != seq || !c->pair_compressed[pair]) return FDKV_ERR_STATE;
+    const Shape& s = c->s;
+    const size_t ut = ((size_t)pair * s.Hkv + h) * 2 + (is_v ? 1 : 0);
+    CU(cudaMemcpyAsync(z0_out, c->work + c->ws.z0 + ut * s.Tmax * s.d * s.esize, (size_t)c->staged_T * s.d * s.esize,
+                       cudaMemcpyDeviceToDevice, S(stream)));
+    CU(cudaStreamSynchronize(S(stream)));
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_get_residual(fdkv_ctx* c, int32_t seq, int32_t pair, int32_t h, int32_t is_v, int32_t* idx_out,
+                              void* val_out, int32_t* count_host, void* stream) {
+    if (!seq_ok(c, seq) || pair < 0 || pair >= c->s.P || h < 0 || h >= c->s.Hkv) return FDKV_ERR_INVALID_ARG;
+    if (c->staged_seq != seq || !c->pair_compressed[pair]) return FDKV_ERR_STATE;
+    const Shape& s = c->s;
+    const size_t ut = ((size_t)pair * s.Hkv + h) * 2 + (is_v ? 1 : 0);
+    const int64_t k = (int64_t)c->staged_T * s.d * s.keep_num / s.keep_den;
+    if (count_host) *count_host = (int32_t)k;
+    if (idx_out && k) CU(cudaMemcpyAsync(idx_out, c->work + c->ws.idx + ut * s.kcap * 4, (size_t)k * 4, cudaMemcpyDeviceToDevice, S(stream)));
+    if (val_out && k) CU(cudaMemcpyAsync(val_out, c->work + c->ws.val + ut * s.kcap * s.esize, (size_t)k * s.esize, cudaMemcpyDeviceToDevice, S(stream)));
+    CU(cudaStreamSynchronize(S(stream)));
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_get_modes(fdkv_ctx* c, int32_t seq, int32_t* modes_host) {
+    if (!seq_ok(c, seq) || !modes_host) return FDKV_ERR_INVALID_ARG;
+    if (!c->seqs[seq].committed && !(c->staged_seq == seq && c->modes_overridden)) return FDKV_ERR_STATE;
+    std::memcpy(modes_host, c->seqs[seq].modes.data(), (size_t)c->s.NU * 4);
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_footprint(fdkv_ctx* c, int32_t seq, size_t* bytes_by_mode_host, size_t* exact_equiv_bytes_host) {
+    if (!seq_ok(c, seq)) return FDKV_ERR_INVALID_ARG;
+    if (!c->seqs[seq].committed) return FDKV_ERR_STATE;
+    if (bytes_by_mode_host)
+        for (int i = 0; i < 3; ++i) bytes_by_mode_host[i] = c->seqs[seq].bytes_by_mode[i];
+    if (exact_equiv_bytes_host)
+        *exact_equiv_bytes_host = (size_t)c->s.NU * 4 * c->seqs[seq].T * c->s.d * c->s.esize;
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_decode_bytes(fdkv_ctx* c, int32_t layer, int32_t batch, size_t* bytes_host) {
+    if (!c || !bytes_host || layer < 0 || layer >= c->s.L || batch < 1 || batch > c->s.max_batch) return FDKV_ERR_INVALID_ARG;
+    const Shape& s = c->s;
+    size_t tot = 0;
+    for (int b = 0; b < batch; ++b) {
+        const SeqState& q = c->seqs[b];
+        if (!q.committed) return FDKV_ERR_STATE;
+        const int64_t k = (int64_t)q.T * s.d * s.keep_num / s.keep_den;
+        const int ntiles = (q.T + kResTile - 1) / kResTile;
+        for (int h = 0; h < s.Hkv; ++h) {
+            const int m = q.modes[(layer / 2) * s.Hkv + h];
+            tot += 2 * (size_t)(q.T + q.tail_len[layer]) * s.d * s.esize;
+            if (m == FDKV_MODE_RESIDUAL) tot += 2 * ((size_t)k * (4 + s.esize) + (size_t)(ntiles + 1) * 4);
+        }
+    }
+    *bytes_host = tot;
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_device_status(fdkv_ctx* c) {
+    if (!c) return FDKV_ERR_INVALID_ARG;
+    int32_t flag = 0;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(&flag, c->work + c->ws.status, 4, cudaMemcpyDeviceToHost));
+    if (flag == kFlagOk) return FDKV_OK;
+    return flag == kFlagTimeout ? FDKV_ERR_TIMEOUT : FDKV_ERR_DEVICE;
+}
+
+int32_t fdkv_last_cuda_error(void) { return g_last_cuda.load(); }
+
+const char* fdkv_status_str(fdkv_status s) {
+    switch (s) {
+        case FDKV_OK: return "ok";
+        case FDKV_ERR_INVALID_ARG: return "invalid argument";
+        case FDKV_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case FDKV_ERR_ARENA_FULL: return "arena full";
+        case FDKV_ERR_WORKSPACE: return "workspace too small";
+        case FDKV_ERR_STATE: return "call order / state";
+        case FDKV_ERR_CUDA: return "CUDA runtime error";
+        case FDKV_ERR_TIMEOUT: return "device wait timed out";
+        case FDKV_ERR_DEVICE: return "device-side check failed";
+    }
+    return "unknown";
+}
+
+int64_t fdkv_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,421 @@
+// Prefill compression kernels: depth split (Eq. 1, B = 2) fused with the magnitude histogram, the
+// radix-select threshold, and the index-ordered compaction of the sparse residual (Eq. 3, entry form).
+#include <algorithm>
+
+#include "fdkv_internal.h"
+
+namespace fdkv {
+
+namespace {
+
+__device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+// ----- storage traits -------------------------------------------------------------------------------
+template <typename T>
+struct Store;
+template <>
+struct Store<float> {
+    static constexpr int VEC = 4;
+    using vec_t = float4;
+    __device__ static void unpack(const vec_t& v, float* f) { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
+    __device__ static vec_t pack(const float* f) { return make_float4(f[0], f[1], f[2], f[3]); }
+};
+template <>
+struct Store<__nv_bfloat16> {
+    static constexpr int VEC = 8;
+    using vec_t = uint4;
+    __device__ static void unpack(const vec_t& v, float* f) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    // f holds float32 values; round each to nearest-even bf16
+    __device__ static vec_t pack(const float* f) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t lo = __bfloat16_as_ushort(__float2bfloat16_rn(f[2 * i]));
+            uint32_t hi = __bfloat16_as_ushort(__float2bfloat16_rn(f[2 * i + 1]));
+            w[i] = lo | (hi << 16);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// value as stored, widened back to float32 (exact)
+template <typename T>
+__device__ __forceinline__ float stored(float x);
+template <>
+__device__ __forceinline__ float stored<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ float stored<__nv_bfloat16>(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+// ----- C1: depth split + histogram of the top 15 magnitude bits of z1 ---------------------------------
+// grid (chunks, Hkv*2); each CTA owns a token range of one unit-tensor and a private 128 KiB histogram.
+template <typename T>
+__global__ void __launch_bounds__(1024) split_hist_kernel(CompressArgs a, int tokens_per_cta) {
+    extern __shared__ uint32_t s_hist[];
+    using S = Store<T>;
+    constexpr int VEC = S::VEC;
+    for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) s_hist[b] = 0;
+    __syncthreads();
+
+    const int h = blockIdx.y >> 1, is_v = blockIdx.y & 1;
+    const int ut = a.ut_base + blockIdx.y;
+    const T* x0 = reinterpret_cast<const T*>(is_v ? a.v0 : a.k0) + (int64_t)h * a.stride_h;
+    const T* x1 = reinterpret_cast<const T*>(is_v ? a.v1 : a.k1) + (int64_t)h * a.stride_h;
+    T* z0 = reinterpret_cast<T*>(a.z0) + (int64_t)ut * a.unit_stride;
+    T* z1 = reinterpret_cast<T*>(a.z1) + (int64_t)ut * a.unit_stride;
+    const float c32 = __uint_as_float(0x3F3504F3u);
+
+    const int t_begin = blockIdx.x * tokens_per_cta;
+    const int t_end = min(a.T, t_begin + tokens_per_cta);
+    const int vpr = a.d / VEC;
+    const int64_t nvec = (int64_t)max(0, t_end - t_begin) * vpr;
+    for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
+        const int t = t_begin + (int)(v / vpr);
+        const int cv = (int)(v % vpr) * VEC;
+        const typename S::vec_t va = *reinterpret_cast<const typename S::vec_t*>(x0 + (int64_t)t * a.stride_t + cv);
+        const typename S::vec_t vb = *reinterpret_cast<const typename S::vec_t*>(x1 + (int64_t)t * a.stride_t + cv);
+        float fa[VEC], fb[VEC], f0[VEC], f1[VEC];
+        S::unpack(va, fa);
+        S::unpack(vb, fb);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            // one float32 add (subtract), one float32 multiply: never contracted into an FMA
+            f0[i] = __fmul_rn(__fadd_rn(fa[i], fb[i]), c32);
+            f1[i] = __fmul_rn(__fsub_rn(fa[i], fb[i]), c32);
+        }
+        *reinterpret_cast<typename S::vec_t*>(z0 + (int64_t)t * a.d + cv) = S::pack(f0);
+        *reinterpret_cast<typename S::vec_t*>(z1 + (int64_t)t * a.d + cv) = S::pack(f1);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) atomicAdd(&s_hist[key_of(stored<T>(f1[i])) >> 16], 1u);
+    }
+    __syncthreads();
+    uint32_t* gh = a.hist + (int64_t)ut * kHistBins;
+    for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) {
+        const uint32_t c = s_hist[b];
+        if (c) atomicAdd(&gh[b], c);
+    }
+}
+
+// ----- C2: threshold from a histogram --------------------------------------------------------------
+// One CTA per unit-tensor.  Scans `nbins` bins from the top: finds the bin where the running count of larger
+// keys first reaches k_rem, appends the bin to the prefix and lowers k_rem.  Clears the bins it read.
+// On the last pass writes tau (prefix left-aligned to 31 bits) and need.
+__global__ void __launch_bounds__(1024) threshold_kernel(uint32_t* hist, SelState* sel, int ut_begin, int nbins,
+                                                         int bits, int first, int last, int shift_final,
+                                                         uint32_t k_init) {
+    __shared__ uint32_t s_part[1024];
+    __shared__ uint32_t s_found_bin, s_found_above;
+    const int ut = ut_begin + blockIdx.x;
+    uint32_t* h = hist + (int64_t)ut * kHistBins;
+    SelState st = sel[ut];
+    if (first) { st.prefix = 0; st.k_rem = k_init; }
+    const int per = nbins / blockDim.x;  // nbins is a multiple of blockDim (32768 or 256 with 256 threads)
+    // thread i owns bins [nbins - (i+1)*per, nbins - i*per): thread 0 owns the largest keys
+    const int hi = nbins - threadIdx.x * per;
+    uint32_t mine = 0;
+    for (int b = hi - 1; b >= hi - per; --b) mine += h[b];
+    s_part[threadIdx.x] = mine;
+    if (threadIdx.x == 0) { s_found_bin = 0xFFFFFFFFu; s_found_above = 0; }
+    __syncthreads();
+    // exclusive prefix over threads (counts of strictly larger bins), simple Hillis-Steele in shared memory
+    uint32_t incl = mine;
+    for (int off = 1; off < blockDim.x; off <<= 1) {
+        uint32_t add = threadIdx.x >= off ? s_part[threadIdx.x - off] : 0;
+        __syncthreads();
+        incl += add;
+        s_part[threadIdx.x] = incl;
+        __syncthreads();
+    }
+    uint32_t above = incl - mine;
+    if (st.k_rem > 0 && above < st.k_rem && st.k_rem <= above + mine) {
+        for (int b = hi - 1; b >= hi - per; --b) {
+            const uint32_t c = h[b];
+            if (st.k_rem <= above + c) { s_found_bin = (uint32_t)b; s_found_above = above; break; }
+            above += c;
+        }
+    }
+    __syncthreads();
+    for (int b = hi - 1; b >= hi - per; --b) h[b] = 0;
+    if (threadIdx.x == 0) {
+        if (st.k_rem == 0 || s_found_bin == 0xFFFFFFFFu) {
+            // nothing (left) to take: a threshold above every key
+            st.prefix = 0xFFFFFFFFu;
+            st.k_rem = 0;
+            if (last) { st.tau = 0xFFFFFFFFu; st.need = 0; }
+        } else {
+            st.prefix = (st.prefix << bits) | s_found_bin;
+            st.k_rem -= s_found_above;
+            if (last) { st.tau = st.prefix << shift_final; st.need = st.k_rem; }
+        }
+        sel[ut] = st;
+    }
+}
+
+// ----- C2b (float32 only): histogram of the next 8 key bits among entries that match the prefix ------
+__global__ void __launch_bounds__(256) refine_hist_kernel(const float* z1, int64_t unit_stride, int64_t n,
+                                                          int ut_begin, const SelState* sel, uint32_t* hist,
+                                                          int shift_prefix, int shift_digit) {
+    __shared__ uint32_t s_h[256];
+    const int ut = ut_begin + blockIdx.y;
+    s_h[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t prefix = sel[ut].prefix;
+    if (prefix != 0xFFFFFFFFu) {
+        const float* z = z1 + (int64_t)ut * unit_stride;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+            const uint32_t key = key_of(z[i]);
+            if ((key >> shift_prefix) == prefix) atomicAdd(&s_h[(key >> shift_digit) & 0xFFu], 1u);
+        }
+    }
+    __syncthreads();
+    if (s_h[threadIdx.x]) atomicAdd(&hist[(int64_t)ut * kHistBins + threadIdx.x], s_h[threadIdx.x]);
+}
+
+// ----- C3: per 32-token tile, how many keys are above / equal to the threshold ------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) tile_count_kernel(SelectArgs a) {
+    using S = Store<T>;
+    constexpr int VEC = S::VEC;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x * 8 + warp;
+    const int ut = a.ut_begin + blockIdx.y;
+    const int ntiles = (a.T + kResTile - 1) / kResTile;
+    if (tile >= ntiles) return;
+    const uint32_t tau = a.sel[ut].tau;
+    const T* z = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride;
+    const int64_t e_begin = (int64_t)tile * kResTile * a.d;
+    const int64_t e_end = min((int64_t)a.T * a.d, e_begin + (int64_t)kResTile * a.d);
+    uint32_t gt = 0, eq = 0;
+    for (int64_t e = e_begin + lane * VEC; e < e_end; e += 32 * VEC) {
+        float f[VEC];
+        S::unpack(*reinterpret_cast<const typename S::vec_t*>(z + e), f);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const uint32_t k = key_of(f[i]);
+            gt += k > tau;
+            eq += k == tau;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o);
+        eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o);
+    }
+    if (lane == 0) {
+        a.tile_cnt[((int64_t)ut * a.ntiles_max + tile) * 2 + 0] = gt;
+        a.tile_cnt[((int64_t)ut * a.ntiles_max + tile) * 2 + 1] = eq;
+    }
+}
+
+// ----- C4: index-ordered scan over tiles ------------------------------------------------------------
+// off[j] = (#keys > tau before tile j) + min(#keys == tau before tile j, need); eq_base[j] = #keys == tau before j.
+__global__ void __launch_bounds__(1024) tile_scan_kernel(SelectArgs a) {
+    __shared__ uint32_t s_gt[1024], s_eq[1024];
+    const int ut = a.ut_begin + blockIdx.x;
+    const int ntiles = (a.T + kResTile - 1) / kResTile;
+    const uint32_t need = a.sel[ut].need;
+    const uint32_t* cnt = a.tile_cnt + (int64_t)ut * a.ntiles_max * 2;
+    uint32_t* eqb = a.tile_eq + (int64_t)ut * a.ntiles_max;
+    int32_t* off = a.tile_off + (int64_t)ut * (a.ntiles_max + 1);
+    uint32_t carry_gt = 0, carry_eq = 0;
+    for (int base = 0; base < ntiles; base += 1024) {
+        const int j = base + threadIdx.x;
+        const uint32_t g = j < ntiles ? cnt[2 * j] : 0, e = j < ntiles ? cnt[2 * j + 1] : 0;
+        uint32_t ig = g, ie = e;
+        s_gt[threadIdx.x] = ig;
+        s_eq[threadIdx.x] = ie;
+        __syncthreads();
+        for (int o = 1; o < 1024; o <<= 1) {
+            const uint32_t ag = threadIdx.x >= o ? s_gt[threadIdx.x - o] : 0;
+            const uint32_t ae = threadIdx.x >= o ? s_eq[threadIdx.x - o] : 0;
+            __syncthreads();
+            ig += ag;
+            ie += ae;
+            s_gt[threadIdx.x] = ig;
+            s_eq[threadIdx.x] = ie;
+            __syncthreads();
+        }
+        if (j < ntiles) {
+            const uint32_t pg = carry_gt + ig - g, pe = carry_eq + ie - e;
+            off[j] = (int32_t)(pg + min(pe, need));
+            eqb[j] = pe;
+        }
+        carry_gt += s_gt[1023];
+        carry_eq += s_eq[1023];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const uint32_t total = carry_gt + min(carry_eq, need);
+        off[ntiles] = (int32_t)total;
+        if ((int64_t)total != a.k) atomicMax(a.status, (int32_t)kFlagCountMismatch);
+    }
+}
+
+// ----- C5: ordered write ---------------------------------------------------------------------------
+// One warp per tile walks its entries in flat-index order; an entry is kept when its key is above the
+// threshold, or equal to it and among the first `need` such entries of the whole unit-tensor.
+template <typename T>
+__global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
+    using S = Store<T>;
+    constexpr int VEC = S::VEC;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x * 8 + warp;
+    const int ut = a.ut_begin + blockIdx.y;
+    const int ntiles = (a.T + kResTile - 1) / kResTile;
+    if (tile >= ntiles) return;
+    const uint32_t tau = a.sel[ut].tau, need = a.sel[ut].need;
+    const T* z = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride;
+    int32_t* idx = a.idx + (int64_t)ut * a.kcap;
+    T* val = reinterpret_cast<T*>(a.val) + (int64_t)ut * a.kcap;
+    uint32_t pos = (uint32_t)a.tile_off[(int64_t)ut * (a.ntiles_max + 1) + tile];
+    uint32_t eq_rank = a.tile_eq[(int64_t)ut * a.ntiles_max + tile];
+    const int64_t e_begin = (int64_t)tile * kResTile * a.d;
+    const int64_t e_end = min((int64_t)a.T * a.d, e_begin + (int64_t)kResTile * a.d);
+    for (int64_t base = e_begin; base < e_end; base += 32 * VEC) {
+        const int64_t e = base + lane * VEC;
+        float f[VEC];
+        uint32_t is_gt = 0, is_eq = 0;
+        if (e < e_end) {
+            S::unpack(*reinterpret_cast<const typename S::vec_t*>(z + e), f);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const uint32_t k = key_of(f[i]);
+                is_gt |= (uint32_t)(k > tau) << i;
+                is_eq |= (uint32_t)(k == tau) << i;
+            }
+        }
+        // rank of this lane's first tie among the unit-tensor's ties
+        uint32_t keep = is_gt;
+        const uint32_t any_eq = __ballot_sync(0xFFFFFFFFu, is_eq != 0);
+        if (any_eq) {
+            const uint32_t n_eq = __popc(is_eq);
+            uint32_t incl = n_eq;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            uint32_t r = eq_rank + incl - n_eq;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i)
+                if (is_eq >> i & 1u) {
+                    if (r < need) keep |= 1u << i;
+                    ++r;
+                }
+            eq_rank += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        }
+        const uint32_t n_keep = __popc(keep);
+        uint32_t incl = n_keep;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        uint32_t w = pos + incl - n_keep;
+#pragma unroll
+        for (int i = 0; i < VEC; ++i)
+            if (keep >> i & 1u) {
+                idx[w] = (int32_t)(e + i);
+                val[w] = z[e + i];
+                ++w;
+            }
+        pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+}
+
+template <typename T>
+__global__ void strided_copy_kernel(const T* src, int64_t stride_t, T* dst, int T_, int d) {
+    using S = Store<T>;
+    constexpr int VEC = S::VEC;
+    const int vpr = d / VEC;
+    const int64_t n = (int64_t)T_ * vpr;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < n; v += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t t = v / vpr;
+        const int cv = (int)(v % vpr) * VEC;
+        *reinterpret_cast<typename S::vec_t*>(dst + t * d + cv) =
+            *reinterpret_cast<const typename S::vec_t*>(src + t * stride_t + cv);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_split_hist(const CompressArgs& a, int dtype, cudaStream_t st) {
+    static bool attr_done = false;
+    const size_t smem = (size_t)kHistBins * sizeof(uint32_t);
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(split_hist_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(split_hist_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    if (a.T <= 0) return cudaSuccess;
+    const int tokens_per_cta = 4096 * 128 / a.d / (dtype == FDKV_BF16 ? 1 : 2);
+    dim3 grid((a.T + tokens_per_cta - 1) / tokens_per_cta, a.Hkv * 2);
+    if (dtype == FDKV_BF16)
+        split_hist_kernel<__nv_bfloat16><<<grid, 1024, smem, st>>>(a, tokens_per_cta);
+    else
+        split_hist_kernel<float><<<grid, 1024, smem, st>>>(a, tokens_per_cta);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream_t st) {
+    if (a.ut_count <= 0) return cudaSuccess;
+    const uint32_t k = (uint32_t)a.k;
+    const int64_t n = (int64_t)a.T * a.d;
+    if (dtype == FDKV_BF16) {
+        threshold_kernel<<<a.ut_count, 1024, 0, st>>>(a.hist, a.sel, a.ut_begin, kHistBins, 15, 1, 1, 16, k);
+        count_launch(1);
+    } else {
+        threshold_kernel<<<a.ut_count, 1024, 0, st>>>(a.hist, a.sel, a.ut_begin, kHistBins, 15, 1, 0, 0, k);
+        const int chunks = (int)std::min<int64_t>(64, (n + 256 * 16 - 1) / (256 * 16));
+        refine_hist_kernel<<<dim3(chunks, a.ut_count), 256, 0, st>>>(reinterpret_cast<const float*>(a.z1), a.unit_stride,
+                                                                     n, a.ut_begin, a.sel, a.hist, 16, 8);
+        threshold_kernel<<<a.ut_count, 256, 0, st>>>(a.hist, a.sel, a.ut_begin, 256, 8, 0, 0, 0, k);
+        refine_hist_kernel<<<dim3(chunks, a.ut_count), 256, 0, st>>>(reinterpret_cast<const float*>(a.z1), a.unit_stride,
+                                                                     n, a.ut_begin, a.sel, a.hist, 8, 0);
+        threshold_kernel<<<a.ut_count, 256, 0, st>>>(a.hist, a.sel, a.ut_begin, 256, 8, 0, 1, 0, k);
+        count_launch(5);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int ntiles = (a.T + kResTile - 1) / kResTile;
+    if (ntiles > 0) {
+        dim3 grid((ntiles + 7) / 8, a.ut_count);
+        if (dtype == FDKV_BF16)
+            tile_count_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a);
+        else
+            tile_count_kernel<float><<<grid, 256, 0, st>>>(a);
+        tile_scan_kernel<<<a.ut_count, 1024, 0, st>>>(a);
+        if (dtype == FDKV_BF16)
+            tile_write_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a);
+        else
+            tile_write_kernel<float><<<grid, 256, 0, st>>>(a);
+        count_launch(3);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st) {
+    if (T <= 0) return cudaSuccess;
+    const int vec = esize == 2 ? 8 : 4;
+    const int64_t n = (int64_t)T * (d / vec);
+    const int blocks = (int)std::min<int64_t>(148 * 8, (n + 255) / 256);
+    if (esize == 2)
+        strided_copy_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(src), stride_t,
+                                                                  reinterpret_cast<__nv_bfloat16*>(dst), T, d);
+    else
+        strided_copy_kernel<float><<<blocks, 256, 0, st>>>(reinterpret_cast<const float*>(src), stride_t,
+                                                           reinterpret_cast<float*>(dst), T, d);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+}  // namespace fdkv

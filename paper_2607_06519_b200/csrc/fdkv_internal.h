@@ -1,0 +1,165 @@
+// Internal declarations shared by the translation units of libfdkv (not part of the public ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "../../include/fdkv.h"
+
+namespace fdkv {
+
+constexpr int kResTile = 32;         // tokens per residual-offset tile: off[j] = first list entry of tokens >= 32 j
+constexpr int kHistBins = 32768;     // one bin per 15-bit magnitude prefix (a whole bf16 key)
+constexpr int kMaxSplits = 128;      // split-K partial slots per (sequence, query head)
+constexpr int kMaxW = 128;           // probe queries
+constexpr int kListPad = 32;         // slack entries after each residual list (aligned over-reads stay in bounds)
+constexpr int kMaxGroup = 8;
+constexpr int kProbeTile = 64;       // tokens per probe CTA (generic kernel)
+
+enum DeviceFlag : int32_t { kFlagOk = 0, kFlagTimeout = 1, kFlagCountMismatch = 2, kFlagTailFull = 3 };
+
+// What decode reads for one (sequence, layer, KV head).
+struct UnitDesc {
+    const void* k_rows;  // [T][d]: Z0 of K (shared / residual) or the layer's original K rows (exact)
+    const void* v_rows;
+    const int32_t* k_idx;  // residual mode only: ascending flat indices t*d + ch
+    const void* k_val;
+    const int32_t* k_off;  // [ceil(T/32) + 1] first entry of each 32-token tile
+    const int32_t* v_idx;
+    const void* v_val;
+    const int32_t* v_off;
+    int32_t mode;
+    int32_t T;
+    float sign;  // +1 for the first layer of the pair, -1 for the second
+    int32_t pad;
+};
+
+struct SelState {
+    uint32_t prefix;  // magnitude-key prefix fixed so far (left-aligned in 31 bits once complete)
+    uint32_t k_rem;   // entries still to take at or below the prefix
+    uint32_t tau;     // final threshold key (31-bit magnitude pattern; bf16 keys are shifted left by 16)
+    uint32_t need;    // entries with key == tau to keep (lowest flat indices first)
+};
+
+struct Shape {
+    int L, P, Hq, Hkv, G, d;
+    int max_batch, Tmax, max_tail;
+    int dtype, esize;
+    int keep_num, keep_den;
+    int64_t kmax;      // floor(Tmax*d*num/den)
+    int64_t kcap;      // list capacity incl. slack
+    int ntiles_max;    // ceil(Tmax/32)
+    int nptiles_max;   // ceil(Tmax/kProbeTile)
+    int NU, NT;        // units and unit-tensors (K and V) of one sequence
+};
+
+struct WsLayout {
+    size_t status, z0, z1, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, probe_part, probe_pos, scores, modes,
+        partials, io_q, io_k, io_v, io_out, total;
+};
+struct ArenaLayout {
+    size_t tail_len, desc, tail_k, tail_v, bump, worst_total;
+};
+
+struct SeqState {
+    bool committed = false;
+    int T = 0;
+    std::vector<int32_t> modes;  // [NU], -1 unknown
+    size_t bytes_by_mode[3] = {0, 0, 0};
+    std::vector<int32_t> tail_len;  // host mirror per layer
+};
+
+}  // namespace fdkv
+
+struct fdkv_ctx {
+    fdkv_config cfg;
+    fdkv::Shape s;
+    fdkv::WsLayout ws;
+    fdkv::ArenaLayout ar;
+    char* arena;
+    size_t arena_bytes;
+    char* work;
+    size_t work_bytes;
+    size_t bump;  // next free arena offset
+    int staged_seq = -1;
+    int staged_T = 0;
+    std::vector<uint8_t> pair_compressed, pair_probed;
+    std::vector<const void*> k_layers, v_layers;
+    int64_t stride_t = 0, stride_h = 0;
+    bool modes_overridden = false;
+    std::vector<fdkv::SeqState> seqs;
+    std::vector<fdkv::UnitDesc> desc_host;  // [max_batch][L][Hkv]
+};
+
+namespace fdkv {
+
+// ---- launchers implemented in compress.cu / probe.cu / decode.cu; each returns cudaGetLastError() ----
+struct CompressArgs {
+    const void *k0, *k1, *v0, *v1;  // the four [T][Hkv][d] strided tensors of one pair
+    int64_t stride_t, stride_h;
+    int T, d, Hkv;
+    int ut_base;  // first unit-tensor of this pair in the stage: (pair*Hkv)*2
+    int64_t unit_stride;  // elements between staged unit-tensors (Tmax*d)
+    void *z0, *z1;
+    uint32_t* hist;
+};
+cudaError_t launch_split_hist(const CompressArgs& a, int dtype, cudaStream_t st);
+
+struct SelectArgs {
+    int ut_begin, ut_count;
+    int T, d;
+    int64_t k;
+    int64_t unit_stride, kcap;
+    int ntiles_max;
+    const void* z1;
+    uint32_t* hist;
+    SelState* sel;
+    uint32_t *tile_cnt, *tile_eq;
+    int32_t* tile_off;
+    int32_t* idx;
+    void* val;
+    int32_t* status;
+};
+cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream_t st);
+
+struct ProbeArgs {
+    int unit_begin, unit_count;  // units of the pair range (unit = pair*Hkv + h)
+    int T, d, Hq, Hkv, G, W;
+    int64_t unit_stride, kcap;
+    int ntiles_max, nptiles_max;
+    const void* z1;  // staged Z1 (unit-tensor ut = unit*2 for K)
+    const int32_t* idx;
+    const int32_t* tile_off;
+    const void* const* q_layers_dev;  // device array [L] of pointers
+    const int32_t* pos;
+    double* part;    // [NU][nptiles_max][2]
+    double* scores;  // [NU][2]
+    int32_t* modes;  // [NU]
+    double lambda, omega[3];
+    int32_t* modes_out;  // user buffers for the pair range, may be null
+    float* scores_out;
+};
+cudaError_t launch_probe(const ProbeArgs& a, int dtype, cudaStream_t st);
+
+struct DecodeArgs {
+    const UnitDesc* desc;  // [batch][.. layer ..] : desc + (b*L + layer)*Hkv + h
+    int L, layer, batch, Hq, Hkv, G, d, max_tail, max_batch;
+    int Tmax_batch;  // largest T among the batch (host side, sizes the grid)
+    const void *q, *k_new, *v_new;
+    void* out;
+    int out_dtype;
+    void *tail_k, *tail_v;  // [L][max_batch][Hkv][max_tail][d]
+    int32_t* tail_len;      // [L][max_batch]
+    float* partials;        // [batch][Hq][kMaxSplits][d+2]
+    int32_t* status;
+};
+cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st);
+cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st);
+
+void count_launch(int n);
+
+}  // namespace fdkv

@@ -1,0 +1,95 @@
+"""Drives a synthetic workload through the library: generate -> upload -> compress -> probe -> commit -> decode.
+
+Used by the GPU tests, the smoke check and the benchmark.  Everything numerical happens inside libfdkv; this
+module only moves seeded inputs to the device and calls the binding.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import synth
+
+
+def to_device(x: np.ndarray, dtype: str, device) -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(device)
+    return t.to(torch.bfloat16) if dtype == "bf16" else t
+
+
+def make_context(w: synth.Workload, max_tail: int | None = None, arena_bytes: int | None = None,
+                 device="cuda:0") -> B.Context:
+    cfg = B.Config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, w.T,
+                   max_tail if max_tail is not None else max(w.n_steps, 1), B.BF16 if w.dtype == "bf16" else B.F32,
+                   w.keep_num, w.keep_den)
+    return B.Context(cfg, device=device, arena_bytes=arena_bytes)
+
+
+class Prefilled:
+    """One workload with every sequence compressed, routed and committed."""
+
+    def __init__(self, w: synth.Workload, ctx: B.Context | None = None, max_tail: int | None = None,
+                 arena_bytes: int | None = None, device="cuda:0"):
+        self.w = w
+        self.device = torch.device(device)
+        self.ctx = ctx or make_context(w, max_tail, arena_bytes, device)
+        self.scores = {}
+        self.probe_modes = {}
+
+    def upload_pair(self, seq: int, pair: int):
+        kv = synth.layer_pair_kv(self.w, seq, pair)
+        return {n: to_device(a, self.w.dtype, self.device) for n, a in kv.items()}
+
+    def upload_probe_q(self, seq: int):
+        return [to_device(synth.probe_q(self.w, seq, l), self.w.dtype, self.device) for l in range(self.w.n_layers)]
+
+    def compress(self, seq: int, keep_inputs: bool = True):
+        """Uploads and compresses every pair of a sequence; returns the per-layer device tensors."""
+        w = self.w
+        k_layers, v_layers = [None] * w.n_layers, [None] * w.n_layers
+        for p in range(w.n_pairs):
+            t = self.upload_pair(seq, p)
+            k_layers[2 * p], k_layers[2 * p + 1] = t["k0"], t["k1"]
+            v_layers[2 * p], v_layers[2 * p + 1] = t["v0"], t["v1"]
+            self.ctx.compress_prefill(seq, p, p + 1, w.T, k_layers, v_layers)
+        return k_layers, v_layers
+
+    def probe(self, seq: int, lam: float):
+        q_layers = self.upload_probe_q(seq)
+        modes, scores = self.ctx.probe(seq, 0, self.w.n_pairs, q_layers, synth.probe_positions(self.w), lam)
+        torch.cuda.synchronize()
+        self.scores[seq] = scores.cpu().numpy().astype(np.float64)
+        self.probe_modes[seq] = modes.cpu().numpy()
+        return self.probe_modes[seq], self.scores[seq]
+
+    def prefill(self, seq: int, modes="quota", lam: float = 0.0):
+        """modes: 'probe' (the rule at lam), 'quota' (benchmark mix from the probe's scores) or an int array."""
+        kv = self.compress(seq)
+        if isinstance(modes, str):
+            pm, sc = self.probe(seq, lam)
+            if modes == "quota":
+                self.ctx.set_modes(seq, synth.quota_modes(sc[..., 0]))
+            elif modes != "probe":
+                raise ValueError(modes)
+        else:
+            self.ctx.set_modes(seq, np.asarray(modes, dtype=np.int32))
+        self.ctx.commit(seq)
+        del kv
+        return self.ctx.get_modes(seq).numpy()
+
+    # ---- decode-side inputs ----
+    def decode_q(self, layer: int, step: int) -> torch.Tensor:
+        w = self.w
+        q = np.stack([synth.decode_q(w, b, layer)[step] for b in range(w.batch)])
+        return to_device(q, w.dtype, self.device)
+
+    def new_rows(self, layer: int, step: int):
+        """k_new, v_new [batch, Hkv, d] of one layer and step."""
+        w = self.w
+        k = np.empty((w.batch, w.n_kv_heads, w.head_dim), np.float32)
+        v = np.empty_like(k)
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                k[b, h] = synth.tail_rows(w, b, layer // 2, h, False)[layer & 1][step]
+                v[b, h] = synth.tail_rows(w, b, layer // 2, h, True)[layer & 1][step]
+        return to_device(k, w.dtype, self.device), to_device(v, w.dtype, self.device)
