@@ -35,6 +35,7 @@ class Prefilled:
         self.ctx = ctx or make_context(w, max_tail, arena_bytes, device)
         self.scores = {}
         self.probe_modes = {}
+        self._inputs = {}  # the library reads exact-mode rows at commit: keep the uploads alive until then
 
     def upload_pair(self, seq: int, pair: int):
         kv = synth.layer_pair_kv(self.w, seq, pair)
@@ -52,7 +53,12 @@ class Prefilled:
             k_layers[2 * p], k_layers[2 * p + 1] = t["k0"], t["k1"]
             v_layers[2 * p], v_layers[2 * p + 1] = t["v0"], t["v1"]
             self.ctx.compress_prefill(seq, p, p + 1, w.T, k_layers, v_layers)
+        self._inputs[seq] = (k_layers, v_layers)
         return k_layers, v_layers
+
+    def commit(self, seq: int):
+        self.ctx.commit(seq)
+        self._inputs.pop(seq, None)
 
     def probe(self, seq: int, lam: float):
         q_layers = self.upload_probe_q(seq)
@@ -64,7 +70,7 @@ class Prefilled:
 
     def prefill(self, seq: int, modes="quota", lam: float = 0.0):
         """modes: 'probe' (the rule at lam), 'quota' (benchmark mix from the probe's scores) or an int array."""
-        kv = self.compress(seq)
+        self.compress(seq)
         if isinstance(modes, str):
             pm, sc = self.probe(seq, lam)
             if modes == "quota":
@@ -73,8 +79,7 @@ class Prefilled:
                 raise ValueError(modes)
         else:
             self.ctx.set_modes(seq, np.asarray(modes, dtype=np.int32))
-        self.ctx.commit(seq)
-        del kv
+        self.commit(seq)
         return self.ctx.get_modes(seq).numpy()
 
     # ---- decode-side inputs ----

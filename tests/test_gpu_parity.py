@@ -68,7 +68,7 @@ def test_tiny_compress_probe_decode(dtype):
         else:
             modes = np.array(forced)
             pf.ctx.set_modes(0, modes)
-        pf.ctx.commit(0)
+        pf.commit(0)
         assert np.array_equal(pf.ctx.get_modes(0).numpy(), modes)
         worst = _decode_all_layers(pf, w, [modes], units, out_dtype=0)
         assert worst <= TOL[dtype], (forced, worst)
@@ -100,7 +100,7 @@ def test_shapes_and_edges(dtype, T, d, Hq, Hkv, keep, tail):
         e = R.probe_error(u.z1["k"], u.kept["k"], pq[0], pq[1], w.group, h, synth.probe_positions(w))
         np.testing.assert_allclose(scores[0, h], e, rtol=1e-4, atol=1e-12)
     pf.ctx.set_modes(0, modes)
-    pf.ctx.commit(0)
+    pf.commit(0)
     for step in range(max(tail, 1)):
         worst = _decode_all_layers(pf, w, [modes], units, step=step, append=tail > 0)
         assert worst <= TOL[dtype], (step, worst)
@@ -152,7 +152,7 @@ def test_llama_shaped_reduced():
             np.testing.assert_allclose(scores[p, h], e, rtol=1e-4)
     modes = synth.quota_modes(scores[..., 0])
     pf.ctx.set_modes(0, modes)
-    pf.ctx.commit(0)
+    pf.commit(0)
     by_mode, exact_equiv = pf.ctx.footprint(0)
     assert exact_equiv == 4 * w.T * w.head_dim * 2 * w.n_pairs * w.n_kv_heads
     assert sum(by_mode) < exact_equiv
