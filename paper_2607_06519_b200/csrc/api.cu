@@ -43,6 +43,7 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.kcap = (int64_t)align_up((size_t)(s.kmax + kListPad), 64);
     s.ntiles_max = (s.Tmax + kResTile - 1) / kResTile;
     s.nptiles_max = (s.Tmax + kProbeTile - 1) / kProbeTile;
+    s.tail_rows = (s.max_tail + kRowPad - 1) / kRowPad * kRowPad;
     s.NU = s.P * s.Hkv;
     s.NT = 2 * s.NU;
     return true;
@@ -76,12 +77,13 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     o = 0;
     a.tail_len = take((size_t)s.L * s.max_batch * 4);
     a.desc = take((size_t)s.max_batch * s.L * s.Hkv * sizeof(UnitDesc));
-    const size_t tail = (size_t)s.L * s.max_batch * s.Hkv * s.max_tail * s.d * s.esize;
+    const size_t tail = (size_t)s.L * s.max_batch * s.Hkv * s.tail_rows * s.d * s.esize;
     a.tail_k = take(tail);
     a.tail_v = take(tail);
     a.bump = o;
-    const size_t exact_unit = 4 * align_up(unit_elems * s.esize);
-    const size_t resid_unit = 2 * align_up(unit_elems * s.esize) + 2 * align_up((size_t)s.kcap * 4) +
+    const size_t rows_pad = align_up((size_t)((s.Tmax + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize);
+    const size_t exact_unit = 4 * rows_pad;
+    const size_t resid_unit = 2 * rows_pad + 2 * align_up((size_t)s.kcap * 4) +
                               2 * align_up((size_t)s.kcap * s.esize) + 2 * align_up((size_t)(s.ntiles_max + 1) * 4);
     a.worst_total = a.bump + (size_t)s.max_batch * s.NU * (exact_unit > resid_unit ? exact_unit : resid_unit);
 }
@@ -142,7 +144,10 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     cudaError_t e = cudaMemset(c->arena + c->ar.tail_len, 0, (size_t)s.L * s.max_batch * 4);
     if (e == cudaSuccess) e = cudaMemset(c->work + c->ws.status, 0, 256);
     if (e == cudaSuccess) e = cudaMemset(c->arena + c->ar.desc, 0, c->desc_host.size() * sizeof(UnitDesc));
+    // tails start as zero rows: the fast decode kernel loads whole 64-row boxes and relies on finite padding
+    if (e == cudaSuccess) e = cudaMemset(c->arena + c->ar.tail_k, 0, c->ar.bump - c->ar.tail_k);
     if (e != cudaSuccess) { delete c; return cuda_fail(e); }
+    if (s.dtype == FDKV_BF16 && s.d == 128) c->has_tmap = make_arena_tensor_map(c->arena, arena_bytes, c->tmap);
     *out = c;
     return FDKV_OK;
 }
@@ -154,6 +159,7 @@ fdkv_status fdkv_reset(fdkv_ctx* c) {
     CU(cudaDeviceSynchronize());
     CU(cudaMemset(c->arena + c->ar.tail_len, 0, (size_t)c->s.L * c->s.max_batch * 4));
     CU(cudaMemset(c->work + c->ws.status, 0, 256));
+    CU(cudaMemset(c->arena + c->ar.tail_k, 0, c->ar.bump - c->ar.tail_k));
     c->bump = c->ar.bump;
     c->staged_seq = -1;
     for (auto& q : c->seqs) {
@@ -293,6 +299,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
         CU(cudaMemcpy(q.modes.data(), c->work + c->ws.modes, (size_t)s.NU * 4, cudaMemcpyDeviceToHost));
     const int T = c->staged_T;
     const size_t rows = (size_t)T * s.d * s.esize;
+    const size_t rows_pad = (size_t)((T + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize;  // zero rows up to a whole box
     const int64_t k = (int64_t)T * s.d * s.keep_num / s.keep_den;
     const int ntiles = (T + kResTile - 1) / kResTile;
     // list copies include the slack so that aligned over-reads of the last tile stay inside the allocation
@@ -301,8 +308,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u];
         if (m < 0 || m > 2) return FDKV_ERR_STATE;
-        if (m == FDKV_MODE_EXACT) need += 4 * align_up(rows);
-        else need += 2 * align_up(rows) + (m == FDKV_MODE_RESIDUAL ? 2 * (align_up(idx_b) + align_up(val_b) + align_up(off_b)) : 0);
+        if (m == FDKV_MODE_EXACT) need += 4 * align_up(rows_pad);
+        else need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * (align_up(idx_b) + align_up(val_b) + align_up(off_b)) : 0);
     }
     if (c->bump + need > c->arena_bytes) return FDKV_ERR_ARENA_FULL;
     size_t o = c->bump;
@@ -323,7 +330,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
             const void* src[4] = {c->k_layers[2 * p], c->k_layers[2 * p + 1], c->v_layers[2 * p], c->v_layers[2 * p + 1]};
             char* dst[4];
             for (int i = 0; i < 4; ++i) {
-                dst[i] = take(rows);
+                dst[i] = take(rows_pad);
+                if (rows_pad > rows) CU(cudaMemsetAsync(dst[i] + rows, 0, rows_pad - rows, st));
                 const char* sp = (const char*)src[i] + (size_t)h * c->stride_h * s.esize;
                 CU(launch_strided_copy(sp, c->stride_t, dst[i], T, s.d, s.esize, st));
             }
@@ -333,7 +341,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
         } else {
             for (int is_v = 0; is_v < 2; ++is_v) {
                 const size_t ut = (size_t)u * 2 + is_v;
-                char* z0 = take(rows);
+                char* z0 = take(rows_pad);
+                if (rows_pad > rows) CU(cudaMemsetAsync(z0 + rows, 0, rows_pad - rows, st));
                 CU(cudaMemcpyAsync(z0, c->work + c->ws.z0 + ut * unit_stride_b, rows, cudaMemcpyDeviceToDevice, st));
                 (is_v ? d0->v_rows : d0->k_rows) = z0;
                 (is_v ? d1->v_rows : d1->k_rows) = z0;
@@ -379,7 +388,17 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
             if (c->seqs[b].tail_len[layer] >= s.max_tail) return FDKV_ERR_STATE;
         for (int b = 0; b < batch; ++b) c->seqs[b].tail_len[layer]++;
     }
+    std::vector<int32_t> host_T(batch), host_modes((size_t)batch * s.Hkv);
+    for (int b = 0; b < batch; ++b) {
+        host_T[b] = c->seqs[b].T;
+        for (int h = 0; h < s.Hkv; ++h) host_modes[(size_t)b * s.Hkv + h] = c->seqs[b].modes[(layer / 2) * s.Hkv + h];
+    }
     DecodeArgs a;
+    a.tail_rows = s.tail_rows;
+    a.host_T = host_T.data(); a.host_modes = host_modes.data();
+    a.tmap = c->has_tmap ? c->tmap : nullptr;
+    a.arena_base = c->arena;
+    a.keep_num = s.keep_num; a.keep_den = s.keep_den;
     a.desc = arp<UnitDesc>(c, c->ar.desc);
     a.L = s.L; a.layer = layer; a.batch = batch; a.Hq = s.Hq; a.Hkv = s.Hkv; a.G = s.G; a.d = s.d;
     a.max_tail = s.max_tail; a.max_batch = s.max_batch; a.Tmax_batch = Tmax;

@@ -55,7 +55,7 @@ __global__ void append_tail_kernel(DecodeArgs a) {
     T* tv = reinterpret_cast<T*>(a.tail_v);
     for (int i = threadIdx.x; i < row; i += blockDim.x) {
         const int h = i / a.d, c = i % a.d;
-        const int64_t o = ((((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.max_tail + n) * a.d + c;
+        const int64_t o = ((((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.tail_rows + n) * a.d + c;
         tk[o] = kn[i];
         tv[o] = vn[i];
     }
@@ -64,6 +64,8 @@ __global__ void append_tail_kernel(DecodeArgs a) {
 }
 
 constexpr int kWarps = 4;
+constexpr int kGTile = 32;                  // tokens per warp tile of the portable kernel
+constexpr int kSub = kGTile / kResTile;     // residual-offset tiles per warp tile
 
 // grid (splits, Hkv, batch); 4 warps; each warp owns whole 32-token tiles and a private online-softmax state.
 template <typename T, int D, int G>
@@ -97,6 +99,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
     const bool coef = u.mode != FDKV_MODE_EXACT;
     const bool resid = u.mode == FDKV_MODE_RESIDUAL;
 
+    const int nres = (u.T + kResTile - 1) / kResTile;
     // ---- one 32-token tile: rows [row0, row0 + nrows) of kbase / vbase ----
     auto tile = [&](const T* kbase, const T* vbase, int nrows, float kscale, float vscale, bool with_res, int jt) {
         float s[G];
@@ -120,9 +123,10 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
 #pragma unroll
             for (int g = 0; g < G; ++g) s_corr[warp][g][lane] = 0.f;
             __syncwarp();
-            const int64_t base = (int64_t)jt * kResTile * D;
+            const int64_t base = (int64_t)jt * kGTile * D;
             const T* val = reinterpret_cast<const T*>(u.k_val);
-            for (int e = u.k_off[jt] + lane; e < u.k_off[jt + 1]; e += 32) {
+            const int ke1 = u.k_off[min(nres, (jt + 1) * kSub)];
+            for (int e = u.k_off[jt * kSub] + lane; e < ke1; e += 32) {
                 const int f = (int)(u.k_idx[e] - base);
                 const float v = ldf<T>(val + e);
 #pragma unroll
@@ -165,9 +169,9 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
 #pragma unroll
             for (int g = 0; g < G; ++g) s_p[warp][g][lane] = p[g];
             __syncwarp();
-            const int64_t base = (int64_t)jt * kResTile * D;
+            const int64_t base = (int64_t)jt * kGTile * D;
             const T* val = reinterpret_cast<const T*>(u.v_val);
-            const int e0 = u.v_off[jt], e1 = u.v_off[jt + 1];
+            const int e0 = u.v_off[jt * kSub], e1 = u.v_off[min(nres, (jt + 1) * kSub)];
             for (int e = e0 + lane; e < e1; e += 32) {
                 const int f = (int)(u.v_idx[e] - base);
                 const float v = ldf<T>(val + e);
@@ -190,7 +194,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
 
     // ---- prefill rows of this split ----
     {
-        const int ntiles = (u.T + kResTile - 1) / kResTile;
+        const int ntiles = (u.T + kGTile - 1) / kGTile;
         const int tiles_per_split = (ntiles + splits - 1) / splits;
         const int j0 = split * tiles_per_split, j1 = min(ntiles, j0 + tiles_per_split);
         const T* kr = reinterpret_cast<const T*>(u.k_rows);
@@ -198,14 +202,14 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
         const float kscale = coef ? c * inv_sqrt_d : inv_sqrt_d;
         const float vscale = coef ? c : 1.f;
         for (int jt = j0 + warp; jt < j1; jt += kWarps) {
-            const int t0 = jt * kResTile;
-            tile(kr + (int64_t)t0 * D, vr + (int64_t)t0 * D, min(kResTile, u.T - t0), kscale, vscale, resid, jt);
+            const int t0 = jt * kGTile;
+            tile(kr + (int64_t)t0 * D, vr + (int64_t)t0 * D, min(kGTile, u.T - t0), kscale, vscale, resid, jt);
         }
     }
     // ---- uncompressed tail rows (last split only) ----
     if (split == splits - 1) {
         const int n = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
-        const int64_t o = (((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.max_tail * D;
+        const int64_t o = (((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.tail_rows * D;
         const T* tk = reinterpret_cast<const T*>(a.tail_k) + o;
         const T* tv = reinterpret_cast<const T*>(a.tail_v) + o;
         for (int t0 = warp * 32; t0 < n; t0 += kWarps * 32)
@@ -304,7 +308,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st) {
     if ((e = launch_decode_fast(a, st, &handled)) != cudaSuccess) return e;
     if (handled) return cudaSuccess;
 
-    const int ntiles = (a.Tmax_batch + kResTile - 1) / kResTile;
+    const int ntiles = (a.Tmax_batch + kGTile - 1) / kGTile;
     int splits = (2 * 148 + a.Hkv * a.batch - 1) / (a.Hkv * a.batch);
     splits = max(1, min(min(splits, kMaxSplits), (ntiles + 7) / 8));
     if (dtype == FDKV_BF16)

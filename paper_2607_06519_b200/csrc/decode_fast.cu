@@ -1,9 +1,609 @@
-// Bulk-copy pipelined decode kernel for bf16, head_dim 128.  Not built yet: the portable kernel handles every shape.
+// Decode attention over the packed cache for bf16 storage, head_dim 128 (the paragraph after Eq. 3: shared
+// coefficients broadcast to both layers of the pair, residual coefficients added only where indexed, the full
+// cache never materialised).
+//
+// One persistent CTA per SM.  A producer warp streams 64-token K and V boxes of the packed cache through a
+// ring of shared-memory stages with TMA (128-byte swizzle, mbarrier completion).  Eight consumer warps (two
+// groups that alternate stages) each own 16 tokens of a stage and a private online-softmax state:
+//   S^T = q K^T   mma.sync m16n8k16 (heads on M, tokens on N; ldmatrix of the swizzled K box),
+//   P = exp2(S - max), split into bf16 hi + lo halves held in rows 0-7 / 8-15 of the next A operand,
+//   O += P V      mma.sync (ldmatrix.trans of the V box).
+// Residual units: the warp scatters its slice's kept Z1 entries into a private zeroed 16x128 bf16 scratch tile
+// and runs the same two products on it with the layer's sign, so the correction is exact in float32.
+// Work is a flat list of (unit, tile) pairs cut into one contiguous range per CTA (byte-weighted), so a CTA may
+// finish one unit and start the next; each (CTA, unit) segment writes one split-K partial.
+#include <cuda.h>
+
+#include <algorithm>
+
 #include "fdkv_internal.h"
 
 namespace fdkv {
-cudaError_t launch_decode_fast(const DecodeArgs&, cudaStream_t, bool* handled) {
-    *handled = false;
-    return cudaSuccess;
+
+namespace {
+
+constexpr int kTT = 64;          // tokens per stage
+constexpr int kStages = 6;
+constexpr int kGroups = 2;       // consumer groups; stage s always belongs to group s % kGroups (kStages % kGroups == 0)
+constexpr int kCW = 4 * kGroups; // consumer warps
+constexpr int kThreads = (kCW + 1) * 32;
+constexpr int kHalfBytes = kTT * 128;        // one 64-channel box of 64 tokens
+constexpr int kStageBytes = 4 * kHalfBytes;  // K ch 0-63, K ch 64-127, V ch 0-63, V ch 64-127
+constexpr int kScratchBytes = 4096;          // per consumer warp: 16 tokens x 128 channels bf16 (or its O tile at merge)
+constexpr int kHeaderBytes = 1024;
+constexpr int kSmemBytes = kHeaderBytes + kStages * kStageBytes + kCW * kScratchBytes;
+constexpr int kMaxCtas = 296;
+constexpr int kMaxUnits = 512;
+constexpr int kPF = 8;  // residual entries prefetched per lane and list
+constexpr uint32_t kSpinCap = 1u << 22;
+static_assert(kStages % kGroups == 0, "stage ownership must be fixed per group");
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+
+struct FastSched {
+    uint32_t start[kMaxCtas + 1];  // unit << 20 | first 64-token tile of CTA c; start[ncta] = units << 20
+    int ncta, units;
+};
+struct CombSched {
+    uint16_t nparts[kMaxUnits];
+};
+
+// header offsets
+constexpr int kOffFull = 0, kOffEmpty = 64, kOffAbort = 128, kOffM = 256, kOffL = 512;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void st_shared_u16(uint32_t addr, uint16_t v) {
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+__device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, %0;" ::"n"(kCW * 32) : "memory"); }
+
+// Bounded wait on an mbarrier phase.  Gives up after kSpinCap polls (or as soon as another thread gave up):
+// raises the CTA abort flag and the device status word, after which every wait returns at once.
+__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* status) {
+    if (*abort_flag) return;
+    for (uint32_t i = 0; i < kSpinCap; ++i) {
+        if (mbar_try_wait(bar, parity)) return;
+        if ((i & 255u) == 255u && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicMax(status, (int32_t)kFlagTimeout);
+}
+
+// byte offset of (row, channel chunk of 8) inside a [rows][64 ch] box with the 128-byte swizzle
+__device__ __forceinline__ uint32_t swz(int row, int chunk8) { return (uint32_t)(row * 128 + (((chunk8 & 7) ^ (row & 7)) << 4)); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastSched sch) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t smem0 = smem_u32(smem_raw);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + kOffAbort);
+    if (smem0 & 1023u) {  // the swizzled boxes need 1024-byte alignment; report instead of computing garbage
+        if (threadIdx.x == 0) atomicMax(a.status, (int32_t)kFlagCountMismatch);
+        return;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem0 + kOffFull + 8 * s, 1);
+            mbar_init(smem0 + kOffEmpty + 8 * s, 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // consumer scratch starts zeroed
+    for (int i = threadIdx.x; i < kCW * kScratchBytes / 16; i += kThreads)
+        st_shared_zero16(smem0 + kHeaderBytes + kStages * kStageBytes + i * 16);
+    __syncthreads();
+
+    const int cta = blockIdx.x;
+    const uint32_t s0 = sch.start[cta], s1 = sch.start[cta + 1];
+    const int u_first = (int)(s0 >> 20), t_first = (int)(s0 & 0xFFFFFu);
+    const int u_last = (int)(s1 >> 20), t_last = (int)(s1 & 0xFFFFFu);
+    const uint64_t arena = reinterpret_cast<uint64_t>(a.arena_base);
+    const uint32_t stage0 = smem0 + kHeaderBytes;
+
+    if (warp == kCW) {
+        // ================= producer =================
+        if (lane == 0) {
+            int it = 0;
+            for (int u = u_first; u <= u_last && u < sch.units; ++u) {
+                const int b = u / a.Hkv, h = u % a.Hkv;
+                const UnitDesc* ud = a.desc + ((int64_t)b * a.L + a.layer) * a.Hkv + h;
+                const int T = ud->T;
+                const int ntiles = (T + kTT - 1) / kTT;
+                const int tb = u == u_first ? t_first : 0;
+                const int te = u == u_last ? t_last : ntiles;
+                if (te <= tb) continue;
+                const int krow0 = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> 8);
+                const int vrow0 = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> 8);
+                int ntail = 0, tkrow0 = 0, tvrow0 = 0;
+                if (te == ntiles) {
+                    const int n = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
+                    ntail = (n + kTT - 1) / kTT;
+                    const int64_t o = (((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.tail_rows;
+                    tkrow0 = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
+                    tvrow0 = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
+                }
+                const int npre = te - tb;
+                for (int j = 0; j < npre + ntail; ++j, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                    wait_bar(smem0 + kOffEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
+                    if (*abort_flag) break;
+                    const int kr = j < npre ? krow0 + (tb + j) * kTT : tkrow0 + (j - npre) * kTT;
+                    const int vr = j < npre ? vrow0 + (tb + j) * kTT : tvrow0 + (j - npre) * kTT;
+                    const uint32_t full = smem0 + kOffFull + 8 * s;
+                    const uint32_t dst = stage0 + s * kStageBytes;
+                    mbar_expect_tx(full, kStageBytes);
+                    tma_load_2d(dst, &tmap, 0, kr, full);
+                    tma_load_2d(dst + kHalfBytes, &tmap, 64, kr, full);
+                    tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
+                    tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
+                }
+                if (*abort_flag) break;
+            }
+        }
+    } else {
+        // ================= consumers =================
+        const int gi = warp >> 2, si = warp & 3;   // group, 16-token slice of the stage
+        const int gid = lane >> 2, tig = lane & 3; // mma fragment coordinates: head row, column pair
+        const int r0 = si * 16;
+        const uint32_t scratch = smem0 + kHeaderBytes + kStages * kStageBytes + warp * kScratchBytes;
+        float* const scratch_f = reinterpret_cast<float*>(smem_raw + kHeaderBytes + kStages * kStageBytes + warp * kScratchBytes);
+        float* const sm_m = reinterpret_cast<float*>(smem_raw + kOffM);
+        float* const sm_l = reinterpret_cast<float*>(smem_raw + kOffL);
+        const float kLog2e = 1.4426950408889634f, kC = 0.70710678118654752440f;
+        const float inv_sqrt_d = 0.08838834764831845f;  // 1/sqrt(128)
+
+        int it = 0;
+        for (int u = u_first; u <= u_last && u < sch.units; ++u) {
+            const int b = u / a.Hkv, h = u % a.Hkv;
+            const UnitDesc ud = a.desc[((int64_t)b * a.L + a.layer) * a.Hkv + h];
+            const int T = ud.T;
+            const int ntiles = (T + kTT - 1) / kTT;
+            const int tb = u == u_first ? t_first : 0;
+            const int te = u == u_last ? t_last : ntiles;
+            if (te <= tb) continue;
+            int ntail = 0, n_tail_rows = 0;
+            if (te == ntiles) {
+                n_tail_rows = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
+                ntail = (n_tail_rows + kTT - 1) / kTT;
+            }
+            const int npre = te - tb, nseg = npre + ntail;
+            const bool coef = ud.mode != FDKV_MODE_EXACT, resid = ud.mode == FDKV_MODE_RESIDUAL;
+            const uint32_t sgn = ud.sign < 0.f ? 0x80008000u : 0u;
+            const int nres = (T + kResTile - 1) / kResTile;
+
+            // q fragments: A operand rows = the G query heads of this KV head, zero elsewhere
+            uint32_t qa[8][2];
+            {
+                const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.Hq + h * a.G + gid) * 128;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    qa[kk][0] = gid < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 2 * tig) : 0u;
+                    qa[kk][1] = gid < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 8 + 2 * tig) : 0u;
+                }
+            }
+            float oacc[16][4];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
+            float m_run = -INFINITY, l_run = 0.f;
+
+            // ---- residual lists: ranges two tiles ahead, entries one tile ahead ----
+            const int32_t* k_idx = ud.k_idx;
+            const int32_t* v_idx = ud.v_idx;
+            const uint16_t* k_val = reinterpret_cast<const uint16_t*>(ud.k_val);
+            const uint16_t* v_val = reinterpret_cast<const uint16_t*>(ud.v_val);
+            int j_my = (((gi - it) % kGroups) + kGroups) % kGroups;  // first tile of the segment owned by this group
+            int cr[4] = {0, 0, 0, 0}, nr[4] = {0, 0, 0, 0};          // {k begin, k end, v begin, v end}
+            int32_t pki[kPF], pvi[kPF];
+            uint16_t pkv[kPF], pvv[kPF];
+            auto load_ranges = [&](int j, int (&r)[4]) {
+                if (resid && j < npre) {
+                    const int o = (tb + j) * (kTT / kResTile) + si;
+                    const int o0 = min(o, nres), o1 = min(o + 1, nres);
+                    r[0] = ud.k_off[o0]; r[1] = ud.k_off[o1];
+                    r[2] = ud.v_off[o0]; r[3] = ud.v_off[o1];
+                } else {
+                    r[0] = r[1] = r[2] = r[3] = 0;
+                }
+            };
+            auto prefetch = [&](const int32_t* idx, const uint16_t* val, int e0, int e1, int32_t (&pi)[kPF], uint16_t (&pv)[kPF]) {
+#pragma unroll
+                for (int i = 0; i < kPF; ++i) {
+                    const int e = e0 + lane + 32 * i;
+                    if (e < e1) { pi[i] = idx[e]; pv[i] = val[e]; }
+                }
+            };
+            // scatter one list slice into the scratch tile (swizzled [2 halves][16 rows][64 ch])
+            auto scatter = [&](const int32_t* idx, const uint16_t* val, int e0, int e1, const int32_t (&pi)[kPF],
+                               const uint16_t (&pv)[kPF], int tok0) {
+                const int base = tok0 * 128;
+#pragma unroll
+                for (int i = 0; i < kPF; ++i) {
+                    const int e = e0 + lane + 32 * i;
+                    if (e < e1) {
+                        const int f = pi[i] - base, row = f >> 7, ch = f & 127;
+                        st_shared_u16(scratch + (ch >> 6) * 2048 + swz(row, ch >> 3) + (ch & 7) * 2, pv[i]);
+                    }
+                }
+                for (int e = e0 + 32 * kPF + lane; e < e1; e += 32) {  // dense slices: direct loads
+                    const int f = idx[e] - base, row = f >> 7, ch = f & 127;
+                    st_shared_u16(scratch + (ch >> 6) * 2048 + swz(row, ch >> 3) + (ch & 7) * 2, val[e]);
+                }
+            };
+            auto zero_scratch = [&]() {
+#pragma unroll
+                for (int i = 0; i < kScratchBytes / 16 / 32; ++i) st_shared_zero16(scratch + (lane + 32 * i) * 16);
+            };
+            if (resid) {
+                load_ranges(j_my, cr);
+                load_ranges(j_my + kGroups, nr);
+                prefetch(k_idx, k_val, cr[0], cr[1], pki, pkv);
+                prefetch(v_idx, v_val, cr[2], cr[3], pvi, pvv);
+            }
+
+            for (int j = j_my; j < nseg; j += kGroups) {
+                const int itj = it + j;
+                const int s = itj % kStages;
+                const uint32_t ph = (uint32_t)(itj / kStages) & 1u;
+                const bool is_tail = j >= npre;
+                const int tile = is_tail ? j - npre : tb + j;
+                const int rows_valid = is_tail ? n_tail_rows - tile * kTT : T - tile * kTT;  // may exceed 64
+                const bool with_res = resid && !is_tail;
+                const float kscale = ((coef && !is_tail) ? kC : 1.f) * inv_sqrt_d * kLog2e;
+                const float vscale = (coef && !is_tail) ? kC : 1.f;
+                const int tok0 = tile * kTT + r0;  // first token of this warp's slice
+                int nnr[4];
+                load_ranges(j + 2 * kGroups, nnr);
+
+                if (with_res && cr[1] > cr[0]) {
+                    scatter(k_idx, k_val, cr[0], cr[1], pki, pkv, tok0);
+                    __syncwarp();
+                }
+                if (resid) prefetch(k_idx, k_val, nr[0], nr[1], pki, pkv);
+
+                wait_bar(smem0 + kOffFull + 8 * s, ph, abort_flag, a.status);
+                const uint32_t kb = stage0 + s * kStageBytes, vb = kb + 2 * kHalfBytes;
+
+                // ---- S^T[head][token] = q . k over 128 channels; two n-tiles of 8 tokens ----
+                float sacc[2][4];
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+                {
+                    const int mi = lane >> 3, rr = lane & 7;
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+                        const int row = r0 + nt * 8 + rr;
+#pragma unroll
+                        for (int kp = 0; kp < 4; ++kp) {
+                            const int c = 4 * kp + mi;  // 16-byte channel chunk 0..15
+                            uint32_t b0, b1, b2, b3;
+                            ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), b0, b1, b2, b3);
+                            mma_bf16(sacc[nt], qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
+                            mma_bf16(sacc[nt], qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b2, b3);
+                        }
+                    }
+                    if (with_res && cr[1] > cr[0]) {
+#pragma unroll
+                        for (int nt = 0; nt < 2; ++nt) {
+                            const int row = nt * 8 + rr;
+#pragma unroll
+                            for (int kp = 0; kp < 4; ++kp) {
+                                const int c = 4 * kp + mi;
+                                uint32_t b0, b1, b2, b3;
+                                ldsm_x4(scratch + (c >> 3) * 2048 + swz(row, c), b0, b1, b2, b3);
+                                mma_bf16(sacc[nt], qa[2 * kp][0] ^ sgn, 0u, qa[2 * kp][1] ^ sgn, 0u, b0, b1);
+                                mma_bf16(sacc[nt], qa[2 * kp + 1][0] ^ sgn, 0u, qa[2 * kp + 1][1] ^ sgn, 0u, b2, b3);
+                            }
+                        }
+                        __syncwarp();
+                        zero_scratch();
+                        __syncwarp();
+                    }
+                }
+                if (with_res && cr[3] > cr[2]) {
+                    scatter(v_idx, v_val, cr[2], cr[3], pvi, pvv, tok0);
+                    __syncwarp();
+                }
+                if (resid) prefetch(v_idx, v_val, nr[2], nr[3], pvi, pvv);
+
+                // ---- online softmax for head gid over this slice's 16 tokens (4 per thread) ----
+                float p[2][2];
+                float mt = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int tl = r0 + nt * 8 + 2 * tig + e;
+                        const float sv = tl < rows_valid ? sacc[nt][e] * kscale : -INFINITY;
+                        p[nt][e] = sv;
+                        mt = fmaxf(mt, sv);
+                    }
+                mt = fmaxf(mt, __shfl_xor_sync(0xFFFFFFFFu, mt, 1));
+                mt = fmaxf(mt, __shfl_xor_sync(0xFFFFFFFFu, mt, 2));
+                const float m_new = fmaxf(m_run, mt);
+                float alpha = 1.f;
+                if (m_new == -INFINITY) {
+                    p[0][0] = p[0][1] = p[1][0] = p[1][1] = 0.f;
+                } else {
+                    alpha = ex2(m_run - m_new);
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) p[nt][e] = ex2(p[nt][e] - m_new);
+                }
+                l_run = l_run * alpha + (p[0][0] + p[0][1] + p[1][0] + p[1][1]);
+                m_run = m_new;
+                if (__any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+#pragma unroll
+                    for (int jn = 0; jn < 16; ++jn) {
+                        oacc[jn][0] *= alpha; oacc[jn][1] *= alpha; oacc[jn][2] *= alpha; oacc[jn][3] *= alpha;
+                    }
+                }
+                // A operand of the second product: rows 0-7 carry the bf16 rounding of P, rows 8-15 its remainder
+                uint32_t pa[4];
+                {
+                    float hi[2][2], lo[2][2];
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float pv_ = p[nt][e] * vscale;
+                            hi[nt][e] = __bfloat162float(__float2bfloat16_rn(pv_));
+                            lo[nt][e] = pv_ - hi[nt][e];
+                        }
+                    pa[0] = pack_bf16(hi[0][0], hi[0][1]);
+                    pa[1] = pack_bf16(lo[0][0], lo[0][1]);
+                    pa[2] = pack_bf16(hi[1][0], hi[1][1]);
+                    pa[3] = pack_bf16(lo[1][0], lo[1][1]);
+                }
+                // ---- O[head][channel] += P . V : 16 n-tiles of 8 channels, k = this slice's 16 tokens ----
+                {
+                    const int mi = lane >> 3, rr = lane & 7;
+                    const int row = r0 + (mi & 1) * 8 + rr;
+#pragma unroll
+                    for (int jp = 0; jp < 8; ++jp) {
+                        const int c = 2 * jp + (mi >> 1);
+                        uint32_t b0, b1, b2, b3;
+                        ldsm_x4_t(vb + (c >> 3) * kHalfBytes + swz(row, c), b0, b1, b2, b3);
+                        mma_bf16(oacc[2 * jp], pa[0], pa[1], pa[2], pa[3], b0, b1);
+                        mma_bf16(oacc[2 * jp + 1], pa[0], pa[1], pa[2], pa[3], b2, b3);
+                    }
+                    if (with_res && cr[3] > cr[2]) {
+                        const int srow = (mi & 1) * 8 + rr;
+#pragma unroll
+                        for (int jp = 0; jp < 8; ++jp) {
+                            const int c = 2 * jp + (mi >> 1);
+                            uint32_t b0, b1, b2, b3;
+                            ldsm_x4_t(scratch + (c >> 3) * 2048 + swz(srow, c), b0, b1, b2, b3);
+                            mma_bf16(oacc[2 * jp], pa[0] ^ sgn, pa[1] ^ sgn, pa[2] ^ sgn, pa[3] ^ sgn, b0, b1);
+                            mma_bf16(oacc[2 * jp + 1], pa[0] ^ sgn, pa[1] ^ sgn, pa[2] ^ sgn, pa[3] ^ sgn, b2, b3);
+                        }
+                        __syncwarp();
+                        zero_scratch();
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem0 + kOffEmpty + 8 * s);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { cr[i] = nr[i]; nr[i] = nnr[i]; }
+            }
+            it += nseg;
+
+            // ---- merge the eight warps' states into this segment's split-K partial ----
+            {
+                float lq = l_run;
+                lq += __shfl_xor_sync(0xFFFFFFFFu, lq, 1);
+                lq += __shfl_xor_sync(0xFFFFFFFFu, lq, 2);
+                if (tig == 0) { sm_m[warp * 8 + gid] = m_run; sm_l[warp * 8 + gid] = lq; }
+#pragma unroll
+                for (int jn = 0; jn < 16; ++jn)
+                    *reinterpret_cast<float2*>(scratch_f + gid * 128 + jn * 8 + 2 * tig) =
+                        make_float2(oacc[jn][0] + oacc[jn][2], oacc[jn][1] + oacc[jn][3]);
+                bar_consumers();
+                // partial slot = number of CTAs that started this unit before this one
+                int slot = 0;
+                for (int c2 = cta - 1; c2 >= 0; --c2) {
+                    const uint32_t ustart = (uint32_t)u << 20, e2 = sch.start[c2 + 1], s2 = sch.start[c2];
+                    if (e2 <= ustart) break;                 // ends before this unit's first tile
+                    if (max(s2, ustart) < e2) ++slot;        // a non-empty range inside this unit
+                    if (s2 <= ustart) break;
+                }
+                const int tid = threadIdx.x;  // 0..255 here
+                for (int i = tid; i < a.G * 128; i += kCW * 32) {
+                    const int g = i >> 7, ch = i & 127;
+                    float M = -INFINITY;
+#pragma unroll
+                    for (int w = 0; w < kCW; ++w) M = fmaxf(M, sm_m[w * 8 + g]);
+                    float L = 0.f, A = 0.f;
+                    if (M != -INFINITY) {
+#pragma unroll
+                        for (int w = 0; w < kCW; ++w) {
+                            const float f = ex2(sm_m[w * 8 + g] - M);
+                            L = fmaf(sm_l[w * 8 + g], f, L);
+                            const float* ow = reinterpret_cast<const float*>(smem_raw + kHeaderBytes + kStages * kStageBytes + w * kScratchBytes);
+                            A = fmaf(ow[g * 128 + ch], f, A);
+                        }
+                    }
+                    float* part = a.partials + (((int64_t)b * a.Hq + h * a.G + g) * kMaxSplits + slot) * (128 + 2);
+                    if (ch == 0) { part[0] = M * 0.6931471805599453f; part[1] = L; }  // the combine step works in natural-log units
+                    part[2 + ch] = A;
+                }
+                bar_consumers();
+                zero_scratch();
+                __syncwarp();
+            }
+        }
+    }
+    // after a timed-out wait: give copies that may still be in flight time to land before the CTA retires
+    if (*abort_flag)
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+}
+
+}  // namespace
+
+// out = sum_s e^{m_s - M} acc_s / sum_s e^{m_s - M} l_s over the unit's parts.  grid (Hq, batch), 128 threads.
+__global__ void combine_fast_kernel(const float* partials, int Hq, int Hkv, CombSched cs, void* out, int out_dtype) {
+    const int i = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
+    const int G = Hq / Hkv;
+    const int n = cs.nparts[b * Hkv + i / G];
+    const float* p = partials + ((int64_t)b * Hq + i) * kMaxSplits * 130;
+    float M = -INFINITY;
+    for (int s = 0; s < n; ++s) M = fmaxf(M, p[s * 130]);
+    float L = 0.f, A = 0.f;
+    for (int s = 0; s < n; ++s) {
+        const float ms = p[s * 130];
+        if (ms == -INFINITY) continue;
+        const float f = __expf(ms - M);
+        L = fmaf(p[s * 130 + 1], f, L);
+        A = fmaf(p[s * 130 + 2 + ch], f, A);
+    }
+    const float r = L > 0.f ? A / L : 0.f;
+    const int64_t o = ((int64_t)b * Hq + i) * 128 + ch;
+    if (out_dtype == FDKV_BF16)
+        reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(r);
+    else
+        reinterpret_cast<float*>(out)[o] = r;
+}
+
+bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    const cuuint64_t rows = arena_bytes / 256;
+    if (rows == 0 || rows > 0x7FFFFFFFull) return false;
+    const cuuint64_t gdim[2] = {128, rows};
+    const cuuint64_t gstride[1] = {256};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTT};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<encode_fn>(fn)(reinterpret_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, arena,
+                                                 gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handled) {
+    *handled = false;
+    const int units = a.batch * a.Hkv;
+    if (!a.tmap || a.d != 128 || units > kMaxUnits || units < 1) return cudaSuccess;
+    static int sm_count = 0;
+    static bool attr_done = false;
+    if (!attr_done) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    // ---- flat byte-weighted schedule: CTA c starts at weight c * W / ncta ----
+    FastSched sch;
+    CombSched cs;
+    std::vector<int64_t> wp(units + 1, 0);
+    std::vector<int> nt(units), wt(units);
+    int64_t total_tiles = 0;
+    for (int u = 0; u < units; ++u) {
+        const int T = a.host_T[u / a.Hkv];
+        nt[u] = (T + kTT - 1) / kTT;
+        if (nt[u] >= (1 << 20)) return cudaSuccess;
+        const int64_t k = (int64_t)T * 128 * a.keep_num / a.keep_den;
+        // bytes per tile in units of 512 B: two 16 KiB boxes, plus the lists' share for residual units
+        wt[u] = 64 + (a.host_modes[u] == FDKV_MODE_RESIDUAL ? (int)((2 * k * 6 / nt[u] + 511) / 512) : 0);
+        wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
+        total_tiles += nt[u];
+    }
+    const int ncta = (int)std::min<int64_t>(std::min(sm_count, kMaxCtas), total_tiles);
+    sch.ncta = ncta;
+    sch.units = units;
+    {
+        int u = 0;
+        for (int c = 0; c < ncta; ++c) {
+            const int64_t target = wp[units] * c / ncta;
+            while (u + 1 < units && wp[u + 1] <= target) ++u;
+            const int tile = (int)((target - wp[u]) / wt[u]);
+            sch.start[c] = ((uint32_t)u << 20) | (uint32_t)tile;
+        }
+        sch.start[ncta] = (uint32_t)units << 20;
+    }
+    // parts per unit = CTAs whose range contains at least one of its tiles
+    for (int u = 0; u < units; ++u) cs.nparts[u] = 0;
+    for (int c = 0; c < ncta; ++c) {
+        const int ua = (int)(sch.start[c] >> 20), ta = (int)(sch.start[c] & 0xFFFFFu);
+        const int ub = (int)(sch.start[c + 1] >> 20), tb = (int)(sch.start[c + 1] & 0xFFFFFu);
+        for (int u = ua; u <= ub && u < units; ++u) {
+            const int b0 = u == ua ? ta : 0, b1 = u == ub ? tb : nt[u];
+            if (b1 > b0) cs.nparts[u]++;
+        }
+    }
+    for (int u = 0; u < units; ++u)
+        if (cs.nparts[u] > kMaxSplits) return cudaSuccess;
+    decode_fast_kernel<<<ncta, kThreads, kSmemBytes, st>>>(*reinterpret_cast<const CUtensorMap*>(a.tmap), a, sch);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    combine_fast_kernel<<<dim3(a.Hq, a.batch), 128, 0, st>>>(a.partials, a.Hq, a.Hkv, cs, a.out, a.out_dtype);
+    count_launch(2);
+    *handled = true;
+    return cudaGetLastError();
+}
+
 }  // namespace fdkv

@@ -12,13 +12,14 @@
 
 namespace fdkv {
 
-constexpr int kResTile = 32;         // tokens per residual-offset tile: off[j] = first list entry of tokens >= 32 j
+constexpr int kResTile = 16;         // tokens per residual-offset tile: off[j] = first list entry of tokens >= 16 j
 constexpr int kHistBins = 32768;     // one bin per 15-bit magnitude prefix (a whole bf16 key)
-constexpr int kMaxSplits = 128;      // split-K partial slots per (sequence, query head)
+constexpr int kMaxSplits = 160;      // split-K partial slots per (sequence, query head)
 constexpr int kMaxW = 128;           // probe queries
 constexpr int kListPad = 32;         // slack entries after each residual list (aligned over-reads stay in bounds)
 constexpr int kMaxGroup = 8;
 constexpr int kProbeTile = 64;       // tokens per probe CTA (generic kernel)
+constexpr int kRowPad = 64;          // packed row blocks and tails are padded (zero rows) to this many tokens
 
 enum DeviceFlag : int32_t { kFlagOk = 0, kFlagTimeout = 1, kFlagCountMismatch = 2, kFlagTailFull = 3 };
 
@@ -28,7 +29,7 @@ struct UnitDesc {
     const void* v_rows;
     const int32_t* k_idx;  // residual mode only: ascending flat indices t*d + ch
     const void* k_val;
-    const int32_t* k_off;  // [ceil(T/32) + 1] first entry of each 32-token tile
+    const int32_t* k_off;  // [ceil(T/16) + 1] first entry of each 16-token tile
     const int32_t* v_idx;
     const void* v_val;
     const int32_t* v_off;
@@ -52,9 +53,10 @@ struct Shape {
     int keep_num, keep_den;
     int64_t kmax;      // floor(Tmax*d*num/den)
     int64_t kcap;      // list capacity incl. slack
-    int ntiles_max;    // ceil(Tmax/32)
+    int ntiles_max;    // ceil(Tmax/16)
     int nptiles_max;   // ceil(Tmax/kProbeTile)
     int NU, NT;        // units and unit-tensors (K and V) of one sequence
+    int tail_rows;     // max_tail rounded up to kRowPad
 };
 
 struct WsLayout {
@@ -93,6 +95,8 @@ struct fdkv_ctx {
     bool modes_overridden = false;
     std::vector<fdkv::SeqState> seqs;
     std::vector<fdkv::UnitDesc> desc_host;  // [max_batch][L][Hkv]
+    alignas(64) unsigned char tmap[128];    // CUtensorMap of the arena (bf16, head_dim 128 only)
+    bool has_tmap = false;
 };
 
 namespace fdkv {
@@ -152,12 +156,21 @@ struct DecodeArgs {
     const void *q, *k_new, *v_new;
     void* out;
     int out_dtype;
-    void *tail_k, *tail_v;  // [L][max_batch][Hkv][max_tail][d]
+    void *tail_k, *tail_v;  // [L][max_batch][Hkv][tail_rows][d], tail_rows = max_tail rounded up to kRowPad
+    int tail_rows;
+    // host-side views used only to plan the launch (valid during the call)
+    const int32_t* host_T;      // [batch]
+    const int32_t* host_modes;  // [batch][Hkv] modes of this layer's pair
+    const void* tmap;           // CUtensorMap over the arena as rows of 256 bytes, or null
+    const void* arena_base;
+    int keep_num, keep_den;
     int32_t* tail_len;      // [L][max_batch]
     float* partials;        // [batch][Hq][kMaxSplits][d+2]
     int32_t* status;
 };
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st);
+// Encodes a 2-D tensor map over the arena viewed as [rows][128] bf16 (256-byte rows), 64x64 boxes, 128-byte swizzle.
+bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out);
 cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st);
 
 void count_launch(int n);
