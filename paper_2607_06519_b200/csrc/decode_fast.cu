@@ -2,9 +2,9 @@
 // coefficients broadcast to both layers of the pair, residual coefficients added only where indexed, the full
 // cache never materialised).
 //
-// One persistent CTA per SM.  A producer warp streams 64-token K and V boxes of the packed cache through a
-// ring of shared-memory stages with TMA (128-byte swizzle, mbarrier completion).  Eight consumer warps (two
-// groups that alternate stages) each own 16 tokens of a stage and a private online-softmax state:
+// One persistent CTA of eight warps per SM.  128-token K and V boxes of the packed cache stream through a ring of
+// shared-memory stages with TMA (128-byte swizzle, mbarrier completion); lane 0 of warp 0 issues the copies two
+// tiles ahead of the compute.  Each warp owns 16 tokens of a stage and a private online-softmax state:
 //   S^T = q K^T   mma.sync m16n8k16 (heads on M, tokens on N; ldmatrix of the swizzled K box),
 //   P = exp2(S - max), split into bf16 hi + lo halves held in rows 0-7 / 8-15 of the next A operand,
 //   O += P V      mma.sync (ldmatrix.trans of the V box).
@@ -22,12 +22,11 @@ namespace fdkv {
 
 namespace {
 
-constexpr int kTT = 64;          // tokens per stage
-constexpr int kStages = 6;
-constexpr int kGroups = 2;       // consumer groups; stage s always belongs to group s % kGroups (kStages % kGroups == 0)
-constexpr int kCW = 4 * kGroups; // consumer warps
-constexpr int kThreads = (kCW + 1) * 32;
-constexpr int kHalfBytes = kTT * 128;        // one 64-channel box of 64 tokens
+constexpr int kTT = 128;         // tokens per stage
+constexpr int kStages = 3;
+constexpr int kCW = kTT / 16;    // warps, 16 tokens of a stage each
+constexpr int kThreads = kCW * 32;  // 256 threads: two warps per scheduler, so up to 255 registers per thread
+constexpr int kHalfBytes = kTT * 128;        // one 64-channel box of 128 tokens
 constexpr int kStageBytes = 4 * kHalfBytes;  // K ch 0-63, K ch 64-127, V ch 0-63, V ch 64-127
 constexpr int kScratchBytes = 4096;          // per consumer warp: 16 tokens x 128 channels bf16 (or its O tile at merge)
 constexpr int kHeaderBytes = 1024;
@@ -36,7 +35,7 @@ constexpr int kMaxCtas = 296;
 constexpr int kMaxUnits = 512;
 constexpr int kPF = 8;  // residual entries prefetched per lane and list
 constexpr uint32_t kSpinCap = 1u << 22;
-static_assert(kStages % kGroups == 0, "stage ownership must be fixed per group");
+static_assert(kTT == kRowPad, "row blocks are padded to whole stages");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct FastSched {
@@ -103,7 +102,6 @@ __device__ __forceinline__ void st_shared_u16(uint32_t addr, uint16_t v) {
 __device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
 }
-__device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, %0;" ::"n"(kCW * 32) : "memory"); }
 
 // Bounded wait on an mbarrier phase.  Gives up after kSpinCap polls (or as soon as another thread gave up):
 // raises the CTA abort flag and the device status word, after which every wait returns at once.
@@ -137,12 +135,12 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem0 + kOffFull + 8 * s, 1);
-            mbar_init(smem0 + kOffEmpty + 8 * s, 4);
+            mbar_init(smem0 + kOffEmpty + 8 * s, kCW);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // consumer scratch starts zeroed
+    // per-warp scratch starts zeroed
     for (int i = threadIdx.x; i < kCW * kScratchBytes / 16; i += kThreads)
         st_shared_zero16(smem0 + kHeaderBytes + kStages * kStageBytes + i * 16);
     __syncthreads();
@@ -153,53 +151,67 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     const int u_last = (int)(s1 >> 20), t_last = (int)(s1 & 0xFFFFFu);
     const uint64_t arena = reinterpret_cast<uint64_t>(a.arena_base);
     const uint32_t stage0 = smem0 + kHeaderBytes;
+    const bool is_producer = threadIdx.x == 0;
 
-    if (warp == kCW) {
-        // ================= producer =================
-        if (lane == 0) {
-            int it = 0;
-            for (int u = u_first; u <= u_last && u < sch.units; ++u) {
-                const int b = u / a.Hkv, h = u % a.Hkv;
-                const UnitDesc* ud = a.desc + ((int64_t)b * a.L + a.layer) * a.Hkv + h;
-                const int T = ud->T;
-                const int ntiles = (T + kTT - 1) / kTT;
-                const int tb = u == u_first ? t_first : 0;
-                const int te = u == u_last ? t_last : ntiles;
-                if (te <= tb) continue;
-                const int krow0 = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> 8);
-                const int vrow0 = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> 8);
-                int ntail = 0, tkrow0 = 0, tvrow0 = 0;
-                if (te == ntiles) {
-                    const int n = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
-                    ntail = (n + kTT - 1) / kTT;
-                    const int64_t o = (((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.tail_rows;
-                    tkrow0 = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
-                    tvrow0 = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
-                }
-                const int npre = te - tb;
-                for (int j = 0; j < npre + ntail; ++j, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-                    wait_bar(smem0 + kOffEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
-                    if (*abort_flag) break;
-                    const int kr = j < npre ? krow0 + (tb + j) * kTT : tkrow0 + (j - npre) * kTT;
-                    const int vr = j < npre ? vrow0 + (tb + j) * kTT : tvrow0 + (j - npre) * kTT;
-                    const uint32_t full = smem0 + kOffFull + 8 * s;
-                    const uint32_t dst = stage0 + s * kStageBytes;
-                    mbar_expect_tx(full, kStageBytes);
-                    tma_load_2d(dst, &tmap, 0, kr, full);
-                    tma_load_2d(dst + kHalfBytes, &tmap, 64, kr, full);
-                    tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
-                    tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
-                }
-                if (*abort_flag) break;
+    // ================= producer cursor (thread 0 only): walks the same tile sequence kStages-1 tiles ahead =================
+    int p_u = u_first, p_j = 0, p_npre = 0, p_nseg = 0, p_tb = 0, p_it = 0;
+    int p_krow = 0, p_vrow = 0, p_tkrow = 0, p_tvrow = 0;
+    bool p_done = !is_producer;
+    auto prod_open_unit = [&]() {
+        for (; p_u <= u_last && p_u < sch.units; ++p_u) {
+            const int b = p_u / a.Hkv, h = p_u % a.Hkv;
+            const UnitDesc* ud = a.desc + ((int64_t)b * a.L + a.layer) * a.Hkv + h;
+            const int T = ud->T;
+            const int ntiles = (T + kTT - 1) / kTT;
+            const int tb = p_u == u_first ? t_first : 0;
+            const int te = p_u == u_last ? t_last : ntiles;
+            if (te <= tb) continue;
+            p_krow = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> 8);
+            p_vrow = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> 8);
+            int ntail = 0;
+            if (te == ntiles) {
+                const int n = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
+                ntail = (n + kTT - 1) / kTT;
+                const int64_t o = (((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.tail_rows;
+                p_tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
+                p_tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
             }
+            p_tb = tb;
+            p_npre = te - tb;
+            p_nseg = p_npre + ntail;
+            p_j = 0;
+            return;
         }
-    } else {
-        // ================= consumers =================
-        const int gi = warp >> 2, si = warp & 3;   // group, 16-token slice of the stage
-        const int gid = lane >> 2, tig = lane & 3; // mma fragment coordinates: head row, column pair
-        const int r0 = si * 16;
+        p_done = true;
+    };
+    auto prod_issue = [&]() {
+        if (p_done) return;
+        const int s = p_it % kStages;
+        const uint32_t ph = (uint32_t)(p_it / kStages) & 1u;
+        wait_bar(smem0 + kOffEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
+        if (*abort_flag) { p_done = true; return; }
+        const int kr = p_j < p_npre ? p_krow + (p_tb + p_j) * kTT : p_tkrow + (p_j - p_npre) * kTT;
+        const int vr = p_j < p_npre ? p_vrow + (p_tb + p_j) * kTT : p_tvrow + (p_j - p_npre) * kTT;
+        const uint32_t full = smem0 + kOffFull + 8 * s;
+        const uint32_t dst = stage0 + s * kStageBytes;
+        mbar_expect_tx(full, kStageBytes);
+        tma_load_2d(dst, &tmap, 0, kr, full);
+        tma_load_2d(dst + kHalfBytes, &tmap, 64, kr, full);
+        tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
+        tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
+        ++p_it;
+        if (++p_j == p_nseg) { ++p_u; prod_open_unit(); }
+    };
+    if (is_producer) {
+        prod_open_unit();
+        for (int i = 0; i < kStages - 1; ++i) prod_issue();
+    }
+    __syncwarp();
+
+    // ================= compute: every warp takes 16 tokens of every stage =================
+    {
+        const int gid = lane >> 2, tig = lane & 3;  // mma fragment coordinates: head row, column pair
+        const int r0 = warp * 16;
         const uint32_t scratch = smem0 + kHeaderBytes + kStages * kStageBytes + warp * kScratchBytes;
         float* const scratch_f = reinterpret_cast<float*>(smem_raw + kHeaderBytes + kStages * kStageBytes + warp * kScratchBytes);
         float* const sm_m = reinterpret_cast<float*>(smem_raw + kOffM);
@@ -246,13 +258,12 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             const int32_t* v_idx = ud.v_idx;
             const uint16_t* k_val = reinterpret_cast<const uint16_t*>(ud.k_val);
             const uint16_t* v_val = reinterpret_cast<const uint16_t*>(ud.v_val);
-            int j_my = (((gi - it) % kGroups) + kGroups) % kGroups;  // first tile of the segment owned by this group
-            int cr[4] = {0, 0, 0, 0}, nr[4] = {0, 0, 0, 0};          // {k begin, k end, v begin, v end}
+            int cr[4] = {0, 0, 0, 0}, nr[4] = {0, 0, 0, 0};  // {k begin, k end, v begin, v end}
             int32_t pki[kPF], pvi[kPF];
             uint16_t pkv[kPF], pvv[kPF];
             auto load_ranges = [&](int j, int (&r)[4]) {
                 if (resid && j < npre) {
-                    const int o = (tb + j) * (kTT / kResTile) + si;
+                    const int o = (tb + j) * (kTT / kResTile) + warp;
                     const int o0 = min(o, nres), o1 = min(o + 1, nres);
                     r[0] = ud.k_off[o0]; r[1] = ud.k_off[o1];
                     r[2] = ud.v_off[o0]; r[3] = ud.v_off[o1];
@@ -289,25 +300,27 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 for (int i = 0; i < kScratchBytes / 16 / 32; ++i) st_shared_zero16(scratch + (lane + 32 * i) * 16);
             };
             if (resid) {
-                load_ranges(j_my, cr);
-                load_ranges(j_my + kGroups, nr);
+                load_ranges(0, cr);
+                load_ranges(1, nr);
                 prefetch(k_idx, k_val, cr[0], cr[1], pki, pkv);
                 prefetch(v_idx, v_val, cr[2], cr[3], pvi, pvv);
             }
 
-            for (int j = j_my; j < nseg; j += kGroups) {
+            for (int j = 0; j < nseg; ++j) {
                 const int itj = it + j;
                 const int s = itj % kStages;
                 const uint32_t ph = (uint32_t)(itj / kStages) & 1u;
                 const bool is_tail = j >= npre;
                 const int tile = is_tail ? j - npre : tb + j;
-                const int rows_valid = is_tail ? n_tail_rows - tile * kTT : T - tile * kTT;  // may exceed 64
+                const int rows_valid = is_tail ? n_tail_rows - tile * kTT : T - tile * kTT;  // may exceed the stage
                 const bool with_res = resid && !is_tail;
                 const float kscale = ((coef && !is_tail) ? kC : 1.f) * inv_sqrt_d * kLog2e;
                 const float vscale = (coef && !is_tail) ? kC : 1.f;
                 const int tok0 = tile * kTT + r0;  // first token of this warp's slice
-                int nnr[4];
-                load_ranges(j + 2 * kGroups, nnr);
+
+                // refill the stage every warp released one tile ago
+                if (is_producer) prod_issue();
+                __syncwarp();
 
                 if (with_res && cr[1] > cr[0]) {
                     scatter(k_idx, k_val, cr[0], cr[1], pki, pkv, tok0);
@@ -439,7 +452,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem0 + kOffEmpty + 8 * s);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) { cr[i] = nr[i]; nr[i] = nnr[i]; }
+                for (int i = 0; i < 4; ++i) cr[i] = nr[i];
+                load_ranges(j + 2, nr);
             }
             it += nseg;
 
@@ -453,8 +467,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 for (int jn = 0; jn < 16; ++jn)
                     *reinterpret_cast<float2*>(scratch_f + gid * 128 + jn * 8 + 2 * tig) =
                         make_float2(oacc[jn][0] + oacc[jn][2], oacc[jn][1] + oacc[jn][3]);
-                bar_consumers();
-                // partial slot = number of CTAs that started this unit before this one
+                __syncthreads();
+                // partial slot = number of CTAs with tiles of this unit before this one
                 int slot = 0;
                 for (int c2 = cta - 1; c2 >= 0; --c2) {
                     const uint32_t ustart = (uint32_t)u << 20, e2 = sch.start[c2 + 1], s2 = sch.start[c2];
@@ -462,8 +476,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     if (max(s2, ustart) < e2) ++slot;        // a non-empty range inside this unit
                     if (s2 <= ustart) break;
                 }
-                const int tid = threadIdx.x;  // 0..255 here
-                for (int i = tid; i < a.G * 128; i += kCW * 32) {
+                for (int i = threadIdx.x; i < a.G * 128; i += kThreads) {
                     const int g = i >> 7, ch = i & 127;
                     float M = -INFINITY;
 #pragma unroll
@@ -482,7 +495,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     if (ch == 0) { part[0] = M * 0.6931471805599453f; part[1] = L; }  // the combine step works in natural-log units
                     part[2 + ch] = A;
                 }
-                bar_consumers();
+                __syncthreads();
                 zero_scratch();
                 __syncwarp();
             }
@@ -534,7 +547,7 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
     if (rows == 0 || rows > 0x7FFFFFFFull) return false;
     const cuuint64_t gdim[2] = {128, rows};
     const cuuint64_t gstride[1] = {256};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kTT};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTT};  // 64 channels x one stage of tokens
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = reinterpret_cast<encode_fn>(fn)(reinterpret_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, arena,
                                                  gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -567,8 +580,8 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         nt[u] = (T + kTT - 1) / kTT;
         if (nt[u] >= (1 << 20)) return cudaSuccess;
         const int64_t k = (int64_t)T * 128 * a.keep_num / a.keep_den;
-        // bytes per tile in units of 512 B: two 16 KiB boxes, plus the lists' share for residual units
-        wt[u] = 64 + (a.host_modes[u] == FDKV_MODE_RESIDUAL ? (int)((2 * k * 6 / nt[u] + 511) / 512) : 0);
+        // bytes per tile in units of 512 B: the K and V boxes, plus the lists' share for residual units
+        wt[u] = 2 * kTT * 256 / 512 + (a.host_modes[u] == FDKV_MODE_RESIDUAL ? (int)((2 * k * 6 / nt[u] + 511) / 512) : 0);
         wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
         total_tiles += nt[u];
     }

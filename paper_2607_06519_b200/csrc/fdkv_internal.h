@@ -19,7 +19,7 @@ constexpr int kMaxW = 128;           // probe queries
 constexpr int kListPad = 32;         // slack entries after each residual list (aligned over-reads stay in bounds)
 constexpr int kMaxGroup = 8;
 constexpr int kProbeTile = 64;       // tokens per probe CTA (generic kernel)
-constexpr int kRowPad = 64;          // packed row blocks and tails are padded (zero rows) to this many tokens
+constexpr int kRowPad = 128;         // packed row blocks and tails are padded (zero rows) to this many tokens
 
 enum DeviceFlag : int32_t { kFlagOk = 0, kFlagTimeout = 1, kFlagCountMismatch = 2, kFlagTailFull = 3 };
 

@@ -87,6 +87,10 @@ WORKLOADS = {
     "decode128k": _llama("decode128k", 1, 131072, 32, 256, 4),
     "prefill32k": _llama("prefill32k", 1, 32768, 16, 64, 2),
 }
+# reduced-depth variants of the 32k / 128k workloads (4 layers): same kernels and per-launch sizes, a few GB on the
+# device; used for profiler captures and quick checks
+WORKLOADS["decode32k_4l"] = WORKLOADS["decode32k"].scaled(n_layers=4, name="decode32k_4l")
+WORKLOADS["decode128k_4l"] = WORKLOADS["decode128k"].scaled(n_layers=4, name="decode128k_4l")
 
 
 def rng(seed: int, seq: int, a: int, b: int, tag: int) -> np.random.Generator:
