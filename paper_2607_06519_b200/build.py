@@ -32,7 +32,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for s in SOURCES:
         obj = os.path.join(HERE, "build", s.replace(".cu", ".o"))
         objs.append(obj)
-        cmd = [nvcc, *[f for f in NVCC_FLAGS if f != "--use_fast_math=false"], "-c", os.path.join(CSRC, s), "-o", obj]
+        extra = os.environ.get("FDKV_EXTRA_NVCC_FLAGS", "").split()
+        cmd = [nvcc, *[f for f in NVCC_FLAGS if f != "--use_fast_math=false"], *extra, "-c", os.path.join(CSRC, s), "-o", obj]
         procs.append((s, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for s, p in procs:

@@ -67,7 +67,8 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.probe_pos = take((size_t)kMaxW * 4 + (size_t)s.L * 8);
     w.scores = take((size_t)s.NU * 16);
     w.modes = take((size_t)s.NU * 4);
-    w.partials = take((size_t)s.max_batch * s.Hq * kMaxSplits * (s.d + 2) * 4);
+    w.partials = take((size_t)s.max_batch * s.Hq * kMaxSplits * (s.d + 4) * 4);
+    w.counters = take((size_t)s.max_batch * s.Hkv * 4);
     w.io_q = take((size_t)s.max_batch * s.Hq * s.d * 4);
     w.io_k = take((size_t)s.max_batch * s.Hkv * s.d * 4);
     w.io_v = take((size_t)s.max_batch * s.Hkv * s.d * 4);
@@ -143,6 +144,7 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     c->desc_host.resize((size_t)s.max_batch * s.L * s.Hkv);
     cudaError_t e = cudaMemset(c->arena + c->ar.tail_len, 0, (size_t)s.L * s.max_batch * 4);
     if (e == cudaSuccess) e = cudaMemset(c->work + c->ws.status, 0, 256);
+    if (e == cudaSuccess) e = cudaMemset(c->work + c->ws.counters, 0, (size_t)s.max_batch * s.Hkv * 4);
     if (e == cudaSuccess) e = cudaMemset(c->arena + c->ar.desc, 0, c->desc_host.size() * sizeof(UnitDesc));
     // tails start as zero rows: the fast decode kernel loads whole 64-row boxes and relies on finite padding
     if (e == cudaSuccess) e = cudaMemset(c->arena + c->ar.tail_k, 0, c->ar.bump - c->ar.tail_k);
@@ -406,6 +408,7 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
     a.tail_k = c->arena + c->ar.tail_k; a.tail_v = c->arena + c->ar.tail_v;
     a.tail_len = arp<int32_t>(c, c->ar.tail_len);
     a.partials = wsp<float>(c, c->ws.partials);
+    a.counters = wsp<int32_t>(c, c->ws.counters);
     a.status = wsp<int32_t>(c, c->ws.status);
     CU(launch_decode(a, s.dtype, st));
     return FDKV_OK;

@@ -41,11 +41,15 @@ __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p) { re
 // Appends k_new / v_new rows of every sequence to the layer's tail and bumps the tail length.
 template <typename T>
 __global__ void append_tail_kernel(DecodeArgs a) {
+    // Programmatic dependent launch: this layer's tail is not touched by the kernels still in flight (they belong
+    // to other layers), so the copy may overlap them; the wait at the end keeps stream order transitive.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int b = blockIdx.x;
     int32_t* len = a.tail_len + a.layer * a.max_batch + b;
     const int n = *len;
     if (n >= a.max_tail) {
         if (threadIdx.x == 0) atomicMax(a.status, (int32_t)kFlagTailFull);
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         return;
     }
     const int row = a.Hkv * a.d;
@@ -61,6 +65,7 @@ __global__ void append_tail_kernel(DecodeArgs a) {
     }
     __syncthreads();
     if (threadIdx.x == 0) *len = n + 1;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 constexpr int kWarps = 4;
@@ -239,9 +244,9 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
             L += M == -INFINITY ? 0.f : s_l[w][g] * __expf(s_m[w][g] - M);
             A += s_vacc[w][g][ch];
         }
-        float* part = a.partials + (((int64_t)b * a.Hq + h * G + g) * kMaxSplits + split) * (D + 2);
+        float* part = a.partials + (((int64_t)b * a.Hq + h * G + g) * kMaxSplits + split) * (D + 4);
         if (ch == 0) { part[0] = M; part[1] = L; }
-        part[2 + ch] = A;
+        part[4 + ch] = A;
     }
 }
 
@@ -249,16 +254,16 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
 template <int D>
 __global__ void combine_kernel(const float* partials, int Hq, int splits, void* out, int out_dtype) {
     const int i = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
-    const float* p = partials + ((int64_t)b * Hq + i) * kMaxSplits * (D + 2);
+    const float* p = partials + ((int64_t)b * Hq + i) * kMaxSplits * (D + 4);
     float M = -INFINITY;
-    for (int s = 0; s < splits; ++s) M = fmaxf(M, p[s * (D + 2)]);
+    for (int s = 0; s < splits; ++s) M = fmaxf(M, p[s * (D + 4)]);
     float L = 0.f, A = 0.f;
     for (int s = 0; s < splits; ++s) {
-        const float ms = p[s * (D + 2)];
+        const float ms = p[s * (D + 4)];
         if (ms == -INFINITY) continue;
         const float f = __expf(ms - M);
-        L = fmaf(p[s * (D + 2) + 1], f, L);
-        A = fmaf(p[s * (D + 2) + 2 + ch], f, A);
+        L = fmaf(p[s * (D + 4) + 1], f, L);
+        A = fmaf(p[s * (D + 4) + 4 + ch], f, A);
     }
     const float r = L > 0.f ? A / L : 0.f;
     const int64_t o = ((int64_t)b * Hq + i) * D + ch;
@@ -297,12 +302,21 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st) {
     cudaError_t e;
     if (a.k_new) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(a.batch);
+        cfg.blockDim = dim3(128);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
         if (dtype == FDKV_BF16)
-            append_tail_kernel<__nv_bfloat16><<<a.batch, 128, 0, st>>>(a);
+            e = cudaLaunchKernelEx(&cfg, append_tail_kernel<__nv_bfloat16>, a);
         else
-            append_tail_kernel<float><<<a.batch, 128, 0, st>>>(a);
+            e = cudaLaunchKernelEx(&cfg, append_tail_kernel<float>, a);
+        if (e != cudaSuccess) return e;
         count_launch(1);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     bool handled = false;
     if ((e = launch_decode_fast(a, st, &handled)) != cudaSuccess) return e;

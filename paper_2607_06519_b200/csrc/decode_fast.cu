@@ -15,6 +15,8 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 
 #include "fdkv_internal.h"
 
@@ -34,20 +36,22 @@ constexpr int kSmemBytes = kHeaderBytes + kStages * kStageBytes + kCW * kScratch
 constexpr int kMaxCtas = 296;
 constexpr int kMaxUnits = 512;
 constexpr int kPF = 8;  // residual entries prefetched per lane and list
+constexpr int kPartStride = 128 + 4;  // floats per split-K part: max, sum, 2 pad, 128 accumulators (16-byte aligned)
 constexpr uint32_t kSpinCap = 1u << 22;
 static_assert(kTT == kRowPad, "row blocks are padded to whole stages");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct FastSched {
     uint32_t start[kMaxCtas + 1];  // unit << 20 | first 64-token tile of CTA c; start[ncta] = units << 20
-    int ncta, units;
+    int ncta, units, tslot;
 };
-struct CombSched {
-    uint16_t nparts[kMaxUnits];
+struct PartCount {
+    uint8_t n[kMaxUnits];  // split-K parts per unit (at most kMaxSplits)
 };
+static_assert(kMaxSplits < 256, "part counts are bytes");
 
 // header offsets
-constexpr int kOffFull = 0, kOffEmpty = 64, kOffAbort = 128, kOffM = 256, kOffL = 512;
+constexpr int kOffFull = 0, kOffEmpty = 64, kOffAbort = 128, kOffTicket = 132, kOffM = 256, kOffL = 512;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -122,9 +126,26 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
 }
 
+#ifdef FDKV_TIMING
+__device__ long long g_timing[64][kMaxCtas][8];
+#define TSTAMP(i) do { if (threadIdx.x == 32) g_timing[sch.tslot][blockIdx.x][i] = clock64(); } while (0)
+#define TADD(i, v) do { t_acc[i - 4] += (v); } while (0)
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TGLOBAL(i) do { if (threadIdx.x == 32) g_timing[sch.tslot][blockIdx.x][i] = gtime(); } while (0)
+#else
+#define TGLOBAL(i)
+#define TSTAMP(i)
+#define TADD(i, v)
+#endif
+
 __global__ void __launch_bounds__(kThreads, 1)
-decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastSched sch) {
+decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastSched sch, PartCount pc) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
+    TSTAMP(0);
+#ifdef FDKV_TIMING
+    long long t_acc[2] = {0, 0};
+#endif
+    TGLOBAL(6);
     const uint32_t smem0 = smem_u32(smem_raw);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + kOffAbort);
     if (smem0 & 1023u) {  // the swizzled boxes need 1024-byte alignment; report instead of computing garbage
@@ -132,6 +153,9 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
         return;
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Let the next kernel in the stream start its own prologue as soon as SMs free up (programmatic dependent
+    // launch); everything this kernel reads before its own griddepcontrol.wait is static since commit.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem0 + kOffFull + 8 * s, 1);
@@ -140,10 +164,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // per-warp scratch starts zeroed
-    for (int i = threadIdx.x; i < kCW * kScratchBytes / 16; i += kThreads)
-        st_shared_zero16(smem0 + kHeaderBytes + kStages * kStageBytes + i * 16);
-    __syncthreads();
 
     const int cta = blockIdx.x;
     const uint32_t s0 = sch.start[cta], s1 = sch.start[cta + 1];
@@ -154,9 +174,9 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     const bool is_producer = threadIdx.x == 0;
 
     // ================= producer cursor (thread 0 only): walks the same tile sequence kStages-1 tiles ahead =================
-    int p_u = u_first, p_j = 0, p_npre = 0, p_nseg = 0, p_tb = 0, p_it = 0;
+    int p_u = u_first, p_j = 0, p_npre = 0, p_nseg = 0, p_tb = 0, p_it = 0, p_b = 0, p_h = 0;
     int p_krow = 0, p_vrow = 0, p_tkrow = 0, p_tvrow = 0;
-    bool p_done = !is_producer;
+    bool p_done = !is_producer, p_tail_pending = false, p_waited = false;
     auto prod_open_unit = [&]() {
         for (; p_u <= u_last && p_u < sch.units; ++p_u) {
             const int b = p_u / a.Hkv, h = p_u % a.Hkv;
@@ -168,24 +188,37 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             if (te <= tb) continue;
             p_krow = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> 8);
             p_vrow = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> 8);
-            int ntail = 0;
-            if (te == ntiles) {
-                const int n = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
-                ntail = (n + kTT - 1) / kTT;
-                const int64_t o = (((int64_t)a.layer * a.max_batch + b) * a.Hkv + h) * a.tail_rows;
-                p_tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
-                p_tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
-            }
+            p_tail_pending = te == ntiles;  // this CTA also streams the unit's tail: length read once the wait is over
+            p_b = b;
+            p_h = h;
             p_tb = tb;
             p_npre = te - tb;
-            p_nseg = p_npre + ntail;
+            p_nseg = p_npre;
             p_j = 0;
             return;
         }
         p_done = true;
     };
+    // the tail (rows and length) may have been written by the kernel right before this one: only after the wait
+    auto prod_tail_info = [&]() {
+        p_tail_pending = false;
+        const int n = min(a.tail_len[a.layer * a.max_batch + p_b], a.max_tail);
+        const int64_t o = (((int64_t)a.layer * a.max_batch + p_b) * a.Hkv + p_h) * a.tail_rows;
+        p_tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
+        p_tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
+        p_nseg = p_npre + (n + kTT - 1) / kTT;
+    };
     auto prod_issue = [&]() {
         if (p_done) return;
+        if (p_j == p_npre && p_tail_pending) {  // prefill tiles of the segment are all issued
+            if (!p_waited) return;              // prologue: never touch the tail before the dependency wait
+            prod_tail_info();
+        }
+        if (p_j >= p_nseg) {
+            ++p_u;
+            prod_open_unit();
+            if (p_done) return;
+        }
         const int s = p_it % kStages;
         const uint32_t ph = (uint32_t)(p_it / kStages) & 1u;
         wait_bar(smem0 + kOffEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
@@ -200,13 +233,20 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
         tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
         tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
         ++p_it;
-        if (++p_j == p_nseg) { ++p_u; prod_open_unit(); }
+        ++p_j;
     };
     if (is_producer) {
         prod_open_unit();
         for (int i = 0; i < kStages - 1; ++i) prod_issue();
     }
-    __syncwarp();
+    // per-warp scratch starts zeroed
+    for (int i = threadIdx.x; i < kCW * kScratchBytes / 16; i += kThreads)
+        st_shared_zero16(smem0 + kHeaderBytes + kStages * kStageBytes + i * 16);
+    // everything below may depend on the kernels launched before this one (q, appended tail rows, partial slots)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    p_waited = true;
+    TGLOBAL(1);
+    __syncthreads();
 
     // ================= compute: every warp takes 16 tokens of every stage =================
     {
@@ -318,8 +358,9 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 const float vscale = (coef && !is_tail) ? kC : 1.f;
                 const int tok0 = tile * kTT + r0;  // first token of this warp's slice
 
-                // refill the stage every warp released one tile ago
-                if (is_producer) prod_issue();
+                // keep the copies kStages-1 tiles ahead: refill the stage every warp released one tile ago
+                if (is_producer)
+                    while (!p_done && p_it < itj + kStages) prod_issue();
                 __syncwarp();
 
                 if (with_res && cr[1] > cr[0]) {
@@ -328,7 +369,14 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 }
                 if (resid) prefetch(k_idx, k_val, nr[0], nr[1], pki, pkv);
 
+#ifdef FDKV_TIMING
+                const long long tw0 = clock64();
+#endif
                 wait_bar(smem0 + kOffFull + 8 * s, ph, abort_flag, a.status);
+#ifdef FDKV_TIMING
+                TADD(4, clock64() - tw0);
+                TADD(5, 1);
+#endif
                 const uint32_t kb = stage0 + s * kStageBytes, vb = kb + 2 * kHalfBytes;
 
                 // ---- S^T[head][token] = q . k over 128 channels; two n-tiles of 8 tokens ----
@@ -456,6 +504,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 load_ranges(j + 2, nr);
             }
             it += nseg;
+            TGLOBAL(2);
 
             // ---- merge the eight warps' states into this segment's split-K partial ----
             {
@@ -491,46 +540,78 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                             A = fmaf(ow[g * 128 + ch], f, A);
                         }
                     }
-                    float* part = a.partials + (((int64_t)b * a.Hq + h * a.G + g) * kMaxSplits + slot) * (128 + 2);
+                    float* part = a.partials + (((int64_t)b * a.Hq + h * a.G + g) * kMaxSplits + slot) * kPartStride;
                     if (ch == 0) { part[0] = M * 0.6931471805599453f; part[1] = L; }  // the combine step works in natural-log units
-                    part[2 + ch] = A;
+                    part[4 + ch] = A;
                 }
+                // ---- split-K combine by whichever CTA finishes this unit last (atomic ticket, nobody waits) ----
+                __threadfence();
                 __syncthreads();
+                int* const s_ticket = reinterpret_cast<int*>(smem_raw + kOffTicket);
+                if (threadIdx.x == 0) *s_ticket = atomicAdd(a.counters + u, 1);
+                __syncthreads();
+                const int nparts = pc.n[u];
+                if (*s_ticket == nparts - 1) {
+                    __threadfence();
+                    // warp w sums parts w, w+8, ... (lane = 4 channels) for every head; the scratch area holds the
+                    // eight per-warp sums, the header the per-head denominators
+                    float* const red = reinterpret_cast<float*>(smem_raw + kHeaderBytes + kStages * kStageBytes);  // [8][G][128]
+                    for (int g = 0; g < a.G; ++g) {
+                        const float* pp = a.partials + ((int64_t)b * a.Hq + h * a.G + g) * kMaxSplits * kPartStride;
+                        float mx = -INFINITY;
+                        for (int sp = lane; sp < nparts; sp += 32) mx = fmaxf(mx, __ldcg(pp + sp * kPartStride));
+#pragma unroll
+                        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+                        float ls = 0.f;
+                        if (mx != -INFINITY)
+                            for (int sp = lane; sp < nparts; sp += 32)
+                                ls = fmaf(__ldcg(pp + sp * kPartStride + 1), __expf(__ldcg(pp + sp * kPartStride) - mx), ls);
+#pragma unroll
+                        for (int o = 16; o; o >>= 1) ls += __shfl_xor_sync(0xFFFFFFFFu, ls, o);
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (mx != -INFINITY)
+                            for (int sp = warp; sp < nparts; sp += kCW) {
+                                const float f = __expf(__ldcg(pp + sp * kPartStride) - mx);
+                                const float4 v = __ldcg(reinterpret_cast<const float4*>(pp + sp * kPartStride + 4) + lane);
+                                acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y);
+                                acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
+                            }
+                        reinterpret_cast<float4*>(red + (warp * a.G + g) * 128)[lane] = acc;
+                        if (warp == 0 && lane == 0) sm_l[g] = ls;
+                    }
+                    __syncthreads();
+                    for (int i = threadIdx.x; i < a.G * 128; i += kThreads) {
+                        const int g = i >> 7, ch = i & 127;
+                        float A = 0.f;
+#pragma unroll
+                        for (int w = 0; w < kCW; ++w) A += red[(w * a.G + g) * 128 + ch];
+                        const float L = sm_l[g];
+                        const float r = L > 0.f ? A / L : 0.f;
+                        const int64_t o = ((int64_t)b * a.Hq + h * a.G + g) * 128 + ch;
+                        if (a.out_dtype == FDKV_BF16)
+                            reinterpret_cast<__nv_bfloat16*>(a.out)[o] = __float2bfloat16_rn(r);
+                        else
+                            reinterpret_cast<float*>(a.out)[o] = r;
+                    }
+                    if (threadIdx.x == 0) a.counters[u] = 0;  // ready for the next launch
+                    __syncthreads();
+                }
                 zero_scratch();
-                __syncwarp();
+                __syncthreads();
             }
         }
     }
+    TSTAMP(3);
+    TGLOBAL(7);
+#ifdef FDKV_TIMING
+    if (threadIdx.x == 32) { g_timing[sch.tslot][blockIdx.x][4] = t_acc[0]; g_timing[sch.tslot][blockIdx.x][5] = t_acc[1]; }
+#endif
     // after a timed-out wait: give copies that may still be in flight time to land before the CTA retires
     if (*abort_flag)
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
 }
 
 }  // namespace
-
-// out = sum_s e^{m_s - M} acc_s / sum_s e^{m_s - M} l_s over the unit's parts.  grid (Hq, batch), 128 threads.
-__global__ void combine_fast_kernel(const float* partials, int Hq, int Hkv, CombSched cs, void* out, int out_dtype) {
-    const int i = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
-    const int G = Hq / Hkv;
-    const int n = cs.nparts[b * Hkv + i / G];
-    const float* p = partials + ((int64_t)b * Hq + i) * kMaxSplits * 130;
-    float M = -INFINITY;
-    for (int s = 0; s < n; ++s) M = fmaxf(M, p[s * 130]);
-    float L = 0.f, A = 0.f;
-    for (int s = 0; s < n; ++s) {
-        const float ms = p[s * 130];
-        if (ms == -INFINITY) continue;
-        const float f = __expf(ms - M);
-        L = fmaf(p[s * 130 + 1], f, L);
-        A = fmaf(p[s * 130 + 2 + ch], f, A);
-    }
-    const float r = L > 0.f ? A / L : 0.f;
-    const int64_t o = ((int64_t)b * Hq + i) * 128 + ch;
-    if (out_dtype == FDKV_BF16)
-        reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(r);
-    else
-        reinterpret_cast<float*>(out)[o] = r;
-}
 
 bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
     typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -569,9 +650,18 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    // ---- flat byte-weighted schedule: CTA c starts at weight c * W / ncta ----
+    static double res_cost = -1.0;
+    static bool use_pdl = true;
+    if (res_cost < 0) {
+        const char* ev = getenv("FDKV_RES_COST");  // tuning knobs for benchmark sweeps
+        res_cost = ev ? atof(ev) : 1.6;
+        if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 1.6;
+        const char* pv = getenv("FDKV_NO_PDL");
+        use_pdl = !(pv && pv[0] == '1');
+    }
+    // ---- flat cost-weighted schedule: CTA c starts at weight c * W / ncta ----
     FastSched sch;
-    CombSched cs;
+    PartCount cs;
     std::vector<int64_t> wp(units + 1, 0);
     std::vector<int> nt(units), wt(units);
     int64_t total_tiles = 0;
@@ -580,12 +670,17 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         nt[u] = (T + kTT - 1) / kTT;
         if (nt[u] >= (1 << 20)) return cudaSuccess;
         const int64_t k = (int64_t)T * 128 * a.keep_num / a.keep_den;
-        // bytes per tile in units of 512 B: the K and V boxes, plus the lists' share for residual units
-        wt[u] = 2 * kTT * 256 / 512 + (a.host_modes[u] == FDKV_MODE_RESIDUAL ? (int)((2 * k * 6 / nt[u] + 511) / 512) : 0);
+        // cost per tile: bytes in units of 512 B (the K and V boxes, plus the lists' share for residual units),
+        // residual tiles scaled by the measured ratio of their compute time to a plain tile's
+        wt[u] = 2 * kTT * 256 / 512;
+        if (a.host_modes[u] == FDKV_MODE_RESIDUAL) wt[u] = (int)((wt[u] + (2 * k * 6 / nt[u] + 511) / 512) * res_cost);
         wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
         total_tiles += nt[u];
     }
     const int ncta = (int)std::min<int64_t>(std::min(sm_count, kMaxCtas), total_tiles);
+    static unsigned g_launch_no = 0;
+    ++g_launch_no;
+    sch.tslot = (int)(g_launch_no % 64);
     sch.ncta = ncta;
     sch.units = units;
     {
@@ -599,23 +694,56 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         sch.start[ncta] = (uint32_t)units << 20;
     }
     // parts per unit = CTAs whose range contains at least one of its tiles
-    for (int u = 0; u < units; ++u) cs.nparts[u] = 0;
+    for (int u = 0; u < kMaxUnits; ++u) cs.n[u] = 0;
     for (int c = 0; c < ncta; ++c) {
         const int ua = (int)(sch.start[c] >> 20), ta = (int)(sch.start[c] & 0xFFFFFu);
         const int ub = (int)(sch.start[c + 1] >> 20), tb = (int)(sch.start[c + 1] & 0xFFFFFu);
         for (int u = ua; u <= ub && u < units; ++u) {
             const int b0 = u == ua ? ta : 0, b1 = u == ub ? tb : nt[u];
-            if (b1 > b0) cs.nparts[u]++;
+            if (b1 > b0 && cs.n[u] < 255) cs.n[u]++;
         }
     }
     for (int u = 0; u < units; ++u)
-        if (cs.nparts[u] > kMaxSplits) return cudaSuccess;
-    decode_fast_kernel<<<ncta, kThreads, kSmemBytes, st>>>(*reinterpret_cast<const CUtensorMap*>(a.tmap), a, sch);
-    cudaError_t e = cudaGetLastError();
+        if (cs.n[u] > kMaxSplits) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ncta);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = use_pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_fast_kernel, *reinterpret_cast<const CUtensorMap*>(a.tmap), a, sch, cs);
     if (e != cudaSuccess) return e;
-    combine_fast_kernel<<<dim3(a.Hq, a.batch), 128, 0, st>>>(a.partials, a.Hq, a.Hkv, cs, a.out, a.out_dtype);
-    count_launch(2);
+    count_launch(1);
     *handled = true;
+#ifdef FDKV_TIMING
+    if (getenv("FDKV_TIMING_DUMP") && (g_launch_no % 64) == 63) {
+        static long long h[64][kMaxCtas][8];
+        cudaStreamSynchronize(st);
+        cudaMemcpyFromSymbol(h, g_timing, sizeof(h));
+        long long base = h[0][0][6];
+        for (int l = 0; l < 64; ++l) {
+            long long g0 = h[l][0][6], g0max = g0, g1 = h[l][0][7], g1min = g1, busy = 0, fd = 0, wf = 0;
+            for (int c = 0; c < ncta; ++c) {
+                g0 = std::min(g0, h[l][c][6]); g0max = std::max(g0max, h[l][c][6]);
+                g1 = std::max(g1, h[l][c][7]); g1min = std::min(g1min, h[l][c][7]);
+                busy += h[l][c][7] - h[l][c][6];
+                fd += h[l][c][1] - h[l][c][0];
+                wf += h[l][c][4];
+            }
+            fprintf(stderr, "launch %2d: first_start %8lld last_start %8lld first_end %8lld last_end %8lld  mean_busy %6lld ns mean_wait_full %6lld cyc\n",
+                    l, g0 - base, g0max - base, g1min - base, g1 - base, busy / ncta, wf / ncta);
+            if (l == 45)
+                for (int c = 0; c < ncta; ++c)
+                    fprintf(stderr, "cta %3d unit %2u mode %d tiles %2lld start %6lld waited %6lld loop_end %6lld end %6lld wait_full_cyc %6lld\n", c,
+                            sch.start[c] >> 20, a.host_modes[sch.start[c] >> 20], h[l][c][5], h[l][c][6] - g0, h[l][c][1] - g0, h[l][c][2] - g0,
+                            h[l][c][7] - g0, h[l][c][4]);
+        }
+    }
+#endif
     return cudaGetLastError();
 }
 

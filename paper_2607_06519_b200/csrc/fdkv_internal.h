@@ -61,7 +61,7 @@ struct Shape {
 
 struct WsLayout {
     size_t status, z0, z1, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, probe_part, probe_pos, scores, modes,
-        partials, io_q, io_k, io_v, io_out, total;
+        partials, counters, io_q, io_k, io_v, io_out, total;
 };
 struct ArenaLayout {
     size_t tail_len, desc, tail_k, tail_v, bump, worst_total;
@@ -165,7 +165,8 @@ struct DecodeArgs {
     const void* arena_base;
     int keep_num, keep_den;
     int32_t* tail_len;      // [L][max_batch]
-    float* partials;        // [batch][Hq][kMaxSplits][d+2]
+    float* partials;        // [batch][Hq][kMaxSplits][d+4]: max, sum, 2 pad, d accumulators
+    int32_t* counters;      // [max_batch][Hkv] split-K arrival tickets, zero between launches
     int32_t* status;
 };
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st);
