@@ -63,6 +63,7 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.tile_off = take((size_t)s.NT * (s.ntiles_max + 1) * 4);
     w.idx = take((size_t)s.NT * s.kcap * 4);
     w.val = take((size_t)s.NT * s.kcap * s.esize);
+    w.packed = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NT * s.kcap * 4 : 0);
     w.probe_part = take((size_t)s.NU * s.nptiles_max * 16);
     w.probe_pos = take((size_t)kMaxW * 4 + (size_t)s.L * 8);
     w.scores = take((size_t)s.NU * 16);
@@ -150,6 +151,7 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     if (e == cudaSuccess) e = cudaMemset(c->arena + c->ar.tail_k, 0, c->ar.bump - c->ar.tail_k);
     if (e != cudaSuccess) { delete c; return cuda_fail(e); }
     if (s.dtype == FDKV_BF16 && s.d == 128) c->has_tmap = make_arena_tensor_map(c->arena, arena_bytes, c->tmap);
+    c->packed_lists = c->has_tmap && s.max_batch * s.Hkv <= kFastMaxUnits;
     *out = c;
     return FDKV_OK;
 }
@@ -228,6 +230,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
     sa.idx = wsp<int32_t>(c, c->ws.idx);
     sa.val = c->work + c->ws.val;
+    sa.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
     sa.status = wsp<int32_t>(c, c->ws.status);
     CU(launch_select_and_compact(sa, s.dtype, st));
     for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; }
@@ -305,7 +308,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     const int64_t k = (int64_t)T * s.d * s.keep_num / s.keep_den;
     const int ntiles = (T + kResTile - 1) / kResTile;
     // list copies include the slack so that aligned over-reads of the last tile stay inside the allocation
-    const size_t idx_b = (size_t)(k + kListPad) * 4, val_b = (size_t)(k + kListPad) * s.esize, off_b = (size_t)(ntiles + 1) * 4;
+    const size_t idx_b = (size_t)(k + kListPad) * 4, off_b = (size_t)(ntiles + 1) * 4;
+    const size_t val_b = c->packed_lists ? 0 : (size_t)(k + kListPad) * s.esize;  // packed entries carry their value
     size_t need = 0;
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u];
@@ -351,17 +355,21 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 by_mode[m] += rows;
                 if (m == FDKV_MODE_RESIDUAL) {
                     char* pi = take(idx_b);
-                    char* pv = take(val_b);
+                    char* pv = val_b ? take(val_b) : nullptr;
                     char* po = take(off_b);
-                    CU(cudaMemcpyAsync(pi, c->work + c->ws.idx + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
-                    CU(cudaMemcpyAsync(pv, c->work + c->ws.val + ut * s.kcap * s.esize, val_b, cudaMemcpyDeviceToDevice, st));
+                    if (c->packed_lists) {
+                        CU(cudaMemcpyAsync(pi, c->work + c->ws.packed + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
+                    } else {
+                        CU(cudaMemcpyAsync(pi, c->work + c->ws.idx + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
+                        CU(cudaMemcpyAsync(pv, c->work + c->ws.val + ut * s.kcap * s.esize, val_b, cudaMemcpyDeviceToDevice, st));
+                    }
                     CU(cudaMemcpyAsync(po, c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, off_b, cudaMemcpyDeviceToDevice, st));
                     for (UnitDesc* d : {d0, d1}) {
                         (is_v ? d->v_idx : d->k_idx) = (const int32_t*)pi;
                         (is_v ? d->v_val : d->k_val) = pv;
                         (is_v ? d->v_off : d->k_off) = (const int32_t*)po;
                     }
-                    by_mode[1] += (size_t)k * (4 + s.esize);
+                    by_mode[1] += (size_t)k * (c->packed_lists ? 4 : 4 + s.esize);
                 }
             }
         }
@@ -401,6 +409,7 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
     a.tmap = c->has_tmap ? c->tmap : nullptr;
     a.arena_base = c->arena;
     a.keep_num = s.keep_num; a.keep_den = s.keep_den;
+    a.packed_lists = c->packed_lists ? 1 : 0;
     a.desc = arp<UnitDesc>(c, c->ar.desc);
     a.L = s.L; a.layer = layer; a.batch = batch; a.Hq = s.Hq; a.Hkv = s.Hkv; a.G = s.G; a.d = s.d;
     a.max_tail = s.max_tail; a.max_batch = s.max_batch; a.Tmax_batch = Tmax;
@@ -510,7 +519,7 @@ fdkv_status fdkv_decode_bytes(fdkv_ctx* c, int32_t layer, int32_t batch, size_t*
         for (int h = 0; h < s.Hkv; ++h) {
             const int m = q.modes[(layer / 2) * s.Hkv + h];
             tot += 2 * (size_t)(q.T + q.tail_len[layer]) * s.d * s.esize;
-            if (m == FDKV_MODE_RESIDUAL) tot += 2 * ((size_t)k * (4 + s.esize) + (size_t)(ntiles + 1) * 4);
+            if (m == FDKV_MODE_RESIDUAL) tot += 2 * ((size_t)k * (c->packed_lists ? 4 : 4 + s.esize) + (size_t)(ntiles + 1) * 4);
         }
     }
     *bytes_host = tot;

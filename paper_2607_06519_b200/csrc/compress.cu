@@ -257,6 +257,20 @@ __global__ void __launch_bounds__(1024) tile_scan_kernel(SelectArgs a) {
     }
 }
 
+// Packed entry of the bf16 / head_dim 128 decode kernel: low half = value bits, high half = (byte offset / 2) of the
+// entry inside a 16-token x 128-channel scratch tile laid out as two 64-channel halves of 128-byte rows whose
+// 16-byte chunks are XOR-swizzled with the row (the layout ldmatrix reads without bank conflicts).
+template <typename T>
+__device__ __forceinline__ uint32_t packed_entry(T v, int flat);
+template <>
+__device__ __forceinline__ uint32_t packed_entry<float>(float, int) { return 0u; }
+template <>
+__device__ __forceinline__ uint32_t packed_entry<__nv_bfloat16>(__nv_bfloat16 v, int flat) {
+    const int row = (flat >> 7) & 15, ch = flat & 127;
+    const uint32_t off = (uint32_t)((ch >> 6) * 2048 + row * 128 + ((((ch >> 3) & 7) ^ (row & 7)) << 4) + (ch & 7) * 2);
+    return (uint32_t)__bfloat16_as_ushort(v) | ((off >> 1) << 16);
+}
+
 // ----- C5: ordered write ---------------------------------------------------------------------------
 // One warp per tile walks its entries in flat-index order; an entry is kept when its key is above the
 // threshold, or equal to it and among the first `need` such entries of the whole unit-tensor.
@@ -273,6 +287,7 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
     const T* z = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride;
     int32_t* idx = a.idx + (int64_t)ut * a.kcap;
     T* val = reinterpret_cast<T*>(a.val) + (int64_t)ut * a.kcap;
+    uint32_t* pk = a.packed ? a.packed + (int64_t)ut * a.kcap : nullptr;
     uint32_t pos = (uint32_t)a.tile_off[(int64_t)ut * (a.ntiles_max + 1) + tile];
     uint32_t eq_rank = a.tile_eq[(int64_t)ut * a.ntiles_max + tile];
     const int64_t e_begin = (int64_t)tile * kResTile * a.d;
@@ -323,6 +338,7 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
             if (keep >> i & 1u) {
                 idx[w] = (int32_t)(e + i);
                 val[w] = z[e + i];
+                if (pk) pk[w] = packed_entry<T>(z[e + i], (int)(e + i));
                 ++w;
             }
         pos += __shfl_sync(0xFFFFFFFFu, incl, 31);

@@ -321,6 +321,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st) {
     bool handled = false;
     if ((e = launch_decode_fast(a, st, &handled)) != cudaSuccess) return e;
     if (handled) return cudaSuccess;
+    if (a.packed_lists) return cudaErrorNotSupported;  // packed residual lists are only read by the kernel above
 
     const int ntiles = (a.Tmax_batch + kGTile - 1) / kGTile;
     int splits = (2 * 148 + a.Hkv * a.batch - 1) / (a.Hkv * a.batch);

@@ -34,7 +34,7 @@ constexpr int kScratchBytes = 4096;          // per consumer warp: 16 tokens x 1
 constexpr int kHeaderBytes = 1024;
 constexpr int kSmemBytes = kHeaderBytes + kStages * kStageBytes + kCW * kScratchBytes;
 constexpr int kMaxCtas = 296;
-constexpr int kMaxUnits = 512;
+constexpr int kMaxUnits = kFastMaxUnits;
 constexpr int kPF = 8;  // residual entries prefetched per lane and list
 constexpr int kPartStride = 128 + 4;  // floats per split-K part: max, sum, 2 pad, 128 accumulators (16-byte aligned)
 constexpr uint32_t kSpinCap = 1u << 22;
@@ -48,7 +48,7 @@ struct FastSched {
 struct PartCount {
     uint8_t n[kMaxUnits];  // split-K parts per unit (at most kMaxSplits)
 };
-static_assert(kMaxSplits < 256, "part counts are bytes");
+static_assert(kMaxSplits < 256 && kMaxSplits % 32 == 0, "part counts are bytes; the combine holds one part per lane and round");
 
 // header offsets
 constexpr int kOffFull = 0, kOffEmpty = 64, kOffAbort = 128, kOffTicket = 132, kOffM = 256, kOffL = 512;
@@ -292,15 +292,20 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
 #pragma unroll
             for (int j = 0; j < 16; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
             float m_run = -INFINITY, l_run = 0.f;
+            // split-K part slot of this segment = number of CTAs with tiles of this unit before this one
+            int slot = 0;
+            for (int c2 = cta - 1; c2 >= 0; --c2) {
+                const uint32_t ustart = (uint32_t)u << 20, e2 = sch.start[c2 + 1], s2 = sch.start[c2];
+                if (e2 <= ustart) break;                 // ends before this unit's first tile
+                if (max(s2, ustart) < e2) ++slot;        // a non-empty range inside this unit
+                if (s2 <= ustart) break;
+            }
 
-            // ---- residual lists: ranges two tiles ahead, entries one tile ahead ----
-            const int32_t* k_idx = ud.k_idx;
-            const int32_t* v_idx = ud.v_idx;
-            const uint16_t* k_val = reinterpret_cast<const uint16_t*>(ud.k_val);
-            const uint16_t* v_val = reinterpret_cast<const uint16_t*>(ud.v_val);
+            // ---- residual lists (packed entries): ranges two tiles ahead, entries one tile ahead ----
+            const uint32_t* k_ent = reinterpret_cast<const uint32_t*>(ud.k_idx);
+            const uint32_t* v_ent = reinterpret_cast<const uint32_t*>(ud.v_idx);
             int cr[4] = {0, 0, 0, 0}, nr[4] = {0, 0, 0, 0};  // {k begin, k end, v begin, v end}
-            int32_t pki[kPF], pvi[kPF];
-            uint16_t pkv[kPF], pvv[kPF];
+            uint32_t pke[kPF], pve[kPF];
             auto load_ranges = [&](int j, int (&r)[4]) {
                 if (resid && j < npre) {
                     const int o = (tb + j) * (kTT / kResTile) + warp;
@@ -311,28 +316,23 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     r[0] = r[1] = r[2] = r[3] = 0;
                 }
             };
-            auto prefetch = [&](const int32_t* idx, const uint16_t* val, int e0, int e1, int32_t (&pi)[kPF], uint16_t (&pv)[kPF]) {
+            auto prefetch = [&](const uint32_t* ent, int e0, int e1, uint32_t (&pe)[kPF]) {
 #pragma unroll
                 for (int i = 0; i < kPF; ++i) {
                     const int e = e0 + lane + 32 * i;
-                    if (e < e1) { pi[i] = idx[e]; pv[i] = val[e]; }
+                    if (e < e1) pe[i] = ent[e];
                 }
             };
-            // scatter one list slice into the scratch tile (swizzled [2 halves][16 rows][64 ch])
-            auto scatter = [&](const int32_t* idx, const uint16_t* val, int e0, int e1, const int32_t (&pi)[kPF],
-                               const uint16_t (&pv)[kPF], int tok0) {
-                const int base = tok0 * 128;
+            // scatter one list slice into the scratch tile: each entry carries its own shared-memory offset
+            auto scatter = [&](const uint32_t* ent, int e0, int e1, const uint32_t (&pe)[kPF]) {
 #pragma unroll
                 for (int i = 0; i < kPF; ++i) {
                     const int e = e0 + lane + 32 * i;
-                    if (e < e1) {
-                        const int f = pi[i] - base, row = f >> 7, ch = f & 127;
-                        st_shared_u16(scratch + (ch >> 6) * 2048 + swz(row, ch >> 3) + (ch & 7) * 2, pv[i]);
-                    }
+                    if (e < e1) st_shared_u16(scratch + ((pe[i] >> 16) << 1), (uint16_t)(pe[i] & 0xFFFFu));
                 }
                 for (int e = e0 + 32 * kPF + lane; e < e1; e += 32) {  // dense slices: direct loads
-                    const int f = idx[e] - base, row = f >> 7, ch = f & 127;
-                    st_shared_u16(scratch + (ch >> 6) * 2048 + swz(row, ch >> 3) + (ch & 7) * 2, val[e]);
+                    const uint32_t w = ent[e];
+                    st_shared_u16(scratch + ((w >> 16) << 1), (uint16_t)(w & 0xFFFFu));
                 }
             };
             auto zero_scratch = [&]() {
@@ -342,8 +342,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             if (resid) {
                 load_ranges(0, cr);
                 load_ranges(1, nr);
-                prefetch(k_idx, k_val, cr[0], cr[1], pki, pkv);
-                prefetch(v_idx, v_val, cr[2], cr[3], pvi, pvv);
+                prefetch(k_ent, cr[0], cr[1], pke);
+                prefetch(v_ent, cr[2], cr[3], pve);
             }
 
             for (int j = 0; j < nseg; ++j) {
@@ -356,7 +356,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 const bool with_res = resid && !is_tail;
                 const float kscale = ((coef && !is_tail) ? kC : 1.f) * inv_sqrt_d * kLog2e;
                 const float vscale = (coef && !is_tail) ? kC : 1.f;
-                const int tok0 = tile * kTT + r0;  // first token of this warp's slice
 
                 // keep the copies kStages-1 tiles ahead: refill the stage every warp released one tile ago
                 if (is_producer)
@@ -364,10 +363,10 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 __syncwarp();
 
                 if (with_res && cr[1] > cr[0]) {
-                    scatter(k_idx, k_val, cr[0], cr[1], pki, pkv, tok0);
+                    scatter(k_ent, cr[0], cr[1], pke);
                     __syncwarp();
                 }
-                if (resid) prefetch(k_idx, k_val, nr[0], nr[1], pki, pkv);
+                if (resid) prefetch(k_ent, nr[0], nr[1], pke);
 
 #ifdef FDKV_TIMING
                 const long long tw0 = clock64();
@@ -398,17 +397,21 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                         }
                     }
                     if (with_res && cr[1] > cr[0]) {
+                        float racc[2][4];  // own accumulators: the two passes' mma chains run side by side
 #pragma unroll
                         for (int nt = 0; nt < 2; ++nt) {
+                            racc[nt][0] = racc[nt][1] = racc[nt][2] = racc[nt][3] = 0.f;
                             const int row = nt * 8 + rr;
 #pragma unroll
                             for (int kp = 0; kp < 4; ++kp) {
                                 const int c = 4 * kp + mi;
                                 uint32_t b0, b1, b2, b3;
                                 ldsm_x4(scratch + (c >> 3) * 2048 + swz(row, c), b0, b1, b2, b3);
-                                mma_bf16(sacc[nt], qa[2 * kp][0] ^ sgn, 0u, qa[2 * kp][1] ^ sgn, 0u, b0, b1);
-                                mma_bf16(sacc[nt], qa[2 * kp + 1][0] ^ sgn, 0u, qa[2 * kp + 1][1] ^ sgn, 0u, b2, b3);
+                                mma_bf16(racc[nt], qa[2 * kp][0] ^ sgn, 0u, qa[2 * kp][1] ^ sgn, 0u, b0, b1);
+                                mma_bf16(racc[nt], qa[2 * kp + 1][0] ^ sgn, 0u, qa[2 * kp + 1][1] ^ sgn, 0u, b2, b3);
                             }
+                            sacc[nt][0] += racc[nt][0];
+                            sacc[nt][1] += racc[nt][1];
                         }
                         __syncwarp();
                         zero_scratch();
@@ -416,10 +419,10 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     }
                 }
                 if (with_res && cr[3] > cr[2]) {
-                    scatter(v_idx, v_val, cr[2], cr[3], pvi, pvv, tok0);
+                    scatter(v_ent, cr[2], cr[3], pve);
                     __syncwarp();
                 }
-                if (resid) prefetch(v_idx, v_val, nr[2], nr[3], pvi, pvv);
+                if (resid) prefetch(v_ent, nr[2], nr[3], pve);
 
                 // ---- online softmax for head gid over this slice's 16 tokens (4 per thread) ----
                 float p[2][2];
@@ -517,14 +520,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     *reinterpret_cast<float2*>(scratch_f + gid * 128 + jn * 8 + 2 * tig) =
                         make_float2(oacc[jn][0] + oacc[jn][2], oacc[jn][1] + oacc[jn][3]);
                 __syncthreads();
-                // partial slot = number of CTAs with tiles of this unit before this one
-                int slot = 0;
-                for (int c2 = cta - 1; c2 >= 0; --c2) {
-                    const uint32_t ustart = (uint32_t)u << 20, e2 = sch.start[c2 + 1], s2 = sch.start[c2];
-                    if (e2 <= ustart) break;                 // ends before this unit's first tile
-                    if (max(s2, ustart) < e2) ++slot;        // a non-empty range inside this unit
-                    if (s2 <= ustart) break;
-                }
                 for (int i = threadIdx.x; i < a.G * 128; i += kThreads) {
                     const int g = i >> 7, ch = i & 127;
                     float M = -INFINITY;
@@ -553,38 +548,52 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 const int nparts = pc.n[u];
                 if (*s_ticket == nparts - 1) {
                     __threadfence();
-                    // warp w sums parts w, w+8, ... (lane = 4 channels) for every head; the scratch area holds the
-                    // eight per-warp sums, the header the per-head denominators
-                    float* const red = reinterpret_cast<float*>(smem_raw + kHeaderBytes + kStages * kStageBytes);  // [8][G][128]
-                    for (int g = 0; g < a.G; ++g) {
+                    // Warp w takes head w % G and every (8/G)-th part of it, 4 channels per lane; the scratch area
+                    // holds the per-warp sums, the header the per-warp denominators.
+                    float* const red = reinterpret_cast<float*>(smem_raw + kHeaderBytes + kStages * kStageBytes);  // [8][128]
+                    {
+                        const int g = warp % a.G, pgi = warp / a.G, npg = kCW / a.G;
                         const float* pp = a.partials + ((int64_t)b * a.Hq + h * a.G + g) * kMaxSplits * kPartStride;
+                        float mreg[kMaxSplits / 32], lreg[kMaxSplits / 32];
                         float mx = -INFINITY;
-                        for (int sp = lane; sp < nparts; sp += 32) mx = fmaxf(mx, __ldcg(pp + sp * kPartStride));
+#pragma unroll
+                        for (int i = 0; i < kMaxSplits / 32; ++i) {
+                            const int sp = lane + 32 * i;
+                            mreg[i] = sp < nparts ? __ldcg(pp + sp * kPartStride) : -INFINITY;
+                            lreg[i] = sp < nparts ? __ldcg(pp + sp * kPartStride + 1) : 0.f;
+                        }
+#pragma unroll
+                        for (int i = 0; i < kMaxSplits / 32; ++i) mx = fmaxf(mx, mreg[i]);
 #pragma unroll
                         for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
                         float ls = 0.f;
-                        if (mx != -INFINITY)
-                            for (int sp = lane; sp < nparts; sp += 32)
-                                ls = fmaf(__ldcg(pp + sp * kPartStride + 1), __expf(__ldcg(pp + sp * kPartStride) - mx), ls);
+#pragma unroll
+                        for (int i = 0; i < kMaxSplits / 32; ++i) {
+                            mreg[i] = mreg[i] == -INFINITY ? 0.f : __expf(mreg[i] - mx);  // now the part's weight
+                            ls = fmaf(lreg[i], mreg[i], ls);
+                        }
 #pragma unroll
                         for (int o = 16; o; o >>= 1) ls += __shfl_xor_sync(0xFFFFFFFFu, ls, o);
                         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (mx != -INFINITY)
-                            for (int sp = warp; sp < nparts; sp += kCW) {
-                                const float f = __expf(__ldcg(pp + sp * kPartStride) - mx);
+#pragma unroll
+                        for (int i = 0; i < kMaxSplits / 32; ++i) {
+                            for (int s32 = pgi; s32 < 32; s32 += npg) {
+                                const int sp = 32 * i + s32;
+                                if (sp >= nparts) break;
+                                const float f = __shfl_sync(0xFFFFFFFFu, mreg[i], s32);
                                 const float4 v = __ldcg(reinterpret_cast<const float4*>(pp + sp * kPartStride + 4) + lane);
                                 acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y);
                                 acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
                             }
-                        reinterpret_cast<float4*>(red + (warp * a.G + g) * 128)[lane] = acc;
-                        if (warp == 0 && lane == 0) sm_l[g] = ls;
+                        }
+                        reinterpret_cast<float4*>(red + warp * 128)[lane] = acc;
+                        if (lane == 0) sm_l[warp] = ls;
                     }
                     __syncthreads();
                     for (int i = threadIdx.x; i < a.G * 128; i += kThreads) {
                         const int g = i >> 7, ch = i & 127;
                         float A = 0.f;
-#pragma unroll
-                        for (int w = 0; w < kCW; ++w) A += red[(w * a.G + g) * 128 + ch];
+                        for (int w = g; w < kCW; w += a.G) A += red[w * 128 + ch];
                         const float L = sm_l[g];
                         const float r = L > 0.f ? A / L : 0.f;
                         const int64_t o = ((int64_t)b * a.Hq + h * a.G + g) * 128 + ch;
@@ -639,7 +648,7 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
 cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handled) {
     *handled = false;
     const int units = a.batch * a.Hkv;
-    if (!a.tmap || a.d != 128 || units > kMaxUnits || units < 1) return cudaSuccess;
+    if (!a.tmap || !a.packed_lists || a.d != 128 || units > kMaxUnits || units < 1) return cudaSuccess;
     static int sm_count = 0;
     static bool attr_done = false;
     if (!attr_done) {
@@ -668,16 +677,16 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     for (int u = 0; u < units; ++u) {
         const int T = a.host_T[u / a.Hkv];
         nt[u] = (T + kTT - 1) / kTT;
-        if (nt[u] >= (1 << 20)) return cudaSuccess;
+        if (nt[u] >= (1 << 20)) return cudaErrorInvalidValue;  // cannot happen: T * 128 < 2^31
         const int64_t k = (int64_t)T * 128 * a.keep_num / a.keep_den;
         // cost per tile: bytes in units of 512 B (the K and V boxes, plus the lists' share for residual units),
         // residual tiles scaled by the measured ratio of their compute time to a plain tile's
         wt[u] = 2 * kTT * 256 / 512;
-        if (a.host_modes[u] == FDKV_MODE_RESIDUAL) wt[u] = (int)((wt[u] + (2 * k * 6 / nt[u] + 511) / 512) * res_cost);
+        if (a.host_modes[u] == FDKV_MODE_RESIDUAL) wt[u] = (int)((wt[u] + (2 * k * 4 / nt[u] + 511) / 512) * res_cost);
         wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
         total_tiles += nt[u];
     }
-    const int ncta = (int)std::min<int64_t>(std::min(sm_count, kMaxCtas), total_tiles);
+    const int ncta = (int)std::min<int64_t>(std::min(std::min(sm_count, kMaxCtas), kMaxSplits), total_tiles);
     static unsigned g_launch_no = 0;
     ++g_launch_no;
     sch.tslot = (int)(g_launch_no % 64);
@@ -704,7 +713,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         }
     }
     for (int u = 0; u < units; ++u)
-        if (cs.n[u] > kMaxSplits) return cudaSuccess;
+        if (cs.n[u] > kMaxSplits) return cudaErrorInvalidValue;  // cannot happen: ncta <= kMaxSplits
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ncta);
     cfg.blockDim = dim3(kThreads);

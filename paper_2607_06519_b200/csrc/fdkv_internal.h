@@ -18,6 +18,7 @@ constexpr int kMaxSplits = 160;      // split-K partial slots per (sequence, que
 constexpr int kMaxW = 128;           // probe queries
 constexpr int kListPad = 32;         // slack entries after each residual list (aligned over-reads stay in bounds)
 constexpr int kMaxGroup = 8;
+constexpr int kFastMaxUnits = 1024;   // (sequences x KV heads) one launch of the bf16 / head_dim 128 decode kernel plans for
 constexpr int kProbeTile = 64;       // tokens per probe CTA (generic kernel)
 constexpr int kRowPad = 128;         // packed row blocks and tails are padded (zero rows) to this many tokens
 
@@ -27,7 +28,10 @@ enum DeviceFlag : int32_t { kFlagOk = 0, kFlagTimeout = 1, kFlagCountMismatch = 
 struct UnitDesc {
     const void* k_rows;  // [T][d]: Z0 of K (shared / residual) or the layer's original K rows (exact)
     const void* v_rows;
-    const int32_t* k_idx;  // residual mode only: ascending flat indices t*d + ch
+    // residual mode only.  Portable layout: ascending flat indices t*d + ch and the stored values.  Packed layout
+    // (bf16, head_dim 128): k_idx holds one 32-bit word per entry, value bits in the low half and the entry's
+    // position inside its 16-token slice (a ready-made shared-memory offset / 2) in the high half; k_val is null.
+    const int32_t* k_idx;
     const void* k_val;
     const int32_t* k_off;  // [ceil(T/16) + 1] first entry of each 16-token tile
     const int32_t* v_idx;
@@ -60,7 +64,7 @@ struct Shape {
 };
 
 struct WsLayout {
-    size_t status, z0, z1, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, probe_part, probe_pos, scores, modes,
+    size_t status, z0, z1, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
         partials, counters, io_q, io_k, io_v, io_out, total;
 };
 struct ArenaLayout {
@@ -97,6 +101,7 @@ struct fdkv_ctx {
     std::vector<fdkv::UnitDesc> desc_host;  // [max_batch][L][Hkv]
     alignas(64) unsigned char tmap[128];    // CUtensorMap of the arena (bf16, head_dim 128 only)
     bool has_tmap = false;
+    bool packed_lists = false;              // decode runs the bf16 / head_dim 128 kernel on packed residual entries
 };
 
 namespace fdkv {
@@ -126,6 +131,7 @@ struct SelectArgs {
     int32_t* tile_off;
     int32_t* idx;
     void* val;
+    uint32_t* packed;  // optional packed entries for the bf16 / head_dim 128 decode kernel (null otherwise)
     int32_t* status;
 };
 cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream_t st);
@@ -164,6 +170,7 @@ struct DecodeArgs {
     const void* tmap;           // CUtensorMap over the arena as rows of 256 bytes, or null
     const void* arena_base;
     int keep_num, keep_den;
+    int packed_lists;
     int32_t* tail_len;      // [L][max_batch]
     float* partials;        // [batch][Hq][kMaxSplits][d+4]: max, sum, 2 pad, d accumulators
     int32_t* counters;      // [max_batch][Hkv] split-K arrival tickets, zero between launches
