@@ -208,7 +208,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
         a.k0 = k_layers[2 * p]; a.k1 = k_layers[2 * p + 1];
         a.v0 = v_layers[2 * p]; a.v1 = v_layers[2 * p + 1];
         a.stride_t = stride_t; a.stride_h = stride_h;
-        a.T = T; a.d = s.d; a.Hkv = s.Hkv;
+        a.T = T; a.d = s.d; a.Hkv = s.Hkv; a.tensors = 2;
         a.ut_base = p * s.Hkv * 2;
         a.unit_stride = (int64_t)s.Tmax * s.d;
         a.z0 = c->work + c->ws.z0; a.z1 = c->work + c->ws.z1;

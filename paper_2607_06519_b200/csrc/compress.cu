@@ -54,7 +54,7 @@ template <>
 __device__ __forceinline__ float stored<__nv_bfloat16>(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
 // ----- C1: depth split + histogram of the top 15 magnitude bits of z1 ---------------------------------
-// grid (chunks, Hkv*2); each CTA owns a token range of one unit-tensor and a private 128 KiB histogram.
+// grid (chunks, Hkv*tensors); each CTA owns a token range of one unit-tensor and a private 128 KiB histogram.
 template <typename T>
 __global__ void __launch_bounds__(1024) split_hist_kernel(CompressArgs a, int tokens_per_cta) {
     extern __shared__ uint32_t s_hist[];
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(1024) split_hist_kernel(CompressArgs a, int to
     for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) s_hist[b] = 0;
     __syncthreads();
 
-    const int h = blockIdx.y >> 1, is_v = blockIdx.y & 1;
+    const int h = blockIdx.y / a.tensors, is_v = blockIdx.y % a.tensors;
     const int ut = a.ut_base + blockIdx.y;
     const T* x0 = reinterpret_cast<const T*>(is_v ? a.v0 : a.k0) + (int64_t)h * a.stride_h;
     const T* x1 = reinterpret_cast<const T*>(is_v ? a.v1 : a.k1) + (int64_t)h * a.stride_h;
@@ -373,7 +373,7 @@ cudaError_t launch_split_hist(const CompressArgs& a, int dtype, cudaStream_t st)
     }
     if (a.T <= 0) return cudaSuccess;
     const int tokens_per_cta = 4096 * 128 / a.d / (dtype == FDKV_BF16 ? 1 : 2);
-    dim3 grid((a.T + tokens_per_cta - 1) / tokens_per_cta, a.Hkv * 2);
+    dim3 grid((a.T + tokens_per_cta - 1) / tokens_per_cta, a.Hkv * a.tensors);
     if (dtype == FDKV_BF16)
         split_hist_kernel<__nv_bfloat16><<<grid, 1024, smem, st>>>(a, tokens_per_cta);
     else

@@ -43,7 +43,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct FastSched {
     uint32_t start[kMaxCtas + 1];  // unit << 20 | first 64-token tile of CTA c; start[ncta] = units << 20
-    int ncta, units, tslot;
+    int ncta, units, tslot, prologue_tiles;
 };
 struct PartCount {
     uint8_t n[kMaxUnits];  // split-K parts per unit (at most kMaxSplits)
@@ -237,7 +237,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     };
     if (is_producer) {
         prod_open_unit();
-        for (int i = 0; i < kStages - 1; ++i) prod_issue();
+        for (int i = 0; i < sch.prologue_tiles; ++i) prod_issue();  // nobody computes yet: stages can all be filled
     }
     // per-warp scratch starts zeroed
     for (int i = threadIdx.x; i < kCW * kScratchBytes / 16; i += kThreads)
@@ -661,12 +661,16 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     }
     static double res_cost = -1.0;
     static bool use_pdl = true;
+    // tiles copied before the dependency wait; more than one takes HBM bandwidth from the kernel still running
+    static int prologue_tiles = 1;
     if (res_cost < 0) {
         const char* ev = getenv("FDKV_RES_COST");  // tuning knobs for benchmark sweeps
         res_cost = ev ? atof(ev) : 1.6;
         if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 1.6;
         const char* pv = getenv("FDKV_NO_PDL");
         use_pdl = !(pv && pv[0] == '1');
+        const char* pt = getenv("FDKV_PROLOGUE_TILES");
+        prologue_tiles = pt ? std::max(0, std::min(kStages, atoi(pt))) : 1;
     }
     // ---- flat cost-weighted schedule: CTA c starts at weight c * W / ncta ----
     FastSched sch;
@@ -691,6 +695,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     ++g_launch_no;
     sch.tslot = (int)(g_launch_no % 64);
     sch.ncta = ncta;
+    sch.prologue_tiles = prologue_tiles;
     sch.units = units;
     {
         int u = 0;

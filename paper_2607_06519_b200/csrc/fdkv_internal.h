@@ -111,6 +111,7 @@ struct CompressArgs {
     const void *k0, *k1, *v0, *v1;  // the four [T][Hkv][d] strided tensors of one pair
     int64_t stride_t, stride_h;
     int T, d, Hkv;
+    int tensors;  // 2: K and V of every head (unit-tensor = head*2 + is_v); 1: K only (unit-tensor = head)
     int ut_base;  // first unit-tensor of this pair in the stage: (pair*Hkv)*2
     int64_t unit_stride;  // elements between staged unit-tensors (Tmax*d)
     void *z0, *z1;
