@@ -43,7 +43,8 @@ typedef enum {
     FDKV_ERR_STATE = 5,       /* call order (probe before compress, decode before commit, tail full)   */
     FDKV_ERR_CUDA = 6,        /* a CUDA runtime call failed; see fdkv_last_cuda_error()                */
     FDKV_ERR_TIMEOUT = 7,     /* a bounded device-side wait gave up (reported by fdkv_device_status)   */
-    FDKV_ERR_DEVICE = 8       /* a device-side consistency check failed (fdkv_device_status)           */
+    FDKV_ERR_DEVICE = 8,      /* a device-side consistency check failed (fdkv_device_status)           */
+    FDKV_ERR_TOO_LARGE = 9    /* fdkv_compress_unit_noalloc: T * head_dim exceeds FDKV_NOALLOC_MAX_ELEMS */
 } fdkv_status;
 
 typedef enum { FDKV_F32 = 0, FDKV_BF16 = 1 } fdkv_dtype;
@@ -156,6 +157,38 @@ fdkv_status fdkv_footprint(fdkv_ctx* ctx, int32_t seq, size_t* bytes_by_mode_hos
 /* Bytes the decode kernels read from the packed cache for one call of `layer` over `batch` sequences
  * (coefficient or exact rows, residual lists and their tile offsets, tails): the roofline numerator.      */
 fdkv_status fdkv_decode_bytes(fdkv_ctx* ctx, int32_t layer, int32_t batch, size_t* bytes_host /*HOST*/);
+
+/*
+ * Compression of ONE [T][head_dim] tensor pair without any allocation.  (The paper has no counterpart: this is
+ * a packaging of the Eq. 1 / Eq. 3 compression step for callers that cannot allocate.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving engine whose memory pool owns
+ * every byte of the device, in a plugin that is only handed tensors, or in a latency-critical path where an
+ * allocation (an implicit device synchronisation) is not acceptable -- and that has no fdkv context, whose
+ * workspace would otherwise provide the scratch.  The scratch this needs (the Z1 temporary, the magnitude
+ * histogram, per-tile counts and offsets; about 4.3 MB) is a static array inside the library's device image:
+ * every GPU that loads libfdkv holds it until the process exits, whether or not this function is ever called.
+ *
+ * Computes exactly what fdkv_compress_prefill computes for one unit-tensor: z0_out[T][head_dim] (storage
+ * dtype, dense), and the k = floor(T*head_dim*keep_num/keep_den) kept entries of Z1 as ascending flat indices
+ * idx_out[k] with their stored values val_out[k] (may be NULL when k == 0).  x0 / x1: rows of layer 2p / 2p+1,
+ * row t at x + t*stride_t (elements).  *count_host (HOST, may be NULL) receives k.  All pointers 16-byte aligned.
+ *
+ * Limits and rules
+ *  - T * head_dim <= FDKV_NOALLOC_MAX_ELEMS, else FDKV_ERR_TOO_LARGE and nothing is enqueued.
+ *  - Calls cudaMalloc / cudaFree or any allocating routine never; it enqueues a memset and kernels on `stream`.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *    current).  Make that first call outside any stream capture.
+ *  - Every call on a device uses the same array, which still holds the previous call's data; the function
+ *    clears what has to start at zero itself.  Two calls whose work overlaps on the GPU (different streams
+ *    without an ordering between them) race on it: serialise them.
+ *  - A device-side count mismatch is not reported here (there is no context to hold a status word the caller
+ *    could read); compare *count_host with what you expect to find in idx_out if in doubt.
+ */
+#define FDKV_NOALLOC_MAX_ELEMS (1 << 20)
+fdkv_status fdkv_compress_unit_noalloc(const void* x0, const void* x1, int64_t stride_t, int32_t T, int32_t head_dim,
+                                       int32_t dtype, int32_t keep_num, int32_t keep_den, void* z0_out,
+                                       int32_t* idx_out, void* val_out, int32_t* count_host /*HOST*/, void* stream);
 
 /* Reads the device status word (synchronises the device): FDKV_OK, FDKV_ERR_TIMEOUT or FDKV_ERR_DEVICE.  */
 fdkv_status fdkv_device_status(fdkv_ctx* ctx);

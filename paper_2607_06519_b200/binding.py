@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libfdkv.so")
 F32, BF16 = 0, 1
 SHARED, RESIDUAL, EXACT = 0, 1, 2
 _STATUS = ["ok", "invalid argument", "unsupported", "arena full", "workspace too small", "state", "cuda error",
-           "device timeout", "device check failed"]
+           "device timeout", "device check failed", "too large for the built-in scratch"]
+NOALLOC_MAX_ELEMS = 1 << 20
 
 
 class FdkvError(RuntimeError):
@@ -56,6 +57,7 @@ def _load():
         "fdkv_footprint": [vp, i32, P(sz), P(sz)],
         "fdkv_decode_bytes": [vp, i32, i32, P(sz)],
         "fdkv_device_status": [vp],
+        "fdkv_compress_unit_noalloc": [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, P(i32), vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -118,6 +120,22 @@ def _stream(stream) -> int:
 
 def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def compress_unit_noalloc(x0, x1, keep_num: int, keep_den: int, z0_out, idx_out, val_out, stream=None) -> int:
+    """Allocation-free compression of one [T, d] pair into caller-owned outputs (no context, no workspace).
+
+    For callers that may not allocate device memory: the scratch is a static array inside the library.  The
+    outputs must already exist (z0_out [T, d], idx_out int32 [k], val_out [k]); returns k.  Calls on one device
+    share the scratch, so do not overlap them on different streams.
+    """
+    T, d = x0.shape
+    dtype = BF16 if x0.dtype == torch.bfloat16 else F32
+    cnt = C.c_int32(0)
+    _check(_lib.fdkv_compress_unit_noalloc(_ptr(x0), _ptr(x1), x0.stride(0), T, d, dtype, keep_num, keep_den, _ptr(z0_out),
+                                           _ptr(idx_out), _ptr(val_out), C.byref(cnt), _stream(stream)),
+           "fdkv_compress_unit_noalloc")
+    return int(cnt.value)
 
 
 class Context:

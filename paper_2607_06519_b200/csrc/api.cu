@@ -102,6 +102,7 @@ bool seq_ok(fdkv_ctx* c, int seq) { return c && seq >= 0 && seq < c->s.max_batch
 
 namespace fdkv {
 void count_launch(int n) { g_launches.fetch_add(n); }
+fdkv_status record_cuda_error(cudaError_t e) { return cuda_fail(e); }
 cudaError_t launch_set_tail_len(int32_t* tail_len, int L, int max_batch, int seq, int n, cudaStream_t st);
 }  // namespace fdkv
 
@@ -548,6 +549,7 @@ const char* fdkv_status_str(fdkv_status s) {
         case FDKV_ERR_CUDA: return "CUDA runtime error";
         case FDKV_ERR_TIMEOUT: return "device wait timed out";
         case FDKV_ERR_DEVICE: return "device-side check failed";
+        case FDKV_ERR_TOO_LARGE: return "input larger than the built-in scratch of the allocation-free entry point";
     }
     return "unknown";
 }

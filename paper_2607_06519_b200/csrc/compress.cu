@@ -1,6 +1,7 @@
 // Prefill compression kernels: depth split (Eq. 1, B = 2) fused with the magnitude histogram, the
 // radix-select threshold, and the index-ordered compaction of the sparse residual (Eq. 3, entry form).
 #include <algorithm>
+#include <mutex>
 
 #include "fdkv_internal.h"
 
@@ -435,3 +436,100 @@ cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, in
 }
 
 }  // namespace fdkv
+
+// ---------------------------------------------------------------------------------------------------------------
+// Allocation-free compression of one [T][d] tensor pair (declared in fdkv.h as fdkv_compress_unit_noalloc).
+// Same kernels as fdkv_compress_prefill; the scratch they need (the Z1 temporary, the magnitude histogram, the
+// select state and the per-tile counts / offsets) lives in the file-scope device array below instead of a
+// caller-provided workspace.  Every GPU that loads this library holds the array until the process exits.
+// ---------------------------------------------------------------------------------------------------------------
+namespace fdkv {
+namespace {
+
+constexpr int64_t kNoAllocMaxElems = FDKV_NOALLOC_MAX_ELEMS;                    // T * head_dim
+constexpr int64_t kNoAllocMaxTiles = kNoAllocMaxElems / 64 / fdkv::kResTile;    // head_dim >= 64
+constexpr size_t kNaZ1 = 0;                                                     // Z1 temporary, float32 worst case
+constexpr size_t kNaHist = kNaZ1 + (size_t)kNoAllocMaxElems * 4;
+constexpr size_t kNaSel = kNaHist + (size_t)fdkv::kHistBins * 4;
+constexpr size_t kNaStatus = kNaSel + 256;
+constexpr size_t kNaCnt = kNaStatus + 256;
+constexpr size_t kNaEq = kNaCnt + (size_t)kNoAllocMaxTiles * 8;
+constexpr size_t kNaOff = kNaEq + (size_t)kNoAllocMaxTiles * 4;
+constexpr size_t kNaBytes = (kNaOff + (size_t)(kNoAllocMaxTiles + 1) * 4 + 255) / 256 * 256;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
+
+// In host code the array's name is only a handle: the device address comes from cudaGetSymbolAddress, once per
+// device, with that device current.
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices] = {};
+std::mutex g_noalloc_mutex;
+
+cudaError_t noalloc_scratch(char** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = static_cast<char*>(g_noalloc_ptr[dev]);
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace fdkv
+
+extern "C" fdkv_status fdkv_compress_unit_noalloc(const void* x0, const void* x1, int64_t stride_t, int32_t T,
+                                                  int32_t head_dim, int32_t dtype, int32_t keep_num, int32_t keep_den,
+                                                  void* z0_out, int32_t* idx_out, void* val_out, int32_t* count_host,
+                                                  void* stream) {
+    using namespace fdkv;
+    if (!x0 || !x1 || !z0_out || T < 1) return FDKV_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return FDKV_ERR_UNSUPPORTED;
+    if (dtype != FDKV_F32 && dtype != FDKV_BF16) return FDKV_ERR_UNSUPPORTED;
+    if (keep_den <= 0 || keep_num < 0 || keep_num > keep_den) return FDKV_ERR_INVALID_ARG;
+    if (stride_t < head_dim || (stride_t % 8)) return FDKV_ERR_INVALID_ARG;
+    if ((int64_t)T * head_dim > kNoAllocMaxElems) return FDKV_ERR_TOO_LARGE;  // the static scratch cannot hold it
+    const int64_t k = (int64_t)T * head_dim * keep_num / keep_den;
+    if (k > 0 && (!idx_out || !val_out)) return FDKV_ERR_INVALID_ARG;
+    for (const void* p : {x0, x1, (const void*)z0_out, (const void*)idx_out, (const void*)val_out})
+        if (reinterpret_cast<uintptr_t>(p) % 16) return FDKV_ERR_INVALID_ARG;
+    if (count_host) *count_host = (int32_t)k;
+
+    char* sc = nullptr;
+    cudaError_t e = noalloc_scratch(&sc);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // the array keeps the previous call's contents: the histogram and the status word must start at zero
+    e = cudaMemsetAsync(sc + kNaHist, 0, (size_t)kHistBins * 4 + 512, st);
+    if (e != cudaSuccess) return record_cuda_error(e);
+
+    CompressArgs a;
+    a.k0 = x0; a.k1 = x1; a.v0 = x0; a.v1 = x1;
+    a.stride_t = stride_t; a.stride_h = 0;
+    a.T = T; a.d = head_dim; a.Hkv = 1; a.tensors = 1;
+    a.ut_base = 0; a.unit_stride = 0;
+    a.z0 = z0_out; a.z1 = sc + kNaZ1;
+    a.hist = reinterpret_cast<uint32_t*>(sc + kNaHist);
+    if ((e = launch_split_hist(a, dtype, st)) != cudaSuccess) return record_cuda_error(e);
+
+    SelectArgs sa;
+    sa.ut_begin = 0; sa.ut_count = 1;
+    sa.T = T; sa.d = head_dim; sa.k = k;
+    sa.unit_stride = 0; sa.kcap = 0; sa.ntiles_max = (int)kNoAllocMaxTiles;
+    sa.z1 = sc + kNaZ1;
+    sa.hist = reinterpret_cast<uint32_t*>(sc + kNaHist);
+    sa.sel = reinterpret_cast<SelState*>(sc + kNaSel);
+    sa.tile_cnt = reinterpret_cast<uint32_t*>(sc + kNaCnt);
+    sa.tile_eq = reinterpret_cast<uint32_t*>(sc + kNaEq);
+    sa.tile_off = reinterpret_cast<int32_t*>(sc + kNaOff);
+    sa.idx = idx_out; sa.val = val_out; sa.packed = nullptr;
+    sa.status = reinterpret_cast<int32_t*>(sc + kNaStatus);
+    if ((e = launch_select_and_compact(sa, dtype, st)) != cudaSuccess) return record_cuda_error(e);
+    return FDKV_OK;
+}

@@ -183,5 +183,7 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out);
 cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st);
 
 void count_launch(int n);
+// Remembers a failed CUDA runtime call for fdkv_last_cuda_error() and returns FDKV_ERR_CUDA.
+fdkv_status record_cuda_error(cudaError_t e);
 
 }  // namespace fdkv
