@@ -31,7 +31,12 @@ if ROOT not in sys.path:
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (None until a capture exists for that workload).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/decode_fast_kernel_decode32k.md: 138.55 MB read + ~6.1 MB written per launch, captured on the 4-layer cut
+    # (same 8 units and bytes per launch as the 32-layer workload)
+    "decode32k": 144.6e6,
+    "decode32k_4l": 144.6e6,
+}
 
 
 def measured_peaks():
