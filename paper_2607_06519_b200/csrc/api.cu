@@ -56,6 +56,7 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.status = take(256);
     w.z0 = take((size_t)s.NT * unit_elems * s.esize);
     w.z1 = take((size_t)s.NT * unit_elems * s.esize);
+    w.z1drop = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NU * unit_elems * s.esize : 0);
     w.hist = take((size_t)s.NT * kHistBins * 4);
     w.sel = take((size_t)s.NT * sizeof(SelState));
     w.tile_cnt = take((size_t)s.NT * s.ntiles_max * 8);
@@ -153,6 +154,9 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     if (e != cudaSuccess) { delete c; return cuda_fail(e); }
     if (s.dtype == FDKV_BF16 && s.d == 128) c->has_tmap = make_arena_tensor_map(c->arena, arena_bytes, c->tmap);
     c->packed_lists = c->has_tmap && s.max_batch * s.Hkv <= kFastMaxUnits;
+    if (s.dtype == FDKV_BF16 && s.d == 128)
+        c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, 128, c->tmap_z1) &&
+                             make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.Tmax * s.d * s.esize, 128, c->tmap_drop);
     *out = c;
     return FDKV_OK;
 }
@@ -232,6 +236,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     sa.idx = wsp<int32_t>(c, c->ws.idx);
     sa.val = c->work + c->ws.val;
     sa.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
+    sa.z1drop = c->has_probe_tmaps ? c->work + c->ws.z1drop : nullptr;
     sa.status = wsp<int32_t>(c, c->ws.status);
     CU(launch_select_and_compact(sa, s.dtype, st));
     for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; }
@@ -277,6 +282,11 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     const double b_sh = 2.0 * Td * e, b_rs = b_sh + 2.0 * k * (e + 4.0), b_ex = 4.0 * Td * e;
     a.omega[0] = b_sh / b_ex; a.omega[1] = b_rs / b_ex; a.omega[2] = 1.0;
     a.modes_out = modes; a.scores_out = scores;
+    a.tmap_z1 = c->has_probe_tmaps ? c->tmap_z1 : nullptr;
+    a.tmap_drop = c->has_probe_tmaps ? c->tmap_drop : nullptr;
+    a.Tmax = s.Tmax;
+    a.pos_host = probe_pos;
+    a.status = wsp<int32_t>(c, c->ws.status);
     CU(launch_probe(a, s.dtype, st));
     for (int p = pb; p < pe; ++p) c->pair_probed[p] = 1;
     return FDKV_OK;

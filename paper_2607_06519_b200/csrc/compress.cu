@@ -289,6 +289,7 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
     int32_t* idx = a.idx + (int64_t)ut * a.kcap;
     T* val = reinterpret_cast<T*>(a.val) + (int64_t)ut * a.kcap;
     uint32_t* pk = a.packed ? a.packed + (int64_t)ut * a.kcap : nullptr;
+    T* drop = (a.z1drop && !(ut & 1)) ? reinterpret_cast<T*>(a.z1drop) + (int64_t)(ut >> 1) * a.unit_stride : nullptr;
     uint32_t pos = (uint32_t)a.tile_off[(int64_t)ut * (a.ntiles_max + 1) + tile];
     uint32_t eq_rank = a.tile_eq[(int64_t)ut * a.ntiles_max + tile];
     const int64_t e_begin = (int64_t)tile * kResTile * a.d;
@@ -342,6 +343,14 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
                 if (pk) pk[w] = packed_entry<T>(z[e + i], (int)(e + i));
                 ++w;
             }
+        // K tensors only: the coefficients the residual candidate drops (Z1 with the kept entries zeroed), the
+        // second B operand of the tensor-core probe
+        if (drop && e < e_end) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i)
+                if (keep >> i & 1u) f[i] = 0.f;
+            *reinterpret_cast<typename S::vec_t*>(drop + e) = S::pack(f);
+        }
         pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
 }
@@ -528,7 +537,7 @@ extern "C" fdkv_status fdkv_compress_unit_noalloc(const void* x0, const void* x1
     sa.tile_cnt = reinterpret_cast<uint32_t*>(sc + kNaCnt);
     sa.tile_eq = reinterpret_cast<uint32_t*>(sc + kNaEq);
     sa.tile_off = reinterpret_cast<int32_t*>(sc + kNaOff);
-    sa.idx = idx_out; sa.val = val_out; sa.packed = nullptr;
+    sa.idx = idx_out; sa.val = val_out; sa.packed = nullptr; sa.z1drop = nullptr;
     sa.status = reinterpret_cast<int32_t*>(sc + kNaStatus);
     if ((e = launch_select_and_compact(sa, dtype, st)) != cudaSuccess) return record_cuda_error(e);
     return FDKV_OK;

@@ -622,7 +622,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
 
 }  // namespace
 
-bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
+bool make_rows_tensor_map(void* base, size_t bytes, int box_rows, void* tmap_out) {
     typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -633,16 +633,20 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
         cudaGetLastError();
         return false;
     }
-    const cuuint64_t rows = arena_bytes / 256;
-    if (rows == 0 || rows > 0x7FFFFFFFull) return false;
+    const cuuint64_t rows = bytes / 256;
+    if (rows == 0 || rows > 0x7FFFFFFFull || box_rows < 1 || box_rows > 256) return false;
     const cuuint64_t gdim[2] = {128, rows};
     const cuuint64_t gstride[1] = {256};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kTT};  // 64 channels x one stage of tokens
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};  // 64 channels x box_rows tokens
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = reinterpret_cast<encode_fn>(fn)(reinterpret_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, arena,
+    CUresult r = reinterpret_cast<encode_fn>(fn)(reinterpret_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base,
                                                  gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+
+bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
+    return make_rows_tensor_map(arena, arena_bytes, kTT, tmap_out);
 }
 
 cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handled) {

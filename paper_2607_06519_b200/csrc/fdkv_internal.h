@@ -64,7 +64,7 @@ struct Shape {
 };
 
 struct WsLayout {
-    size_t status, z0, z1, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
+    size_t status, z0, z1, z1drop, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
         partials, counters, io_q, io_k, io_v, io_out, total;
 };
 struct ArenaLayout {
@@ -101,6 +101,8 @@ struct fdkv_ctx {
     std::vector<fdkv::UnitDesc> desc_host;  // [max_batch][L][Hkv]
     alignas(64) unsigned char tmap[128];    // CUtensorMap of the arena (bf16, head_dim 128 only)
     bool has_tmap = false;
+    alignas(64) unsigned char tmap_z1[128], tmap_drop[128];  // probe operands (bf16, head_dim 128 only)
+    bool has_probe_tmaps = false;
     bool packed_lists = false;              // decode runs the bf16 / head_dim 128 kernel on packed residual entries
 };
 
@@ -132,6 +134,7 @@ struct SelectArgs {
     int32_t* tile_off;
     int32_t* idx;
     void* val;
+    void* z1drop;      // optional [unit][Tmax*d]: Z1 of K with the kept entries zeroed (tensor-core probe), or null
     uint32_t* packed;  // optional packed entries for the bf16 / head_dim 128 decode kernel (null otherwise)
     int32_t* status;
 };
@@ -153,6 +156,12 @@ struct ProbeArgs {
     double lambda, omega[3];
     int32_t* modes_out;  // user buffers for the pair range, may be null
     float* scores_out;
+    // tensor-core path (bf16, head_dim 128): tensor maps over the staged Z1 and the dropped copy, viewed as
+    // [rows][128] bf16 with 128-token x 64-channel boxes; null when unavailable
+    const void *tmap_z1, *tmap_drop;
+    int Tmax;
+    const int32_t* pos_host;
+    int32_t* status;
 };
 cudaError_t launch_probe(const ProbeArgs& a, int dtype, cudaStream_t st);
 
@@ -180,6 +189,8 @@ struct DecodeArgs {
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st);
 // Encodes a 2-D tensor map over the arena viewed as [rows][128] bf16 (256-byte rows), 64x64 boxes, 128-byte swizzle.
 bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out);
+// Same view ([rows][128] bf16, 64-channel x box_rows boxes, 128-byte swizzle) over any 256-byte aligned region.
+bool make_rows_tensor_map(void* base, size_t bytes, int box_rows, void* tmap_out);
 cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st);
 
 void count_launch(int n);

@@ -1,9 +1,319 @@
-// Tensor-core (tcgen05) probe kernel for bf16, head_dim 128.  Not built yet: the portable kernel handles every shape.
+// Routing probe on the 5th-generation tensor cores (bf16 storage, head_dim 128): the error term of Eq. 2.
+//
+// For a unit and a candidate (shared: R = Z1 of K; residual: R = Z1 of K with the kept entries zeroed) the probe
+// needs sum_{rows, keys j <= pos(row)} (Q_row . R_j)^2 over the 2*G*W probe rows (2 layers x G group heads x W
+// probe queries).  That is a dense [rows x 128] x [128 x T] contraction whose result is squared, masked causally
+// and summed without ever leaving the SM:
+//   * work item = (unit, layer of the pair, block of 256 probe rows, candidate, range of 128-token key tiles);
+//     one CTA per item, 6 warps: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner), warps 2-5 = epilogue;
+//   * A (the item's 256 Q rows, 64 KiB) is gathered once into shared memory in the 128-byte-swizzled K-major
+//     layout; B tiles (128 tokens x 128 channels) stream through a 4-stage TMA ring;
+//   * per key tile 16 tcgen05.mma (M = 128, N = 128, K = 16, kind::f16, bf16 x bf16 -> f32) fill two 128x128 f32
+//     accumulators in TMEM (256 columns); two such accumulator sets alternate so the epilogue of tile i overlaps
+//     the MMAs of tile i+1;
+//   * epilogue: tcgen05.ld (32 lanes x 32 columns per instruction), square, mask keys after the row's probe
+//     position, accumulate; one float64 sum per item, summed across items in a fixed order by the finalize kernel.
+// Every mbarrier wait is bounded; on expiry the CTA flags the device status word, stops waiting and still frees
+// its tensor memory before it retires.
+#include <cuda.h>
+
+#include <algorithm>
+#include <cstdlib>
+
 #include "fdkv_internal.h"
 
 namespace fdkv {
-cudaError_t launch_probe_tc(const ProbeArgs&, int, cudaStream_t, bool* handled, int*) {
+
+namespace {
+
+constexpr int kBN = 128;                       // key tokens per tile
+constexpr int kBStages = 4;
+constexpr int kBHalf = kBN * 128;              // one 64-channel half of a B tile: 16 KiB
+constexpr int kBStageBytes = 2 * kBHalf;       // 32 KiB
+constexpr int kAHalf = 128 * 128;              // one 64-channel half of a 128-row A tile: 16 KiB
+constexpr int kATile = 2 * kAHalf;             // 32 KiB per 128 rows
+constexpr int kABytes = 2 * kATile;            // 256 rows
+constexpr int kHdr = 1024;
+constexpr int kProbeSmem = kHdr + kABytes + kBStages * kBStageBytes;  // 193 KiB
+constexpr int kPThreads = 6 * 32;
+constexpr uint32_t kSpin = 1u << 22;
+constexpr int kTmemCols = 512;
+// header: full[4] @0, empty[4] @32, tfull[2] @64, tempty[2] @80, tmem slot @96, abort @100, reduce @128 (4 doubles)
+constexpr int oFull = 0, oEmpty = 32, oTFull = 64, oTEmpty = 80, oSlot = 96, oAbort = 100, oRed = 128;
+
+__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mb_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mb_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mb_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mb_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ void mb_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* status) {
+    if (*abort_flag) return;
+    for (uint32_t i = 0; i < kSpin; ++i) {
+        if (mb_try(bar, parity)) return;
+        if ((i & 255u) == 255u && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicMax(status, (int32_t)kFlagTimeout);
+}
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address
+    d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+    d |= (uint64_t)1 << 46;                            // descriptor version
+    d |= (uint64_t)2 << 61;                            // 128-byte swizzle
+    return d;
+}
+// instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 128
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(da), "l"(db), "r"(kIdesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+
+struct TcPlan {
+    int items_per_unit;  // 2 layers x mblocks x 2 candidates x nsplits
+    int mblocks, nsplits, ntiles, tiles_per_split;
+    int pos_min, pos_max;
+};
+
+__global__ void __launch_bounds__(kPThreads, 1)
+probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_constant__ CUtensorMap tmap_drop, ProbeArgs a, TcPlan pl) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sm0 = s_u32(smem);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + oAbort);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (sm0 & 1023u) {
+        if (threadIdx.x == 0) atomicMax(a.status, (int32_t)kFlagCountMismatch);
+        return;
+    }
+    // ---- decode the work item ----
+    int it = blockIdx.x;
+    const int unit = a.unit_begin + it / pl.items_per_unit;
+    it %= pl.items_per_unit;
+    const int split = it % pl.nsplits; it /= pl.nsplits;
+    const int cand = it & 1; it >>= 1;
+    const int mblock = it % pl.mblocks; it /= pl.mblocks;
+    const int layer = it;  // 0 or 1
+    const int h = unit % a.Hkv, pair = unit / a.Hkv;
+    const int tile0 = split * pl.tiles_per_split;
+    const int tile1 = min(pl.ntiles, tile0 + pl.tiles_per_split);
+    const int ntile = max(0, tile1 - tile0);
+    const int rows_layer = a.G * a.W;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kBStages; ++s) { mb_init(sm0 + oFull + 8 * s, 1); mb_init(sm0 + oEmpty + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { mb_init(sm0 + oTFull + 8 * s, 1); mb_init(sm0 + oTEmpty + 8 * s, 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // ---- A: rows r = mblock*256 + i of this layer's probe block, row = g*W + qi -> Q[layer][qi][h*G+g][:] ----
+    {
+        const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[2 * pair + layer]);
+        for (int v = threadIdx.x; v < 256 * 16; v += kPThreads) {
+            const int i = v >> 4, chunk = v & 15;  // row in block, 16-byte chunk of 8 channels
+            const int r = mblock * 256 + i;
+            uint4 val = make_uint4(0u, 0u, 0u, 0u);
+            if (r < rows_layer) {
+                const int g = r / a.W, qi = r % a.W;
+                val = *reinterpret_cast<const uint4*>(q + ((int64_t)qi * a.Hq + h * a.G + g) * 128 + chunk * 8);
+            }
+            const int mt = i >> 7, rr = i & 127;
+            uint8_t* dst = smem + kHdr + mt * kATile + (chunk >> 3) * kAHalf + rr * 128 + (((chunk & 7) ^ (rr & 7)) << 4);
+            *reinterpret_cast<uint4*>(dst) = val;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA's async reads
+    }
+    if (warp == 1) {  // tensor memory: all 512 columns (two sets of two 128x128 f32 accumulators)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sm0 + oSlot), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + oSlot);
+    const uint32_t b0 = sm0 + kHdr + kABytes;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            const CUtensorMap* map = cand ? &tmap_drop : &tmap_z1;
+            // rows of this unit's K coefficients: staged Z1 holds K and V per unit (unit-tensor 2*unit), the dropped copy K only
+            const int64_t row0 = (cand ? (int64_t)unit : (int64_t)unit * 2) * a.Tmax;
+            for (int i = 0; i < ntile; ++i) {
+                const int s = i % kBStages;
+                const uint32_t ph = (uint32_t)(i / kBStages) & 1u;
+                mb_wait(sm0 + oEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
+                if (*abort_flag) break;
+                const uint32_t full = sm0 + oFull + 8 * s, dst = b0 + s * kBStageBytes;
+                const int y = (int)(row0 + (int64_t)(tile0 + i) * kBN);
+                mb_expect_tx(full, kBStageBytes);
+                tma_2d(dst, map, 0, y, full);
+                tma_2d(dst + kBHalf, map, 64, y, full);
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            for (int i = 0; i < ntile; ++i) {
+                const int s = i % kBStages, as = i & 1;
+                mb_wait(sm0 + oTEmpty + 8 * as, (((uint32_t)i >> 1) & 1u) ^ 1u, abort_flag, a.status);
+                mb_wait(sm0 + oFull + 8 * s, (uint32_t)(i / kBStages) & 1u, abort_flag, a.status);
+                if (*abort_flag) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(as * 256 + mt * 128);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {  // 8 steps of 16 channels: 4 per 64-channel half, 32 bytes apart inside the swizzle atom
+                        const uint64_t da = smem_desc(sm0 + kHdr + mt * kATile + (k >> 2) * kAHalf + (k & 3) * 32);
+                        const uint64_t db = smem_desc(b0 + s * kBStageBytes + (k >> 2) * kBHalf + (k & 3) * 32);
+                        umma(d_tmem, da, db, k > 0 ? 1u : 0u);
+                    }
+                }
+                umma_commit(sm0 + oEmpty + 8 * s);    // the B stage is free once these MMAs have read it
+                umma_commit(sm0 + oTFull + 8 * as);   // the accumulators are complete
+            }
+        }
+    } else {
+        // ================= epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 =================
+        const int lq = warp & 3;
+        const int rl = lq * 32 + lane;  // row within a 128-row M tile == TMEM lane
+        int pos_row[2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const int r = mblock * 256 + mt * 128 + rl;
+            pos_row[mt] = r < rows_layer ? a.pos[r % a.W] : -1;  // padding rows never count
+        }
+        double total = 0.0;
+        for (int i = 0; i < ntile; ++i) {
+            const int as = i & 1;
+            const int t0 = (tile0 + i) * kBN;
+            mb_wait(sm0 + oTFull + 8 * as, ((uint32_t)i >> 1) & 1u, abort_flag, a.status);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float acc = 0.f;
+            if (!*abort_flag) {
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    const bool all_visible = t0 + kBN - 1 <= pl.pos_min;  // every key of the tile precedes every probe position
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(as * 256 + mt * 128 + cc * 32), r);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (all_visible && pos_row[mt] >= 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) { const float v = __uint_as_float(r[j]); acc = fmaf(v, v, acc); }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float v = __uint_as_float(r[j]);
+                                if (t0 + cc * 32 + j <= pos_row[mt]) acc = fmaf(v, v, acc);
+                            }
+                        }
+                    }
+                }
+            }
+            total += (double)acc;
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mb_arrive(sm0 + oTEmpty + 8 * as);
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+        if (lane == 0) reinterpret_cast<double*>(smem + oRed)[lq] = total;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (*abort_flag)
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let copies and MMAs in flight finish before the memory goes away
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    }
+    if (threadIdx.x == 0) {
+        const double* red = reinterpret_cast<const double*>(smem + oRed);
+        // part slot of this item inside its unit: (layer, mblock, split); candidate selects the column
+        const int slot = (layer * pl.mblocks + mblock) * pl.nsplits + split;
+        a.part[((int64_t)unit * a.nptiles_max + slot) * 2 + cand] = red[0] + red[1] + red[2] + red[3];
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_probe_tc(const ProbeArgs& a, int dtype, cudaStream_t st, bool* handled, int* nparts) {
     *handled = false;
+    if (dtype != FDKV_BF16 || a.d != 128 || !a.tmap_z1 || !a.tmap_drop) return cudaSuccess;
+    static int enabled = -1, sm_count = 148;
+    if (enabled < 0) {
+        const char* ev = getenv("FDKV_NO_TC_PROBE");
+        enabled = (ev && ev[0] == '1') ? 0 : 1;
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(probe_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kProbeSmem);
+        if (e != cudaSuccess) return e;
+    }
+    if (!enabled) return cudaSuccess;
+    TcPlan pl;
+    pl.pos_min = a.pos_host[0];
+    pl.pos_max = a.pos_host[a.W - 1];
+    pl.ntiles = pl.pos_max / kBN + 1;  // keys after the last probe position never count
+    pl.mblocks = (a.G * a.W + 255) / 256;
+    const int base_items = a.unit_count * 2 * pl.mblocks * 2;
+    // split the key range so that the grid fills the machine several times over, but keep >= 8 tiles per item
+    int nsplits = std::max(1, std::min((4 * sm_count + base_items - 1) / base_items, (pl.ntiles + 7) / 8));
+    pl.tiles_per_split = (pl.ntiles + nsplits - 1) / nsplits;
+    nsplits = (pl.ntiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
+    pl.nsplits = nsplits;
+    pl.items_per_unit = 2 * pl.mblocks * 2 * nsplits;
+    const int slots = 2 * pl.mblocks * nsplits;
+    if (slots > a.nptiles_max) return cudaSuccess;  // the part array is sized for the portable kernel's tiles
+    probe_tc_kernel<<<a.unit_count * pl.items_per_unit, kPThreads, kProbeSmem, st>>>(
+        *reinterpret_cast<const CUtensorMap*>(a.tmap_z1), *reinterpret_cast<const CUtensorMap*>(a.tmap_drop), a, pl);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    count_launch(1);
+    *nparts = slots;
+    *handled = true;
     return cudaSuccess;
 }
+
 }  // namespace fdkv
