@@ -234,18 +234,27 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
                 for (int mt = 0; mt < 2; ++mt) {
                     const bool all_visible = t0 + kBN - 1 <= pl.pos_min;  // every key of the tile precedes every probe position
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(as * 256 + mt * 128 + cc * 32), r);
+                    for (int cp = 0; cp < 2; ++cp) {  // two 32-column loads in flight per wait
+                        uint32_t r0[32], r1[32];
+                        const uint32_t ta = tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(as * 256 + mt * 128 + cp * 64);
+                        tmem_ld32(ta, r0);
+                        tmem_ld32(ta + 32, r1);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                         if (all_visible && pos_row[mt] >= 0) {
+                            float acc1 = 0.f;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) { const float v = __uint_as_float(r[j]); acc = fmaf(v, v, acc); }
+                            for (int j = 0; j < 32; ++j) {
+                                const float v = __uint_as_float(r0[j]), w = __uint_as_float(r1[j]);
+                                acc = fmaf(v, v, acc);
+                                acc1 = fmaf(w, w, acc1);
+                            }
+                            acc += acc1;
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                const float v = __uint_as_float(r[j]);
-                                if (t0 + cc * 32 + j <= pos_row[mt]) acc = fmaf(v, v, acc);
+                                const float v = __uint_as_float(r0[j]), w = __uint_as_float(r1[j]);
+                                if (t0 + cp * 64 + j <= pos_row[mt]) acc = fmaf(v, v, acc);
+                                if (t0 + cp * 64 + 32 + j <= pos_row[mt]) acc = fmaf(w, w, acc);
                             }
                         }
                     }
