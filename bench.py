@@ -179,6 +179,9 @@ def run_ours(args, w):
         for p in range(w.n_pairs):
             t = pf.upload_pair(b, p)
             k_layers[2 * p], k_layers[2 * p + 1], v_layers[2 * p], v_layers[2 * p + 1] = t["k0"], t["k1"], t["v0"], t["v1"]
+        if b == 0:  # untimed pass: first launches pay the lazy loading of every kernel
+            ctx.compress_prefill(b, 0, w.n_pairs, w.T, k_layers, v_layers)
+            ctx.probe(b, 0, w.n_pairs, pf.upload_probe_q(b), synth.probe_positions(w), 0.0)
         torch.cuda.synchronize()
         e0, e1 = ev(), ev()
         e0.record()

@@ -155,8 +155,8 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     if (s.dtype == FDKV_BF16 && s.d == 128) c->has_tmap = make_arena_tensor_map(c->arena, arena_bytes, c->tmap);
     c->packed_lists = c->has_tmap && s.max_batch * s.Hkv <= kFastMaxUnits;
     if (s.dtype == FDKV_BF16 && s.d == 128)
-        c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, 128, c->tmap_z1) &&
-                             make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.Tmax * s.d * s.esize, 128, c->tmap_drop);
+        c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_z1) &&
+                             make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_drop);
     *out = c;
     return FDKV_OK;
 }

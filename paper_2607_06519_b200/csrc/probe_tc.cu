@@ -6,11 +6,12 @@
 // and summed without ever leaving the SM:
 //   * work item = (unit, layer of the pair, block of 256 probe rows, candidate, range of 128-token key tiles);
 //     one CTA per item, 6 warps: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner), warps 2-5 = epilogue;
-//   * A (the item's 256 Q rows, 64 KiB) is gathered once into shared memory in the 128-byte-swizzled K-major
-//     layout; B tiles (128 tokens x 128 channels) stream through a 4-stage TMA ring;
-//   * per key tile 16 tcgen05.mma (M = 128, N = 128, K = 16, kind::f16, bf16 x bf16 -> f32) fill two 128x128 f32
-//     accumulators in TMEM (256 columns); two such accumulator sets alternate so the epilogue of tile i overlaps
-//     the MMAs of tile i+1;
+//   * A (the item's 256 Q rows) is written once into tensor memory (128 columns: lane = row, two bf16 channels per
+//     column) by the threads that own the lanes; B tiles (192 tokens x 128 channels, 128-byte-swizzled K-major)
+//     stream through a 4-stage TMA ring;
+//   * per key tile 16 tcgen05.mma (M = 128, N = 192, K = 16, kind::f16, A from TMEM, bf16 x bf16 -> f32) fill two
+//     128x192 f32 accumulators in TMEM (384 columns).  (With N = 96 two accumulator sets alternate; measured
+//     slightly slower: the tensor pipe, not the epilogue, is the limit.);
 //   * epilogue: tcgen05.ld (32 lanes x 32 columns per instruction), square, mask keys after the row's probe
 //     position, accumulate; one float64 sum per item, summed across items in a fixed order by the finalize kernel.
 // Every mbarrier wait is bounded; on expiry the CTA flags the device status word, stops waiting and still frees
@@ -18,6 +19,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdio>
 #include <cstdlib>
 
 #include "fdkv_internal.h"
@@ -26,20 +28,22 @@ namespace fdkv {
 
 namespace {
 
-constexpr int kBN = 128;                       // key tokens per tile
-constexpr int kBStages = 4;
-constexpr int kBHalf = kBN * 128;              // one 64-channel half of a B tile: 16 KiB
-constexpr int kBStageBytes = 2 * kBHalf;       // 32 KiB
-constexpr int kAHalf = 128 * 128;              // one 64-channel half of a 128-row A tile: 16 KiB
-constexpr int kATile = 2 * kAHalf;             // 32 KiB per 128 rows
-constexpr int kABytes = 2 * kATile;            // 256 rows
+constexpr int kBN = kProbeBoxRows;             // key tokens per tile (N of the MMA): 96 (two accumulator sets) or 192 (one)
+constexpr int kBStages = kBN == 96 ? 8 : 4;
+constexpr int kAccSets = kBN == 96 ? 2 : 1;
+constexpr int kBHalf = kBN * 128;              // one 64-channel half of a B tile: 12 KiB
+constexpr int kBStageBytes = 2 * kBHalf;       // 24 KiB
 constexpr int kHdr = 1024;
-constexpr int kProbeSmem = kHdr + kABytes + kBStages * kBStageBytes;  // 193 KiB
+constexpr int kProbeSmem = kHdr + kBStages * kBStageBytes;  // 193 KiB
 constexpr int kPThreads = 6 * 32;
 constexpr uint32_t kSpin = 1u << 22;
+// Tensor memory (512 columns): the item's 256 Q rows as the A operand (2 M tiles x 64 columns: 128 channels, two bf16
+// per column) and two alternating sets of two 128 x 96 f32 accumulators.
 constexpr int kTmemCols = 512;
-// header: full[4] @0, empty[4] @32, tfull[2] @64, tempty[2] @80, tmem slot @96, abort @100, reduce @128 (4 doubles)
-constexpr int oFull = 0, oEmpty = 32, oTFull = 64, oTEmpty = 80, oSlot = 96, oAbort = 100, oRed = 128;
+constexpr int kTmemA = 0, kTmemAcc = 128, kAccSet = 2 * kBN;
+static_assert(kTmemAcc + kAccSets * kAccSet <= kTmemCols && kBN % 96 == 0, "tensor memory budget");
+// header: full[8] @0, empty[8] @64, tfull[2] @128, tempty[2] @144, tmem slot @160, abort @164, reduce @192 (4 doubles)
+constexpr int oFull = 0, oEmpty = 64, oTFull = 128, oTEmpty = 144, oSlot = 160, oAbort = 164, oRed = 192;
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mb_init(uint32_t bar, uint32_t count) {
@@ -85,13 +89,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;                            // 128-byte swizzle
     return d;
 }
-// instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 128
+// instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = kBN
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] * B[smem]^T; ACC = 0 overwrites D
+template <int ACC>
+__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(da), "l"(db), "r"(kIdesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(db), "r"(kIdesc), "n"(ACC)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -108,10 +114,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr));
 }
 
+// 64 consecutive 32-bit columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_st64(uint32_t taddr, const uint32_t (&r)[64]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x64.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,"
+        "%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63,%64};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+          "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+          "r"(r[30]), "r"(r[31]), "r"(r[32]), "r"(r[33]), "r"(r[34]), "r"(r[35]), "r"(r[36]), "r"(r[37]), "r"(r[38]), "r"(r[39]),
+          "r"(r[40]), "r"(r[41]), "r"(r[42]), "r"(r[43]), "r"(r[44]), "r"(r[45]), "r"(r[46]), "r"(r[47]), "r"(r[48]), "r"(r[49]),
+          "r"(r[50]), "r"(r[51]), "r"(r[52]), "r"(r[53]), "r"(r[54]), "r"(r[55]), "r"(r[56]), "r"(r[57]), "r"(r[58]), "r"(r[59]),
+          "r"(r[60]), "r"(r[61]), "r"(r[62]), "r"(r[63])
+        : "memory");
+}
+
 struct TcPlan {
     int items_per_unit;  // 2 layers x mblocks x 2 candidates x nsplits
     int mblocks, nsplits, ntiles, tiles_per_split;
     int pos_min, pos_max;
+    int experiment;  // timing experiments only (FDKV_PROBE_EXPERIMENT): 1 = epilogue skips the accumulator reads
 };
 
 __global__ void __launch_bounds__(kPThreads, 1)
@@ -124,6 +147,8 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         if (threadIdx.x == 0) atomicMax(a.status, (int32_t)kFlagCountMismatch);
         return;
     }
+    long long dbg_c0 = 0, dbg_g0 = 0;
+    if (pl.experiment >= 8 && threadIdx.x == 0) { dbg_c0 = clock64(); asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(dbg_g0)); }
     // ---- decode the work item ----
     int it = blockIdx.x;
     const int unit = a.unit_begin + it / pl.items_per_unit;
@@ -144,24 +169,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // ---- A: rows r = mblock*256 + i of this layer's probe block, row = g*W + qi -> Q[layer][qi][h*G+g][:] ----
-    {
-        const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[2 * pair + layer]);
-        for (int v = threadIdx.x; v < 256 * 16; v += kPThreads) {
-            const int i = v >> 4, chunk = v & 15;  // row in block, 16-byte chunk of 8 channels
-            const int r = mblock * 256 + i;
-            uint4 val = make_uint4(0u, 0u, 0u, 0u);
-            if (r < rows_layer) {
-                const int g = r / a.W, qi = r % a.W;
-                val = *reinterpret_cast<const uint4*>(q + ((int64_t)qi * a.Hq + h * a.G + g) * 128 + chunk * 8);
-            }
-            const int mt = i >> 7, rr = i & 127;
-            uint8_t* dst = smem + kHdr + mt * kATile + (chunk >> 3) * kAHalf + rr * 128 + (((chunk & 7) ^ (rr & 7)) << 4);
-            *reinterpret_cast<uint4*>(dst) = val;
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA's async reads
-    }
-    if (warp == 1) {  // tensor memory: all 512 columns (two sets of two 128x128 f32 accumulators)
+    if (warp == 1) {  // tensor memory: all 512 columns
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sm0 + oSlot), "r"((uint32_t)kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -169,7 +177,34 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + oSlot);
-    const uint32_t b0 = sm0 + kHdr + kABytes;
+    // ---- A operand: row r = mblock*256 + mt*128 + lane-row of this layer's probe block, r = g*W + qi ->
+    //      Q[layer][qi][h*G+g][:], written by the thread that owns that TMEM lane (two bf16 channels per column) ----
+    if (warp >= 2) {
+        const int lq = warp & 3, rl = lq * 32 + lane;
+        const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[2 * pair + layer]);
+#pragma unroll 1
+        for (int mt = 0; mt < 2; ++mt) {
+            const int r = mblock * 256 + mt * 128 + rl;
+            uint32_t w[64];
+            if (r < rows_layer) {
+                const uint4* src = reinterpret_cast<const uint4*>(q + ((int64_t)(r % a.W) * a.Hq + h * a.G + r / a.W) * 128);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const uint4 v = src[i];
+                    w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 64; ++i) w[i] = 0u;  // padding rows contribute nothing
+            }
+            tmem_st64(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(kTmemA + mt * 64), w);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t b0 = sm0 + kHdr;
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -177,7 +212,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
             const CUtensorMap* map = cand ? &tmap_drop : &tmap_z1;
             // rows of this unit's K coefficients: staged Z1 holds K and V per unit (unit-tensor 2*unit), the dropped copy K only
             const int64_t row0 = (cand ? (int64_t)unit : (int64_t)unit * 2) * a.Tmax;
-            for (int i = 0; i < ntile; ++i) {
+            for (int i = 0; i < ntile && pl.experiment != 2; ++i) {
                 const int s = i % kBStages;
                 const uint32_t ph = (uint32_t)(i / kBStages) & 1u;
                 mb_wait(sm0 + oEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
@@ -193,19 +228,23 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         // ================= MMA issuer =================
         if (lane == 0) {
             for (int i = 0; i < ntile; ++i) {
-                const int s = i % kBStages, as = i & 1;
-                mb_wait(sm0 + oTEmpty + 8 * as, (((uint32_t)i >> 1) & 1u) ^ 1u, abort_flag, a.status);
-                mb_wait(sm0 + oFull + 8 * s, (uint32_t)(i / kBStages) & 1u, abort_flag, a.status);
+                const int s = i % kBStages, as = i % kAccSets;
+                mb_wait(sm0 + oTEmpty + 8 * as, ((uint32_t)(i / kAccSets) & 1u) ^ 1u, abort_flag, a.status);
+                if (pl.experiment != 2) mb_wait(sm0 + oFull + 8 * s, (uint32_t)(i / kBStages) & 1u, abort_flag, a.status);
                 if (*abort_flag) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                // one descriptor per stage; the k steps and the two M tiles only add compile-time constants
+                const uint64_t db_stage = smem_desc(b0 + s * kBStageBytes);
+                const uint32_t d0 = tmem_base + (uint32_t)(kTmemAcc + as * kAccSet);
+                if (pl.experiment != 3)
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(as * 256 + mt * 128);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {  // 8 steps of 16 channels: 4 per 64-channel half, 32 bytes apart inside the swizzle atom
-                        const uint64_t da = smem_desc(sm0 + kHdr + mt * kATile + (k >> 2) * kAHalf + (k & 3) * 32);
-                        const uint64_t db = smem_desc(b0 + s * kBStageBytes + (k >> 2) * kBHalf + (k & 3) * 32);
-                        umma(d_tmem, da, db, k > 0 ? 1u : 0u);
+                    for (int k = 0; k < 8; ++k) {  // 8 steps of 16 channels: 8 TMEM columns of A, 32 bytes of B inside the swizzle atom
+                        const uint64_t db = db_stage + (uint64_t)(((k >> 2) * kBHalf + (k & 3) * 32) >> 4);
+                        const uint32_t ta = tmem_base + (uint32_t)(kTmemA + mt * 64 + k * 8);
+                        if (k == 0) umma_ts<0>(d0 + mt * kBN, ta, db);
+                        else umma_ts<1>(d0 + mt * kBN, ta, db);
                     }
                 }
                 umma_commit(sm0 + oEmpty + 8 * s);    // the B stage is free once these MMAs have read it
@@ -224,37 +263,41 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         }
         double total = 0.0;
         for (int i = 0; i < ntile; ++i) {
-            const int as = i & 1;
+            const int as = i % kAccSets;
             const int t0 = (tile0 + i) * kBN;
-            mb_wait(sm0 + oTFull + 8 * as, ((uint32_t)i >> 1) & 1u, abort_flag, a.status);
+            mb_wait(sm0 + oTFull + 8 * as, (uint32_t)(i / kAccSets) & 1u, abort_flag, a.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float acc = 0.f;
-            if (!*abort_flag) {
+            if (!*abort_flag && pl.experiment != 1) {
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
                     const bool all_visible = t0 + kBN - 1 <= pl.pos_min;  // every key of the tile precedes every probe position
 #pragma unroll
-                    for (int cp = 0; cp < 2; ++cp) {  // two 32-column loads in flight per wait
-                        uint32_t r0[32], r1[32];
-                        const uint32_t ta = tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(as * 256 + mt * 128 + cp * 64);
+                    for (int cg = 0; cg < kBN / 96; ++cg) {  // 96 accumulator columns of this lane per round, three loads in flight
+                        uint32_t r0[32], r1[32], r2[32];
+                        const uint32_t ta = tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(kTmemAcc + as * kAccSet + mt * kBN + cg * 96);
+                        const int tc = t0 + cg * 96;
                         tmem_ld32(ta, r0);
                         tmem_ld32(ta + 32, r1);
+                        tmem_ld32(ta + 64, r2);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                         if (all_visible && pos_row[mt] >= 0) {
-                            float acc1 = 0.f;
+                            float acc1 = 0.f, acc2 = 0.f;
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                const float v = __uint_as_float(r0[j]), w = __uint_as_float(r1[j]);
-                                acc = fmaf(v, v, acc);
-                                acc1 = fmaf(w, w, acc1);
+                                const float u = __uint_as_float(r0[j]), v = __uint_as_float(r1[j]), w = __uint_as_float(r2[j]);
+                                acc = fmaf(u, u, acc);
+                                acc1 = fmaf(v, v, acc1);
+                                acc2 = fmaf(w, w, acc2);
                             }
-                            acc += acc1;
+                            acc += acc1 + acc2;
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                const float v = __uint_as_float(r0[j]), w = __uint_as_float(r1[j]);
-                                if (t0 + cp * 64 + j <= pos_row[mt]) acc = fmaf(v, v, acc);
-                                if (t0 + cp * 64 + 32 + j <= pos_row[mt]) acc = fmaf(w, w, acc);
+                                const float u = __uint_as_float(r0[j]), v = __uint_as_float(r1[j]), w = __uint_as_float(r2[j]);
+                                if (tc + j <= pos_row[mt]) acc = fmaf(u, u, acc);
+                                if (tc + 32 + j <= pos_row[mt]) acc = fmaf(v, v, acc);
+                                if (tc + 64 + j <= pos_row[mt]) acc = fmaf(w, w, acc);
                             }
                         }
                     }
@@ -276,6 +319,12 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let copies and MMAs in flight finish before the memory goes away
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    }
+    if (pl.experiment >= 8 && threadIdx.x == 0 && (blockIdx.x % 257) == 0) {
+        long long c1 = clock64(), g1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1));
+        printf("item %d: %lld cycles in %lld ns = %.0f MHz, %d tiles, %.0f cycles per tile\n", blockIdx.x, c1 - dbg_c0, g1 - dbg_g0,
+               1e3 * (double)(c1 - dbg_c0) / (double)(g1 - dbg_g0), ntile, (double)(c1 - dbg_c0) / ntile);
     }
     if (threadIdx.x == 0) {
         const double* red = reinterpret_cast<const double*>(smem + oRed);
@@ -302,6 +351,7 @@ cudaError_t launch_probe_tc(const ProbeArgs& a, int dtype, cudaStream_t st, bool
     }
     if (!enabled) return cudaSuccess;
     TcPlan pl;
+    { const char* ex = getenv("FDKV_PROBE_EXPERIMENT"); pl.experiment = ex ? atoi(ex) : 0; }
     pl.pos_min = a.pos_host[0];
     pl.pos_max = a.pos_host[a.W - 1];
     pl.ntiles = pl.pos_max / kBN + 1;  // keys after the last probe position never count
