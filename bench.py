@@ -153,7 +153,7 @@ def run_reference(args, w):
 def run_ours(args, w):
     import torch
 
-    from paper_2607_06519_b200 import binding as B, runner, synth
+    from paper_2607_06519_b200 import binding as B, replicas, runner, synth
 
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -263,8 +263,7 @@ def run_ours(args, w):
         for _ in range(args.warmup):
             run_step()
     stream.synchronize()
-    if dist:
-        dist.barrier()
+    replicas.barrier(dist)
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     if rank == 0:
@@ -287,12 +286,9 @@ def run_ours(args, w):
                     run_step()
             stream.synchronize()
         clocks = sampler.stop()
-    if dist:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    value, total_s = replicas.whole_job_rate(w.batch * args.steps, total_ms * 1e-3, dist, dev)
+    total_ms = total_s * 1e3
     ms_per_step = total_ms / args.steps
-    value = world * w.batch * args.steps / (total_ms * 1e-3)
 
     # ---------------- end to end: host buffers through the C ABI, copies inside the timed region ----------------
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
@@ -325,11 +321,7 @@ def run_ours(args, w):
         host_step()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if dist:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_val = world * w.batch * args.steps / e2e_s
+    e2e_val, e2e_s = replicas.whole_job_rate(w.batch * args.steps, e2e_s, dist, dev)
     h2d = sum(q.numel() * q.element_size() for q in hq)
     if append:
         h2d += sum(2 * t[0].numel() * t[0].element_size() for t in hk)
