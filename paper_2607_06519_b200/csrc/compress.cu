@@ -20,6 +20,12 @@ struct Store<float> {
     using vec_t = float4;
     __device__ static void unpack(const vec_t& v, float* f) { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
     __device__ static vec_t pack(const float* f) { return make_float4(f[0], f[1], f[2], f[3]); }
+    // element i of the vector (i only known at run time: select, never index, so the vector stays in registers)
+    __device__ static float element(const vec_t& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+    // the vector with the elements whose bit is set in `mask` zeroed
+    __device__ static vec_t clear(const vec_t& v, uint32_t mask) {
+        return make_float4(mask & 1u ? 0.f : v.x, mask & 2u ? 0.f : v.y, mask & 4u ? 0.f : v.z, mask & 8u ? 0.f : v.w);
+    }
 };
 template <>
 struct Store<__nv_bfloat16> {
@@ -41,6 +47,19 @@ struct Store<__nv_bfloat16> {
             uint32_t lo = __bfloat16_as_ushort(__float2bfloat16_rn(f[2 * i]));
             uint32_t hi = __bfloat16_as_ushort(__float2bfloat16_rn(f[2 * i + 1]));
             w[i] = lo | (hi << 16);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __device__ static __nv_bfloat16 element(const vec_t& v, int i) {
+        const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
+        return __ushort_as_bfloat16((unsigned short)((i & 1) ? (w >> 16) : (w & 0xFFFFu)));
+    }
+    __device__ static vec_t clear(const vec_t& v, uint32_t mask) {
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (mask >> (2 * j) & 1u) w[j] &= 0xFFFF0000u;
+            if (mask >> (2 * j + 1) & 1u) w[j] &= 0x0000FFFFu;
         }
         return make_uint4(w[0], w[1], w[2], w[3]);
     }
@@ -76,24 +95,41 @@ __global__ void __launch_bounds__(1024) split_hist_kernel(CompressArgs a, int to
     const int t_end = min(a.T, t_begin + tokens_per_cta);
     const int vpr = a.d / VEC;
     const int64_t nvec = (int64_t)max(0, t_end - t_begin) * vpr;
-    for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
-        const int t = t_begin + (int)(v / vpr);
-        const int cv = (int)(v % vpr) * VEC;
-        const typename S::vec_t va = *reinterpret_cast<const typename S::vec_t*>(x0 + (int64_t)t * a.stride_t + cv);
-        const typename S::vec_t vb = *reinterpret_cast<const typename S::vec_t*>(x1 + (int64_t)t * a.stride_t + cv);
-        float fa[VEC], fb[VEC], f0[VEC], f1[VEC];
-        S::unpack(va, fa);
-        S::unpack(vb, fb);
+    // two vector pairs in flight per thread: all four loads are issued before the first is used
+    for (int64_t v0 = threadIdx.x; v0 < nvec; v0 += 2 * (int64_t)blockDim.x) {
+        typename S::vec_t va[2], vb[2];
+        int64_t off_in[2], off_out[2];
+        bool live[2];
 #pragma unroll
-        for (int i = 0; i < VEC; ++i) {
-            // one float32 add (subtract), one float32 multiply: never contracted into an FMA
-            f0[i] = __fmul_rn(__fadd_rn(fa[i], fb[i]), c32);
-            f1[i] = __fmul_rn(__fsub_rn(fa[i], fb[i]), c32);
+        for (int u = 0; u < 2; ++u) {
+            const int64_t v = v0 + (int64_t)u * blockDim.x;
+            live[u] = v < nvec;
+            const int t = t_begin + (int)(v / vpr);
+            const int cv = (int)(v % vpr) * VEC;
+            off_in[u] = (int64_t)t * a.stride_t + cv;
+            off_out[u] = (int64_t)t * a.d + cv;
+            if (live[u]) {
+                va[u] = *reinterpret_cast<const typename S::vec_t*>(x0 + off_in[u]);
+                vb[u] = *reinterpret_cast<const typename S::vec_t*>(x1 + off_in[u]);
+            }
         }
-        *reinterpret_cast<typename S::vec_t*>(z0 + (int64_t)t * a.d + cv) = S::pack(f0);
-        *reinterpret_cast<typename S::vec_t*>(z1 + (int64_t)t * a.d + cv) = S::pack(f1);
 #pragma unroll
-        for (int i = 0; i < VEC; ++i) atomicAdd(&s_hist[key_of(stored<T>(f1[i])) >> 16], 1u);
+        for (int u = 0; u < 2; ++u) {
+            if (!live[u]) continue;
+            float fa[VEC], fb[VEC], f0[VEC], f1[VEC];
+            S::unpack(va[u], fa);
+            S::unpack(vb[u], fb);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                // one float32 add (subtract), one float32 multiply: never contracted into an FMA
+                f0[i] = __fmul_rn(__fadd_rn(fa[i], fb[i]), c32);
+                f1[i] = __fmul_rn(__fsub_rn(fa[i], fb[i]), c32);
+            }
+            *reinterpret_cast<typename S::vec_t*>(z0 + off_out[u]) = S::pack(f0);
+            *reinterpret_cast<typename S::vec_t*>(z1 + off_out[u]) = S::pack(f1);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) atomicAdd(&s_hist[key_of(stored<T>(f1[i])) >> 16], 1u);
+        }
     }
     __syncthreads();
     uint32_t* gh = a.hist + (int64_t)ut * kHistBins;
@@ -294,64 +330,71 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
     uint32_t eq_rank = a.tile_eq[(int64_t)ut * a.ntiles_max + tile];
     const int64_t e_begin = (int64_t)tile * kResTile * a.d;
     const int64_t e_end = min((int64_t)a.T * a.d, e_begin + (int64_t)kResTile * a.d);
-    for (int64_t base = e_begin; base < e_end; base += 32 * VEC) {
-        const int64_t e = base + lane * VEC;
-        float f[VEC];
-        uint32_t is_gt = 0, is_eq = 0;
-        if (e < e_end) {
-            S::unpack(*reinterpret_cast<const typename S::vec_t*>(z + e), f);
+    constexpr int CH = 8;  // vectors in flight per lane: all loads of a round are issued before any is used
+    for (int64_t base0 = e_begin; base0 < e_end; base0 += (int64_t)CH * 32 * VEC) {
+        typename S::vec_t vreg[CH];
 #pragma unroll
-            for (int i = 0; i < VEC; ++i) {
-                const uint32_t k = key_of(f[i]);
-                is_gt |= (uint32_t)(k > tau) << i;
-                is_eq |= (uint32_t)(k == tau) << i;
-            }
+        for (int c = 0; c < CH; ++c) {
+            const int64_t e = base0 + ((int64_t)c * 32 + lane) * VEC;
+            if (e < e_end) vreg[c] = *reinterpret_cast<const typename S::vec_t*>(z + e);
         }
-        // rank of this lane's first tie among the unit-tensor's ties
-        uint32_t keep = is_gt;
-        const uint32_t any_eq = __ballot_sync(0xFFFFFFFFu, is_eq != 0);
-        if (any_eq) {
-            const uint32_t n_eq = __popc(is_eq);
-            uint32_t incl = n_eq;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const int64_t e = base0 + ((int64_t)c * 32 + lane) * VEC;
+            if (base0 + (int64_t)c * 32 * VEC >= e_end) break;  // warp-uniform
+            float f[VEC];
+            uint32_t is_gt = 0, is_eq = 0;
+            if (e < e_end) {
+                S::unpack(vreg[c], f);
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) {
+                    const uint32_t k = key_of(f[i]);
+                    is_gt |= (uint32_t)(k > tau) << i;
+                    is_eq |= (uint32_t)(k == tau) << i;
+                }
+            }
+            // rank of this lane's first tie among the unit-tensor's ties
+            uint32_t keep = is_gt;
+            const uint32_t any_eq = __ballot_sync(0xFFFFFFFFu, is_eq != 0);
+            if (any_eq) {
+                const uint32_t n_eq = __popc(is_eq);
+                uint32_t incl = n_eq;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                uint32_t r = eq_rank + incl - n_eq;
+#pragma unroll
+                for (int i = 0; i < VEC; ++i)
+                    if (is_eq >> i & 1u) {
+                        if (r < need) keep |= 1u << i;
+                        ++r;
+                    }
+                eq_rank += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            }
+            const uint32_t n_keep = __popc(keep);
+            uint32_t incl = n_keep;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
                 if (lane >= o) incl += v;
             }
-            uint32_t r = eq_rank + incl - n_eq;
-#pragma unroll
-            for (int i = 0; i < VEC; ++i)
-                if (is_eq >> i & 1u) {
-                    if (r < need) keep |= 1u << i;
-                    ++r;
-                }
-            eq_rank += __shfl_sync(0xFFFFFFFFu, incl, 31);
-        }
-        const uint32_t n_keep = __popc(keep);
-        uint32_t incl = n_keep;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        uint32_t w = pos + incl - n_keep;
-#pragma unroll
-        for (int i = 0; i < VEC; ++i)
-            if (keep >> i & 1u) {
+            uint32_t w = pos + incl - n_keep;
+            // most lanes keep nothing, few keep more than one or two of their elements: walk the set bits
+            for (uint32_t kk = keep; kk; kk &= kk - 1) {
+                const int i = __ffs((int)kk) - 1;
+                const T v = S::element(vreg[c], i);
                 idx[w] = (int32_t)(e + i);
-                val[w] = z[e + i];
-                if (pk) pk[w] = packed_entry<T>(z[e + i], (int)(e + i));
+                val[w] = v;
+                if (pk) pk[w] = packed_entry<T>(v, (int)(e + i));
                 ++w;
             }
-        // K tensors only: the coefficients the residual candidate drops (Z1 with the kept entries zeroed), the
-        // second B operand of the tensor-core probe
-        if (drop && e < e_end) {
-#pragma unroll
-            for (int i = 0; i < VEC; ++i)
-                if (keep >> i & 1u) f[i] = 0.f;
-            *reinterpret_cast<typename S::vec_t*>(drop + e) = S::pack(f);
+            // K tensors only: the coefficients the residual candidate drops (Z1 with the kept entries zeroed), the
+            // second B operand of the tensor-core probe
+            if (drop && e < e_end) *reinterpret_cast<typename S::vec_t*>(drop + e) = S::clear(vreg[c], keep);
+            pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
         }
-        pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
 }
 
