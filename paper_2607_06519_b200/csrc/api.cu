@@ -208,19 +208,23 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     cudaStream_t st = S(stream);
     const int ut_begin = pb * s.Hkv * 2, ut_count = (pe - pb) * s.Hkv * 2;
     CU(cudaMemsetAsync(wsp<uint32_t>(c, c->ws.hist) + (size_t)ut_begin * kHistBins, 0, (size_t)ut_count * kHistBins * 4, st));
-    for (int p = pb; p < pe; ++p) {
+    for (int p0 = pb; p0 < pe; p0 += kSplitPairs) {
         CompressArgs a;
-        a.k0 = k_layers[2 * p]; a.k1 = k_layers[2 * p + 1];
-        a.v0 = v_layers[2 * p]; a.v1 = v_layers[2 * p + 1];
+        a.n_pairs = pe - p0 < kSplitPairs ? pe - p0 : kSplitPairs;
+        for (int j = 0; j < a.n_pairs; ++j) {
+            const int p = p0 + j;
+            a.k0[j] = k_layers[2 * p]; a.k1[j] = k_layers[2 * p + 1];
+            a.v0[j] = v_layers[2 * p]; a.v1[j] = v_layers[2 * p + 1];
+            c->k_layers[2 * p] = a.k0[j]; c->k_layers[2 * p + 1] = a.k1[j];
+            c->v_layers[2 * p] = a.v0[j]; c->v_layers[2 * p + 1] = a.v1[j];
+        }
         a.stride_t = stride_t; a.stride_h = stride_h;
         a.T = T; a.d = s.d; a.Hkv = s.Hkv; a.tensors = 2;
-        a.ut_base = p * s.Hkv * 2;
+        a.ut_base = p0 * s.Hkv * 2;
         a.unit_stride = (int64_t)s.Tmax * s.d;
         a.z0 = c->work + c->ws.z0; a.z1 = c->work + c->ws.z1;
         a.hist = wsp<uint32_t>(c, c->ws.hist);
         CU(launch_split_hist(a, s.dtype, st));
-        c->k_layers[2 * p] = a.k0; c->k_layers[2 * p + 1] = a.k1;
-        c->v_layers[2 * p] = a.v0; c->v_layers[2 * p + 1] = a.v1;
     }
     SelectArgs sa;
     sa.ut_begin = ut_begin; sa.ut_count = ut_count;

@@ -74,7 +74,7 @@ template <>
 __device__ __forceinline__ float stored<__nv_bfloat16>(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
 // ----- C1: depth split + histogram of the top 15 magnitude bits of z1 ---------------------------------
-// grid (chunks, Hkv*tensors); each CTA owns a token range of one unit-tensor and a private 128 KiB histogram.
+// grid (chunks, Hkv*tensors, pairs); each CTA owns a token range of one unit-tensor and a private 128 KiB histogram.
 template <typename T>
 __global__ void __launch_bounds__(1024) split_hist_kernel(CompressArgs a, int tokens_per_cta) {
     extern __shared__ uint32_t s_hist[];
@@ -83,10 +83,10 @@ __global__ void __launch_bounds__(1024) split_hist_kernel(CompressArgs a, int to
     for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) s_hist[b] = 0;
     __syncthreads();
 
-    const int h = blockIdx.y / a.tensors, is_v = blockIdx.y % a.tensors;
-    const int ut = a.ut_base + blockIdx.y;
-    const T* x0 = reinterpret_cast<const T*>(is_v ? a.v0 : a.k0) + (int64_t)h * a.stride_h;
-    const T* x1 = reinterpret_cast<const T*>(is_v ? a.v1 : a.k1) + (int64_t)h * a.stride_h;
+    const int h = blockIdx.y / a.tensors, is_v = blockIdx.y % a.tensors, pj = blockIdx.z;
+    const int ut = a.ut_base + pj * a.Hkv * a.tensors + blockIdx.y;
+    const T* x0 = reinterpret_cast<const T*>(is_v ? a.v0[pj] : a.k0[pj]) + (int64_t)h * a.stride_h;
+    const T* x1 = reinterpret_cast<const T*>(is_v ? a.v1[pj] : a.k1[pj]) + (int64_t)h * a.stride_h;
     T* z0 = reinterpret_cast<T*>(a.z0) + (int64_t)ut * a.unit_stride;
     T* z1 = reinterpret_cast<T*>(a.z1) + (int64_t)ut * a.unit_stride;
     const float c32 = __uint_as_float(0x3F3504F3u);
@@ -424,9 +424,9 @@ cudaError_t launch_split_hist(const CompressArgs& a, int dtype, cudaStream_t st)
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    if (a.T <= 0) return cudaSuccess;
+    if (a.T <= 0 || a.n_pairs <= 0) return cudaSuccess;
     const int tokens_per_cta = 4096 * 128 / a.d / (dtype == FDKV_BF16 ? 1 : 2);
-    dim3 grid((a.T + tokens_per_cta - 1) / tokens_per_cta, a.Hkv * a.tensors);
+    dim3 grid((a.T + tokens_per_cta - 1) / tokens_per_cta, a.Hkv * a.tensors, a.n_pairs);
     if (dtype == FDKV_BF16)
         split_hist_kernel<__nv_bfloat16><<<grid, 1024, smem, st>>>(a, tokens_per_cta);
     else
@@ -562,7 +562,8 @@ extern "C" fdkv_status fdkv_compress_unit_noalloc(const void* x0, const void* x1
     if (e != cudaSuccess) return record_cuda_error(e);
 
     CompressArgs a;
-    a.k0 = x0; a.k1 = x1; a.v0 = x0; a.v1 = x1;
+    a.k0[0] = x0; a.k1[0] = x1; a.v0[0] = x0; a.v1[0] = x1;
+    a.n_pairs = 1;
     a.stride_t = stride_t; a.stride_h = 0;
     a.T = T; a.d = head_dim; a.Hkv = 1; a.tensors = 1;
     a.ut_base = 0; a.unit_stride = 0;

@@ -113,12 +113,15 @@ struct fdkv_ctx {
 namespace fdkv {
 
 // ---- launchers implemented in compress.cu / probe.cu / decode.cu; each returns cudaGetLastError() ----
+constexpr int kSplitPairs = 32;  // layer pairs one launch of the split kernel covers
 struct CompressArgs {
-    const void *k0, *k1, *v0, *v1;  // the four [T][Hkv][d] strided tensors of one pair
+    // the four [T][Hkv][d] strided tensors (K and V of layers 2p, 2p+1) of each pair of the launch
+    const void *k0[kSplitPairs], *k1[kSplitPairs], *v0[kSplitPairs], *v1[kSplitPairs];
+    int n_pairs;
     int64_t stride_t, stride_h;
     int T, d, Hkv;
     int tensors;  // 2: K and V of every head (unit-tensor = head*2 + is_v); 1: K only (unit-tensor = head)
-    int ut_base;  // first unit-tensor of this pair in the stage: (pair*Hkv)*2
+    int ut_base;  // first unit-tensor of the first pair in the stage; pair j adds j*Hkv*tensors
     int64_t unit_stride;  // elements between staged unit-tensors (Tmax*d)
     void *z0, *z1;
     uint32_t* hist;
