@@ -667,16 +667,19 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     static bool use_pdl = true;
     // tiles copied before the dependency wait; more than one takes HBM bandwidth from the kernel still running
     static int prologue_tiles = 1;
+    static bool whole_ctas = true;
     if (res_cost < 0) {
         const char* ev = getenv("FDKV_RES_COST");  // tuning knobs for benchmark sweeps
         res_cost = ev ? atof(ev) : 1.6;
         if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 1.6;
         const char* pv = getenv("FDKV_NO_PDL");
         use_pdl = !(pv && pv[0] == '1');
+        const char* wc = getenv("FDKV_NO_WHOLE_CTAS");
+        whole_ctas = !(wc && wc[0] == '1');
         const char* pt = getenv("FDKV_PROLOGUE_TILES");
         prologue_tiles = pt ? std::max(0, std::min(kStages, atoi(pt))) : 1;
     }
-    // ---- flat cost-weighted schedule: CTA c starts at weight c * W / ncta ----
+    // ---- cost-weighted schedule: whole CTAs per unit when there are enough CTAs, else a flat cut of the (unit, tile) list ----
     FastSched sch;
     PartCount cs;
     std::vector<int64_t> wp(units + 1, 0);
@@ -701,7 +704,36 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     sch.ncta = ncta;
     sch.prologue_tiles = prologue_tiles;
     sch.units = units;
-    {
+    bool whole = whole_ctas && units <= ncta;
+    std::vector<int> nc(units, 1);
+    if (whole) {
+        // Whole CTAs per unit (no CTA pays a second merge + ticket): shares proportional to the unit's cost, at least
+        // one each, the remainder to the units with the largest cost per CTA; never more CTAs than tiles.
+        int given = units;
+        for (int u = 0; u < units; ++u) {
+            const int extra = std::min<int64_t>((int64_t)nt[u] - 1, (int64_t)((double)(ncta - units) * (double)(wp[u + 1] - wp[u]) / (double)wp[units]));
+            nc[u] += std::max(0, extra);
+            given += std::max(0, extra);
+        }
+        while (given < ncta) {
+            int best = -1;
+            double best_load = 0.0;
+            for (int u = 0; u < units; ++u) {
+                const double load = (double)(wp[u + 1] - wp[u]) / nc[u];
+                if (nc[u] < nt[u] && load > best_load) { best_load = load; best = u; }
+            }
+            if (best < 0) break;
+            ++nc[best];
+            ++given;
+        }
+        if (given != ncta) whole = false;
+    }
+    if (whole) {
+        int c = 0;
+        for (int u = 0; u < units; ++u)
+            for (int j = 0; j < nc[u]; ++j) sch.start[c++] = ((uint32_t)u << 20) | (uint32_t)((int64_t)nt[u] * j / nc[u]);
+        sch.start[ncta] = (uint32_t)units << 20;
+    } else {
         int u = 0;
         for (int c = 0; c < ncta; ++c) {
             const int64_t target = wp[units] * c / ncta;
