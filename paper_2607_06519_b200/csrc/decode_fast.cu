@@ -736,6 +736,10 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
             ++given;
         }
         if (given != ncta) whole = false;
+        // with few CTAs per unit the integer shares are too uneven (2 vs 3 CTAs is +50 %): cut the flat list instead
+        double worst = 0.0;
+        for (int u = 0; u < units; ++u) worst = std::max(worst, (double)(wp[u + 1] - wp[u]) / nc[u]);
+        if (worst > 1.06 * (double)wp[units] / ncta) whole = false;
     }
     if (whole) {
         int c = 0;
