@@ -579,16 +579,28 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                         }
 #pragma unroll
                         for (int o = 16; o; o >>= 1) ls += __shfl_xor_sync(0xFFFFFFFFu, ls, o);
-                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        // part weights to shared memory (one row per warp, after the eight 128-float sums), then the
+                        // accumulator rows in batches of eight independent loads
+                        float* const wts = red + kCW * 128 + warp * kMaxSplits;
 #pragma unroll
-                        for (int i = 0; i < kMaxSplits / 32; ++i) {
-                            for (int s32 = pgi; s32 < 32; s32 += npg) {
-                                const int sp = 32 * i + s32;
-                                if (sp >= nparts) break;
-                                const float f = __shfl_sync(0xFFFFFFFFu, mreg[i], s32);
-                                const float4 v = __ldcg(reinterpret_cast<const float4*>(pp + sp * kPartStride + 4) + lane);
-                                acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y);
-                                acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
+                        for (int i = 0; i < kMaxSplits / 32; ++i) wts[lane + 32 * i] = mreg[i];
+                        __syncwarp();
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int base = pgi; base < nparts; base += 8 * npg) {
+                            float4 v[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int sp = base + j * npg;
+                                if (sp < nparts) v[j] = __ldcg(reinterpret_cast<const float4*>(pp + sp * kPartStride + 4) + lane);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int sp = base + j * npg;
+                                if (sp < nparts) {
+                                    const float f = wts[sp];
+                                    acc.x = fmaf(v[j].x, f, acc.x); acc.y = fmaf(v[j].y, f, acc.y);
+                                    acc.z = fmaf(v[j].z, f, acc.z); acc.w = fmaf(v[j].w, f, acc.w);
+                                }
                             }
                         }
                         reinterpret_cast<float4*>(red + warp * 128)[lane] = acc;
