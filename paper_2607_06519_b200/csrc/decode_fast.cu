@@ -545,14 +545,18 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     part[4 + ch] = A;
                 }
                 // ---- split-K combine by whichever CTA finishes this unit last (atomic ticket, nobody waits) ----
-                __threadfence();
+                // The block barrier orders every thread's part stores before thread 0's fence, which is cumulative: the
+                // ticket increment publishes the whole part at device scope; the last CTA's reads go to L2 (ld.cg).
                 __syncthreads();
                 int* const s_ticket = reinterpret_cast<int*>(smem_raw + kOffTicket);
-                if (threadIdx.x == 0) *s_ticket = atomicAdd(a.counters + u, 1);
+                if (threadIdx.x == 0) {
+                    __threadfence();
+                    *s_ticket = atomicAdd(a.counters + u, 1);
+                    __threadfence();
+                }
                 __syncthreads();
                 const int nparts = pc.n[u];
                 if (*s_ticket == nparts - 1) {
-                    __threadfence();
                     // Warp w takes head w % G and every (8/G)-th part of it, 4 channels per lane; the scratch area
                     // holds the per-warp sums, the header the per-warp denominators.
                     float* const red = reinterpret_cast<float*>(smem_raw + kHeaderBytes + kStages * kStageBytes);  // [8][128]
