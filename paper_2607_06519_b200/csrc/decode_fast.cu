@@ -141,7 +141,6 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
 __global__ void __launch_bounds__(kThreads, 1)
 decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastSched sch, PartCount pc) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    TSTAMP(0);
 #ifdef FDKV_TIMING
     long long t_acc[2] = {0, 0};
 #endif
@@ -525,6 +524,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     *reinterpret_cast<float2*>(scratch_f + gid * 128 + jn * 8 + 2 * tig) =
                         make_float2(oacc[jn][0] + oacc[jn][2], oacc[jn][1] + oacc[jn][3]);
                 __syncthreads();
+                TGLOBAL(0);
                 for (int i = threadIdx.x; i < a.G * 128; i += kThreads) {
                     const int g = i >> 7, ch = i & 127;
                     float M = -INFINITY;
@@ -550,11 +550,12 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 __syncthreads();
                 int* const s_ticket = reinterpret_cast<int*>(smem_raw + kOffTicket);
                 if (threadIdx.x == 0) {
-                    __threadfence();
-                    *s_ticket = atomicAdd(a.counters + u, 1);
-                    __threadfence();
+                    int t;  // one release+acquire read-modify-write instead of fence, atomic, fence
+                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(t) : "l"(a.counters + u) : "memory");
+                    *s_ticket = t;
                 }
                 __syncthreads();
+                TGLOBAL(3);
                 const int nparts = pc.n[u];
                 if (*s_ticket == nparts - 1) {
                     // Warp w takes head w % G and every (8/G)-th part of it, 4 channels per lane; the scratch area
@@ -631,7 +632,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             }
         }
     }
-    TSTAMP(3);
     TGLOBAL(7);
 #ifdef FDKV_TIMING
     if (threadIdx.x == 32) { g_timing[sch.tslot][blockIdx.x][4] = t_acc[0]; g_timing[sch.tslot][blockIdx.x][5] = t_acc[1]; }
@@ -817,9 +817,9 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
                     l, g0 - base, g0max - base, g1min - base, g1 - base, busy / ncta, wf / ncta);
             if (l == 45)
                 for (int c = 0; c < ncta; ++c)
-                    fprintf(stderr, "cta %3d unit %2u mode %d tiles %2lld start %6lld waited %6lld loop_end %6lld end %6lld wait_full_cyc %6lld\n", c,
+                    fprintf(stderr, "cta %3d unit %2u mode %d tiles %2lld start %6lld waited %6lld loop_end %6lld end %6lld wait_full_cyc %6lld merged %6lld ticket %6lld\n", c,
                             sch.start[c] >> 20, a.host_modes[sch.start[c] >> 20], h[l][c][5], h[l][c][6] - g0, h[l][c][1] - g0, h[l][c][2] - g0,
-                            h[l][c][7] - g0, h[l][c][4]);
+                            h[l][c][7] - g0, h[l][c][4], h[l][c][0] - g0, h[l][c][3] - g0);
         }
     }
 #endif

@@ -1,0 +1,101 @@
+"""Argument and call-order errors are reported by the host side of the C ABI before anything is launched
+(no test here makes the GPU fault, trap or hang): status codes, and the context stays usable afterwards."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+def _ctx(**kw):
+    from paper_2607_06519_b200 import binding as B
+
+    cfg = dict(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, max_batch=2, max_prefill=256, max_tail=2, dtype=B.F32,
+               keep_num=1, keep_den=8)
+    cfg.update(kw)
+    return B, B.Context(B.Config(**cfg))
+
+
+def _kv(T=256, H=2, d=64, dtype=torch.float32):
+    g = torch.Generator(device="cuda").manual_seed(0)
+    return [torch.randn((T, H, d), device="cuda", generator=g).to(dtype) for _ in range(4)]
+
+
+def _code(B, fn):
+    with pytest.raises(B.FdkvError) as e:
+        fn()
+    return e.value.code
+
+
+def test_call_order_and_argument_checks():
+    B, ctx = _ctx()
+    k0, k1, v0, v1 = _kv()
+    q = torch.randn((1, 4, 64), device="cuda")
+    # decode before anything is committed
+    assert _code(B, lambda: ctx.decode_attn(0, q)) == 5
+    # probe before compress
+    pq = [torch.randn((8, 4, 64), device="cuda") for _ in range(2)]
+    assert _code(B, lambda: ctx.probe(0, 0, 1, pq, list(range(248, 256)), 1.0)) == 5
+    # bad ranges and sizes
+    assert _code(B, lambda: ctx.compress_prefill(0, 0, 2, 256, [k0, k1], [v0, v1])) == 1      # pair range beyond n_layers/2
+    assert _code(B, lambda: ctx.compress_prefill(5, 0, 1, 256, [k0, k1], [v0, v1])) == 1      # sequence slot
+    assert _code(B, lambda: ctx.compress_prefill(0, 0, 1, 257, [k0, k1], [v0, v1])) == 1      # T > max_prefill
+    # misaligned pointer (offset by one element) is rejected, not dereferenced
+    flat = torch.randn(256 * 2 * 64 + 8, device="cuda")
+    bad = flat[1:1 + 256 * 2 * 64].view(256, 2, 64)
+    assert _code(B, lambda: ctx.compress_prefill(0, 0, 1, 256, [bad, k1], [v0, v1])) == 1
+    # a good compress, then probe argument checks
+    ctx.compress_prefill(0, 0, 1, 256, [k0, k1], [v0, v1])
+    assert _code(B, lambda: ctx.probe(0, 0, 1, pq, [5, 5, 6, 7, 8, 9, 10, 11], 1.0)) == 1       # not strictly ascending
+    assert _code(B, lambda: ctx.probe(0, 0, 1, pq, list(range(249, 257)), 1.0)) == 1            # position >= T
+    assert _code(B, lambda: ctx.probe(0, 0, 1, pq, list(range(248, 256)), -1.0)) == 1           # negative lambda
+    # commit without modes
+    assert _code(B, lambda: ctx.commit(0)) == 5
+    assert _code(B, lambda: ctx.set_modes(0, [0, 3])) == 1                                       # mode out of range
+    ctx.set_modes(0, [1, 2])
+    ctx.commit(0)
+    assert _code(B, lambda: ctx.commit(0)) == 5                                                  # already committed
+    assert _code(B, lambda: ctx.decode_attn(0, torch.randn((2, 4, 64), device="cuda"))) == 5     # slot 1 not committed
+    assert _code(B, lambda: ctx.decode_attn(2, q)) == 1                                          # layer out of range
+    # the tail holds max_tail rows per layer; the next append is refused on the host
+    kn = torch.randn((1, 2, 64), device="cuda")
+    ctx.decode_attn(0, q, kn, kn)
+    ctx.decode_attn(0, q, kn, kn)
+    assert _code(B, lambda: ctx.decode_attn(0, q, kn, kn)) == 5
+    # still usable
+    out = ctx.decode_attn(1, q)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all()
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_arena_too_small_is_reported_at_commit():
+    B, _ = _ctx()
+    _.close()
+    cfg = B.Config(2, 4, 2, 64, 1, 4096, 1, B.F32, 1, 8)
+    worst, _w = B.sizes(cfg)
+    ctx = B.Context(cfg, arena_bytes=worst * 3 // 4)  # room for a shared-mode sequence, not for an exact-mode one
+    k0, k1, v0, v1 = _kv(T=4096)
+    ctx.compress_prefill(0, 0, 1, 4096, [k0, k1], [v0, v1])
+    ctx.set_modes(0, [2, 2])
+    with pytest.raises(B.FdkvError) as e:
+        ctx.commit(0)
+    assert e.value.code == 3
+    ctx.set_modes(0, [0, 0])
+    ctx.commit(0)  # the cheaper modes fit
+    by_mode, exact_equiv = ctx.footprint(0)
+    assert by_mode[0] == exact_equiv // 2 and by_mode[1] == by_mode[2] == 0
+    ctx.close()
+
+
+def test_reset_frees_the_arena():
+    B, ctx = _ctx()
+    k0, k1, v0, v1 = _kv()
+    for _ in range(3):
+        ctx.compress_prefill(0, 0, 1, 256, [k0, k1], [v0, v1])
+        ctx.set_modes(0, [2, 2])
+        ctx.commit(0)
+        assert ctx.get_modes(0).tolist() == [[2, 2]]
+        ctx.reset()
+    ctx.close()
