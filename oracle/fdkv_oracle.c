@@ -199,6 +199,18 @@ void fdkv_ref_omega(int64_t T, int64_t d, int64_t e_bytes, int64_t k, double* om
     omega[2] = b_ex / b_ex;
 }
 
+/* Same with the paper's token-granular residual (the paragraph before Eq. 3): the k_tok selected tokens keep all d
+ * high-frequency coefficients of K and of V, one int32 token index each (the set is shared by K and V):
+ *   residual 2*T*d*e + 2*k_tok*d*e + 4*k_tok.                                                                */
+void fdkv_ref_omega_tokens(int64_t T, int64_t d, int64_t e_bytes, int64_t k_tok, double* omega) {
+    double b_sh = 2.0 * (double)T * (double)d * (double)e_bytes;
+    double b_rs = b_sh + 2.0 * (double)k_tok * (double)d * (double)e_bytes + 4.0 * (double)k_tok;
+    double b_ex = 4.0 * (double)T * (double)d * (double)e_bytes;
+    omega[0] = b_sh / b_ex;
+    omega[1] = b_rs / b_ex;
+    omega[2] = b_ex / b_ex;
+}
+
 int fdkv_ref_mode(double e_shared, double e_residual, const double* omega, double lambda, double* loss_out,
                   double* margin_out) {
     double L[3];

@@ -28,6 +28,7 @@ _lib.fdkv_ref_select_entries.restype = _i64
 _lib.fdkv_ref_reconstruct.argtypes = [_f32p, _f32p, _i32p, _i64, _i64, C.c_int, C.c_int, _f32p, _f64p]
 _lib.fdkv_ref_probe_error.argtypes = [_f32p, _i32p, _i64, _i64, _i64, _f32p, _f32p, _i64, _i64, _i64, _i32p, _i64, _f64p]
 _lib.fdkv_ref_omega.argtypes = [_i64, _i64, _i64, _i64, _f64p]
+_lib.fdkv_ref_omega_tokens.argtypes = [_i64, _i64, _i64, _i64, _f64p]
 _lib.fdkv_ref_mode.argtypes = [C.c_double, C.c_double, _f64p, C.c_double, _f64p, C.POINTER(C.c_double)]
 _lib.fdkv_ref_mode.restype = C.c_int
 _lib.fdkv_ref_attention.argtypes = [_f64p, _f64p, _i64, _i64, _f32p, _f64p]
@@ -109,6 +110,18 @@ def omega(T: int, d: int, e_bytes: int, k: int) -> np.ndarray:
     return om
 
 
+def omega_tokens(T: int, d: int, e_bytes: int, k_tok: int) -> np.ndarray:
+    om = np.zeros(3, dtype=np.float64)
+    _lib.fdkv_ref_omega_tokens(T, d, e_bytes, k_tok, om)
+    return om
+
+
+def token_entries(tokens, d: int) -> np.ndarray:
+    """Flat entry indices t*d + ch of every channel of the given tokens (ascending when the tokens are)."""
+    t = np.asarray(tokens, dtype=np.int64)
+    return (t[:, None] * d + np.arange(d, dtype=np.int64)[None, :]).reshape(-1).astype(np.int32)
+
+
 def mode_rule(e_shared: float, e_residual: float, om, lam: float):
     loss = np.zeros(3, dtype=np.float64)
     margin = C.c_double(0.0)
@@ -145,18 +158,32 @@ def select_tokens(s, k_tok: int) -> np.ndarray:
 
 
 class Unit:
-    """Compressed state of one (pair, KV head): coefficients, kept sets, originals, and the exact tails."""
+    """Compressed state of one (pair, KV head): coefficients, kept sets, originals, and the exact tails.
 
-    def __init__(self, k0, k1, v0, v1, bf16: bool, keep_num: int, keep_den: int):
+    Entry rule (default): K and V each keep their k largest-magnitude Z1 entries.  Token rule (`tokens` given, or
+    chosen later with `use_tokens`): the listed tokens keep every Z1 coefficient of K and of V.
+    """
+
+    def __init__(self, k0, k1, v0, v1, bf16: bool, keep_num: int, keep_den: int, tokens=None, select: bool = True):
         self.x = {"k": (_c32(k0), _c32(k1)), "v": (_c32(v0), _c32(v1))}
         self.T, self.d = self.x["k"][0].shape
         self.bf16 = bf16
         self.k_keep = keep_count(self.T, self.d, keep_num, keep_den)
+        self.k_tok = (self.T * keep_num) // keep_den
         self.z0, self.z1, self.kept = {}, {}, {}
         for name in ("k", "v"):
             self.z0[name], self.z1[name] = depth_split(self.x[name][0], self.x[name][1], bf16)
-            self.kept[name] = select_entries(self.z1[name], self.k_keep)
+            if tokens is None and select:
+                self.kept[name] = select_entries(self.z1[name], self.k_keep)
         self.tail = {("k", 0): [], ("k", 1): [], ("v", 0): [], ("v", 1): []}
+        if tokens is not None:
+            self.use_tokens(tokens)
+
+    def use_tokens(self, tokens):
+        """Token rule: the same token set for K and V, all d coefficients of each."""
+        self.tokens = np.asarray(tokens, dtype=np.int32)
+        ent = token_entries(self.tokens, self.d)
+        self.kept = {"k": ent, "v": ent}
 
     def append(self, layer_in_pair: int, k_row, v_row):
         self.tail[("k", layer_in_pair)].append(_c32(k_row))

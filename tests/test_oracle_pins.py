@@ -335,3 +335,40 @@ def test_token_rule_vs_bruteforce_and_needles():
         order = np.lexsort((np.arange(w.T), -s))
         assert np.array_equal(tok, np.sort(order[: w.T // 8]))
         assert set(synth.needle_positions(w, 0, 0, h).tolist()) <= set(tok.tolist())
+
+
+# ---------------------------------------------------------------- token-granular residual (the paper's own rule)
+def test_token_rule_candidates_probe_and_attention_vs_bruteforce():
+    w = synth.WORKLOADS["tiny"]
+    pos = synth.probe_positions(w)
+    pq = (synth.probe_q(w, 0, 0), synth.probe_q(w, 0, 1))
+    h = 1
+    k0, k1 = synth.unit_tensor(w, 0, 0, h, False)
+    v0, v1 = synth.unit_tensor(w, 0, 0, h, True)
+    u = R.Unit(k0, k1, v0, v1, False, 1, 8, select=False)
+    s = R.token_scores(u.z1["k"], pq[0], pq[1], w.group, h, pos)
+    tok = R.select_tokens(s, u.k_tok)
+    assert tok.size == w.T // 8 and np.all(np.diff(tok) > 0)
+    u.use_tokens(tok)
+    mask = np.zeros((w.T, w.head_dim))
+    mask[tok] = 1.0  # Eq. 3's indicator 1[t in S]: whole rows
+    assert np.array_equal(np.flatnonzero(mask.ravel()), u.kept["k"])
+    e_sh, e_rs = R.probe_error(u.z1["k"], u.kept["k"], pq[0], pq[1], w.group, h, pos)
+    b_sh, b_rs = bf.probe_errors(u.z0["k"], u.z1["k"], mask, pq, w.group, h, pos)
+    assert e_sh == pytest.approx(b_sh, rel=1e-10) and e_rs == pytest.approx(b_rs, rel=1e-10)
+    assert e_rs < e_sh
+    Kc = bf.candidates(u.z0["k"], u.z1["k"], mask, (k0, k1))
+    Vc = bf.candidates(u.z0["v"], u.z1["v"], mask, (v0, v1))
+    q = synth.decode_q(w, 0, 1)[0][h * w.group:(h + 1) * w.group]
+    got = u.attend(R.RESIDUAL, 1, q)
+    for g in range(w.group):
+        np.testing.assert_allclose(got[g], bf.attention(Kc[1][1], Vc[1][1], q[g]), rtol=1e-10, atol=1e-12)
+    # memory cost of the token form: rows of K and V plus one index per token
+    om = R.omega_tokens(w.T, w.head_dim, 4, u.k_tok)
+    Td = w.T * w.head_dim
+    np.testing.assert_allclose(om, [0.5, (2 * Td * 4 + 2 * u.k_tok * w.head_dim * 4 + 4 * u.k_tok) / (4 * Td * 4), 1.0])
+    # keeping every token is lossless, keeping none is the shared cache
+    u.use_tokens(np.arange(w.T))
+    assert np.max(np.abs(u.rows("k", R.RESIDUAL, 1) - k1)) <= 2e-7 * np.max(np.abs(k1))
+    u.use_tokens(np.zeros(0, np.int32))
+    assert np.array_equal(u.rows("k", R.RESIDUAL, 0), u.rows("k", R.SHARED, 0))
