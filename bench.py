@@ -204,8 +204,14 @@ def run_ours(args, w):
     units = w.batch * w.n_pairs * w.n_kv_heads
     n_ut = 2 * units
     N = w.T * w.head_dim
-    compress_min_bytes = n_ut * (2 * N * esize + N * esize + w.k_keep * (4 + esize))
-    probe_flops = 2.0 * units * 2 * (2 * w.group * w.W) * w.T * w.head_dim
+    if w.residual_rule == 1:
+        # token rule: compression is the depth split alone (the probe selects); the probe runs three products
+        # (token scores, then the two candidates' errors)
+        compress_min_bytes = n_ut * (2 * N * esize + N * esize) + units * (2 * w.k_tok * w.head_dim * esize + 4 * w.k_tok)
+        probe_flops = 2.0 * units * 3 * (2 * w.group * w.W) * w.T * w.head_dim
+    else:
+        compress_min_bytes = n_ut * (2 * N * esize + N * esize + w.k_keep * (4 + esize))
+        probe_flops = 2.0 * units * 2 * (2 * w.group * w.W) * w.T * w.head_dim
     modes_all = np.stack([ctx.get_modes(b).numpy() for b in range(w.batch)])
     mix = [int((modes_all == m).sum()) for m in range(3)]
     torch.cuda.empty_cache()
@@ -354,7 +360,7 @@ def run_ours(args, w):
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "context": w.T, "batch": w.batch, "layers": w.n_layers, "q_heads": w.n_q_heads,
                    "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "keep": f"{w.keep_num}/{w.keep_den}",
-                   "mode_mix_shared_residual_exact": mix, "launch": "cuda_graph" if graph is not None else "stream",
+                   "residual_rule": "tokens" if w.residual_rule == 1 else "entries", "mode_mix_shared_residual_exact": mix, "launch": "cuda_graph" if graph is not None else "stream",
                    "l2": "inputs larger than L2 (each step streams the whole packed cache)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,

@@ -61,7 +61,20 @@ typedef struct {
     int32_t dtype;       /* fdkv_dtype: storage type of K, V, Q and of the stored coefficients         */
     int32_t keep_num;    /* residual keep fraction: k = floor(T * head_dim * keep_num / keep_den)      */
     int32_t keep_den;    /*   entries per (unit, K or V); 0 <= keep_num <= keep_den                    */
+    int32_t residual_rule; /* fdkv_residual_rule: how the sparse high-frequency residual is chosen     */
 } fdkv_config;
+
+/*
+ * FDKV_RESIDUAL_ENTRIES (default): the k largest-magnitude entries of Z1, K and V independently (chosen in
+ *   fdkv_compress_prefill; indices bit-reproducible).
+ * FDKV_RESIDUAL_TOKENS: the paper's rule (Method, the unnumbered score between Eq. 2 and Eq. 3): token t of a
+ *   unit is scored s_t = max over the pair's two layers, the group's query heads and the probe queries q with
+ *   probe_pos[q] >= t of | Q . (c * Z1K[t,:]) |; the k_tok = floor(T * keep_num / keep_den) tokens with the
+ *   largest score (ties: lowest t) keep ALL head_dim high-frequency coefficients of K and of V.  The scores
+ *   need the probe queries, so the set is chosen inside fdkv_probe (which is then mandatory before commit, even
+ *   when modes are overridden); Omega(residual) counts 2*k_tok*d*e + 4*k_tok bytes.  bf16, head_dim 128 only.
+ */
+typedef enum { FDKV_RESIDUAL_ENTRIES = 0, FDKV_RESIDUAL_TOKENS = 1 } fdkv_residual_rule;
 
 typedef struct fdkv_ctx fdkv_ctx;
 
@@ -149,6 +162,10 @@ fdkv_status fdkv_get_shared(fdkv_ctx* ctx, int32_t seq, int32_t pair, int32_t kv
 fdkv_status fdkv_get_residual(fdkv_ctx* ctx, int32_t seq, int32_t pair, int32_t kv_head, int32_t is_v,
                               int32_t* idx_out /*DEVICE [k]*/, void* val_out /*DEVICE [k] storage dtype*/,
                               int32_t* count_host /*HOST*/, void* stream);
+/* Token rule only: the selected tokens of a staged unit (ascending, DEVICE int32[k_tok], may be NULL), the scores of
+ * all T tokens (DEVICE float[T], may be NULL) and the count (HOST).  Valid after fdkv_probe.  Synchronous.          */
+fdkv_status fdkv_get_token_set(fdkv_ctx* ctx, int32_t seq, int32_t pair, int32_t kv_head, int32_t* tok_out,
+                               float* score_out, int32_t* count_host /*HOST*/, void* stream);
 /* Modes of a committed (or mode-overridden) sequence: HOST int32[n_layers/2][n_kv_heads]. */
 fdkv_status fdkv_get_modes(fdkv_ctx* ctx, int32_t seq, int32_t* modes_host /*HOST*/);
 /* Bytes a committed sequence holds in the arena per mode, and what the uncompressed cache would take. */

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libfdkv.so")
 
 F32, BF16 = 0, 1
 SHARED, RESIDUAL, EXACT = 0, 1, 2
+RESIDUAL_ENTRIES, RESIDUAL_TOKENS = 0, 1
 _STATUS = ["ok", "invalid argument", "unsupported", "arena full", "workspace too small", "state", "cuda error",
            "device timeout", "device check failed", "too large for the built-in scratch"]
 NOALLOC_MAX_ELEMS = 1 << 20
@@ -30,7 +31,7 @@ class FdkvError(RuntimeError):
 
 class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "max_batch", "max_prefill",
-                                         "max_tail", "dtype", "keep_num", "keep_den")]
+                                         "max_tail", "dtype", "keep_num", "keep_den", "residual_rule")]
 
 
 def _load():
@@ -54,6 +55,7 @@ def _load():
         "fdkv_get_shared": [vp, i32, i32, i32, i32, vp, vp],
         "fdkv_get_residual": [vp, i32, i32, i32, i32, vp, vp, P(i32), vp],
         "fdkv_get_modes": [vp, i32, P(i32)],
+        "fdkv_get_token_set": [vp, i32, i32, i32, vp, vp, P(i32), vp],
         "fdkv_footprint": [vp, i32, P(sz), P(sz)],
         "fdkv_decode_bytes": [vp, i32, i32, P(sz)],
         "fdkv_device_status": [vp],
@@ -95,6 +97,7 @@ class Config:
     dtype: int
     keep_num: int
     keep_den: int
+    residual_rule: int = 0  # 0: largest-magnitude entries; 1: the paper's probe-scored tokens
 
     def c(self) -> _Config:
         return _Config(*(int(getattr(self, f[0])) for f in _Config._fields_))
@@ -242,6 +245,16 @@ class Context:
         _check(_lib.fdkv_get_residual(self.h, seq, pair, kv_head, int(is_v), _ptr(idx), _ptr(val), C.byref(cnt),
                                       _stream(stream)), "fdkv_get_residual")
         return idx, val
+
+    def get_token_set(self, seq, pair, kv_head, T, stream=None):
+        """Token rule: (selected tokens int32 [k_tok] ascending, scores float32 [T]) of a staged, probed unit."""
+        cnt = C.c_int32(0)
+        _check(_lib.fdkv_get_token_set(self.h, seq, pair, kv_head, None, None, C.byref(cnt), _stream(stream)), "fdkv_get_token_set")
+        tok = torch.empty(cnt.value, dtype=torch.int32, device=self.device)
+        score = torch.empty(T, dtype=torch.float32, device=self.device)
+        _check(_lib.fdkv_get_token_set(self.h, seq, pair, kv_head, _ptr(tok), _ptr(score), C.byref(cnt), _stream(stream)),
+               "fdkv_get_token_set")
+        return tok, score
 
     def get_modes(self, seq):
         n = self.n_pairs * self.cfg.n_kv_heads

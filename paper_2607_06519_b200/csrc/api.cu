@@ -44,6 +44,11 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.ntiles_max = (s.Tmax + kResTile - 1) / kResTile;
     s.nptiles_max = (s.Tmax + kProbeTile - 1) / kProbeTile;
     s.tail_rows = (s.max_tail + kRowPad - 1) / kRowPad * kRowPad;
+    if (c.residual_rule != FDKV_RESIDUAL_ENTRIES && c.residual_rule != FDKV_RESIDUAL_TOKENS) return false;
+    s.tok_rule = c.residual_rule == FDKV_RESIDUAL_TOKENS;
+    if (s.tok_rule && !(c.dtype == FDKV_BF16 && c.head_dim == 128)) return false;  // tensor-core kernels only
+    s.ktok_max = (int64_t)s.Tmax * s.keep_num / s.keep_den;
+    s.ktok_cap = (int64_t)align_up((size_t)(s.ktok_max + 32), 64);
     s.NU = s.P * s.Hkv;
     s.NT = 2 * s.NU;
     return true;
@@ -65,6 +70,10 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.idx = take((size_t)s.NT * s.kcap * 4);
     w.val = take((size_t)s.NT * s.kcap * s.esize);
     w.packed = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NT * s.kcap * 4 : 0);
+    w.tok_score = take(s.tok_rule ? (size_t)s.NU * s.Tmax * 4 : 0);
+    w.tok_flag = take(s.tok_rule ? (size_t)s.NU * s.Tmax : 0);
+    w.tok_list = take(s.tok_rule ? (size_t)s.NU * s.ktok_cap * 4 : 0);
+    w.tok_off = take(s.tok_rule ? (size_t)s.NU * (s.ntiles_max + 1) * 4 : 0);
     w.probe_part = take((size_t)s.NU * s.nptiles_max * 16);
     w.probe_pos = take((size_t)kMaxW * 4 + (size_t)s.L * 8);
     w.scores = take((size_t)s.NU * 16);
@@ -86,8 +95,11 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     a.bump = o;
     const size_t rows_pad = align_up((size_t)((s.Tmax + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize);
     const size_t exact_unit = 4 * rows_pad;
-    const size_t resid_unit = 2 * rows_pad + 2 * align_up((size_t)s.kcap * 4) +
-                              2 * align_up((size_t)s.kcap * s.esize) + 2 * align_up((size_t)(s.ntiles_max + 1) * 4);
+    const size_t resid_unit = s.tok_rule
+                                  ? 2 * rows_pad + 2 * align_up((size_t)s.ktok_cap * s.d * s.esize) + align_up((size_t)s.ktok_cap * 4) +
+                                        align_up((size_t)(s.ntiles_max + 1) * 4)
+                                  : 2 * rows_pad + 2 * align_up((size_t)s.kcap * 4) + 2 * align_up((size_t)s.kcap * s.esize) +
+                                        2 * align_up((size_t)(s.ntiles_max + 1) * 4);
     a.worst_total = a.bump + (size_t)s.max_batch * s.NU * (exact_unit > resid_unit ? exact_unit : resid_unit);
 }
 
@@ -140,6 +152,7 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     c->bump = c->ar.bump;
     c->pair_compressed.assign(s.P, 0);
     c->pair_probed.assign(s.P, 0);
+    c->pair_scored.assign(s.P, 0);
     c->k_layers.assign(s.L, nullptr);
     c->v_layers.assign(s.L, nullptr);
     c->seqs.resize(s.max_batch);
@@ -154,9 +167,14 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     if (e != cudaSuccess) { delete c; return cuda_fail(e); }
     if (s.dtype == FDKV_BF16 && s.d == 128) c->has_tmap = make_arena_tensor_map(c->arena, arena_bytes, c->tmap);
     c->packed_lists = c->has_tmap && s.max_batch * s.Hkv <= kFastMaxUnits;
+    if (s.tok_rule) {
+        const bool ok = c->packed_lists && make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
+        if (!ok) { delete c; return FDKV_ERR_UNSUPPORTED; }
+    }
     if (s.dtype == FDKV_BF16 && s.d == 128)
         c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_z1) &&
                              make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_drop);
+    if (s.tok_rule && !c->has_probe_tmaps) { delete c; return FDKV_ERR_UNSUPPORTED; }
     *out = c;
     return FDKV_OK;
 }
@@ -198,6 +216,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
         c->staged_T = T;
         std::fill(c->pair_compressed.begin(), c->pair_compressed.end(), 0);
         std::fill(c->pair_probed.begin(), c->pair_probed.end(), 0);
+        std::fill(c->pair_scored.begin(), c->pair_scored.end(), 0);
         c->modes_overridden = false;
         c->seqs[seq].modes.assign(s.NU, -1);
         c->stride_t = stride_t;
@@ -242,8 +261,8 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     sa.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
     sa.z1drop = c->has_probe_tmaps ? c->work + c->ws.z1drop : nullptr;
     sa.status = wsp<int32_t>(c, c->ws.status);
-    CU(launch_select_and_compact(sa, s.dtype, st));
-    for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; }
+    if (!s.tok_rule) CU(launch_select_and_compact(sa, s.dtype, st));  // the token rule selects inside fdkv_probe
+    for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; c->pair_scored[p] = 0; }
     return FDKV_OK;
 }
 
@@ -283,7 +302,9 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     a.lambda = lambda;
     const double e = s.esize, Td = (double)T * s.d;
     const double k = (double)((int64_t)T * s.d * s.keep_num / s.keep_den);
-    const double b_sh = 2.0 * Td * e, b_rs = b_sh + 2.0 * k * (e + 4.0), b_ex = 4.0 * Td * e;
+    const double k_tok = (double)((int64_t)T * s.keep_num / s.keep_den);
+    const double b_sh = 2.0 * Td * e, b_ex = 4.0 * Td * e;
+    const double b_rs = s.tok_rule ? b_sh + 2.0 * k_tok * s.d * e + 4.0 * k_tok : b_sh + 2.0 * k * (e + 4.0);
     a.omega[0] = b_sh / b_ex; a.omega[1] = b_rs / b_ex; a.omega[2] = 1.0;
     a.modes_out = modes; a.scores_out = scores;
     a.tmap_z1 = c->has_probe_tmaps ? c->tmap_z1 : nullptr;
@@ -291,6 +312,20 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     a.Tmax = s.Tmax;
     a.pos_host = probe_pos;
     a.status = wsp<int32_t>(c, c->ws.status);
+    if (s.tok_rule) {
+        TokenArgs t;
+        t.unit_begin = a.unit_begin; t.unit_count = a.unit_count;
+        t.T = T; t.Tmax = s.Tmax; t.Hq = s.Hq; t.Hkv = s.Hkv; t.G = s.G; t.W = W; t.ntiles_max = s.ntiles_max;
+        t.k_tok = (int64_t)T * s.keep_num / s.keep_den; t.ktok_cap = s.ktok_cap; t.unit_stride = (int64_t)s.Tmax * s.d;
+        t.z1 = c->work + c->ws.z1; t.z1drop = c->work + c->ws.z1drop;
+        t.q_layers_dev = qptr_dev; t.pos = pos_dev; t.pos_host = probe_pos;
+        t.score = wsp<uint32_t>(c, c->ws.tok_score); t.flag = wsp<uint8_t>(c, c->ws.tok_flag);
+        t.list = wsp<int32_t>(c, c->ws.tok_list); t.off = wsp<int32_t>(c, c->ws.tok_off);
+        t.tmap_z1_128 = c->tmap_z1_128;
+        t.status = wsp<int32_t>(c, c->ws.status);
+        CU(launch_token_select(t, st));
+        for (int p = pb; p < pe; ++p) c->pair_scored[p] = 1;
+    }
     CU(launch_probe(a, s.dtype, st));
     for (int p = pb; p < pe; ++p) c->pair_probed[p] = 1;
     return FDKV_OK;
@@ -311,7 +346,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     if (c->staged_seq != seq || c->seqs[seq].committed) return FDKV_ERR_STATE;
     const Shape& s = c->s;
     for (int p = 0; p < s.P; ++p)
-        if (!c->pair_compressed[p] || (!c->modes_overridden && !c->pair_probed[p])) return FDKV_ERR_STATE;
+        if (!c->pair_compressed[p] || (!c->modes_overridden && !c->pair_probed[p]) || (s.tok_rule && !c->pair_scored[p]))
+            return FDKV_ERR_STATE;
     cudaStream_t st = S(stream);
     SeqState& q = c->seqs[seq];
     CU(cudaStreamSynchronize(st));
@@ -325,11 +361,14 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     // list copies include the slack so that aligned over-reads of the last tile stay inside the allocation
     const size_t idx_b = (size_t)(k + kListPad) * 4, off_b = (size_t)(ntiles + 1) * 4;
     const size_t val_b = c->packed_lists ? 0 : (size_t)(k + kListPad) * s.esize;  // packed entries carry their value
+    const int64_t k_tok = (int64_t)T * s.keep_num / s.keep_den;
+    const size_t trow_b = (size_t)(k_tok + 4) * s.d * s.esize, tlist_b = (size_t)(k_tok + 32) * 4;  // token rows, token list
     size_t need = 0;
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u];
         if (m < 0 || m > 2) return FDKV_ERR_STATE;
         if (m == FDKV_MODE_EXACT) need += 4 * align_up(rows_pad);
+        else if (s.tok_rule) need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * align_up(trow_b) + align_up(tlist_b) + align_up(off_b) : 0);
         else need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * (align_up(idx_b) + align_up(val_b) + align_up(off_b)) : 0);
     }
     if (c->bump + need > c->arena_bytes) return FDKV_ERR_ARENA_FULL;
@@ -360,6 +399,14 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
             d0->v_rows = dst[2]; d1->v_rows = dst[3];
             by_mode[2] += 4 * rows;
         } else {
+            char *tl = nullptr, *to = nullptr;
+            if (s.tok_rule && m == FDKV_MODE_RESIDUAL) {  // one token list and one offset table serve K and V
+                tl = take(tlist_b);
+                to = take(off_b);
+                CU(cudaMemcpyAsync(tl, c->work + c->ws.tok_list + (size_t)u * s.ktok_cap * 4, (size_t)k_tok * 4, cudaMemcpyDeviceToDevice, st));
+                CU(cudaMemcpyAsync(to, c->work + c->ws.tok_off + (size_t)u * (s.ntiles_max + 1) * 4, off_b, cudaMemcpyDeviceToDevice, st));
+                by_mode[1] += (size_t)k_tok * 4;
+            }
             for (int is_v = 0; is_v < 2; ++is_v) {
                 const size_t ut = (size_t)u * 2 + is_v;
                 char* z0 = take(rows_pad);
@@ -368,7 +415,17 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 (is_v ? d0->v_rows : d0->k_rows) = z0;
                 (is_v ? d1->v_rows : d1->k_rows) = z0;
                 by_mode[m] += rows;
-                if (m == FDKV_MODE_RESIDUAL) {
+                if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
+                    char* rows_res = take(trow_b);
+                    CU(launch_token_gather(c->work + c->ws.z1 + ut * unit_stride_b, (const int32_t*)tl, k_tok, rows_res, st));
+                    for (UnitDesc* d : {d0, d1}) {
+                        d->res_kind = 1;
+                        d->k_idx = (const int32_t*)tl;
+                        d->k_off = (const int32_t*)to;
+                        (is_v ? d->v_val : d->k_val) = rows_res;
+                    }
+                    by_mode[1] += (size_t)k_tok * s.d * s.esize;
+                } else if (m == FDKV_MODE_RESIDUAL) {
                     char* pi = take(idx_b);
                     char* pv = val_b ? take(val_b) : nullptr;
                     char* po = take(off_b);
@@ -425,6 +482,7 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
     a.arena_base = c->arena;
     a.keep_num = s.keep_num; a.keep_den = s.keep_den;
     a.packed_lists = c->packed_lists ? 1 : 0;
+    a.tok_rule = s.tok_rule;
     a.desc = arp<UnitDesc>(c, c->ar.desc);
     a.L = s.L; a.layer = layer; a.batch = batch; a.Hq = s.Hq; a.Hkv = s.Hkv; a.G = s.G; a.d = s.d;
     a.max_tail = s.max_tail; a.max_batch = s.max_batch; a.Tmax_batch = Tmax;
@@ -496,11 +554,27 @@ fdkv_status fdkv_get_residual(fdkv_ctx* c, int32_t seq, int32_t pair, int32_t h,
     if (!seq_ok(c, seq) || pair < 0 || pair >= c->s.P || h < 0 || h >= c->s.Hkv) return FDKV_ERR_INVALID_ARG;
     if (c->staged_seq != seq || !c->pair_compressed[pair]) return FDKV_ERR_STATE;
     const Shape& s = c->s;
+    if (s.tok_rule) return FDKV_ERR_UNSUPPORTED;  // token rule: see fdkv_get_token_set
     const size_t ut = ((size_t)pair * s.Hkv + h) * 2 + (is_v ? 1 : 0);
     const int64_t k = (int64_t)c->staged_T * s.d * s.keep_num / s.keep_den;
     if (count_host) *count_host = (int32_t)k;
     if (idx_out && k) CU(cudaMemcpyAsync(idx_out, c->work + c->ws.idx + ut * s.kcap * 4, (size_t)k * 4, cudaMemcpyDeviceToDevice, S(stream)));
     if (val_out && k) CU(cudaMemcpyAsync(val_out, c->work + c->ws.val + ut * s.kcap * s.esize, (size_t)k * s.esize, cudaMemcpyDeviceToDevice, S(stream)));
+    CU(cudaStreamSynchronize(S(stream)));
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_get_token_set(fdkv_ctx* c, int32_t seq, int32_t pair, int32_t h, int32_t* tok_out, float* score_out,
+                               int32_t* count_host, void* stream) {
+    if (!seq_ok(c, seq) || pair < 0 || pair >= c->s.P || h < 0 || h >= c->s.Hkv) return FDKV_ERR_INVALID_ARG;
+    const Shape& s = c->s;
+    if (!s.tok_rule) return FDKV_ERR_UNSUPPORTED;
+    if (c->staged_seq != seq || !c->pair_scored[pair]) return FDKV_ERR_STATE;
+    const size_t u = (size_t)pair * s.Hkv + h;
+    const int64_t k_tok = (int64_t)c->staged_T * s.keep_num / s.keep_den;
+    if (count_host) *count_host = (int32_t)k_tok;
+    if (tok_out && k_tok) CU(cudaMemcpyAsync(tok_out, c->work + c->ws.tok_list + u * s.ktok_cap * 4, (size_t)k_tok * 4, cudaMemcpyDeviceToDevice, S(stream)));
+    if (score_out) CU(cudaMemcpyAsync(score_out, c->work + c->ws.tok_score + u * s.Tmax * 4, (size_t)c->staged_T * 4, cudaMemcpyDeviceToDevice, S(stream)));
     CU(cudaStreamSynchronize(S(stream)));
     return FDKV_OK;
 }
@@ -534,7 +608,11 @@ fdkv_status fdkv_decode_bytes(fdkv_ctx* c, int32_t layer, int32_t batch, size_t*
         for (int h = 0; h < s.Hkv; ++h) {
             const int m = q.modes[(layer / 2) * s.Hkv + h];
             tot += 2 * (size_t)(q.T + q.tail_len[layer]) * s.d * s.esize;
-            if (m == FDKV_MODE_RESIDUAL) tot += 2 * ((size_t)k * (c->packed_lists ? 4 : 4 + s.esize) + (size_t)(ntiles + 1) * 4);
+            if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
+                const size_t kt = (size_t)((int64_t)q.T * s.keep_num / s.keep_den);
+                tot += 2 * kt * s.d * s.esize + kt * 4 + (size_t)(ntiles + 1) * 4;
+            } else if (m == FDKV_MODE_RESIDUAL)
+                tot += 2 * ((size_t)k * (c->packed_lists ? 4 : 4 + s.esize) + (size_t)(ntiles + 1) * 4);
         }
     }
     *bytes_host = tot;

@@ -103,6 +103,9 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ void st_shared_u16(uint32_t addr, uint16_t v) {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
 }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 __device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
 }
@@ -310,12 +313,19 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             const uint32_t* v_ent = reinterpret_cast<const uint32_t*>(ud.v_idx);
             int cr[4] = {0, 0, 0, 0}, nr[4] = {0, 0, 0, 0};  // {k begin, k end, v begin, v end}
             uint32_t pke[kPF], pve[kPF];
+            // token-granular residual: one ascending token list (k_idx) with per-slice counts (k_off) for K and V,
+            // and the selected tokens' Z1 rows packed densely (k_val / v_val, 256 bytes each)
+            const bool tokmode = resid && ud.res_kind == 1;
+            const uint4* t_krows = reinterpret_cast<const uint4*>(ud.k_val);
+            const uint4* t_vrows = reinterpret_cast<const uint4*>(ud.v_val);
+            int ptk[2] = {0, 0}, ptv[2] = {0, 0};
             auto load_ranges = [&](int j, int (&r)[4]) {
                 if (resid && j < npre) {
                     const int o = (rev ? tb + npre - 1 - j : tb + j) * (kTT / kResTile) + warp;
                     const int o0 = min(o, nres), o1 = min(o + 1, nres);
                     r[0] = ud.k_off[o0]; r[1] = ud.k_off[o1];
-                    r[2] = ud.v_off[o0]; r[3] = ud.v_off[o1];
+                    if (tokmode) { r[2] = r[0]; r[3] = r[1]; }
+                    else { r[2] = ud.v_off[o0]; r[3] = ud.v_off[o1]; }
                 } else {
                     r[0] = r[1] = r[2] = r[3] = 0;
                 }
@@ -339,6 +349,34 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     st_shared_u16(scratch + ((w >> 16) << 1), (uint16_t)(w & 0xFFFFu));
                 }
             };
+            // token rows: two tokens per round (half a warp each, 16 bytes per lane), two rounds in registers
+            auto prefetch_tok = [&](const uint4* rows, int e0, int e1, uint32_t (&pe)[kPF], int (&pt)[2]) {
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int j = e0 + 2 * r + (lane >> 4);
+                    if (j < e1) {
+                        const uint4 v = rows[(int64_t)j * 16 + (lane & 15)];
+                        pe[4 * r] = v.x; pe[4 * r + 1] = v.y; pe[4 * r + 2] = v.z; pe[4 * r + 3] = v.w;
+                        pt[r] = k_ent[j];  // the token list sits where the packed layout keeps the K entries
+                    }
+                }
+            };
+            auto scatter_tok = [&](const uint4* rows, int e0, int e1, const uint32_t (&pe)[kPF], const int (&pt)[2]) {
+                const int chunk = lane & 15;
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int j = e0 + 2 * r + (lane >> 4);
+                    if (j < e1) {
+                        const int row = pt[r] & 15;
+                        st_shared_v4(scratch + (chunk >> 3) * 2048 + swz(row, chunk), pe[4 * r], pe[4 * r + 1], pe[4 * r + 2], pe[4 * r + 3]);
+                    }
+                }
+                for (int j = e0 + 4 + (lane >> 4); j < e1; j += 2) {  // more than four selected tokens in the slice
+                    const int row = (int)k_ent[j] & 15;
+                    const uint4 v = rows[(int64_t)j * 16 + chunk];
+                    st_shared_v4(scratch + (chunk >> 3) * 2048 + swz(row, chunk), v.x, v.y, v.z, v.w);
+                }
+            };
             auto zero_scratch = [&]() {
 #pragma unroll
                 for (int i = 0; i < kScratchBytes / 16 / 32; ++i) st_shared_zero16(scratch + (lane + 32 * i) * 16);
@@ -346,8 +384,13 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             if (resid) {
                 load_ranges(0, cr);
                 load_ranges(1, nr);
-                prefetch(k_ent, cr[0], cr[1], pke);
-                prefetch(v_ent, cr[2], cr[3], pve);
+                if (tokmode) {
+                    prefetch_tok(t_krows, cr[0], cr[1], pke, ptk);
+                    prefetch_tok(t_vrows, cr[2], cr[3], pve, ptv);
+                } else {
+                    prefetch(k_ent, cr[0], cr[1], pke);
+                    prefetch(v_ent, cr[2], cr[3], pve);
+                }
             }
 
             for (int j = 0; j < nseg; ++j) {
@@ -367,10 +410,12 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 __syncwarp();
 
                 if (with_res && cr[1] > cr[0]) {
-                    scatter(k_ent, cr[0], cr[1], pke);
+                    if (tokmode) scatter_tok(t_krows, cr[0], cr[1], pke, ptk);
+                    else scatter(k_ent, cr[0], cr[1], pke);
                     __syncwarp();
                 }
-                if (resid) prefetch(k_ent, nr[0], nr[1], pke);
+                if (tokmode) prefetch_tok(t_krows, nr[0], nr[1], pke, ptk);
+                else if (resid) prefetch(k_ent, nr[0], nr[1], pke);
 
 #ifdef FDKV_TIMING
                 const long long tw0 = clock64();
@@ -423,10 +468,12 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     }
                 }
                 if (with_res && cr[3] > cr[2]) {
-                    scatter(v_ent, cr[2], cr[3], pve);
+                    if (tokmode) scatter_tok(t_vrows, cr[2], cr[3], pve, ptv);
+                    else scatter(v_ent, cr[2], cr[3], pve);
                     __syncwarp();
                 }
-                if (resid) prefetch(v_ent, nr[2], nr[3], pve);
+                if (tokmode) prefetch_tok(t_vrows, nr[2], nr[3], pve, ptv);
+                else if (resid) prefetch(v_ent, nr[2], nr[3], pve);
 
                 // ---- online softmax for head gid over this slice's 16 tokens (4 per thread) ----
                 float p[2][2];
@@ -717,7 +764,10 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         // cost per tile: bytes in units of 512 B (the K and V boxes, plus the lists' share for residual units),
         // residual tiles scaled by the measured ratio of their compute time to a plain tile's
         wt[u] = 2 * kTT * 256 / 512;
-        if (a.host_modes[u] == FDKV_MODE_RESIDUAL) wt[u] = (int)((wt[u] + (2 * k * 4 / nt[u] + 511) / 512) * res_cost);
+        if (a.host_modes[u] == FDKV_MODE_RESIDUAL) {
+            const int64_t res_bytes = a.tok_rule ? 2 * ((int64_t)T * a.keep_num / a.keep_den) * 260 : 2 * k * 4;  // rows + index, or packed entries
+            wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * res_cost);
+        }
         wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
         total_tiles += nt[u];
     }

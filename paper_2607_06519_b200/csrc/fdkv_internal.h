@@ -44,7 +44,7 @@ struct UnitDesc {
     int32_t mode;
     int32_t T;
     float sign;  // +1 for the first layer of the pair, -1 for the second
-    int32_t pad;
+    int32_t res_kind;  // residual layout: 0 packed entries (k_idx / v_idx), 1 token rows (k_idx = token list, k_val / v_val = rows, k_off = per-slice counts)
 };
 
 struct SelState {
@@ -65,9 +65,12 @@ struct Shape {
     int nptiles_max;   // ceil(Tmax/kProbeTile)
     int NU, NT;        // units and unit-tensors (K and V) of one sequence
     int tail_rows;     // max_tail rounded up to kRowPad
+    int tok_rule;      // 1: token-granular residual chosen by the probe
+    int64_t ktok_max, ktok_cap;  // floor(Tmax*num/den) and the list capacity incl. slack
 };
 
 struct WsLayout {
+    size_t tok_score, tok_flag, tok_list, tok_off;
     size_t status, z0, z1, z1drop, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
         partials, counters, io_q, io_k, io_v, io_out, total;
 };
@@ -107,6 +110,8 @@ struct fdkv_ctx {
     bool has_tmap = false;
     alignas(64) unsigned char tmap_z1[128], tmap_drop[128];  // probe operands (bf16, head_dim 128 only)
     bool has_probe_tmaps = false;
+    alignas(64) unsigned char tmap_z1_128[128];  // staged Z1 with 128-token boxes (token-score kernel)
+    std::vector<uint8_t> pair_scored;            // token rule: the probe has chosen this pair's token sets
     bool packed_lists = false;              // decode runs the bf16 / head_dim 128 kernel on packed residual entries
 };
 
@@ -188,6 +193,7 @@ struct DecodeArgs {
     const void* arena_base;
     int keep_num, keep_den;
     int packed_lists;
+    int tok_rule;
     int32_t* tail_len;      // [L][max_batch]
     float* partials;        // [batch][Hq][kMaxSplits][d+4]: max, sum, 2 pad, d accumulators
     int32_t* counters;      // [max_batch][Hkv] split-K arrival tickets, zero between launches
@@ -199,6 +205,26 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out);
 // Same view ([rows][128] bf16, 64-channel x box_rows boxes, 128-byte swizzle) over any 256-byte aligned region.
 bool make_rows_tensor_map(void* base, size_t bytes, int box_rows, void* tmap_out);
 cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st);
+
+// ---- token-granular residual (token_rule.cu) ----
+struct TokenArgs {
+    int unit_begin, unit_count;
+    int T, Tmax, Hq, Hkv, G, W, ntiles_max;
+    int64_t k_tok, ktok_cap, unit_stride;
+    const void* z1;                    // staged Z1 (K of unit u at unit-tensor 2u)
+    void* z1drop;                      // [unit][Tmax*128] Z1 of K with the selected rows zeroed
+    const void* const* q_layers_dev;
+    const int32_t* pos;
+    const int32_t* pos_host;
+    uint32_t* score;                   // [unit][Tmax] float bits (non-negative)
+    uint8_t* flag;                     // [unit][Tmax]
+    int32_t* list;                     // [unit][ktok_cap]
+    int32_t* off;                      // [unit][ntiles_max + 1]
+    const void* tmap_z1_128;
+    int32_t* status;
+};
+cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st);
+cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, cudaStream_t st);
 
 void count_launch(int n);
 // Remembers a failed CUDA runtime call for fdkv_last_cuda_error() and returns FDKV_ERR_CUDA.

@@ -21,7 +21,7 @@ def make_context(w: synth.Workload, max_tail: int | None = None, arena_bytes: in
                  device="cuda:0") -> B.Context:
     cfg = B.Config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, w.T,
                    max_tail if max_tail is not None else max(w.n_steps, 1), B.BF16 if w.dtype == "bf16" else B.F32,
-                   w.keep_num, w.keep_den)
+                   w.keep_num, w.keep_den, w.residual_rule)
     return B.Context(cfg, device=device, arena_bytes=arena_bytes)
 
 
@@ -78,6 +78,8 @@ class Prefilled:
             elif modes != "probe":
                 raise ValueError(modes)
         else:
+            if self.w.residual_rule == 1:
+                self.probe(seq, lam)  # the token rule chooses its sets inside the probe
             self.ctx.set_modes(seq, np.asarray(modes, dtype=np.int32))
         self.commit(seq)
         return self.ctx.get_modes(seq).numpy()

@@ -46,6 +46,7 @@ class Workload:
     fixed_rho: float | None = None
     n_steps: int = 1
     seq_seeds: tuple | None = None  # per-sequence seed override (batched workload)
+    residual_rule: int = 0  # 0: largest-magnitude entries; 1: probe-scored tokens (the paper's rule)
 
     @property
     def n_pairs(self) -> int:
@@ -54,6 +55,10 @@ class Workload:
     @property
     def group(self) -> int:
         return self.n_q_heads // self.n_kv_heads
+
+    @property
+    def k_tok(self) -> int:
+        return (self.T * self.keep_num) // self.keep_den
 
     @property
     def k_keep(self) -> int:
@@ -91,6 +96,9 @@ WORKLOADS = {
 # device; used for profiler captures and quick checks
 WORKLOADS["decode32k_4l"] = WORKLOADS["decode32k"].scaled(n_layers=4, name="decode32k_4l")
 WORKLOADS["decode128k_4l"] = WORKLOADS["decode128k"].scaled(n_layers=4, name="decode128k_4l")
+# the same 32k workload with the paper's token-granular residual (probe-scored tokens keep whole rows)
+WORKLOADS["decode32k_tok"] = WORKLOADS["decode32k"].scaled(residual_rule=1, name="decode32k_tok")
+WORKLOADS["decode32k_tok_4l"] = WORKLOADS["decode32k_tok"].scaled(n_layers=4, name="decode32k_tok_4l")
 
 
 def rng(seed: int, seq: int, a: int, b: int, tag: int) -> np.random.Generator:

@@ -123,3 +123,49 @@ def test_batch8_decode_with_tail_appends():
     assert worst <= TOL["bf16"], worst
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_decode32k_token_rule():
+    """The 32k benchmark shape with the paper's token-granular residual: token sets by score band, probe errors and
+    attention on the GPU's own sets, sampled units."""
+    from paper_2607_06519_b200 import runner
+
+    w = synth.WORKLOADS["decode32k_tok"]
+    sample = [(0, 2, 1), (0, 11, 6)]
+    pf = runner.Prefilled(w, max_tail=1)
+    pf.compress(0)
+    pmodes, scores = pf.probe(0, 0.0)
+    pos = synth.probe_positions(w)
+    units = {}
+    for (b, p, h) in sample:
+        k0, k1 = synth.unit_tensor(w, 0, p, h, False)
+        v0, v1 = synth.unit_tensor(w, 0, p, h, True)
+        u = R.Unit(k0, k1, v0, v1, True, w.keep_num, w.keep_den, select=False)
+        pq = (synth.probe_q(w, 0, 2 * p), synth.probe_q(w, 0, 2 * p + 1))
+        tok, sc = pf.ctx.get_token_set(0, p, h, w.T)
+        tok, sc = tok.cpu().numpy(), f32(sc).astype(np.float64)
+        s_ref = R.token_scores(u.z1["k"], pq[0], pq[1], w.group, h, pos)
+        np.testing.assert_allclose(sc, s_ref, rtol=1e-5, atol=1e-6 * s_ref.max())
+        kth = np.sort(s_ref)[::-1][w.k_tok - 1]
+        assert tok.size == w.k_tok and np.all(np.diff(tok) > 0)
+        assert set(np.flatnonzero(s_ref > kth * (1 + 2e-5)).tolist()) <= set(tok.tolist()) <= set(np.flatnonzero(s_ref >= kth * (1 - 2e-5)).tolist())
+        assert set(synth.needle_positions(w, 0, p, h).tolist()) <= set(tok.tolist())  # the planted needles are all kept
+        u.use_tokens(tok)
+        e = R.probe_error(u.z1["k"], u.kept["k"], pq[0], pq[1], w.group, h, pos)
+        np.testing.assert_allclose(scores[p, h], e, rtol=1e-4)
+        units[(b, p, h)] = u
+    modes = synth.quota_modes(scores[..., 0])
+    for (b, p, h) in sample:
+        modes[p, h] = 1  # make sure the sampled units exercise the residual path
+    pf.ctx.set_modes(0, modes)
+    pf.commit(0)
+    worst = 0.0
+    for layer in range(w.n_layers):
+        q = pf.decode_q(layer, 0)
+        out = pf.ctx.decode_attn(layer, q)
+        torch.cuda.synchronize()
+        assert torch.isfinite(out.float()).all()
+        worst = max(worst, _check_layer(pf, w, layer, 0, units, [modes], q, out))
+    assert worst <= TOL["bf16"], worst
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
