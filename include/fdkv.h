@@ -124,6 +124,20 @@ fdkv_status fdkv_probe(fdkv_ctx* ctx, int32_t seq, int32_t pair_begin, int32_t p
                        const void* const* q_layers /*HOST*/, const int32_t* probe_pos /*HOST*/, int32_t W,
                        double lambda, int32_t* modes, float* scores, void* stream);
 
+/*
+ * Budgeted routing (Method: the memory budget is enforced by increasing lambda until the estimated KV footprint fits).
+ * Uses the probe errors fdkv_probe left for the staged sequence (every pair must have been probed; waits for the
+ * stream) and finds the smallest lambda >= 0 whose routing -- mode = argmin E(m) + lambda * Omega(m) per unit, ties to
+ * the lowest id -- has sum over units of Omega(mode) * bytes(exact) <= budget_bytes.  The footprint can only change
+ * where two of a unit's loss lines cross, so the candidates are 0 and every crossing, ascending; each is tried at
+ * crossing * (1 + 2^-40).  The modes found replace the probe's (as fdkv_set_modes would) and are what fdkv_commit
+ * packs.  *lambda_host (HOST, may be NULL) receives lambda; modes_host (HOST int32[n_layers/2][n_kv_heads], may be
+ * NULL) the modes.  If even the all-shared routing exceeds the budget: FDKV_ERR_ARENA_FULL, lambda = +inf, all shared.
+ * The estimate counts the prefill cache in canonical bytes (as Omega does), not the generated-token tails.
+ */
+fdkv_status fdkv_route_budget(fdkv_ctx* ctx, int32_t seq, size_t budget_bytes, double* lambda_host /*HOST*/,
+                              int32_t* modes_host /*HOST*/, void* stream);
+
 /* Overrides the modes of the staged sequence (forced-mode tests, ablations, benchmark mode mix).
  * modes_host: HOST int32[n_layers/2][n_kv_heads], each 0, 1 or 2.                                        */
 fdkv_status fdkv_set_modes(fdkv_ctx* ctx, int32_t seq, const int32_t* modes_host /*HOST*/);

@@ -297,3 +297,45 @@ int64_t fdkv_ref_select_tokens(const double* s, int64_t T, int64_t k_tok, int32_
     qsort(tok_out, (size_t)k_tok, sizeof(int32_t), cmp_i32);
     return k_tok;
 }
+
+/* ---- budgeted routing (Method: "the memory budget is enforced by increasing lambda until the estimated peak KV
+ * footprint satisfies the requested budget") ------------------------------------------------------------------
+ * Footprint(lambda) = sum over units of Omega(mode_u(lambda)) * bytes_exact_unit, with the mode rule above; it can only
+ * change where two of a unit's three loss lines cross, so the smallest lambda that fits is 0 or (just above) one of
+ * those crossings.  Candidates are visited in ascending order; each is tried at lambda = crossing * (1 + 2^-40) so
+ * that the unit that crosses there has already taken its cheaper mode.  Returns 1 and the first lambda that fits
+ * (with its modes), or 0 with lambda = +inf and every unit shared when even that does not fit.                   */
+static int cmp_f64(const void* a, const void* b) {
+    double x = *(const double*)a, y = *(const double*)b;
+    return (x > y) - (x < y);
+}
+int fdkv_ref_route_budget(const double* e_shared, const double* e_residual, int64_t n_units, const double* omega,
+                          double bytes_exact_unit, double budget_bytes, double* lambda_out, int32_t* modes_out) {
+    int64_t n_cand = 3 * n_units + 1;
+    double* cand = (double*)malloc((size_t)n_cand * sizeof(double));
+    cand[0] = 0.0;
+    for (int64_t u = 0; u < n_units; ++u) {
+        cand[1 + 3 * u] = (e_shared[u] - e_residual[u]) / (omega[1] - omega[0]); /* shared <-> residual */
+        cand[2 + 3 * u] = e_residual[u] / (omega[2] - omega[1]);                 /* residual <-> exact  */
+        cand[3 + 3 * u] = e_shared[u] / (omega[2] - omega[0]);                   /* shared <-> exact    */
+    }
+    qsort(cand, (size_t)n_cand, sizeof(double), cmp_f64);
+    int fits = 0;
+    for (int64_t i = 0; i < n_cand && !fits; ++i) {
+        if (!(cand[i] >= 0.0) || isinf(cand[i])) continue;
+        double lam = cand[i] * (1.0 + ldexp(1.0, -40));
+        double total = 0.0;
+        for (int64_t u = 0; u < n_units; ++u) {
+            int m = fdkv_ref_mode(e_shared[u], e_residual[u], omega, lam, NULL, NULL);
+            modes_out[u] = m;
+            total += omega[m] * bytes_exact_unit;
+        }
+        if (total <= budget_bytes) { fits = 1; *lambda_out = lam; }
+    }
+    if (!fits) {
+        *lambda_out = INFINITY;
+        for (int64_t u = 0; u < n_units; ++u) modes_out[u] = 0;
+    }
+    free(cand);
+    return fits;
+}

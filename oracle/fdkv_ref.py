@@ -31,6 +31,8 @@ _lib.fdkv_ref_omega.argtypes = [_i64, _i64, _i64, _i64, _f64p]
 _lib.fdkv_ref_omega_tokens.argtypes = [_i64, _i64, _i64, _i64, _f64p]
 _lib.fdkv_ref_mode.argtypes = [C.c_double, C.c_double, _f64p, C.c_double, _f64p, C.POINTER(C.c_double)]
 _lib.fdkv_ref_mode.restype = C.c_int
+_lib.fdkv_ref_route_budget.argtypes = [_f64p, _f64p, _i64, _f64p, C.c_double, C.c_double, C.POINTER(C.c_double), _i32p]
+_lib.fdkv_ref_route_budget.restype = C.c_int
 _lib.fdkv_ref_attention.argtypes = [_f64p, _f64p, _i64, _i64, _f32p, _f64p]
 _lib.fdkv_ref_token_scores.argtypes = [_f32p, _i64, _i64, _f32p, _f32p, _i64, _i64, _i64, _i32p, _i64, _f64p]
 _lib.fdkv_ref_select_tokens.argtypes = [_f64p, _i64, _i64, _i32p]
@@ -128,6 +130,17 @@ def mode_rule(e_shared: float, e_residual: float, om, lam: float):
     m = _lib.fdkv_ref_mode(float(e_shared), float(e_residual), np.ascontiguousarray(om, dtype=np.float64),
                            float(lam), loss, C.byref(margin))
     return int(m), loss, float(margin.value)
+
+
+def route_budget(e_shared, e_residual, om, bytes_exact_unit: float, budget_bytes: float):
+    """Smallest lambda whose routing fits the budget: (fits, lambda, modes)."""
+    e_sh = np.ascontiguousarray(e_shared, dtype=np.float64).ravel()
+    e_rs = np.ascontiguousarray(e_residual, dtype=np.float64).ravel()
+    modes = np.zeros(e_sh.size, dtype=np.int32)
+    lam = C.c_double(0.0)
+    fits = _lib.fdkv_ref_route_budget(e_sh, e_rs, e_sh.size, np.ascontiguousarray(om, dtype=np.float64), float(bytes_exact_unit),
+                                      float(budget_bytes), C.byref(lam), modes)
+    return bool(fits), float(lam.value), modes
 
 
 def attention(khat, vhat, q) -> np.ndarray:

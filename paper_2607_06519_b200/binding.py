@@ -48,6 +48,7 @@ def _load():
         "fdkv_compress_prefill": [vp, i32, i32, i32, i32, P(vp), P(vp), i64, i64, vp],
         "fdkv_probe": [vp, i32, i32, i32, P(vp), P(i32), i32, C.c_double, vp, vp, vp],
         "fdkv_set_modes": [vp, i32, P(i32)],
+        "fdkv_route_budget": [vp, i32, sz, P(C.c_double), P(i32), vp],
         "fdkv_commit": [vp, i32, vp],
         "fdkv_decode_attn": [vp, i32, i32, vp, vp, vp, vp, i32, vp],
         "fdkv_decode_attn_host": [vp, i32, i32, vp, vp, vp, vp, i32, vp],
@@ -207,6 +208,16 @@ class Context:
         if len(flat) != self.n_pairs * self.cfg.n_kv_heads:
             raise ValueError("modes must have n_pairs * n_kv_heads entries")
         _check(_lib.fdkv_set_modes(self.h, seq, arr), "fdkv_set_modes")
+
+    def route_budget(self, seq, budget_bytes, stream=None):
+        """Smallest lambda whose routing fits the byte budget: (fits, lambda, modes int32 [pairs, Hkv]); sets the modes."""
+        n = self.n_pairs * self.cfg.n_kv_heads
+        lam = C.c_double(0.0)
+        arr = (C.c_int32 * n)()
+        st = _lib.fdkv_route_budget(self.h, seq, int(budget_bytes), C.byref(lam), arr, _stream(stream))
+        if st not in (0, 3):
+            raise FdkvError(st, "fdkv_route_budget")
+        return st == 0, float(lam.value), torch.tensor(list(arr), dtype=torch.int32).view(self.n_pairs, -1)
 
     def commit(self, seq, stream=None):
         _check(_lib.fdkv_commit(self.h, seq, _stream(stream)), "fdkv_commit")

@@ -1,5 +1,7 @@
 // Host side of the C ABI: argument checks, workspace / arena bookkeeping, launch sequencing.
+#include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstring>
 #include <new>
 
@@ -329,6 +331,62 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     CU(launch_probe(a, s.dtype, st));
     for (int p = pb; p < pe; ++p) c->pair_probed[p] = 1;
     return FDKV_OK;
+}
+
+fdkv_status fdkv_route_budget(fdkv_ctx* c, int32_t seq, size_t budget_bytes, double* lambda_host, int32_t* modes_host,
+                              void* stream) {
+    if (!seq_ok(c, seq)) return FDKV_ERR_INVALID_ARG;
+    if (c->staged_seq != seq) return FDKV_ERR_STATE;
+    const Shape& s = c->s;
+    for (int p = 0; p < s.P; ++p)
+        if (!c->pair_probed[p]) return FDKV_ERR_STATE;
+    CU(cudaStreamSynchronize(S(stream)));
+    std::vector<double> e((size_t)s.NU * 2);
+    CU(cudaMemcpy(e.data(), c->work + c->ws.scores, e.size() * sizeof(double), cudaMemcpyDeviceToHost));
+    // Omega of the staged sequence, as in fdkv_probe
+    const int T = c->staged_T;
+    const double eb = s.esize, Td = (double)T * s.d;
+    const double k = (double)((int64_t)T * s.d * s.keep_num / s.keep_den), k_tok = (double)((int64_t)T * s.keep_num / s.keep_den);
+    const double b_sh = 2.0 * Td * eb, b_ex = 4.0 * Td * eb;
+    const double b_rs = s.tok_rule ? b_sh + 2.0 * k_tok * s.d * eb + 4.0 * k_tok : b_sh + 2.0 * k * (eb + 4.0);
+    const double om[3] = {b_sh / b_ex, b_rs / b_ex, 1.0};
+    auto mode_at = [&](int u, double lam) {
+        const double L0 = e[2 * u] + lam * om[0], L1 = e[2 * u + 1] + lam * om[1], L2 = lam * om[2];
+        int m = 0;
+        double best = L0;
+        if (L1 < best) { best = L1; m = 1; }
+        if (L2 < best) { best = L2; m = 2; }
+        return m;
+    };
+    // the footprint only changes where two loss lines of a unit cross: try 0 and every crossing, in ascending order
+    std::vector<double> cand;
+    cand.reserve((size_t)s.NU * 3 + 1);
+    cand.push_back(0.0);
+    for (int u = 0; u < s.NU; ++u) {
+        cand.push_back((e[2 * u] - e[2 * u + 1]) / (om[1] - om[0]));
+        cand.push_back(e[2 * u + 1] / (om[2] - om[1]));
+        cand.push_back(e[2 * u] / (om[2] - om[0]));
+    }
+    std::sort(cand.begin(), cand.end());
+    std::vector<int32_t> modes(s.NU, 0);
+    bool fits = false;
+    double lam_found = INFINITY;
+    for (double cv : cand) {
+        if (!(cv >= 0.0) || std::isinf(cv)) continue;
+        const double lam = cv * (1.0 + std::ldexp(1.0, -40));  // just past the crossing: that unit already took its cheaper mode
+        double total = 0.0;
+        for (int u = 0; u < s.NU; ++u) {
+            modes[u] = mode_at(u, lam);
+            total += om[modes[u]] * b_ex;
+        }
+        if (total <= (double)budget_bytes) { fits = true; lam_found = lam; break; }
+    }
+    if (!fits) std::fill(modes.begin(), modes.end(), 0);
+    c->seqs[seq].modes = modes;
+    c->modes_overridden = true;
+    if (lambda_host) *lambda_host = lam_found;
+    if (modes_host) std::memcpy(modes_host, modes.data(), (size_t)s.NU * 4);
+    return fits ? FDKV_OK : FDKV_ERR_ARENA_FULL;
 }
 
 fdkv_status fdkv_set_modes(fdkv_ctx* c, int32_t seq, const int32_t* modes_host) {

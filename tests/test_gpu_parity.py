@@ -161,3 +161,39 @@ def test_llama_shaped_reduced():
         assert worst <= TOL["bf16"], (step, worst)
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_budgeted_routing_matches_oracle():
+    """Smallest lambda that fits a byte budget: the library's search on its own probe errors against the oracle's
+    search on the oracle's errors (same modes; lambda equal up to the probe errors' float32 accumulation)."""
+    runner = _runner()
+    w = synth.WORKLOADS["decode32k"].scaled(n_layers=8, T=1024 + 5, n_needles=8, name="budget")
+    pf = runner.Prefilled(w, max_tail=1)
+    pf.compress(0)
+    pf.probe(0, 0.0)
+    pos = synth.probe_positions(w)
+    e = np.zeros((w.n_pairs, w.n_kv_heads, 2))
+    for p in range(w.n_pairs):
+        pq = (synth.probe_q(w, 0, 2 * p), synth.probe_q(w, 0, 2 * p + 1))
+        for h in range(w.n_kv_heads):
+            u = oracle_unit(w, 0, p, h)
+            e[p, h] = R.probe_error(u.z1["k"], u.kept["k"], pq[0], pq[1], w.group, h, pos)
+    om = R.omega(w.T, w.head_dim, 2, w.k_keep)
+    unit_bytes = 4.0 * w.T * w.head_dim * 2
+    n = w.n_pairs * w.n_kv_heads
+    for frac in (1.0, 0.8, 0.62, 0.55, 0.5):
+        budget = int(frac * n * unit_bytes)
+        fits, lam, modes = pf.ctx.route_budget(0, budget)
+        rf, rl, rm = R.route_budget(e[..., 0], e[..., 1], om, unit_bytes, budget)
+        assert fits and rf
+        assert np.array_equal(modes.numpy().ravel(), rm), frac
+        assert lam == pytest.approx(rl, rel=1e-4, abs=1e-12)
+        assert sum(om[m] for m in rm) * unit_bytes <= budget
+    fits, lam, modes = pf.ctx.route_budget(0, int(0.4 * n * unit_bytes))
+    assert not fits and np.isinf(lam) and int(modes.sum()) == 0
+    fits, lam, modes = pf.ctx.route_budget(0, int(0.62 * n * unit_bytes))
+    pf.commit(0)  # commit packs the budgeted modes
+    assert np.array_equal(pf.ctx.get_modes(0).numpy(), modes.numpy())
+    by_mode, exact_equiv = pf.ctx.footprint(0)
+    assert exact_equiv == int(n * unit_bytes)
+    pf.ctx.close()

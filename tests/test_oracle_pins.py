@@ -372,3 +372,40 @@ def test_token_rule_candidates_probe_and_attention_vs_bruteforce():
     assert np.max(np.abs(u.rows("k", R.RESIDUAL, 1) - k1)) <= 2e-7 * np.max(np.abs(k1))
     u.use_tokens(np.zeros(0, np.int32))
     assert np.array_equal(u.rows("k", R.RESIDUAL, 0), u.rows("k", R.SHARED, 0))
+
+
+# ---------------------------------------------------------------- budgeted routing
+def test_route_budget_is_the_smallest_lambda_that_fits():
+    rng = np.random.default_rng(90)
+    n = 40
+    e_sh = rng.lognormal(3.0, 1.0, n)
+    e_rs = e_sh * rng.uniform(0.05, 0.4, n)
+    om = R.omega(32768, 128, 2, 262144)
+    unit = 4.0 * 32768 * 128 * 2
+
+    def footprint(lam):
+        return sum(om[R.mode_rule(a, b, om, lam)[0]] * unit for a, b in zip(e_sh, e_rs))
+
+    # footprint is monotone non-increasing in lambda (the premise of "increase lambda until it fits")
+    grid = np.concatenate([[0.0], np.geomspace(1e-3, 1e6, 400)])
+    fp = np.array([footprint(l) for l in grid])
+    assert np.all(np.diff(fp) <= 1e-6)
+    for frac in (1.0, 0.9, 0.7, 0.6, 0.55, 0.5):
+        budget = frac * n * unit
+        fits, lam, modes = R.route_budget(e_sh, e_rs, om, unit, budget)
+        assert fits
+        assert footprint(lam) <= budget
+        assert [R.mode_rule(a, b, om, lam)[0] for a, b in zip(e_sh, e_rs)] == modes.tolist()
+        if lam > 0:
+            assert footprint(lam * (1 - 1e-9)) > budget            # minimal: anything smaller does not fit
+            assert not np.any((grid < lam * (1 - 1e-9)) & (fp <= budget))
+        else:
+            assert np.all(modes == R.EXACT)
+    # below the all-shared footprint nothing fits
+    fits, lam, modes = R.route_budget(e_sh, e_rs, om, unit, 0.49 * n * unit)
+    assert not fits and np.isinf(lam) and np.all(modes == 0)
+    # one unit, by hand: shared<->residual crossing at (100-10)/(0.59375-0.5) = 960, residual<->exact at 10/0.40625
+    fits, lam, modes = R.route_budget([100.0], [10.0], om, unit, 0.6 * unit)
+    assert fits and modes.tolist() == [1] and lam == pytest.approx(10.0 / (1 - 0.59375), rel=1e-9)
+    fits, lam, modes = R.route_budget([100.0], [10.0], om, unit, 0.5 * unit)
+    assert fits and modes.tolist() == [0] and lam == pytest.approx(90.0 / 0.09375, rel=1e-9)
