@@ -12,7 +12,7 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libfdkv.so")
+LIB_PATH = os.environ.get("FDKV_LIB_PATH", os.path.join(_HERE, "libfdkv.so"))  # override: A/B runs of two builds
 
 F32, BF16 = 0, 1
 SHARED, RESIDUAL, EXACT = 0, 1, 2

@@ -43,7 +43,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct FastSched {
     uint32_t start[kMaxCtas + 1];  // unit << 20 | first 64-token tile of CTA c; start[ncta] = units << 20
-    int ncta, units, tslot, prologue_tiles, reverse_odd;
+    int ncta, units, tslot, prologue_tiles, reverse_odd, experiment;
 };
 struct PartCount {
     uint8_t n[kMaxUnits];  // split-K parts per unit (at most kMaxSplits)
@@ -426,6 +426,11 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 TADD(5, 1);
 #endif
                 const uint32_t kb = stage0 + s * kStageBytes, vb = kb + 2 * kHalfBytes;
+                if (sch.experiment == 1) {  // timing experiment only: stream the tiles, compute nothing
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem0 + kOffEmpty + 8 * s);
+                    continue;
+                }
 
                 // ---- S^T[head][token] = q . k over 128 channels; two n-tiles of 8 tokens ----
                 float sacc[2][4];
@@ -778,6 +783,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     sch.ncta = ncta;
     sch.prologue_tiles = prologue_tiles;
     sch.reverse_odd = reverse_odd ? 1 : 0;
+    { const char* ex = getenv("FDKV_DECODE_EXPERIMENT"); sch.experiment = ex ? atoi(ex) : 0; }
     sch.units = units;
     bool whole = whole_ctas && units <= ncta;
     std::vector<int> nc(units, 1);
