@@ -31,7 +31,8 @@ constexpr int kThreads = kCW * 32;  // 256 threads: two warps per scheduler, so 
 constexpr int kHalfBytes = kTT * 128;        // one 64-channel box of 128 tokens
 constexpr int kStageBytes = 4 * kHalfBytes;  // K ch 0-63, K ch 64-127, V ch 0-63, V ch 64-127
 constexpr int kScratchBytes = 4096;          // per consumer warp: 16 tokens x 128 channels bf16 (or its O tile at merge)
-constexpr int kHeaderBytes = 1024;
+constexpr int kHeaderBytes = 2048;
+constexpr int kMaxSeg = 24;  // (unit, range) segments one CTA can walk: at most units / CTAs + 2
 constexpr int kSmemBytes = kHeaderBytes + kStages * kStageBytes + kCW * kScratchBytes;
 constexpr int kMaxCtas = 296;
 constexpr int kMaxUnits = kFastMaxUnits;
@@ -51,7 +52,14 @@ struct PartCount {
 static_assert(kMaxSplits < 256 && kMaxSplits % 32 == 0, "part counts are bytes; the combine holds one part per lane and round");
 
 // header offsets
-constexpr int kOffFull = 0, kOffEmpty = 64, kOffAbort = 128, kOffTicket = 132, kOffM = 256, kOffL = 512;
+constexpr int kOffFull = 0, kOffAbort = 128, kOffTicket = 132, kOffM = 256, kOffL = 512, kOffSeg = 1024, kOffSegInfo = 1920,
+              kOffCnt = 1936;
+// one (unit, tile range) segment of a CTA: arena rows of its K / V boxes and tail, first tile, prefill tiles, first
+// index in the CTA's tile sequence, and the sequence / head whose tail it also streams (or -1)
+struct Seg {
+    int krow, vrow, tkrow, tvrow, tb, npre, it0, tail_b, tail_h;
+};
+static_assert(kMaxSeg * sizeof(Seg) <= 896, "segment table fits its header slot");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -161,7 +169,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem0 + kOffFull + 8 * s, 1);
-            mbar_init(smem0 + kOffEmpty + 8 * s, kCW);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -179,59 +186,22 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     // (Measured: 1.4 % per step; L2 eviction hints on the TMA loads did not add to it.)
     const bool rev = sch.reverse_odd && (a.layer & 1);
 
-    // ================= producer cursor (thread 0 only): walks the same tile sequence kStages-1 tiles ahead =================
-    int p_u = u_first, p_j = 0, p_npre = 0, p_nseg = 0, p_tb = 0, p_it = 0, p_b = 0, p_h = 0;
-    int p_krow = 0, p_vrow = 0, p_tkrow = 0, p_tvrow = 0;
-    bool p_done = !is_producer, p_tail_pending = false, p_waited = false;
-    auto prod_open_unit = [&]() {
-        for (; p_u <= u_last && p_u < sch.units; ++p_u) {
-            const int b = p_u / a.Hkv, h = p_u % a.Hkv;
-            const UnitDesc* ud = a.desc + ((int64_t)b * a.L + a.layer) * a.Hkv + h;
-            const int T = ud->T;
-            const int ntiles = (T + kTT - 1) / kTT;
-            const int tb = p_u == u_first ? t_first : 0;
-            const int te = p_u == u_last ? t_last : ntiles;
-            if (te <= tb) continue;
-            p_krow = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> 8);
-            p_vrow = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> 8);
-            p_tail_pending = te == ntiles;  // this CTA also streams the unit's tail: length read once the wait is over
-            p_b = b;
-            p_h = h;
-            p_tb = tb;
-            p_npre = te - tb;
-            p_nseg = p_npre;
-            p_j = 0;
-            return;
-        }
-        p_done = true;
-    };
-    // the tail (rows and length) may have been written by the kernel right before this one: only after the wait
-    auto prod_tail_info = [&]() {
-        p_tail_pending = false;
-        const int n = min(a.tail_len[a.layer * a.max_batch + p_b], a.max_tail);
-        const int64_t o = (((int64_t)a.layer * a.max_batch + p_b) * a.Hkv + p_h) * a.tail_rows;
-        p_tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
-        p_tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
-        p_nseg = p_npre + (n + kTT - 1) / kTT;
-    };
-    auto prod_issue = [&]() {
-        if (p_done) return;
-        if (p_j == p_npre && p_tail_pending) {  // prefill tiles of the segment are all issued
-            if (!p_waited) return;              // prologue: never touch the tail before the dependency wait
-            prod_tail_info();
-        }
-        if (p_j >= p_nseg) {
-            ++p_u;
-            prod_open_unit();
-            if (p_done) return;
-        }
-        const int s = p_it % kStages;
-        const uint32_t ph = (uint32_t)(p_it / kStages) & 1u;
-        wait_bar(smem0 + kOffEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
-        if (*abort_flag) { p_done = true; return; }
-        const int p_tile = rev ? p_tb + p_npre - 1 - p_j : p_tb + p_j;
-        const int kr = p_j < p_npre ? p_krow + p_tile * kTT : p_tkrow + (p_j - p_npre) * kTT;
-        const int vr = p_j < p_npre ? p_vrow + p_tile * kTT : p_tvrow + (p_j - p_npre) * kTT;
+    // ================= the CTA's tile sequence: a small segment table in shared memory =================
+    // Tile `it` of the CTA (all segments, prefill tiles then tail tiles of each) always lands in stage it % kStages.
+    // Whichever warp is the last to finish a tile refills its stage with tile it + kStages at once (a counter per
+    // stage, no waiting producer), so copies are issued the moment a stage is free.
+    Seg* const segs = reinterpret_cast<Seg*>(smem_raw + kOffSeg);
+    int* const seg_info = reinterpret_cast<int*>(smem_raw + kOffSegInfo);  // [0] segments, [1] tiles in total
+    int* const stage_cnt = reinterpret_cast<int*>(smem_raw + kOffCnt);
+    auto issue_tile = [&](int it) {
+        int si = 0;
+        while (si + 1 < seg_info[0] && it >= segs[si + 1].it0) ++si;
+        const Seg g = segs[si];
+        const int j = it - g.it0;
+        const int tile = rev ? g.tb + g.npre - 1 - j : g.tb + j;
+        const int kr = j < g.npre ? g.krow + tile * kTT : g.tkrow + (j - g.npre) * kTT;
+        const int vr = j < g.npre ? g.vrow + tile * kTT : g.tvrow + (j - g.npre) * kTT;
+        const int s = it % kStages;
         const uint32_t full = smem0 + kOffFull + 8 * s;
         const uint32_t dst = stage0 + s * kStageBytes;
         mbar_expect_tx(full, kStageBytes);
@@ -239,20 +209,74 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
         tma_load_2d(dst + kHalfBytes, &tmap, 64, kr, full);
         tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
         tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
-        ++p_it;
-        ++p_j;
     };
+    // a warp is done reading stage s (tile it): the last of the eight refills it
+    auto release_stage = [&](int s, int it) {
+        __syncwarp();
+        if (lane == 0) {
+            const int old = atomicAdd(stage_cnt + s, 1);
+            if (old == kCW - 1) {
+                stage_cnt[s] = 0;
+                if (it + kStages < seg_info[1]) issue_tile(it + kStages);
+            }
+        }
+    };
+    int prologue_issued = 0;
     if (is_producer) {
-        prod_open_unit();
-        for (int i = 0; i < sch.prologue_tiles; ++i) prod_issue();  // nobody computes yet: stages can all be filled
+        // static part (packed cache, fixed since commit): may run before the dependency wait
+        int n = 0, it0 = 0;
+        for (int u = u_first; u <= u_last && u < sch.units; ++u) {
+            const int b = u / a.Hkv, h = u % a.Hkv;
+            const UnitDesc* ud = a.desc + ((int64_t)b * a.L + a.layer) * a.Hkv + h;
+            const int ntiles = (ud->T + kTT - 1) / kTT;
+            const int tb = u == u_first ? t_first : 0;
+            const int te = u == u_last ? t_last : ntiles;
+            if (te <= tb) continue;
+            if (n == kMaxSeg) { atomicMax(a.status, (int32_t)kFlagCountMismatch); break; }  // cannot happen: see the launcher
+            Seg g;
+            g.krow = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> 8);
+            g.vrow = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> 8);
+            g.tkrow = g.tvrow = 0;
+            g.tb = tb;
+            g.npre = te - tb;
+            g.it0 = it0;
+            g.tail_b = te == ntiles ? b : -1;  // this CTA also streams the unit's tail (length known after the wait)
+            g.tail_h = h;
+            segs[n++] = g;
+            it0 += g.npre;
+        }
+        seg_info[0] = n;
+        seg_info[1] = it0;
+        for (int s = 0; s < kStages; ++s) stage_cnt[s] = 0;
+        if (n > 0)
+            for (; prologue_issued < sch.prologue_tiles && prologue_issued < kStages && prologue_issued < segs[0].npre; ++prologue_issued)
+                issue_tile(prologue_issued);
     }
     // per-warp scratch starts zeroed
     for (int i = threadIdx.x; i < kCW * kScratchBytes / 16; i += kThreads)
         st_shared_zero16(smem0 + kHeaderBytes + kStages * kStageBytes + i * 16);
     // everything below may depend on the kernels launched before this one (q, appended tail rows, partial slots)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    p_waited = true;
     TGLOBAL(1);
+    if (is_producer) {
+        // tails: rows and lengths may have been written by the kernel right before this one
+        int it0 = 0;
+        for (int i = 0; i < seg_info[0]; ++i) {
+            Seg g = segs[i];
+            g.it0 = it0;
+            if (g.tail_b >= 0) {
+                const int n = min(a.tail_len[a.layer * a.max_batch + g.tail_b], a.max_tail);
+                const int64_t o = (((int64_t)a.layer * a.max_batch + g.tail_b) * a.Hkv + g.tail_h) * a.tail_rows;
+                g.tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
+                g.tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
+                it0 += (n + kTT - 1) / kTT;
+            }
+            it0 += g.npre;
+            segs[i] = g;
+        }
+        seg_info[1] = it0;
+        for (int it = prologue_issued; it < kStages && it < it0; ++it) issue_tile(it);  // nobody computes yet: fill every stage
+    }
     __syncthreads();
 
     // ================= compute: every warp takes 16 tokens of every stage =================
@@ -281,7 +305,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 ntail = (n_tail_rows + kTT - 1) / kTT;
             }
             const int npre = te - tb, nseg = npre + ntail;
-            const bool coef = ud.mode != FDKV_MODE_EXACT, resid = ud.mode == FDKV_MODE_RESIDUAL;
+            const bool coef = ud.mode != FDKV_MODE_EXACT, resid = ud.mode == FDKV_MODE_RESIDUAL && sch.experiment != 5;  // (experiment 5: no residual work)
             const uint32_t sgn = ud.sign < 0.f ? 0x80008000u : 0u;
             const int nres = (T + kResTile - 1) / kResTile;
 
@@ -404,10 +428,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 const float kscale = ((coef && !is_tail) ? kC : 1.f) * inv_sqrt_d * kLog2e;
                 const float vscale = (coef && !is_tail) ? kC : 1.f;
 
-                // keep the copies kStages-1 tiles ahead: refill the stage every warp released one tile ago
-                if (is_producer)
-                    while (!p_done && p_it < itj + kStages) prod_issue();
-                __syncwarp();
 
                 if (with_res && cr[1] > cr[0]) {
                     if (tokmode) scatter_tok(t_krows, cr[0], cr[1], pke, ptk);
@@ -427,8 +447,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
 #endif
                 const uint32_t kb = stage0 + s * kStageBytes, vb = kb + 2 * kHalfBytes;
                 if (sch.experiment == 1) {  // timing experiment only: stream the tiles, compute nothing
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem0 + kOffEmpty + 8 * s);
+                    release_stage(s, itj);
                     continue;
                 }
 
@@ -438,6 +457,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 for (int nt = 0; nt < 2; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
                 {
                     const int mi = lane >> 3, rr = lane & 7;
+                    if (sch.experiment != 3)  // (timing experiment 3 skips this product)
 #pragma unroll
                     for (int nt = 0; nt < 2; ++nt) {
                         const int row = r0 + nt * 8 + rr;
@@ -534,6 +554,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 {
                     const int mi = lane >> 3, rr = lane & 7;
                     const int row = r0 + (mi & 1) * 8 + rr;
+                    if (sch.experiment != 2)  // (timing experiment 2 skips this product)
 #pragma unroll
                     for (int jp = 0; jp < 8; ++jp) {
                         const int c = 2 * jp + (mi >> 1);
@@ -556,8 +577,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                         zero_scratch();
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem0 + kOffEmpty + 8 * s);
+                release_stage(s, itj);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) cr[i] = nr[i];
                 load_ranges(j + 2, nr);
@@ -833,10 +853,13 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     for (int c = 0; c < ncta; ++c) {
         const int ua = (int)(sch.start[c] >> 20), ta = (int)(sch.start[c] & 0xFFFFFu);
         const int ub = (int)(sch.start[c + 1] >> 20), tb = (int)(sch.start[c + 1] & 0xFFFFFu);
+        int nseg_cta = 0;
         for (int u = ua; u <= ub && u < units; ++u) {
             const int b0 = u == ua ? ta : 0, b1 = u == ub ? tb : nt[u];
+            if (b1 > b0) ++nseg_cta;
             if (b1 > b0 && cs.n[u] < 255) cs.n[u]++;
         }
+        if (nseg_cta > kMaxSeg) return cudaErrorInvalidValue;  // more one-tile units per CTA than the segment table holds
     }
     for (int u = 0; u < units; ++u)
         if (cs.n[u] > kMaxSplits) return cudaErrorInvalidValue;  // cannot happen: ncta <= kMaxSplits
