@@ -103,6 +103,11 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {  // transpose an 8 x 8 matrix of 16-bit elements held by the warp
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -143,7 +148,10 @@ __device__ long long g_timing[64][kMaxCtas][8];
 #define TADD(i, v) do { t_acc[i - 4] += (v); } while (0)
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define TGLOBAL(i) do { if (threadIdx.x == 32) g_timing[sch.tslot][blockIdx.x][i] = gtime(); } while (0)
+__device__ unsigned g_phase[kMaxCtas][12];
+#define TPH(i) do { const unsigned now_ = (unsigned)clock(); t_ph[i] += now_ - t_mark; t_mark = now_; } while (0)
 #else
+#define TPH(i)
 #define TGLOBAL(i)
 #define TSTAMP(i)
 #define TADD(i, v)
@@ -154,6 +162,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     extern __shared__ __align__(1024) uint8_t smem_raw[];
 #ifdef FDKV_TIMING
     long long t_acc[2] = {0, 0};
+    unsigned t_ph[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, t_mark = 0;
 #endif
     TGLOBAL(6);
     const uint32_t smem0 = smem_u32(smem_raw);
@@ -309,20 +318,24 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             const uint32_t sgn = ud.sign < 0.f ? 0x80008000u : 0u;
             const int nres = (T + kResTile - 1) / kResTile;
 
-            // q fragments: A operand rows = the G query heads of this KV head, zero elsewhere
-            uint32_t qa[8][2];
+            // q fragments: B operand columns = the G query heads of this KV head.  With G <= 4 columns 4-7 repeat
+            // them: in the second product those columns carry the bf16 rounding remainder of P, so P acts in ~16 bits.
+            const bool split = a.G <= 4;
+            const int qcol = split ? (gid & 3) : gid;
+            uint32_t qb[8][2];
             {
-                const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.Hq + h * a.G + gid) * 128;
+                const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.Hq + h * a.G + qcol) * 128;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    qa[kk][0] = gid < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 2 * tig) : 0u;
-                    qa[kk][1] = gid < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 8 + 2 * tig) : 0u;
+                    qb[kk][0] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 2 * tig) : 0u;
+                    qb[kk][1] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 8 + 2 * tig) : 0u;
                 }
             }
-            float oacc[16][4];
+            // O^T[channel][column]: eight 16-channel m-tiles; this thread holds columns 2 tig, 2 tig + 1
+            float oacc[8][4];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
-            float m_run = -INFINITY, l_run = 0.f;
+            for (int j = 0; j < 8; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
+            float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};  // per held column; l is this thread's share
             // split-K part slot of this segment = number of CTAs with tiles of this unit before this one
             int slot = 0;
             for (int c2 = cta - 1; c2 >= 0; --c2) {
@@ -427,7 +440,9 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 const bool with_res = resid && !is_tail;
                 const float kscale = ((coef && !is_tail) ? kC : 1.f) * inv_sqrt_d * kLog2e;
                 const float vscale = (coef && !is_tail) ? kC : 1.f;
-
+#ifdef FDKV_TIMING
+                t_mark = (unsigned)clock();
+#endif
 
                 if (with_res && cr[1] > cr[0]) {
                     if (tokmode) scatter_tok(t_krows, cr[0], cr[1], pke, ptk);
@@ -437,10 +452,12 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 if (tokmode) prefetch_tok(t_krows, nr[0], nr[1], pke, ptk);
                 else if (resid) prefetch(k_ent, nr[0], nr[1], pke);
 
+                TPH(0);
 #ifdef FDKV_TIMING
                 const long long tw0 = clock64();
 #endif
                 wait_bar(smem0 + kOffFull + 8 * s, ph, abort_flag, a.status);
+                TPH(1);
 #ifdef FDKV_TIMING
                 TADD(4, clock64() - tw0);
                 TADD(5, 1);
@@ -451,47 +468,40 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                     continue;
                 }
 
-                // ---- S^T[head][token] = q . k over 128 channels; two n-tiles of 8 tokens ----
+                // ---- S[token][column] = k . q over 128 channels: one 16 x 8 tile, two accumulator chains ----
                 float sacc[2][4];
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+                for (int i = 0; i < 2; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
                 {
                     const int mi = lane >> 3, rr = lane & 7;
+                    const int row = r0 + (mi & 1) * 8 + rr;  // ldmatrix: matrices = (tokens 0-7 | 8-15) x (chunk | chunk + 1)
                     if (sch.experiment != 3)  // (timing experiment 3 skips this product)
 #pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) {
-                        const int row = r0 + nt * 8 + rr;
-#pragma unroll
-                        for (int kp = 0; kp < 4; ++kp) {
-                            const int c = 4 * kp + mi;  // 16-byte channel chunk 0..15
-                            uint32_t b0, b1, b2, b3;
-                            ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), b0, b1, b2, b3);
-                            mma_bf16(sacc[nt], qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
-                            mma_bf16(sacc[nt], qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b2, b3);
-                        }
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const int c = 2 * kk + (mi >> 1);  // 16-byte channel chunk 0..15
+                        uint32_t a0, a1, a2, a3;
+                        ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
+                        mma_bf16(sacc[kk & 1], a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
                     }
+                    TPH(2);
                     if (with_res && cr[1] > cr[0]) {
-                        float racc[2][4];  // own accumulators: the two passes' mma chains run side by side
+                        float racc[4] = {0.f, 0.f, 0.f, 0.f};  // own accumulator: this chain runs beside the two above
+                        const int srow = (mi & 1) * 8 + rr;
 #pragma unroll
-                        for (int nt = 0; nt < 2; ++nt) {
-                            racc[nt][0] = racc[nt][1] = racc[nt][2] = racc[nt][3] = 0.f;
-                            const int row = nt * 8 + rr;
-#pragma unroll
-                            for (int kp = 0; kp < 4; ++kp) {
-                                const int c = 4 * kp + mi;
-                                uint32_t b0, b1, b2, b3;
-                                ldsm_x4(scratch + (c >> 3) * 2048 + swz(row, c), b0, b1, b2, b3);
-                                mma_bf16(racc[nt], qa[2 * kp][0] ^ sgn, 0u, qa[2 * kp][1] ^ sgn, 0u, b0, b1);
-                                mma_bf16(racc[nt], qa[2 * kp + 1][0] ^ sgn, 0u, qa[2 * kp + 1][1] ^ sgn, 0u, b2, b3);
-                            }
-                            sacc[nt][0] += racc[nt][0];
-                            sacc[nt][1] += racc[nt][1];
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const int c = 2 * kk + (mi >> 1);
+                            uint32_t a0, a1, a2, a3;
+                            ldsm_x4(scratch + (c >> 3) * 2048 + swz(srow, c), a0, a1, a2, a3);
+                            mma_bf16(racc, a0, a1, a2, a3, qb[kk][0] ^ sgn, qb[kk][1] ^ sgn);
                         }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) sacc[0][i] += racc[i];
                         __syncwarp();
                         zero_scratch();
                         __syncwarp();
                     }
                 }
+                TPH(3);
                 if (with_res && cr[3] > cr[2]) {
                     if (tokmode) scatter_tok(t_vrows, cr[2], cr[3], pve, ptv);
                     else scatter(v_ent, cr[2], cr[3], pve);
@@ -500,101 +510,131 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 if (tokmode) prefetch_tok(t_vrows, nr[2], nr[3], pve, ptv);
                 else if (resid) prefetch(v_ent, nr[2], nr[3], pve);
 
-                // ---- online softmax for head gid over this slice's 16 tokens (4 per thread) ----
-                float p[2][2];
-                float mt = -INFINITY;
+                TPH(4);
+                // ---- online softmax per column over this slice's 16 tokens (this thread: tokens gid, gid + 8) ----
+                float p[2][2];  // [token half][column 2 tig + e]
+                float mt[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
+                for (int hh = 0; hh < 2; ++hh) {
+                    const bool valid = r0 + gid + 8 * hh < rows_valid;
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
-                        const int tl = r0 + nt * 8 + 2 * tig + e;
-                        const float sv = tl < rows_valid ? sacc[nt][e] * kscale : -INFINITY;
-                        p[nt][e] = sv;
-                        mt = fmaxf(mt, sv);
-                    }
-                mt = fmaxf(mt, __shfl_xor_sync(0xFFFFFFFFu, mt, 1));
-                mt = fmaxf(mt, __shfl_xor_sync(0xFFFFFFFFu, mt, 2));
-                const float m_new = fmaxf(m_run, mt);
-                float alpha = 1.f;
-                if (m_new == -INFINITY) {
-                    p[0][0] = p[0][1] = p[1][0] = p[1][1] = 0.f;
-                } else {
-                    alpha = ex2(m_run - m_new);
-#pragma unroll
-                    for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) p[nt][e] = ex2(p[nt][e] - m_new);
-                }
-                l_run = l_run * alpha + (p[0][0] + p[0][1] + p[1][0] + p[1][1]);
-                m_run = m_new;
-                if (__any_sync(0xFFFFFFFFu, alpha != 1.f)) {
-#pragma unroll
-                    for (int jn = 0; jn < 16; ++jn) {
-                        oacc[jn][0] *= alpha; oacc[jn][1] *= alpha; oacc[jn][2] *= alpha; oacc[jn][3] *= alpha;
+                        const float sv = valid ? (sacc[0][2 * hh + e] + sacc[1][2 * hh + e]) * kscale : -INFINITY;
+                        p[hh][e] = sv;
+                        mt[e] = fmaxf(mt[e], sv);
                     }
                 }
-                // A operand of the second product: rows 0-7 carry the bf16 rounding of P, rows 8-15 its remainder
-                uint32_t pa[4];
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) {
+                    mt[0] = fmaxf(mt[0], __shfl_xor_sync(0xFFFFFFFFu, mt[0], o));
+                    mt[1] = fmaxf(mt[1], __shfl_xor_sync(0xFFFFFFFFu, mt[1], o));
+                }
+                float alpha[2];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const float m_new = fmaxf(m_run[e], mt[e]);
+                    if (m_new == -INFINITY) {
+                        alpha[e] = 1.f;
+                        p[0][e] = p[1][e] = 0.f;
+                    } else {
+                        alpha[e] = ex2(m_run[e] - m_new);
+                        p[0][e] = ex2(p[0][e] - m_new);
+                        p[1][e] = ex2(p[1][e] - m_new);
+                    }
+                    l_run[e] = l_run[e] * alpha[e] + (p[0][e] + p[1][e]);
+                    m_run[e] = m_new;
+                }
+                if (__any_sync(0xFFFFFFFFu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+#pragma unroll
+                    for (int jm = 0; jm < 8; ++jm) {
+                        oacc[jm][0] *= alpha[0]; oacc[jm][1] *= alpha[1]; oacc[jm][2] *= alpha[0]; oacc[jm][3] *= alpha[1];
+                    }
+                }
+                // B operand of the second product, P^T[token][column]: columns 0-3 carry the bf16 rounding of P and
+                // (G <= 4) columns 4-7 its remainder; an 8 x 8 register transpose turns the accumulator layout
+                // (token row, column pair) into the operand layout (column, token pair).
+                uint32_t pb[2];
                 {
-                    float hi[2][2], lo[2][2];
+                    const bool lo_part = split && tig >= 2;
 #pragma unroll
-                    for (int nt = 0; nt < 2; ++nt)
+                    for (int hh = 0; hh < 2; ++hh) {
+                        float v[2];
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const float pv_ = p[nt][e] * vscale;
-                            hi[nt][e] = __bfloat162float(__float2bfloat16_rn(pv_));
-                            lo[nt][e] = pv_ - hi[nt][e];
+                            const float pv_ = p[hh][e] * vscale;
+                            const float hi = __bfloat162float(__float2bfloat16_rn(pv_));
+                            v[e] = lo_part ? pv_ - hi : hi;
                         }
-                    pa[0] = pack_bf16(hi[0][0], hi[0][1]);
-                    pa[1] = pack_bf16(lo[0][0], lo[0][1]);
-                    pa[2] = pack_bf16(hi[1][0], hi[1][1]);
-                    pa[3] = pack_bf16(lo[1][0], lo[1][1]);
+                        pb[hh] = movmatrix_t(pack_bf16(v[0], v[1]));
+                    }
                 }
-                // ---- O[head][channel] += P . V : 16 n-tiles of 8 channels, k = this slice's 16 tokens ----
+                TPH(5);
+                // ---- O^T[channel][column] += V^T . P^T : eight m-tiles of 16 channels, k = this slice's 16 tokens ----
                 {
                     const int mi = lane >> 3, rr = lane & 7;
-                    const int row = r0 + (mi & 1) * 8 + rr;
+                    const int row = r0 + (mi >> 1) * 8 + rr;  // ldmatrix.trans: matrices = (chunk | chunk + 1) x (tokens 0-7 | 8-15)
                     if (sch.experiment != 2)  // (timing experiment 2 skips this product)
 #pragma unroll
-                    for (int jp = 0; jp < 8; ++jp) {
-                        const int c = 2 * jp + (mi >> 1);
-                        uint32_t b0, b1, b2, b3;
-                        ldsm_x4_t(vb + (c >> 3) * kHalfBytes + swz(row, c), b0, b1, b2, b3);
-                        mma_bf16(oacc[2 * jp], pa[0], pa[1], pa[2], pa[3], b0, b1);
-                        mma_bf16(oacc[2 * jp + 1], pa[0], pa[1], pa[2], pa[3], b2, b3);
+                    for (int jm = 0; jm < 8; ++jm) {
+                        const int c = 2 * jm + (mi & 1);
+                        uint32_t a0, a1, a2, a3;
+                        ldsm_x4_t(vb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
+                        mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0], pb[1]);
                     }
+                    TPH(6);
                     if (with_res && cr[3] > cr[2]) {
-                        const int srow = (mi & 1) * 8 + rr;
+                        const int srow = (mi >> 1) * 8 + rr;
 #pragma unroll
-                        for (int jp = 0; jp < 8; ++jp) {
-                            const int c = 2 * jp + (mi >> 1);
-                            uint32_t b0, b1, b2, b3;
-                            ldsm_x4_t(scratch + (c >> 3) * 2048 + swz(srow, c), b0, b1, b2, b3);
-                            mma_bf16(oacc[2 * jp], pa[0] ^ sgn, pa[1] ^ sgn, pa[2] ^ sgn, pa[3] ^ sgn, b0, b1);
-                            mma_bf16(oacc[2 * jp + 1], pa[0] ^ sgn, pa[1] ^ sgn, pa[2] ^ sgn, pa[3] ^ sgn, b2, b3);
+                        for (int jm = 0; jm < 8; ++jm) {
+                            const int c = 2 * jm + (mi & 1);
+                            uint32_t a0, a1, a2, a3;
+                            ldsm_x4_t(scratch + (c >> 3) * 2048 + swz(srow, c), a0, a1, a2, a3);
+                            mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0] ^ sgn, pb[1] ^ sgn);
                         }
                         __syncwarp();
                         zero_scratch();
                     }
                 }
+                TPH(7);
                 release_stage(s, itj);
+                TPH(8);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) cr[i] = nr[i];
                 load_ranges(j + 2, nr);
+                TPH(9);
             }
             it += nseg;
             TGLOBAL(2);
 
             // ---- merge the eight warps' states into this segment's split-K partial ----
             {
-                float lq = l_run;
-                lq += __shfl_xor_sync(0xFFFFFFFFu, lq, 1);
-                lq += __shfl_xor_sync(0xFFFFFFFFu, lq, 2);
-                if (tig == 0) { sm_m[warp * 8 + gid] = m_run; sm_l[warp * 8 + gid] = lq; }
+                float lq[2] = {l_run[0], l_run[1]};
 #pragma unroll
-                for (int jn = 0; jn < 16; ++jn)
-                    *reinterpret_cast<float2*>(scratch_f + gid * 128 + jn * 8 + 2 * tig) =
-                        make_float2(oacc[jn][0] + oacc[jn][2], oacc[jn][1] + oacc[jn][3]);
+                for (int o = 4; o < 32; o <<= 1) {
+                    lq[0] += __shfl_xor_sync(0xFFFFFFFFu, lq[0], o);
+                    lq[1] += __shfl_xor_sync(0xFFFFFFFFu, lq[1], o);
+                }
+                if (gid == 0) {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) { sm_m[warp * 8 + 2 * tig + e] = m_run[e]; sm_l[warp * 8 + 2 * tig + e] = lq[e]; }
+                }
+                // O[head][channel]: column g plus (G <= 4) its remainder column g + 4, held by the lane two over
+#pragma unroll
+                for (int jm = 0; jm < 8; ++jm) {
+                    float v[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        v[i] = oacc[jm][i];
+                        if (split) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
+                    }
+                    if (!split || tig < 2) {
+                        const int ch = 16 * jm + gid, col = 2 * tig;
+                        scratch_f[col * 128 + ch] = v[0];
+                        scratch_f[(col + 1) * 128 + ch] = v[1];
+                        scratch_f[col * 128 + ch + 8] = v[2];
+                        scratch_f[(col + 1) * 128 + ch + 8] = v[3];
+                    }
+                }
                 __syncthreads();
                 TGLOBAL(0);
                 for (int i = threadIdx.x; i < a.G * 128; i += kThreads) {
@@ -706,7 +746,10 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
     }
     TGLOBAL(7);
 #ifdef FDKV_TIMING
-    if (threadIdx.x == 32) { g_timing[sch.tslot][blockIdx.x][4] = t_acc[0]; g_timing[sch.tslot][blockIdx.x][5] = t_acc[1]; }
+    if (threadIdx.x == 32) {
+        g_timing[sch.tslot][blockIdx.x][4] = t_acc[0]; g_timing[sch.tslot][blockIdx.x][5] = t_acc[1];
+        for (int i = 0; i < 10; ++i) g_phase[blockIdx.x][i] = t_ph[i];
+    }
 #endif
     // after a timed-out wait: give copies that may still be in flight time to land before the CTA retires
     if (*abort_flag)
@@ -894,6 +937,15 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
             }
             fprintf(stderr, "launch %2d: first_start %8lld last_start %8lld first_end %8lld last_end %8lld  mean_busy %6lld ns mean_wait_full %6lld cyc\n",
                     l, g0 - base, g0max - base, g1min - base, g1 - base, busy / ncta, wf / ncta);
+            if (l == 63) {
+                static unsigned hp[kMaxCtas][12];
+                cudaMemcpyFromSymbol(hp, g_phase, sizeof(hp));
+                for (int c = 0; c < ncta; c += 6) {
+                    fprintf(stderr, "phase cta %3d tiles %3lld:", c, h[l][c][5]);
+                    for (int i = 0; i < 10; ++i) fprintf(stderr, " %6u", hp[c][i] / (unsigned)std::max(1ll, h[l][c][5]));
+                    fprintf(stderr, "\n");
+                }
+            }
             if (l == 45)
                 for (int c = 0; c < ncta; ++c)
                     fprintf(stderr, "cta %3d unit %2u mode %d tiles %2lld start %6lld waited %6lld loop_end %6lld end %6lld wait_full_cyc %6lld merged %6lld ticket %6lld\n", c,
