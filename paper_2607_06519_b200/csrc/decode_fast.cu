@@ -356,16 +356,42 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             const uint4* t_krows = reinterpret_cast<const uint4*>(ud.k_val);
             const uint4* t_vrows = reinterpret_cast<const uint4*>(ud.v_val);
             int ptk[2] = {0, 0}, ptv[2] = {0, 0};
-            auto load_ranges = [&](int j, int (&r)[4]) {
-                if (resid && j < npre) {
-                    const int o = (rev ? tb + npre - 1 - j : tb + j) * (kTT / kResTile) + warp;
+            // List ranges of this warp's slice, one tile per lane: lane l of a batch holds tile rb + l of the segment
+            // ({begin, end} of the K and of the V list), loaded 32 to 64 tiles before use and handed out by shuffle.
+            int rb = 0, rk[2] = {0, 0}, rv[2] = {0, 0}, rk_n[2] = {0, 0}, rv_n[2] = {0, 0};
+            auto load_batch = [&](int jb, int (&k)[2], int (&v)[2]) {
+                const int jj = jb + lane;
+                k[0] = k[1] = v[0] = v[1] = 0;
+                if (resid && jj < npre) {
+                    const int o = (rev ? tb + npre - 1 - jj : tb + jj) * (kTT / kResTile) + warp;
                     const int o0 = min(o, nres), o1 = min(o + 1, nres);
-                    r[0] = ud.k_off[o0]; r[1] = ud.k_off[o1];
-                    if (tokmode) { r[2] = r[0]; r[3] = r[1]; }
-                    else { r[2] = ud.v_off[o0]; r[3] = ud.v_off[o1]; }
-                } else {
-                    r[0] = r[1] = r[2] = r[3] = 0;
+                    k[0] = ud.k_off[o0]; k[1] = ud.k_off[o1];
+                    if (tokmode) { v[0] = k[0]; v[1] = k[1]; }
+                    else { v[0] = ud.v_off[o0]; v[1] = ud.v_off[o1]; }
                 }
+            };
+            auto get_ranges = [&](int j, int (&r)[4]) {  // rb <= j < rb + 64
+                const bool nx = j - rb >= 32;
+                const int src = (j - rb) & 31;
+                r[0] = __shfl_sync(0xFFFFFFFFu, nx ? rk_n[0] : rk[0], src);
+                r[1] = __shfl_sync(0xFFFFFFFFu, nx ? rk_n[1] : rk[1], src);
+                r[2] = __shfl_sync(0xFFFFFFFFu, nx ? rv_n[0] : rv[0], src);
+                r[3] = __shfl_sync(0xFFFFFFFFu, nx ? rv_n[1] : rv[1], src);
+            };
+            // pull a tile's list slices (or selected token rows) into L2 a few tiles ahead: lanes 0-15 the K side,
+            // lanes 16-31 the V side, one 128-byte line each
+            auto l2_prefetch = [&](const int (&r)[4]) {
+                const int hl = lane & 15;
+                const void* ptr = nullptr;
+                if (tokmode) {
+                    const int j = r[0] + (hl >> 1);
+                    if (j < r[1]) ptr = reinterpret_cast<const char*>(lane < 16 ? t_krows : t_vrows) + (int64_t)j * 256 + (hl & 1) * 128;
+                } else {
+                    const int e0 = lane < 16 ? r[0] : r[2], e1 = lane < 16 ? r[1] : r[3];
+                    const int e = (e0 & ~31) + 32 * hl;
+                    if (e < e1) ptr = (lane < 16 ? k_ent : v_ent) + e;
+                }
+                if (ptr) asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
             };
             auto prefetch = [&](const uint32_t* ent, int e0, int e1, uint32_t (&pe)[kPF]) {
 #pragma unroll
@@ -419,8 +445,16 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 for (int i = 0; i < kScratchBytes / 16 / 32; ++i) st_shared_zero16(scratch + (lane + 32 * i) * 16);
             };
             if (resid) {
-                load_ranges(0, cr);
-                load_ranges(1, nr);
+                load_batch(0, rk, rv);
+                load_batch(32, rk_n, rv_n);
+                get_ranges(0, cr);
+                get_ranges(1, nr);
+                {
+                    int fr[4];
+                    get_ranges(2, fr);
+                    l2_prefetch(nr);
+                    l2_prefetch(fr);
+                }
                 if (tokmode) {
                     prefetch_tok(t_krows, cr[0], cr[1], pke, ptk);
                     prefetch_tok(t_vrows, cr[2], cr[3], pve, ptv);
@@ -600,7 +634,17 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 TPH(8);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) cr[i] = nr[i];
-                load_ranges(j + 2, nr);
+                if (resid) {
+                    if (j + 1 - rb == 32) {  // the next tile opens a new batch
+                        rk[0] = rk_n[0]; rk[1] = rk_n[1]; rv[0] = rv_n[0]; rv[1] = rv_n[1];
+                        rb += 32;
+                        load_batch(rb + 32, rk_n, rv_n);
+                    }
+                    int fr[4];
+                    get_ranges(j + 2, nr);
+                    get_ranges(j + 3, fr);
+                    l2_prefetch(fr);
+                }
                 TPH(9);
             }
             it += nseg;
@@ -801,14 +845,15 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     }
     static double res_cost = -1.0;
     static bool use_pdl = true;
-    // tiles copied before the dependency wait; more than one takes HBM bandwidth from the kernel still running
-    static int prologue_tiles = 1;
+    // tiles copied to shared memory before the dependency wait (measured: filling every stage is best; prefetching
+    // further tiles to L2 as well takes bandwidth from the CTAs of the previous kernel that are still streaming)
+    static int prologue_tiles = kStages;
     static bool whole_ctas = true;
     static bool reverse_odd = true;
     if (res_cost < 0) {
         const char* ev = getenv("FDKV_RES_COST");  // tuning knobs for benchmark sweeps
-        res_cost = ev ? atof(ev) : 1.6;
-        if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 1.6;
+        res_cost = ev ? atof(ev) : 2.0;
+        if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 2.0;
         const char* pv = getenv("FDKV_NO_PDL");
         use_pdl = !(pv && pv[0] == '1');
         const char* ro = getenv("FDKV_NO_REVERSE");
@@ -816,7 +861,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         const char* wc = getenv("FDKV_NO_WHOLE_CTAS");
         whole_ctas = !(wc && wc[0] == '1');
         const char* pt = getenv("FDKV_PROLOGUE_TILES");
-        prologue_tiles = pt ? std::max(0, std::min(kStages, atoi(pt))) : 1;
+        prologue_tiles = pt ? std::max(0, std::min(kStages, atoi(pt))) : kStages;
     }
     // ---- cost-weighted schedule: whole CTAs per unit when there are enough CTAs, else a flat cut of the (unit, tile) list ----
     FastSched sch;
