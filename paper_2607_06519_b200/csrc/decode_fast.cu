@@ -3,15 +3,23 @@
 // cache never materialised).
 //
 // One persistent CTA of eight warps per SM.  128-token K and V boxes of the packed cache stream through a ring of
-// shared-memory stages with TMA (128-byte swizzle, mbarrier completion); lane 0 of warp 0 issues the copies two
-// tiles ahead of the compute.  Each warp owns 16 tokens of a stage and a private online-softmax state:
-//   S^T = q K^T   mma.sync m16n8k16 (heads on M, tokens on N; ldmatrix of the swizzled K box),
-//   P = exp2(S - max), split into bf16 hi + lo halves held in rows 0-7 / 8-15 of the next A operand,
-//   O += P V      mma.sync (ldmatrix.trans of the V box).
+// shared-memory stages with TMA (128-byte swizzle, mbarrier completion).  The CTA's tile sequence sits in a small
+// segment table in shared memory; whichever warp finishes a tile last re-arms its stage with the tile three ahead,
+// so no warp is a dedicated producer.  Each warp owns 16 tokens of a stage and a private online-softmax state:
+//   S = K q^T        mma.sync m16n8k16, tokens on M (ldmatrix of the swizzled K box), the G query heads on N;
+//   P = exp2(S - max) per column; for G <= 4 columns 4-7 repeat the heads and carry the bf16 rounding remainder of
+//                    P, so P acts with ~16 bits; movmatrix turns the accumulator layout into the next B operand;
+//   O^T += V^T P^T   mma.sync, channels on M (ldmatrix.trans of the V box).
+// (Heads on M, as in a prefill kernel, would use 4 of 16 rows and twice the instructions: mma.sync runs at a quarter
+// of the tcgen05 rate on this part and was the limiter in that form.)
 // Residual units: the warp scatters its slice's kept Z1 entries into a private zeroed 16x128 bf16 scratch tile
-// and runs the same two products on it with the layer's sign, so the correction is exact in float32.
-// Work is a flat list of (unit, tile) pairs cut into one contiguous range per CTA (byte-weighted), so a CTA may
-// finish one unit and start the next; each (CTA, unit) segment writes one split-K partial.
+// and runs the same two products on it with the layer's sign, so the correction is exact in float32.  (Adding the
+// entries into the landed rows in place, rounded to bf16, was faster to write but quadrupled the output error.)
+// The list ranges are loaded one tile per lane 32-64 tiles ahead and handed out by shuffle; the lists themselves
+// are pulled into L2 three tiles ahead and into registers one tile ahead.
+// Work is a flat list of (unit, tile) pairs cut into one contiguous range per CTA (cost-weighted), so a CTA may
+// finish one unit and start the next; each (CTA, unit) segment writes one split-K partial and the CTA that takes
+// the unit's last ticket combines them.
 #include <cuda.h>
 
 #include <algorithm>
@@ -348,7 +356,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             // ---- residual lists (packed entries): ranges two tiles ahead, entries one tile ahead ----
             const uint32_t* k_ent = reinterpret_cast<const uint32_t*>(ud.k_idx);
             const uint32_t* v_ent = reinterpret_cast<const uint32_t*>(ud.v_idx);
-            int cr[4] = {0, 0, 0, 0}, nr[4] = {0, 0, 0, 0};  // {k begin, k end, v begin, v end}
+            int cr[4] = {0, 0, 0, 0}, nr[4] = {0, 0, 0, 0}, fr[4] = {0, 0, 0, 0};  // {k begin, k end, v begin, v end}: this tile, next, the one after
             uint32_t pke[kPF], pve[kPF];
             // token-granular residual: one ascending token list (k_idx) with per-slice counts (k_off) for K and V,
             // and the selected tokens' Z1 rows packed densely (k_val / v_val, 256 bytes each)
@@ -449,12 +457,9 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 load_batch(32, rk_n, rv_n);
                 get_ranges(0, cr);
                 get_ranges(1, nr);
-                {
-                    int fr[4];
-                    get_ranges(2, fr);
-                    l2_prefetch(nr);
-                    l2_prefetch(fr);
-                }
+                get_ranges(2, fr);
+                l2_prefetch(nr);
+                l2_prefetch(fr);
                 if (tokmode) {
                     prefetch_tok(t_krows, cr[0], cr[1], pke, ptk);
                     prefetch_tok(t_vrows, cr[2], cr[3], pve, ptv);
@@ -509,31 +514,33 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 {
                     const int mi = lane >> 3, rr = lane & 7;
                     const int row = r0 + (mi & 1) * 8 + rr;  // ldmatrix: matrices = (tokens 0-7 | 8-15) x (chunk | chunk + 1)
-                    if (sch.experiment != 3)  // (timing experiment 3 skips this product)
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const int c = 2 * kk + (mi >> 1);  // 16-byte channel chunk 0..15
-                        uint32_t a0, a1, a2, a3;
-                        ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
-                        mma_bf16(sacc[kk & 1], a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
-                    }
-                    TPH(2);
                     if (with_res && cr[1] > cr[0]) {
-                        float racc[4] = {0.f, 0.f, 0.f, 0.f};  // own accumulator: this chain runs beside the two above
+                        float racc[4] = {0.f, 0.f, 0.f, 0.f};  // the residual's own chain, interleaved with the two main ones
                         const int srow = (mi & 1) * 8 + rr;
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const int c = 2 * kk + (mi >> 1);
-                            uint32_t a0, a1, a2, a3;
-                            ldsm_x4(scratch + (c >> 3) * 2048 + swz(srow, c), a0, a1, a2, a3);
-                            mma_bf16(racc, a0, a1, a2, a3, qb[kk][0] ^ sgn, qb[kk][1] ^ sgn);
+                            uint32_t a0, a1, a2, a3, e0, e1, e2, e3;
+                            ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
+                            ldsm_x4(scratch + (c >> 3) * 2048 + swz(srow, c), e0, e1, e2, e3);
+                            mma_bf16(sacc[kk & 1], a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
+                            mma_bf16(racc, e0, e1, e2, e3, qb[kk][0] ^ sgn, qb[kk][1] ^ sgn);
                         }
 #pragma unroll
                         for (int i = 0; i < 4; ++i) sacc[0][i] += racc[i];
                         __syncwarp();
                         zero_scratch();
                         __syncwarp();
+                    } else if (sch.experiment != 3) {  // (timing experiment 3 skips this product)
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const int c = 2 * kk + (mi >> 1);
+                            uint32_t a0, a1, a2, a3;
+                            ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
+                            mma_bf16(sacc[kk & 1], a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
+                        }
                     }
+                    TPH(2);
                 }
                 TPH(3);
                 if (with_res && cr[3] > cr[2]) {
@@ -640,8 +647,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                         rb += 32;
                         load_batch(rb + 32, rk_n, rv_n);
                     }
-                    int fr[4];
-                    get_ranges(j + 2, nr);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) nr[i] = fr[i];
                     get_ranges(j + 3, fr);
                     l2_prefetch(fr);
                 }
@@ -852,8 +859,8 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     static bool reverse_odd = true;
     if (res_cost < 0) {
         const char* ev = getenv("FDKV_RES_COST");  // tuning knobs for benchmark sweeps
-        res_cost = ev ? atof(ev) : 2.0;
-        if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 2.0;
+        res_cost = ev ? atof(ev) : 1.7;
+        if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 1.7;
         const char* pv = getenv("FDKV_NO_PDL");
         use_pdl = !(pv && pv[0] == '1');
         const char* ro = getenv("FDKV_NO_REVERSE");
