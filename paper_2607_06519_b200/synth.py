@@ -24,6 +24,7 @@ import os
 import numpy as np
 
 TAG_K, TAG_V, TAG_NEEDLE, TAG_PROBE_Q, TAG_DECODE_Q, TAG_TAIL_K, TAG_TAIL_V, TAG_RHO = range(8)
+TAG_BLOCK_K, TAG_BLOCK_V, TAG_BLOCK_TAIL_K, TAG_BLOCK_TAIL_V = range(8, 12)  # four-layer blocks
 
 
 @dataclass(frozen=True)
@@ -47,10 +48,15 @@ class Workload:
     n_steps: int = 1
     seq_seeds: tuple | None = None  # per-sequence seed override (batched workload)
     residual_rule: int = 0  # 0: largest-magnitude entries; 1: probe-scored tokens (the paper's rule)
+    block_size: int = 2  # layers per depth block (2 or 4)
 
     @property
     def n_pairs(self) -> int:
         return self.n_layers // 2
+
+    @property
+    def n_blocks(self) -> int:
+        return self.n_layers // self.block_size
 
     @property
     def group(self) -> int:
@@ -99,6 +105,10 @@ WORKLOADS["decode128k_4l"] = WORKLOADS["decode128k"].scaled(n_layers=4, name="de
 # the same 32k workload with the paper's token-granular residual (probe-scored tokens keep whole rows)
 WORKLOADS["decode32k_tok"] = WORKLOADS["decode32k"].scaled(residual_rule=1, name="decode32k_tok")
 WORKLOADS["decode32k_tok_4l"] = WORKLOADS["decode32k_tok"].scaled(n_layers=4, name="decode32k_tok_4l")
+# depth blocks of four layers (the paper's default block size): tiny correctness case and the 32k shape
+WORKLOADS["tiny_b4"] = WORKLOADS["tiny"].scaled(n_layers=4, block_size=4, name="tiny_b4")
+WORKLOADS["decode32k_b4"] = WORKLOADS["decode32k"].scaled(block_size=4, name="decode32k_b4")
+WORKLOADS["decode32k_b4_8l"] = WORKLOADS["decode32k"].scaled(n_layers=8, block_size=4, name="decode32k_b4_8l")
 
 
 def rng(seed: int, seq: int, a: int, b: int, tag: int) -> np.random.Generator:
@@ -162,6 +172,74 @@ def unit_tensor(w: Workload, seq: int, pair: int, h: int, is_v: bool):
     u0 *= sigma
     x1 = _rs(u0, w.dtype)
     return x0, x1
+
+
+def block_tensor(w: Workload, seq: int, blk: int, h: int, is_v: bool):
+    """[x0, x1, x2, x3]: the [T, d] K (or V) tensors of the four layers of block `blk` for KV head h.
+
+    A first-order chain in unit-variance space: u_0 ~ N(0,1), u_l = rho u_{l-1} + sqrt(1-rho^2) m n_l, each layer
+    scaled by the head's per-channel sigma; m is 8 on the planted needle tokens."""
+    T, d = w.T, w.head_dim
+    r = rng(w.seed_of(seq), seq, blk, h, TAG_BLOCK_V if is_v else TAG_BLOCK_K)
+    sigma = np.exp(r.standard_normal(d)).astype(np.float32)
+    u = r.standard_normal((T, d), dtype=np.float32)
+    rho = rho_of(w, seq, blk)
+    rho32 = np.float32(rho)
+    beta32 = np.float32(np.sqrt(1.0 - rho * rho))
+    m = np.ones((T, 1), dtype=np.float32)
+    m[needle_positions(w, seq, blk, h), 0] = np.float32(8.0)
+    out = [_rs(u * sigma, w.dtype)]
+    for _ in range(3):
+        n = r.standard_normal((T, d), dtype=np.float32)
+        n *= m
+        n *= beta32
+        u = u * rho32
+        u += n
+        out.append(_rs(u * sigma, w.dtype))
+    return out
+
+
+def block_sigma(w: Workload, seq: int, blk: int, h: int, is_v: bool) -> np.ndarray:
+    r = rng(w.seed_of(seq), seq, blk, h, TAG_BLOCK_V if is_v else TAG_BLOCK_K)
+    return np.exp(r.standard_normal(w.head_dim)).astype(np.float32)
+
+
+def block_tail_rows(w: Workload, seq: int, blk: int, h: int, is_v: bool):
+    """[x0_new .. x3_new]: [n_steps, d] generated-token rows for the four layers of a block (same chain, m = 1)."""
+    sigma = block_sigma(w, seq, blk, h, is_v)
+    r = rng(w.seed_of(seq), seq, blk, h, TAG_BLOCK_TAIL_V if is_v else TAG_BLOCK_TAIL_K)
+    rho = rho_of(w, seq, blk)
+    rho32 = np.float32(rho)
+    beta32 = np.float32(np.sqrt(1.0 - rho * rho))
+    u = r.standard_normal((w.n_steps, w.head_dim), dtype=np.float32)
+    out = [_rs(u * sigma, w.dtype)]
+    for _ in range(3):
+        n = r.standard_normal((w.n_steps, w.head_dim), dtype=np.float32)
+        u = rho32 * u + beta32 * n
+        out.append(_rs(u * sigma, w.dtype))
+    return out
+
+
+def layer_block_kv(w: Workload, seq: int, blk: int, threads: int | None = None):
+    """K and V of the four layers of a block in model layout: dict k0..k3, v0..v3, each [T, Hkv, d] float32."""
+    T, H, d = w.T, w.n_kv_heads, w.head_dim
+    out = {f"{n}{l}": np.empty((T, H, d), dtype=np.float32) for n in ("k", "v") for l in range(4)}
+
+    def fill(job):
+        h, is_v = job
+        xs = block_tensor(w, seq, blk, h, is_v)
+        for l in range(4):
+            out[f"{'v' if is_v else 'k'}{l}"][:, h, :] = xs[l]
+
+    jobs = [(h, is_v) for h in range(H) for is_v in (False, True)]
+    n = threads or min(len(jobs), os.cpu_count() or 1)
+    if n <= 1:
+        for j in jobs:
+            fill(j)
+    else:
+        with ThreadPoolExecutor(n) as ex:
+            list(ex.map(fill, jobs))
+    return out
 
 
 def probe_q(w: Workload, seq: int, layer: int) -> np.ndarray:
