@@ -51,7 +51,7 @@ typedef enum { FDKV_F32 = 0, FDKV_BF16 = 1 } fdkv_dtype;
 typedef enum { FDKV_MODE_SHARED = 0, FDKV_MODE_RESIDUAL = 1, FDKV_MODE_EXACT = 2 } fdkv_mode;
 
 typedef struct {
-    int32_t n_layers;    /* even; pair p = layers 2p, 2p+1 (block size B = 2 of Eq. 1)                 */
+    int32_t n_layers;    /* multiple of the block size B of Eq. 1; block p = layers B p .. B p + B - 1   */
     int32_t n_q_heads;   /* multiple of n_kv_heads; group size n_q_heads / n_kv_heads <= 8             */
     int32_t n_kv_heads;
     int32_t head_dim;    /* 64 or 128                                                                  */
@@ -62,7 +62,25 @@ typedef struct {
     int32_t keep_num;    /* residual keep fraction: k = floor(T * head_dim * keep_num / keep_den)      */
     int32_t keep_den;    /*   entries per (unit, K or V); 0 <= keep_num <= keep_den                    */
     int32_t residual_rule; /* fdkv_residual_rule: how the sparse high-frequency residual is chosen     */
+    int32_t block_size;  /* B of Eq. 1: 2 (also when 0) or 4 layers per depth block                    */
 } fdkv_config;
+
+/*
+ * Block size 4 (Method, Eq. 1 with the orthonormal DCT-II of size 4; the paper's default for middle layers).
+ * Wherever this header says "pair" read "block": pair ranges index blocks, a unit is (block, KV head), modes and
+ * scores have one entry per unit.  What is stored per tensor (K or V) of a unit, in float32 arithmetic that is
+ * never contracted, rs = rounding to the storage type:
+ *     s = (x0 + x1) + (x2 + x3);   Z0 = rs(0.5 s)                the shared coefficient (first DCT row = 1/2 each)
+ *     dev_l = rs(x_l - 0.5 Z0),  l = 0..3                         layer l's high-frequency part in layer space:
+ *                                                                 sum_{j>=1} F_4[j][l] Z_j = x_l - mean(x)
+ *     e = (dev_0^2 + dev_1^2) + (dev_2^2 + dev_3^2)               the position's high-frequency energy (Parseval)
+ * The three high-frequency groups share one kept set per tensor (Eq. 3): the k positions of largest e, ties to the
+ * lowest flat index; the four values dev_l are kept there (instead of three coefficients), so that a decode call of
+ * layer l reads one value per kept position.  Candidates: shared = Z0 / 2, residual = Z0 / 2 + dev_l on the kept
+ * positions, exact = x_l.  Eq. 2 averages over the block's four layers; Omega(residual) counts four values and one
+ * int32 index per kept position, Omega(exact) four layers.  The mixed schedule of the paper (B = 4 in the middle,
+ * B = 2 for the first and last layers) is two contexts, one per block size.  Entry residual rule only.
+ */
 
 /*
  * FDKV_RESIDUAL_ENTRIES (default): the k largest-magnitude entries of Z1, K and V independently (chosen in

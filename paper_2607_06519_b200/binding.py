@@ -31,7 +31,7 @@ class FdkvError(RuntimeError):
 
 class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "max_batch", "max_prefill",
-                                         "max_tail", "dtype", "keep_num", "keep_den", "residual_rule")]
+                                         "max_tail", "dtype", "keep_num", "keep_den", "residual_rule", "block_size")]
 
 
 def _load():
@@ -99,6 +99,7 @@ class Config:
     keep_num: int
     keep_den: int
     residual_rule: int = 0  # 0: largest-magnitude entries; 1: the paper's probe-scored tokens
+    block_size: int = 2  # layers per depth block (B of Eq. 1): 2 or 4; "pair" arguments then index blocks
 
     def c(self) -> _Config:
         return _Config(*(int(getattr(self, f[0])) for f in _Config._fields_))
@@ -161,7 +162,8 @@ class Context:
             _check(_lib.fdkv_create(C.byref(cfg.c()), self.arena.data_ptr(), self.arena_bytes, self.work.data_ptr(), work,
                                     C.byref(h)), "fdkv_create")
         self.h = h
-        self.n_pairs = cfg.n_layers // 2
+        self.block_size = cfg.block_size or 2
+        self.n_pairs = cfg.n_layers // self.block_size  # depth blocks (pairs when the block size is 2)
 
     def close(self):
         if getattr(self, "h", None):
@@ -252,7 +254,8 @@ class Context:
                "fdkv_get_residual")
         k = cnt.value
         idx = torch.empty(k, dtype=torch.int32, device=self.device)
-        val = torch.empty(k, dtype=self.tdtype, device=self.device)
+        # a block of four layers keeps four values per position: [4, k]
+        val = torch.empty((4, k) if self.block_size == 4 else (k,), dtype=self.tdtype, device=self.device)
         _check(_lib.fdkv_get_residual(self.h, seq, pair, kv_head, int(is_v), _ptr(idx), _ptr(val), C.byref(cnt),
                                       _stream(stream)), "fdkv_get_residual")
         return idx, val

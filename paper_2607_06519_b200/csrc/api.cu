@@ -28,7 +28,9 @@ fdkv_status cuda_fail(cudaError_t e) {
     } while (0)
 
 bool make_shape(const fdkv_config& c, Shape& s) {
-    if (c.n_layers <= 0 || (c.n_layers & 1) || c.n_layers > 1024) return false;
+    const int B = c.block_size == 0 ? 2 : c.block_size;
+    if (B != 2 && B != 4) return false;
+    if (c.n_layers <= 0 || (c.n_layers % B) || c.n_layers > 1024) return false;
     if (c.n_kv_heads <= 0 || c.n_q_heads <= 0 || c.n_q_heads % c.n_kv_heads) return false;
     const int G = c.n_q_heads / c.n_kv_heads;
     if (!(G == 1 || G == 2 || G == 4 || G == 8)) return false;
@@ -37,7 +39,7 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     if ((int64_t)c.max_prefill * c.head_dim >= (int64_t)1 << 31) return false;
     if (c.dtype != FDKV_F32 && c.dtype != FDKV_BF16) return false;
     if (c.keep_den <= 0 || c.keep_num < 0 || c.keep_num > c.keep_den) return false;
-    s.L = c.n_layers; s.P = c.n_layers / 2; s.Hq = c.n_q_heads; s.Hkv = c.n_kv_heads; s.G = G; s.d = c.head_dim;
+    s.L = c.n_layers; s.B = B; s.NB = B == 4 ? 4 : 1; s.P = c.n_layers / B; s.Hq = c.n_q_heads; s.Hkv = c.n_kv_heads; s.G = G; s.d = c.head_dim;
     s.max_batch = c.max_batch; s.Tmax = c.max_prefill; s.max_tail = c.max_tail;
     s.dtype = c.dtype; s.esize = c.dtype == FDKV_BF16 ? 2 : 4;
     s.keep_num = c.keep_num; s.keep_den = c.keep_den;
@@ -49,6 +51,7 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     if (c.residual_rule != FDKV_RESIDUAL_ENTRIES && c.residual_rule != FDKV_RESIDUAL_TOKENS) return false;
     s.tok_rule = c.residual_rule == FDKV_RESIDUAL_TOKENS;
     if (s.tok_rule && !(c.dtype == FDKV_BF16 && c.head_dim == 128)) return false;  // tensor-core kernels only
+    if (s.tok_rule && B != 2) return false;
     s.ktok_max = (int64_t)s.Tmax * s.keep_num / s.keep_den;
     s.ktok_cap = (int64_t)align_up((size_t)(s.ktok_max + 32), 64);
     s.NU = s.P * s.Hkv;
@@ -62,16 +65,18 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     const size_t unit_elems = (size_t)s.Tmax * s.d;
     w.status = take(256);
     w.z0 = take((size_t)s.NT * unit_elems * s.esize);
-    w.z1 = take((size_t)s.NT * unit_elems * s.esize);
-    w.z1drop = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NU * unit_elems * s.esize : 0);
+    w.z1 = take((size_t)s.NT * s.NB * unit_elems * s.esize);  // Z1 of a pair, or the four layers' deviations of a block
+    w.z1drop = take(s.B == 2 && s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NU * unit_elems * s.esize : 0);
+    w.energy = take(s.B == 4 ? (size_t)s.NT * unit_elems * 4 : 0);
+    w.eval = take(s.B == 4 ? (size_t)s.NT * s.kcap * 4 : 0);
     w.hist = take((size_t)s.NT * kHistBins * 4);
     w.sel = take((size_t)s.NT * sizeof(SelState));
     w.tile_cnt = take((size_t)s.NT * s.ntiles_max * 8);
     w.tile_eq = take((size_t)s.NT * s.ntiles_max * 4);
     w.tile_off = take((size_t)s.NT * (s.ntiles_max + 1) * 4);
     w.idx = take((size_t)s.NT * s.kcap * 4);
-    w.val = take((size_t)s.NT * s.kcap * s.esize);
-    w.packed = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NT * s.kcap * 4 : 0);
+    w.val = take((size_t)s.NT * s.NB * s.kcap * s.esize);
+    w.packed = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NT * s.NB * s.kcap * 4 : 0);
     w.tok_score = take(s.tok_rule ? (size_t)s.NU * s.Tmax * 4 : 0);
     w.tok_flag = take(s.tok_rule ? (size_t)s.NU * s.Tmax : 0);
     w.tok_list = take(s.tok_rule ? (size_t)s.NU * s.ktok_cap * 4 : 0);
@@ -96,12 +101,12 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     a.tail_v = take(tail);
     a.bump = o;
     const size_t rows_pad = align_up((size_t)((s.Tmax + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize);
-    const size_t exact_unit = 4 * rows_pad;
+    const size_t exact_unit = 2 * (size_t)s.B * rows_pad;
     const size_t resid_unit = s.tok_rule
                                   ? 2 * rows_pad + 2 * align_up((size_t)s.ktok_cap * s.d * s.esize) + align_up((size_t)s.ktok_cap * 4) +
                                         align_up((size_t)(s.ntiles_max + 1) * 4)
-                                  : 2 * rows_pad + 2 * align_up((size_t)s.kcap * 4) + 2 * align_up((size_t)s.kcap * s.esize) +
-                                        2 * align_up((size_t)(s.ntiles_max + 1) * 4);
+                                  : 2 * rows_pad + 2 * (size_t)s.NB * (align_up((size_t)s.kcap * 4) + align_up((size_t)s.kcap * s.esize)) +
+                                        2 * align_up((size_t)s.kcap * 4) + 2 * align_up((size_t)(s.ntiles_max + 1) * 4);
     a.worst_total = a.bump + (size_t)s.max_batch * s.NU * (exact_unit > resid_unit ? exact_unit : resid_unit);
 }
 
@@ -112,6 +117,21 @@ template <typename T>
 inline T* arp(fdkv_ctx* c, size_t off) { return reinterpret_cast<T*>(c->arena + off); }
 
 bool seq_ok(fdkv_ctx* c, int seq) { return c && seq >= 0 && seq < c->s.max_batch; }
+
+// Omega(m) of Eq. 2 for one unit (K and V together): bytes of the mode / bytes of the exact mode.  Returns the latter.
+// Residual bytes per kept position: one value and one int32 index (pair), four layer values and one index (block of
+// four); token rule: d values per kept token and one index.
+double omega_of(const Shape& s, int T, double (&om)[3]) {
+    const double e = s.esize, Td = (double)T * s.d;
+    const double k = (double)((int64_t)T * s.d * s.keep_num / s.keep_den);
+    const double k_tok = (double)((int64_t)T * s.keep_num / s.keep_den);
+    const double b_sh = 2.0 * Td * e, b_ex = 2.0 * s.B * Td * e;
+    double b_rs;
+    if (s.tok_rule) b_rs = b_sh + 2.0 * k_tok * s.d * e + 4.0 * k_tok;
+    else b_rs = b_sh + 2.0 * k * (s.NB * e + 4.0);
+    om[0] = b_sh / b_ex; om[1] = b_rs / b_ex; om[2] = 1.0;
+    return b_ex;
+}
 
 }  // namespace
 
@@ -173,7 +193,7 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
         const bool ok = c->packed_lists && make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
         if (!ok) { delete c; return FDKV_ERR_UNSUPPORTED; }
     }
-    if (s.dtype == FDKV_BF16 && s.d == 128)
+    if (s.B == 2 && s.dtype == FDKV_BF16 && s.d == 128)
         c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_z1) &&
                              make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_drop);
     if (s.tok_rule && !c->has_probe_tmaps) { delete c; return FDKV_ERR_UNSUPPORTED; }
@@ -209,7 +229,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     if (pb < 0 || pe > s.P || pb >= pe) return FDKV_ERR_INVALID_ARG;
     if (T < 1 || T > s.Tmax) return FDKV_ERR_INVALID_ARG;
     if (stride_h < s.d || stride_t < s.d || (stride_t % 8) || (stride_h % 8)) return FDKV_ERR_INVALID_ARG;
-    for (int l = 2 * pb; l < 2 * pe; ++l)
+    for (int l = s.B * pb; l < s.B * pe; ++l)
         if (!k_layers[l] || !v_layers[l] || !aligned(k_layers[l], 16) || !aligned(v_layers[l], 16))
             return FDKV_ERR_INVALID_ARG;
     if (c->seqs[seq].committed) return FDKV_ERR_STATE;
@@ -229,6 +249,54 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     cudaStream_t st = S(stream);
     const int ut_begin = pb * s.Hkv * 2, ut_count = (pe - pb) * s.Hkv * 2;
     CU(cudaMemsetAsync(wsp<uint32_t>(c, c->ws.hist) + (size_t)ut_begin * kHistBins, 0, (size_t)ut_count * kHistBins * 4, st));
+    if (s.B == 4) {
+        // blocks of four layers: Z0, the layers' deviations and the positions' energies; one kept set per tensor from
+        // the float32 radix select on the energies; then the four layers' values at the kept positions
+        for (int p = pb; p < pe; ++p) {
+            Split4Args a4;
+            for (int l = 0; l < 4; ++l) {
+                a4.k[l] = k_layers[4 * p + l];
+                a4.v[l] = v_layers[4 * p + l];
+                c->k_layers[4 * p + l] = a4.k[l];
+                c->v_layers[4 * p + l] = a4.v[l];
+            }
+            a4.stride_t = stride_t; a4.stride_h = stride_h;
+            a4.T = T; a4.d = s.d; a4.Hkv = s.Hkv;
+            a4.ut_base = p * s.Hkv * 2;
+            a4.unit_stride = (int64_t)s.Tmax * s.d;
+            a4.z0 = c->work + c->ws.z0; a4.dev = c->work + c->ws.z1;
+            a4.energy = wsp<float>(c, c->ws.energy);
+            a4.hist = wsp<uint32_t>(c, c->ws.hist);
+            CU(launch_split4_hist(a4, s.dtype, st));
+        }
+        SelectArgs sa;
+        sa.ut_begin = ut_begin; sa.ut_count = ut_count;
+        sa.T = T; sa.d = s.d;
+        sa.k = (int64_t)T * s.d * s.keep_num / s.keep_den;
+        sa.unit_stride = (int64_t)s.Tmax * s.d; sa.kcap = s.kcap; sa.ntiles_max = s.ntiles_max;
+        sa.z1 = c->work + c->ws.energy;
+        sa.hist = wsp<uint32_t>(c, c->ws.hist);
+        sa.sel = wsp<SelState>(c, c->ws.sel);
+        sa.tile_cnt = wsp<uint32_t>(c, c->ws.tile_cnt);
+        sa.tile_eq = wsp<uint32_t>(c, c->ws.tile_eq);
+        sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
+        sa.idx = wsp<int32_t>(c, c->ws.idx);
+        sa.val = c->work + c->ws.eval;
+        sa.packed = nullptr;
+        sa.z1drop = nullptr;
+        sa.status = wsp<int32_t>(c, c->ws.status);
+        CU(launch_select_and_compact(sa, FDKV_F32, st));
+        Gather4Args g;
+        g.ut_begin = ut_begin; g.ut_count = ut_count;
+        g.k = sa.k; g.kcap = s.kcap; g.unit_stride = (int64_t)s.Tmax * s.d;
+        g.dev = c->work + c->ws.z1;
+        g.idx = wsp<int32_t>(c, c->ws.idx);
+        g.val = c->work + c->ws.val;
+        g.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
+        CU(launch_gather4(g, s.dtype, st));
+        for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; c->pair_scored[p] = 0; }
+        return FDKV_OK;
+    }
     for (int p0 = pb; p0 < pe; p0 += kSplitPairs) {
         CompressArgs a;
         a.n_pairs = pe - p0 < kSplitPairs ? pe - p0 : kSplitPairs;
@@ -281,14 +349,15 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     const int T = c->staged_T;
     for (int i = 0; i < W; ++i)
         if (probe_pos[i] < 0 || probe_pos[i] >= T || (i && probe_pos[i] <= probe_pos[i - 1])) return FDKV_ERR_INVALID_ARG;
-    for (int l = 2 * pb; l < 2 * pe; ++l)
+    for (int l = s.B * pb; l < s.B * pe; ++l)
         if (!q_layers[l] || !aligned(q_layers[l], 16)) return FDKV_ERR_INVALID_ARG;
     cudaStream_t st = S(stream);
     int32_t* pos_dev = wsp<int32_t>(c, c->ws.probe_pos);
     const void** qptr_dev = reinterpret_cast<const void**>(c->work + c->ws.probe_pos + kMaxW * 4);
     CU(cudaMemcpyAsync(pos_dev, probe_pos, (size_t)W * 4, cudaMemcpyHostToDevice, st));
-    CU(cudaMemcpyAsync(qptr_dev + 2 * pb, q_layers + 2 * pb, (size_t)(pe - pb) * 2 * sizeof(void*), cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(qptr_dev + s.B * pb, q_layers + s.B * pb, (size_t)(pe - pb) * s.B * sizeof(void*), cudaMemcpyHostToDevice, st));
     ProbeArgs a;
+    a.B = s.B;
     a.unit_begin = pb * s.Hkv; a.unit_count = (pe - pb) * s.Hkv;
     a.T = T; a.d = s.d; a.Hq = s.Hq; a.Hkv = s.Hkv; a.G = s.G; a.W = W;
     a.unit_stride = (int64_t)s.Tmax * s.d; a.kcap = s.kcap;
@@ -302,12 +371,7 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     a.scores = wsp<double>(c, c->ws.scores);
     a.modes = wsp<int32_t>(c, c->ws.modes);
     a.lambda = lambda;
-    const double e = s.esize, Td = (double)T * s.d;
-    const double k = (double)((int64_t)T * s.d * s.keep_num / s.keep_den);
-    const double k_tok = (double)((int64_t)T * s.keep_num / s.keep_den);
-    const double b_sh = 2.0 * Td * e, b_ex = 4.0 * Td * e;
-    const double b_rs = s.tok_rule ? b_sh + 2.0 * k_tok * s.d * e + 4.0 * k_tok : b_sh + 2.0 * k * (e + 4.0);
-    a.omega[0] = b_sh / b_ex; a.omega[1] = b_rs / b_ex; a.omega[2] = 1.0;
+    omega_of(s, T, a.omega);
     a.modes_out = modes; a.scores_out = scores;
     a.tmap_z1 = c->has_probe_tmaps ? c->tmap_z1 : nullptr;
     a.tmap_drop = c->has_probe_tmaps ? c->tmap_drop : nullptr;
@@ -345,11 +409,8 @@ fdkv_status fdkv_route_budget(fdkv_ctx* c, int32_t seq, size_t budget_bytes, dou
     CU(cudaMemcpy(e.data(), c->work + c->ws.scores, e.size() * sizeof(double), cudaMemcpyDeviceToHost));
     // Omega of the staged sequence, as in fdkv_probe
     const int T = c->staged_T;
-    const double eb = s.esize, Td = (double)T * s.d;
-    const double k = (double)((int64_t)T * s.d * s.keep_num / s.keep_den), k_tok = (double)((int64_t)T * s.keep_num / s.keep_den);
-    const double b_sh = 2.0 * Td * eb, b_ex = 4.0 * Td * eb;
-    const double b_rs = s.tok_rule ? b_sh + 2.0 * k_tok * s.d * eb + 4.0 * k_tok : b_sh + 2.0 * k * (eb + 4.0);
-    const double om[3] = {b_sh / b_ex, b_rs / b_ex, 1.0};
+    double om[3];
+    const double b_ex = omega_of(s, T, om);
     auto mode_at = [&](int u, double lam) {
         const double L0 = e[2 * u] + lam * om[0], L1 = e[2 * u + 1] + lam * om[1], L2 = lam * om[2];
         int m = 0;
@@ -422,12 +483,15 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     const int64_t k_tok = (int64_t)T * s.keep_num / s.keep_den;
     const size_t trow_b = (size_t)(k_tok + 4) * s.d * s.esize, tlist_b = (size_t)(k_tok + 32) * 4;  // token rows, token list
     size_t need = 0;
+    // residual lists of one tensor: packed layout = one entry list per stored high-frequency tensor (one for a pair,
+    // four for a block of four layers); portable layout = one index list and one value list per such tensor
+    const size_t lists_b = c->packed_lists ? (size_t)s.NB * align_up(idx_b) : align_up(idx_b) + (size_t)s.NB * align_up(val_b);
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u];
         if (m < 0 || m > 2) return FDKV_ERR_STATE;
-        if (m == FDKV_MODE_EXACT) need += 4 * align_up(rows_pad);
+        if (m == FDKV_MODE_EXACT) need += 2 * (size_t)s.B * align_up(rows_pad);
         else if (s.tok_rule) need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * align_up(trow_b) + align_up(tlist_b) + align_up(off_b) : 0);
-        else need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * (align_up(idx_b) + align_up(val_b) + align_up(off_b)) : 0);
+        else need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * (lists_b + align_up(off_b)) : 0);
     }
     if (c->bump + need > c->arena_bytes) return FDKV_ERR_ARENA_FULL;
     size_t o = c->bump;
@@ -436,26 +500,26 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     const size_t unit_stride_b = (size_t)s.Tmax * s.d * s.esize;
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u], p = u / s.Hkv, h = u % s.Hkv;
-        UnitDesc* d0 = &c->desc_host[((size_t)seq * s.L + 2 * p) * s.Hkv + h];
-        UnitDesc* d1 = &c->desc_host[((size_t)seq * s.L + 2 * p + 1) * s.Hkv + h];
-        std::memset(d0, 0, sizeof(UnitDesc));
-        std::memset(d1, 0, sizeof(UnitDesc));
-        d0->mode = d1->mode = m;
-        d0->T = d1->T = T;
-        d0->sign = 1.f;
-        d1->sign = -1.f;
+        UnitDesc* dl[4] = {nullptr, nullptr, nullptr, nullptr};
+        for (int l = 0; l < s.B; ++l) {
+            dl[l] = &c->desc_host[((size_t)seq * s.L + (size_t)s.B * p + l) * s.Hkv + h];
+            std::memset(dl[l], 0, sizeof(UnitDesc));
+            dl[l]->mode = m;
+            dl[l]->T = T;
+            dl[l]->sign = s.B == 2 ? (l == 0 ? 1.f : -1.f) : 2.f;
+            dl[l]->scale = m == FDKV_MODE_EXACT ? 1.f : (s.B == 2 ? 0.70710678118654752440f : 0.5f);
+        }
         if (m == FDKV_MODE_EXACT) {
-            const void* src[4] = {c->k_layers[2 * p], c->k_layers[2 * p + 1], c->v_layers[2 * p], c->v_layers[2 * p + 1]};
-            char* dst[4];
-            for (int i = 0; i < 4; ++i) {
-                dst[i] = take(rows_pad);
-                if (rows_pad > rows) CU(cudaMemsetAsync(dst[i] + rows, 0, rows_pad - rows, st));
-                const char* sp = (const char*)src[i] + (size_t)h * c->stride_h * s.esize;
-                CU(launch_strided_copy(sp, c->stride_t, dst[i], T, s.d, s.esize, st));
-            }
-            d0->k_rows = dst[0]; d1->k_rows = dst[1];
-            d0->v_rows = dst[2]; d1->v_rows = dst[3];
-            by_mode[2] += 4 * rows;
+            for (int l = 0; l < s.B; ++l)
+                for (int is_v = 0; is_v < 2; ++is_v) {
+                    const void* src = is_v ? c->v_layers[s.B * p + l] : c->k_layers[s.B * p + l];
+                    char* dst = take(rows_pad);
+                    if (rows_pad > rows) CU(cudaMemsetAsync(dst + rows, 0, rows_pad - rows, st));
+                    const char* sp = (const char*)src + (size_t)h * c->stride_h * s.esize;
+                    CU(launch_strided_copy(sp, c->stride_t, dst, T, s.d, s.esize, st));
+                    (is_v ? dl[l]->v_rows : dl[l]->k_rows) = dst;
+                }
+            by_mode[2] += 2 * (size_t)s.B * rows;
         } else {
             char *tl = nullptr, *to = nullptr;
             if (s.tok_rule && m == FDKV_MODE_RESIDUAL) {  // one token list and one offset table serve K and V
@@ -470,13 +534,13 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 char* z0 = take(rows_pad);
                 if (rows_pad > rows) CU(cudaMemsetAsync(z0 + rows, 0, rows_pad - rows, st));
                 CU(cudaMemcpyAsync(z0, c->work + c->ws.z0 + ut * unit_stride_b, rows, cudaMemcpyDeviceToDevice, st));
-                (is_v ? d0->v_rows : d0->k_rows) = z0;
-                (is_v ? d1->v_rows : d1->k_rows) = z0;
+                for (int l = 0; l < s.B; ++l) (is_v ? dl[l]->v_rows : dl[l]->k_rows) = z0;
                 by_mode[m] += rows;
                 if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
                     char* rows_res = take(trow_b);
                     CU(launch_token_gather(c->work + c->ws.z1 + ut * unit_stride_b, (const int32_t*)tl, k_tok, rows_res, st));
-                    for (UnitDesc* d : {d0, d1}) {
+                    for (int l = 0; l < s.B; ++l) {
+                        UnitDesc* d = dl[l];
                         d->res_kind = 1;
                         d->k_idx = (const int32_t*)tl;
                         d->k_off = (const int32_t*)to;
@@ -484,22 +548,33 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                     }
                     by_mode[1] += (size_t)k_tok * s.d * s.esize;
                 } else if (m == FDKV_MODE_RESIDUAL) {
-                    char* pi = take(idx_b);
-                    char* pv = val_b ? take(val_b) : nullptr;
                     char* po = take(off_b);
-                    if (c->packed_lists) {
-                        CU(cudaMemcpyAsync(pi, c->work + c->ws.packed + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
-                    } else {
-                        CU(cudaMemcpyAsync(pi, c->work + c->ws.idx + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
-                        CU(cudaMemcpyAsync(pv, c->work + c->ws.val + ut * s.kcap * s.esize, val_b, cudaMemcpyDeviceToDevice, st));
-                    }
                     CU(cudaMemcpyAsync(po, c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, off_b, cudaMemcpyDeviceToDevice, st));
-                    for (UnitDesc* d : {d0, d1}) {
-                        (is_v ? d->v_idx : d->k_idx) = (const int32_t*)pi;
-                        (is_v ? d->v_val : d->k_val) = pv;
+                    char* pi_shared = nullptr;
+                    if (!c->packed_lists) {
+                        pi_shared = take(idx_b);
+                        CU(cudaMemcpyAsync(pi_shared, c->work + c->ws.idx + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
+                    }
+                    char *pi_l[4] = {nullptr, nullptr, nullptr, nullptr}, *pv_l[4] = {nullptr, nullptr, nullptr, nullptr};
+                    for (int j = 0; j < s.NB; ++j) {  // one list per stored high-frequency tensor
+                        const size_t lt = ut * s.NB + j;
+                        if (c->packed_lists) {
+                            pi_l[j] = take(idx_b);
+                            CU(cudaMemcpyAsync(pi_l[j], c->work + c->ws.packed + lt * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
+                        } else {
+                            pi_l[j] = pi_shared;
+                            pv_l[j] = take(val_b);
+                            CU(cudaMemcpyAsync(pv_l[j], c->work + c->ws.val + lt * s.kcap * s.esize, val_b, cudaMemcpyDeviceToDevice, st));
+                        }
+                    }
+                    for (int l = 0; l < s.B; ++l) {
+                        UnitDesc* d = dl[l];
+                        const int j = s.NB == 1 ? 0 : l;  // a pair's two layers read the same Z1 list with opposite signs
+                        (is_v ? d->v_idx : d->k_idx) = (const int32_t*)pi_l[j];
+                        (is_v ? d->v_val : d->k_val) = pv_l[j];
                         (is_v ? d->v_off : d->k_off) = (const int32_t*)po;
                     }
-                    by_mode[1] += (size_t)k * (c->packed_lists ? 4 : 4 + s.esize);
+                    by_mode[1] += (size_t)k * (c->packed_lists ? (size_t)4 * s.NB : 4 + (size_t)s.NB * s.esize);
                 }
             }
         }
@@ -531,7 +606,7 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
     std::vector<int32_t> host_T(batch), host_modes((size_t)batch * s.Hkv);
     for (int b = 0; b < batch; ++b) {
         host_T[b] = c->seqs[b].T;
-        for (int h = 0; h < s.Hkv; ++h) host_modes[(size_t)b * s.Hkv + h] = c->seqs[b].modes[(layer / 2) * s.Hkv + h];
+        for (int h = 0; h < s.Hkv; ++h) host_modes[(size_t)b * s.Hkv + h] = c->seqs[b].modes[(layer / s.B) * s.Hkv + h];
     }
     DecodeArgs a;
     a.tail_rows = s.tail_rows;
@@ -617,7 +692,9 @@ fdkv_status fdkv_get_residual(fdkv_ctx* c, int32_t seq, int32_t pair, int32_t h,
     const int64_t k = (int64_t)c->staged_T * s.d * s.keep_num / s.keep_den;
     if (count_host) *count_host = (int32_t)k;
     if (idx_out && k) CU(cudaMemcpyAsync(idx_out, c->work + c->ws.idx + ut * s.kcap * 4, (size_t)k * 4, cudaMemcpyDeviceToDevice, S(stream)));
-    if (val_out && k) CU(cudaMemcpyAsync(val_out, c->work + c->ws.val + ut * s.kcap * s.esize, (size_t)k * s.esize, cudaMemcpyDeviceToDevice, S(stream)));
+    for (int j = 0; j < s.NB && val_out && k; ++j)  // a block of four returns its four layers' values as [4][count]
+        CU(cudaMemcpyAsync((char*)val_out + (size_t)j * k * s.esize, c->work + c->ws.val + (ut * s.NB + j) * s.kcap * s.esize,
+                           (size_t)k * s.esize, cudaMemcpyDeviceToDevice, S(stream)));
     CU(cudaStreamSynchronize(S(stream)));
     return FDKV_OK;
 }
@@ -650,7 +727,7 @@ fdkv_status fdkv_footprint(fdkv_ctx* c, int32_t seq, size_t* bytes_by_mode_host,
     if (bytes_by_mode_host)
         for (int i = 0; i < 3; ++i) bytes_by_mode_host[i] = c->seqs[seq].bytes_by_mode[i];
     if (exact_equiv_bytes_host)
-        *exact_equiv_bytes_host = (size_t)c->s.NU * 4 * c->seqs[seq].T * c->s.d * c->s.esize;
+        *exact_equiv_bytes_host = (size_t)c->s.NU * 2 * c->s.B * c->seqs[seq].T * c->s.d * c->s.esize;
     return FDKV_OK;
 }
 
@@ -664,7 +741,7 @@ fdkv_status fdkv_decode_bytes(fdkv_ctx* c, int32_t layer, int32_t batch, size_t*
         const int64_t k = (int64_t)q.T * s.d * s.keep_num / s.keep_den;
         const int ntiles = (q.T + kResTile - 1) / kResTile;
         for (int h = 0; h < s.Hkv; ++h) {
-            const int m = q.modes[(layer / 2) * s.Hkv + h];
+            const int m = q.modes[(layer / s.B) * s.Hkv + h];
             tot += 2 * (size_t)(q.T + q.tail_len[layer]) * s.d * s.esize;
             if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
                 const size_t kt = (size_t)((int64_t)q.T * s.keep_num / s.keep_den);

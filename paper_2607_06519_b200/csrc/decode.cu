@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
     }
 
     const float inv_sqrt_d = rsqrtf((float)D);
-    const float c = 0.70710678118654752440f;
+    const float c = u.scale;  // what the stored rows are multiplied by (1/sqrt 2 for a pair, 1/2 for a block of four)
     const bool coef = u.mode != FDKV_MODE_EXACT;
     const bool resid = u.mode == FDKV_MODE_RESIDUAL;
 

@@ -304,7 +304,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
         float* const scratch_f = reinterpret_cast<float*>(smem_raw + kHeaderBytes + kStages * kStageBytes + warp * kScratchBytes);
         float* const sm_m = reinterpret_cast<float*>(smem_raw + kOffM);
         float* const sm_l = reinterpret_cast<float*>(smem_raw + kOffL);
-        const float kLog2e = 1.4426950408889634f, kC = 0.70710678118654752440f;
+        const float kLog2e = 1.4426950408889634f;
         const float inv_sqrt_d = 0.08838834764831845f;  // 1/sqrt(128)
 
         int it = 0;
@@ -477,8 +477,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 const int tile = is_tail ? j - npre : (rev ? tb + npre - 1 - j : tb + j);
                 const int rows_valid = is_tail ? n_tail_rows - tile * kTT : T - tile * kTT;  // may exceed the stage
                 const bool with_res = resid && !is_tail;
-                const float kscale = ((coef && !is_tail) ? kC : 1.f) * inv_sqrt_d * kLog2e;
-                const float vscale = (coef && !is_tail) ? kC : 1.f;
+                const float kscale = ((coef && !is_tail) ? ud.scale : 1.f) * inv_sqrt_d * kLog2e;
+                const float vscale = (coef && !is_tail) ? ud.scale : 1.f;
 #ifdef FDKV_TIMING
                 t_mark = (unsigned)clock();
 #endif

@@ -43,8 +43,11 @@ struct UnitDesc {
     const int32_t* v_off;
     int32_t mode;
     int32_t T;
-    float sign;  // +1 for the first layer of the pair, -1 for the second
+    float sign;  // multiplier of the residual values relative to the rows: +1 / -1 for the two layers of a pair,
+                 // 2 for a layer of a four-layer block (rows scaled by 1/2, deviations by 1)
     int32_t res_kind;  // residual layout: 0 packed entries (k_idx / v_idx), 1 token rows (k_idx = token list, k_val / v_val = rows, k_off = per-slice counts)
+    float scale;       // what the stored rows are multiplied by: 1/sqrt 2 (pair coefficients), 1/2 (block of four), 1 (exact)
+    int32_t pad_;
 };
 
 struct SelState {
@@ -66,11 +69,14 @@ struct Shape {
     int NU, NT;        // units and unit-tensors (K and V) of one sequence
     int tail_rows;     // max_tail rounded up to kRowPad
     int tok_rule;      // 1: token-granular residual chosen by the probe
+    int B;             // layers per depth block: 2 or 4
+    int NB;            // staged high-frequency tensors per unit-tensor: 1 (Z1 of a pair) or 4 (the layers' deviations)
     int64_t ktok_max, ktok_cap;  // floor(Tmax*num/den) and the list capacity incl. slack
 };
 
 struct WsLayout {
     size_t tok_score, tok_flag, tok_list, tok_off;
+    size_t energy, eval;  // four-layer blocks: per-position high-frequency energy (float32) and the kept energies
     size_t status, z0, z1, z1drop, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
         partials, counters, io_q, io_k, io_v, io_out, total;
 };
@@ -152,7 +158,32 @@ struct SelectArgs {
 };
 cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream_t st);
 
+// ---- four-layer blocks (block4.cu) ----
+struct Split4Args {
+    const void* k[4];  // the block's four [T][Hkv][d] strided K tensors, layer order
+    const void* v[4];
+    int64_t stride_t, stride_h;
+    int T, d, Hkv;
+    int ut_base;          // first unit-tensor of the block (unit-tensor = head*2 + is_v)
+    int64_t unit_stride;  // elements between staged tensors (Tmax*d)
+    void* z0;             // [NT][unit_stride]
+    void* dev;            // [NT][4][unit_stride]: deviation of each layer from the block mean
+    float* energy;        // [NT][unit_stride]
+    uint32_t* hist;
+};
+cudaError_t launch_split4_hist(const Split4Args& a, int dtype, cudaStream_t st);
+struct Gather4Args {
+    int ut_begin, ut_count;
+    int64_t k, kcap, unit_stride;
+    const void* dev;     // [NT][4][unit_stride]
+    const int32_t* idx;  // [NT][kcap] ascending kept positions
+    void* val;           // [NT][4][kcap] the four layers' values at the kept positions
+    uint32_t* packed;    // optional [NT][4][kcap] packed entries (value doubled: the rows are scaled by 1/2), or null
+};
+cudaError_t launch_gather4(const Gather4Args& a, int dtype, cudaStream_t st);
+
 struct ProbeArgs {
+    int B;  // layers per block: 2 (one Z1 operand, both layers' queries) or 4 (one deviation operand per layer)
     int unit_begin, unit_count;  // units of the pair range (unit = pair*Hkv + h)
     int T, d, Hq, Hkv, G, W;
     int64_t unit_stride, kcap;

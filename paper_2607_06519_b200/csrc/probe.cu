@@ -31,67 +31,70 @@ __global__ void __launch_bounds__(256) probe_tile_kernel(ProbeArgs a) {
     const int nt = min(kProbeTile, a.T - t0);
     const int h = unit % a.Hkv, pair = unit / a.Hkv;
     const int ut = unit * 2;  // K
-    const T* z1 = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride + (int64_t)t0 * d;
-
-    for (int i = threadIdx.x; i < kProbeTile * d; i += blockDim.x) {
-        const int t = i / d, c = i % d;
-        const float v = t < nt ? ldf<T>(z1 + i) : 0.f;
-        full[t * ld + c] = v;
-        drop[t * ld + c] = v;
-    }
-    __syncthreads();
-    {
-        const int32_t* off = a.tile_off + (int64_t)ut * (a.ntiles_max + 1);
-        const int ntiles = (a.T + kResTile - 1) / kResTile;
-        const int j0 = t0 / kResTile, j1 = min(ntiles, (t0 + kProbeTile) / kResTile);
-        const int32_t* idx = a.idx + (int64_t)ut * a.kcap;
-        for (int e = off[j0] + threadIdx.x; e < off[j1]; e += blockDim.x) {
-            const int f = idx[e] - t0 * d;
-            drop[(f / d) * ld + (f % d)] = 0.f;
-        }
-    }
-    __syncthreads();
-
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j = (warp & 1) * 32 + lane;  // token within the tile
     const int rg = warp >> 1;              // 4 row groups
-    const int M = 2 * a.G * a.W;
+    // A pair has one high-frequency operand (Z1) that both layers' queries see; a block of four layers has one
+    // operand per layer (its deviation from the block mean), seen by that layer's queries only.
+    const int n_ops = a.B == 4 ? 4 : 1;
+    const int M = (a.B == 4 ? 1 : 2) * a.G * a.W;  // probe rows per operand
     float sum_f = 0.f, sum_d = 0.f;
-    for (int rb = 0; rb < M; rb += kRowsBlk) {
-        // stage 16 probe rows: row r = (layer*G + g)*W + qi  ->  Q[layer][qi][h*G + g][:]
-        for (int i = threadIdx.x; i < kRowsBlk * d; i += blockDim.x) {
-            const int r = rb + i / d, c = i % d;
-            float v = 0.f;
-            if (r < M) {
-                const int layer = r / (a.G * a.W), g = (r / a.W) % a.G, qi = r % a.W;
-                const T* q = reinterpret_cast<const T*>(a.q_layers_dev[2 * pair + layer]);
-                v = ldf<T>(q + ((int64_t)qi * a.Hq + h * a.G + g) * d + c);
-            }
-            qs[i] = v;
+    for (int op = 0; op < n_ops; ++op) {
+        const T* z1 = reinterpret_cast<const T*>(a.z1) + ((int64_t)ut * n_ops + op) * a.unit_stride + (int64_t)t0 * d;
+        for (int i = threadIdx.x; i < kProbeTile * d; i += blockDim.x) {
+            const int t = i / d, c = i % d;
+            const float v = t < nt ? ldf<T>(z1 + i) : 0.f;
+            full[t * ld + c] = v;
+            drop[t * ld + c] = v;
         }
         __syncthreads();
-        float af[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
-        const float* zf = full + j * ld;
-        const float* zd = drop + j * ld;
-        const float* qr = qs + rg * 4 * d;
-        for (int c = 0; c < d; ++c) {
-            const float vf = zf[c], vd = zd[c];
+        {
+            const int32_t* off = a.tile_off + (int64_t)ut * (a.ntiles_max + 1);
+            const int ntiles = (a.T + kResTile - 1) / kResTile;
+            const int j0 = t0 / kResTile, j1 = min(ntiles, (t0 + kProbeTile) / kResTile);
+            const int32_t* idx = a.idx + (int64_t)ut * a.kcap;
+            for (int e = off[j0] + threadIdx.x; e < off[j1]; e += blockDim.x) {
+                const int f = idx[e] - t0 * d;
+                drop[(f / d) * ld + (f % d)] = 0.f;
+            }
+        }
+        __syncthreads();
+        for (int rb = 0; rb < M; rb += kRowsBlk) {
+            // stage 16 probe rows: row r = (layer*G + g)*W + qi  ->  Q[layer][qi][h*G + g][:]
+            for (int i = threadIdx.x; i < kRowsBlk * d; i += blockDim.x) {
+                const int r = rb + i / d, c = i % d;
+                float v = 0.f;
+                if (r < M) {
+                    const int layer = a.B == 4 ? op : r / (a.G * a.W), g = (r / a.W) % a.G, qi = r % a.W;
+                    const T* q = reinterpret_cast<const T*>(a.q_layers_dev[a.B * pair + layer]);
+                    v = ldf<T>(q + ((int64_t)qi * a.Hq + h * a.G + g) * d + c);
+                }
+                qs[i] = v;
+            }
+            __syncthreads();
+            float af[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
+            const float* zf = full + j * ld;
+            const float* zd = drop + j * ld;
+            const float* qr = qs + rg * 4 * d;
+            for (int c = 0; c < d; ++c) {
+                const float vf = zf[c], vd = zd[c];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float qv = qr[i * d + c];
+                    af[i] = fmaf(qv, vf, af[i]);
+                    ad[i] = fmaf(qv, vd, ad[i]);
+                }
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const float qv = qr[i * d + c];
-                af[i] = fmaf(qv, vf, af[i]);
-                ad[i] = fmaf(qv, vd, ad[i]);
+                const int r = rb + rg * 4 + i;
+                if (r < M && j < nt && t0 + j <= a.pos[r % a.W]) {  // causal: keys at or before the probe position
+                    sum_f = fmaf(af[i], af[i], sum_f);
+                    sum_d = fmaf(ad[i], ad[i], sum_d);
+                }
             }
+            __syncthreads();
         }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int r = rb + rg * 4 + i;
-            if (r < M && j < nt && t0 + j <= a.pos[r % a.W]) {  // causal: keys at or before the probe position
-                sum_f = fmaf(af[i], af[i], sum_f);
-                sum_d = fmaf(ad[i], ad[i], sum_d);
-            }
-        }
-        __syncthreads();
     }
     double df = sum_f, dd = sum_d;
 #pragma unroll
@@ -127,7 +130,8 @@ __global__ void __launch_bounds__(256) probe_finalize_kernel(ProbeArgs a, int np
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        const double norm = 0.5 / (double)a.d / (double)(2 * a.G * a.W);
+        // (c / sqrt d)^2 over 2 G W rows for a pair's Z1; (1 / sqrt d)^2 over 4 G W rows for a block's deviations
+        const double norm = a.B == 4 ? 1.0 / (double)a.d / (double)(4 * a.G * a.W) : 0.5 / (double)a.d / (double)(2 * a.G * a.W);
         const double e_sh = s0[0] * norm, e_rs = s1[0] * norm;
         a.scores[2 * unit] = e_sh;
         a.scores[2 * unit + 1] = e_rs;

@@ -21,7 +21,7 @@ def make_context(w: synth.Workload, max_tail: int | None = None, arena_bytes: in
                  device="cuda:0") -> B.Context:
     cfg = B.Config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, w.T,
                    max_tail if max_tail is not None else max(w.n_steps, 1), B.BF16 if w.dtype == "bf16" else B.F32,
-                   w.keep_num, w.keep_den, w.residual_rule)
+                   w.keep_num, w.keep_den, w.residual_rule, w.block_size)
     return B.Context(cfg, device=device, arena_bytes=arena_bytes)
 
 
@@ -38,7 +38,8 @@ class Prefilled:
         self._inputs = {}  # the library reads exact-mode rows at commit: keep the uploads alive until then
 
     def upload_pair(self, seq: int, pair: int):
-        kv = synth.layer_pair_kv(self.w, seq, pair)
+        """Device tensors k0.., v0.. of one depth block (a pair, or four layers)."""
+        kv = synth.layer_block_kv(self.w, seq, pair) if self.w.block_size == 4 else synth.layer_pair_kv(self.w, seq, pair)
         return {n: to_device(a, self.w.dtype, self.device) for n, a in kv.items()}
 
     def upload_probe_q(self, seq: int):
@@ -48,10 +49,11 @@ class Prefilled:
         """Uploads and compresses every pair of a sequence; returns the per-layer device tensors."""
         w = self.w
         k_layers, v_layers = [None] * w.n_layers, [None] * w.n_layers
-        for p in range(w.n_pairs):
+        nb = w.block_size
+        for p in range(w.n_blocks):
             t = self.upload_pair(seq, p)
-            k_layers[2 * p], k_layers[2 * p + 1] = t["k0"], t["k1"]
-            v_layers[2 * p], v_layers[2 * p + 1] = t["v0"], t["v1"]
+            for l in range(nb):
+                k_layers[nb * p + l], v_layers[nb * p + l] = t[f"k{l}"], t[f"v{l}"]
             self.ctx.compress_prefill(seq, p, p + 1, w.T, k_layers, v_layers)
         self._inputs[seq] = (k_layers, v_layers)
         return k_layers, v_layers
@@ -62,7 +64,7 @@ class Prefilled:
 
     def probe(self, seq: int, lam: float):
         q_layers = self.upload_probe_q(seq)
-        modes, scores = self.ctx.probe(seq, 0, self.w.n_pairs, q_layers, synth.probe_positions(self.w), lam)
+        modes, scores = self.ctx.probe(seq, 0, self.w.n_blocks, q_layers, synth.probe_positions(self.w), lam)
         torch.cuda.synchronize()
         self.scores[seq] = scores.cpu().numpy().astype(np.float64)
         self.probe_modes[seq] = modes.cpu().numpy()
@@ -95,8 +97,10 @@ class Prefilled:
         w = self.w
         k = np.empty((w.batch, w.n_kv_heads, w.head_dim), np.float32)
         v = np.empty_like(k)
+        nb = w.block_size
+        rows = synth.block_tail_rows if nb == 4 else synth.tail_rows
         for b in range(w.batch):
             for h in range(w.n_kv_heads):
-                k[b, h] = synth.tail_rows(w, b, layer // 2, h, False)[layer & 1][step]
-                v[b, h] = synth.tail_rows(w, b, layer // 2, h, True)[layer & 1][step]
+                k[b, h] = rows(w, b, layer // nb, h, False)[layer % nb][step]
+                v[b, h] = rows(w, b, layer // nb, h, True)[layer % nb][step]
         return to_device(k, w.dtype, self.device), to_device(v, w.dtype, self.device)
