@@ -102,12 +102,17 @@ def oracle_sample(w, n_units: int):
     from paper_2607_06519_b200 import synth
 
     rng = np.random.default_rng(12345)
-    picks = [(int(p), int(h)) for p, h in zip(rng.integers(0, w.n_pairs, n_units), rng.integers(0, w.n_kv_heads, n_units))]
+    picks = [(int(p), int(h)) for p, h in zip(rng.integers(0, w.n_blocks, n_units), rng.integers(0, w.n_kv_heads, n_units))]
     units = []
     for i, (p, h) in enumerate(picks):
-        k0, k1 = synth.unit_tensor(w, 0, p, h, False)
-        v0, v1 = synth.unit_tensor(w, 0, p, h, True)
-        u = R.Unit(k0, k1, v0, v1, w.dtype == "bf16", w.keep_num, w.keep_den)
+        if w.block_size == 4:
+            from oracle import fdkv_ref_b4 as R4
+            u = R4.Unit4(synth.block_tensor(w, 0, p, h, False), synth.block_tensor(w, 0, p, h, True), w.dtype == "bf16",
+                         w.keep_num, w.keep_den)
+        else:
+            k0, k1 = synth.unit_tensor(w, 0, p, h, False)
+            v0, v1 = synth.unit_tensor(w, 0, p, h, True)
+            u = R.Unit(k0, k1, v0, v1, w.dtype == "bf16", w.keep_num, w.keep_den)
         mode = (0, 1, 0, 2, 1, 0, 1, 0)[i % 8]  # close to the 50/35/15 benchmark mix
         units.append((p, h, mode, u))
     return units
@@ -119,8 +124,8 @@ def oracle_step(w, units):
 
     t0 = time.perf_counter()
     for p, h, mode, u in units:
-        for lp in range(2):
-            q = synth.decode_q(w, 0, 2 * p + lp)[0][h * w.group:(h + 1) * w.group]
+        for lp in range(w.block_size):
+            q = synth.decode_q(w, 0, w.block_size * p + lp)[0][h * w.group:(h + 1) * w.group]
             u.attend(mode, lp, q)
     return time.perf_counter() - t0
 
@@ -136,9 +141,9 @@ def run_reference(args, w):
     total_calls = w.n_layers * w.n_kv_heads * w.batch
     times = [oracle_step(w, units) for _ in range(args.warmup + args.steps)][args.warmup:]
     t_step_sample = float(np.mean(times))
-    t_full = t_step_sample * total_calls / (2 * len(units))
+    t_full = t_step_sample * total_calls / (w.block_size * len(units))
     val = w.batch / t_full
-    sample = (f"{2 * len(units)} of {total_calls} (layer, KV head) attention units of one decode step, "
+    sample = (f"{w.block_size * len(units)} of {total_calls} (layer, KV head) attention units of one decode step, "
               f"scaled to the full step")
     line = {"impl": "reference", "metric": "compressed-KV decode attention tokens/s", "value": val, "unit": "tokens/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_full * 1e3,
@@ -176,16 +181,18 @@ def run_ours(args, w):
     esize = 2 if w.dtype == "bf16" else 4
     for b in range(w.batch):
         k_layers, v_layers = [None] * w.n_layers, [None] * w.n_layers
-        for p in range(w.n_pairs):
+        nb = w.block_size
+        for p in range(w.n_blocks):
             t = pf.upload_pair(b, p)
-            k_layers[2 * p], k_layers[2 * p + 1], v_layers[2 * p], v_layers[2 * p + 1] = t["k0"], t["k1"], t["v0"], t["v1"]
+            for lb in range(nb):
+                k_layers[nb * p + lb], v_layers[nb * p + lb] = t[f"k{lb}"], t[f"v{lb}"]
         if b == 0:  # untimed pass: first launches pay the lazy loading of every kernel
-            ctx.compress_prefill(b, 0, w.n_pairs, w.T, k_layers, v_layers)
-            ctx.probe(b, 0, w.n_pairs, pf.upload_probe_q(b), synth.probe_positions(w), 0.0)
+            ctx.compress_prefill(b, 0, w.n_blocks, w.T, k_layers, v_layers)
+            ctx.probe(b, 0, w.n_blocks, pf.upload_probe_q(b), synth.probe_positions(w), 0.0)
         torch.cuda.synchronize()
         e0, e1 = ev(), ev()
         e0.record()
-        ctx.compress_prefill(b, 0, w.n_pairs, w.T, k_layers, v_layers)
+        ctx.compress_prefill(b, 0, w.n_blocks, w.T, k_layers, v_layers)
         e1.record()
         torch.cuda.synchronize()
         compress_ms += e0.elapsed_time(e1)
@@ -193,7 +200,7 @@ def run_ours(args, w):
         torch.cuda.synchronize()
         e0, e1 = ev(), ev()
         e0.record()
-        modes, scores = ctx.probe(b, 0, w.n_pairs, q_layers, synth.probe_positions(w), 0.0)
+        modes, scores = ctx.probe(b, 0, w.n_blocks, q_layers, synth.probe_positions(w), 0.0)
         e1.record()
         torch.cuda.synchronize()
         probe_ms += e0.elapsed_time(e1)
@@ -201,7 +208,7 @@ def run_ours(args, w):
         ctx.commit(b)
         del k_layers, v_layers, q_layers, t
     launches_prefill = B.launch_count() - launches_prefill
-    units = w.batch * w.n_pairs * w.n_kv_heads
+    units = w.batch * w.n_blocks * w.n_kv_heads
     n_ut = 2 * units
     N = w.T * w.head_dim
     if w.residual_rule == 1:
@@ -210,8 +217,10 @@ def run_ours(args, w):
         compress_min_bytes = n_ut * (2 * N * esize + N * esize) + units * (2 * w.k_tok * w.head_dim * esize + 4 * w.k_tok)
         probe_flops = 2.0 * units * 3 * (2 * w.group * w.W) * w.T * w.head_dim
     else:
-        compress_min_bytes = n_ut * (2 * N * esize + N * esize + w.k_keep * (4 + esize))
-        probe_flops = 2.0 * units * 2 * (2 * w.group * w.W) * w.T * w.head_dim
+        # read the block's layers, write the shared coefficient, the index and the kept values
+        nbl = w.block_size
+        compress_min_bytes = n_ut * (nbl * N * esize + N * esize + w.k_keep * (4 + (1 if nbl == 2 else 4) * esize))
+        probe_flops = 2.0 * units * 2 * (nbl * w.group * w.W) * w.T * w.head_dim
     modes_all = np.stack([ctx.get_modes(b).numpy() for b in range(w.batch)])
     mix = [int((modes_all == m).sum()) for m in range(3)]
     torch.cuda.empty_cache()
@@ -227,12 +236,13 @@ def run_ours(args, w):
     if append:
         args.no_graph = True  # the tail length advances on the device and in the host mirror: launch directly
         args.steps = min(args.steps, w.n_steps - args.warmup - 1)
-        rows = {(b, p, h, v): synth.tail_rows(w, b, p, h, bool(v)) for b in range(w.batch) for p in range(w.n_pairs)
+        tail_fn = synth.block_tail_rows if w.block_size == 4 else synth.tail_rows
+        rows = {(b, p, h, v): tail_fn(w, b, p, h, bool(v)) for b in range(w.batch) for p in range(w.n_blocks)
                 for h in range(w.n_kv_heads) for v in (0, 1)}
         new_k, new_v = [], []
         for l in range(w.n_layers):
             for v, dst in ((0, new_k), (1, new_v)):
-                a = np.stack([[rows[(b, l // 2, h, v)][l & 1] for h in range(w.n_kv_heads)] for b in range(w.batch)])
+                a = np.stack([[rows[(b, l // w.block_size, h, v)][l % w.block_size] for h in range(w.n_kv_heads)] for b in range(w.batch)])
                 dst.append(runner.to_device(np.ascontiguousarray(a.transpose(2, 0, 1, 3)), w.dtype, dev))  # [step][b][h][d]
 
     def step():
@@ -346,9 +356,9 @@ def run_ours(args, w):
         reps = 3
         t_s = min(oracle_step(w, ou) for _ in range(reps))
         total_calls = w.n_layers * w.n_kv_heads * w.batch
-        t_full = t_s * total_calls / (2 * len(ou))
+        t_full = t_s * total_calls / (w.block_size * len(ou))
         cpu = {"value": w.batch / t_full, "unit": "tokens/s", "cores": R.threads(), "kind": "oracle",
-               "sample": f"{2 * len(ou)} of {total_calls} (layer, KV head) attention units of one decode step (float64), "
+               "sample": f"{w.block_size * len(ou)} of {total_calls} (layer, KV head) attention units of one decode step (float64), "
                          f"best of {reps}, scaled to the full step"}
 
     layer_calls = w.n_layers

@@ -66,7 +66,7 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.status = take(256);
     w.z0 = take((size_t)s.NT * unit_elems * s.esize);
     w.z1 = take((size_t)s.NT * s.NB * unit_elems * s.esize);  // Z1 of a pair, or the four layers' deviations of a block
-    w.z1drop = take(s.B == 2 && s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NU * unit_elems * s.esize : 0);
+    w.z1drop = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NU * s.NB * unit_elems * s.esize : 0);
     w.energy = take(s.B == 4 ? (size_t)s.NT * unit_elems * 4 : 0);
     w.eval = take(s.B == 4 ? (size_t)s.NT * s.kcap * 4 : 0);
     w.hist = take((size_t)s.NT * kHistBins * 4);
@@ -193,9 +193,9 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
         const bool ok = c->packed_lists && make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
         if (!ok) { delete c; return FDKV_ERR_UNSUPPORTED; }
     }
-    if (s.B == 2 && s.dtype == FDKV_BF16 && s.d == 128)
-        c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_z1) &&
-                             make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_drop);
+    if (s.dtype == FDKV_BF16 && s.d == 128)
+        c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.NB * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_z1) &&
+                             make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.NB * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_drop);
     if (s.tok_rule && !c->has_probe_tmaps) { delete c; return FDKV_ERR_UNSUPPORTED; }
     *out = c;
     return FDKV_OK;
@@ -266,6 +266,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
             a4.unit_stride = (int64_t)s.Tmax * s.d;
             a4.z0 = c->work + c->ws.z0; a4.dev = c->work + c->ws.z1;
             a4.energy = wsp<float>(c, c->ws.energy);
+            a4.drop = c->has_probe_tmaps ? c->work + c->ws.z1drop : nullptr;
             a4.hist = wsp<uint32_t>(c, c->ws.hist);
             CU(launch_split4_hist(a4, s.dtype, st));
         }
@@ -293,6 +294,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
         g.idx = wsp<int32_t>(c, c->ws.idx);
         g.val = c->work + c->ws.val;
         g.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
+        g.drop = c->has_probe_tmaps ? c->work + c->ws.z1drop : nullptr;  // tensor-core probe: the K deviations without the kept positions
         CU(launch_gather4(g, s.dtype, st));
         for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; c->pair_scored[p] = 0; }
         return FDKV_OK;

@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(512) split4_hist_kernel(Split4Args a, int toke
     T* z0 = reinterpret_cast<T*>(a.z0) + (int64_t)ut * a.unit_stride;
     T* dev = reinterpret_cast<T*>(a.dev) + (int64_t)ut * 4 * a.unit_stride;
     float* en = a.energy + (int64_t)ut * a.unit_stride;
+    T* drop = (a.drop && !is_v) ? reinterpret_cast<T*>(a.drop) + (int64_t)(ut >> 1) * 4 * a.unit_stride : nullptr;
 
     const int t_begin = blockIdx.x * tokens_per_cta;
     const int t_end = min(a.T, t_begin + tokens_per_cta);
@@ -93,7 +94,11 @@ __global__ void __launch_bounds__(512) split4_hist_kernel(Split4Args a, int toke
         }
         *reinterpret_cast<typename V::raw*>(z0 + off_out) = V::pack(z);
 #pragma unroll
-        for (int l = 0; l < 4; ++l) *reinterpret_cast<typename V::raw*>(dev + (int64_t)l * a.unit_stride + off_out) = V::pack(dv[l]);
+        for (int l = 0; l < 4; ++l) {
+            const typename V::raw pk = V::pack(dv[l]);
+            *reinterpret_cast<typename V::raw*>(dev + (int64_t)l * a.unit_stride + off_out) = pk;
+            if (drop) *reinterpret_cast<typename V::raw*>(drop + (int64_t)l * a.unit_stride + off_out) = pk;
+        }
 #pragma unroll
         for (int i = 0; i < N; i += 4)
             *reinterpret_cast<float4*>(en + off_out + i) = make_float4(e[i], e[i + 1], e[i + 2], e[i + 3]);
@@ -126,10 +131,13 @@ __global__ void __launch_bounds__(256) gather4_kernel(Gather4Args a) {
     const int i = a.idx[(int64_t)ut * a.kcap + w];
     const T* dev = reinterpret_cast<const T*>(a.dev) + (int64_t)ut * 4 * a.unit_stride;
     T* val = reinterpret_cast<T*>(a.val) + (int64_t)ut * 4 * a.kcap;
+    // K tensors: the copy of the deviations that the residual candidate of the probe misses loses its kept positions
+    T* drop = (a.drop && !(ut & 1)) ? reinterpret_cast<T*>(a.drop) + (int64_t)(ut >> 1) * 4 * a.unit_stride : nullptr;
 #pragma unroll
     for (int l = 0; l < 4; ++l) {
         const T v = dev[(int64_t)l * a.unit_stride + i];
         val[(int64_t)l * a.kcap + w] = v;
+        if (drop) drop[(int64_t)l * a.unit_stride + i] = T(0.f);
         if constexpr (sizeof(T) == 2) {
             // the decode kernel scales the rows by 1/2 and the residual by the same factor: store twice the deviation
             if (a.packed) a.packed[((int64_t)ut * 4 + l) * a.kcap + w] = packed_entry_bf16(2.f * __bfloat162float(v), i);

@@ -169,6 +169,7 @@ struct Split4Args {
     void* z0;             // [NT][unit_stride]
     void* dev;            // [NT][4][unit_stride]: deviation of each layer from the block mean
     float* energy;        // [NT][unit_stride]
+    void* drop;           // optional [NU][4][unit_stride]: second copy of the K deviations (the gather zeroes its kept positions)
     uint32_t* hist;
 };
 cudaError_t launch_split4_hist(const Split4Args& a, int dtype, cudaStream_t st);
@@ -179,6 +180,7 @@ struct Gather4Args {
     const int32_t* idx;  // [NT][kcap] ascending kept positions
     void* val;           // [NT][4][kcap] the four layers' values at the kept positions
     uint32_t* packed;    // optional [NT][4][kcap] packed entries (value doubled: the rows are scaled by 1/2), or null
+    void* drop;          // optional [NU][4][unit_stride]: the K deviations (copied there beforehand); kept positions get zeroed
 };
 cudaError_t launch_gather4(const Gather4Args& a, int dtype, cudaStream_t st);
 

@@ -131,7 +131,7 @@ __device__ __forceinline__ void tmem_st64(uint32_t taddr, const uint32_t (&r)[64
 }
 
 struct TcPlan {
-    int items_per_unit;  // 2 layers x mblocks x 2 candidates x nsplits
+    int items_per_unit;  // B layers x mblocks x 2 candidates x nsplits
     int mblocks, nsplits, ntiles, tiles_per_split;
     int pos_min, pos_max;
     int experiment;  // timing experiments only (FDKV_PROBE_EXPERIMENT): 1 = epilogue skips the accumulator reads
@@ -156,7 +156,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
     const int split = it % pl.nsplits; it /= pl.nsplits;
     const int cand = it & 1; it >>= 1;
     const int mblock = it % pl.mblocks; it /= pl.mblocks;
-    const int layer = it;  // 0 or 1
+    const int layer = it;  // layer inside the depth block: 0 .. B-1
     const int h = unit % a.Hkv, pair = unit / a.Hkv;
     const int tile0 = split * pl.tiles_per_split;
     const int tile1 = min(pl.ntiles, tile0 + pl.tiles_per_split);
@@ -181,7 +181,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
     //      Q[layer][qi][h*G+g][:], written by the thread that owns that TMEM lane (two bf16 channels per column) ----
     if (warp >= 2) {
         const int lq = warp & 3, rl = lq * 32 + lane;
-        const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[2 * pair + layer]);
+        const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[a.B * pair + layer]);
 #pragma unroll 1
         for (int mt = 0; mt < 2; ++mt) {
             const int r = mblock * 256 + mt * 128 + rl;
@@ -211,7 +211,9 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         if (lane == 0) {
             const CUtensorMap* map = cand ? &tmap_drop : &tmap_z1;
             // rows of this unit's K coefficients: staged Z1 holds K and V per unit (unit-tensor 2*unit), the dropped copy K only
-            const int64_t row0 = (cand ? (int64_t)unit : (int64_t)unit * 2) * a.Tmax;
+            // (a block of four layers stages one operand per layer: [unit-tensor][4] and [unit][4])
+            const int64_t row0 = a.B == 4 ? ((cand ? (int64_t)unit : (int64_t)unit * 2) * 4 + layer) * a.Tmax
+                                          : (cand ? (int64_t)unit : (int64_t)unit * 2) * a.Tmax;
             for (int i = 0; i < ntile && pl.experiment != 2; ++i) {
                 const int s = i % kBStages;
                 const uint32_t ph = (uint32_t)(i / kBStages) & 1u;
@@ -356,14 +358,14 @@ cudaError_t launch_probe_tc(const ProbeArgs& a, int dtype, cudaStream_t st, bool
     pl.pos_max = a.pos_host[a.W - 1];
     pl.ntiles = pl.pos_max / kBN + 1;  // keys after the last probe position never count
     pl.mblocks = (a.G * a.W + 255) / 256;
-    const int base_items = a.unit_count * 2 * pl.mblocks * 2;
+    const int base_items = a.unit_count * a.B * pl.mblocks * 2;
     // split the key range so that the grid fills the machine several times over, but keep >= 8 tiles per item
     int nsplits = std::max(1, std::min((4 * sm_count + base_items - 1) / base_items, (pl.ntiles + 7) / 8));
     pl.tiles_per_split = (pl.ntiles + nsplits - 1) / nsplits;
     nsplits = (pl.ntiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
     pl.nsplits = nsplits;
-    pl.items_per_unit = 2 * pl.mblocks * 2 * nsplits;
-    const int slots = 2 * pl.mblocks * nsplits;
+    pl.items_per_unit = a.B * pl.mblocks * 2 * nsplits;
+    const int slots = a.B * pl.mblocks * nsplits;
     if (slots > a.nptiles_max) return cudaSuccess;  // the part array is sized for the portable kernel's tiles
     probe_tc_kernel<<<a.unit_count * pl.items_per_unit, kPThreads, kProbeSmem, st>>>(
         *reinterpret_cast<const CUtensorMap*>(a.tmap_z1), *reinterpret_cast<const CUtensorMap*>(a.tmap_drop), a, pl);
