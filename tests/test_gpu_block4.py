@@ -118,3 +118,43 @@ def test_block4_all_modes_each(request):
         assert worst <= TOL["bf16"], (mode, worst)
         assert pf.ctx.device_status() == 0
         pf.ctx.close()
+
+
+def test_block4_benchmark_workload_sampled():
+    """decode32k_b4 (32 layers = 8 blocks, 32k, bf16, quota mode mix) through the calls bench.py times; sampled
+    units are checked against the oracle: stored values bit-exact, probe errors, one decode step of all layers."""
+    runner = _runner()
+    w = synth.WORKLOADS["decode32k_b4"]
+    sample = [(0, 2), (3, 5), (7, 7)]
+    pf = runner.Prefilled(w, max_tail=1)
+    pf.compress(0)
+    units = {(b, h): check_compression4(pf.ctx, w, 0, b, h) for (b, h) in sample}
+    pmodes, scores = pf.probe(0, 0.0)
+    pos = synth.probe_positions(w)
+    for (b, h) in sample[:2]:
+        u = units[(b, h)]
+        e = R4.probe_error4(u.dev["k"], u.kept["k"], [synth.probe_q(w, 0, 4 * b + l) for l in range(4)], w.group, h, pos)
+        np.testing.assert_allclose(scores[b, h], e, rtol=1e-4)
+    modes = synth.quota_modes(scores[..., 0])
+    pf.ctx.set_modes(0, modes)
+    pf.commit(0)
+    assert np.bincount(modes.ravel(), minlength=3).tolist() == [32, 22, 10]
+    torch.cuda.empty_cache()
+    worst = 0.0
+    G = w.group
+    for layer in range(w.n_layers):
+        blk, lb = divmod(layer, 4)
+        q = pf.decode_q(layer, 0)
+        out = pf.ctx.decode_attn(layer, q)
+        torch.cuda.synchronize()
+        assert torch.isfinite(out.float()).all()
+        for (b, h), u in units.items():
+            if b != blk:
+                continue
+            ref = u.attend(int(modes[b][h]), lb, f32(q)[0][h * G:(h + 1) * G])
+            worst = max(worst, float(vector_errors(f32(out)[0][h * G:(h + 1) * G], ref).max()))
+    assert worst <= TOL["bf16"], worst
+    by_mode, exact_equiv = pf.ctx.footprint(0)
+    assert sum(by_mode) < 0.5 * exact_equiv  # a shared unit stores one of four layers
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
