@@ -202,6 +202,27 @@ class Unit:
         self.tail[("k", layer_in_pair)].append(_c32(k_row))
         self.tail[("v", layer_in_pair)].append(_c32(v_row))
 
+    def fold(self, n: int, keep_num: int, keep_den: int):
+        """Periodic refresh (Method, last paragraph: routing is decided once; the cache may be refreshed every fixed
+        number of tokens): the first n generated tokens of both layers leave the exact tail and join the compressed
+        form under the unit's mode.  The chunk is transformed by Eq. 1 and keeps its own k = floor(n d num / den)
+        largest-magnitude Z1 entries per tensor (Eq. 3 applied to the chunk); its originals stay available to the
+        exact mode.  Entry rule only."""
+        assert not hasattr(self, "tokens")
+        for name in ("k", "v"):
+            t0, t1 = self.tail[(name, 0)], self.tail[(name, 1)]
+            assert len(t0) >= n and len(t1) >= n
+            x0c, x1c = np.stack(t0[:n]), np.stack(t1[:n])
+            z0c, z1c = depth_split(x0c, x1c, self.bf16)
+            keptc = select_entries(z1c, keep_count(n, self.d, keep_num, keep_den))
+            self.kept[name] = np.concatenate([self.kept[name], keptc + np.int32(self.T * self.d)]).astype(np.int32)
+            self.x[name] = (np.concatenate([self.x[name][0], x0c]), np.concatenate([self.x[name][1], x1c]))
+            self.z0[name] = np.concatenate([self.z0[name], z0c])
+            self.z1[name] = np.concatenate([self.z1[name], z1c])
+            self.tail[(name, 0)], self.tail[(name, 1)] = t0[n:], t1[n:]
+        self.T += n
+        self.k_keep = self.kept["k"].size
+
     def rows(self, name: str, mode: int, layer_in_pair: int) -> np.ndarray:
         pre = reconstruct(self.z0[name], self.z1[name], self.kept[name], mode, layer_in_pair,
                           self.x[name][layer_in_pair])

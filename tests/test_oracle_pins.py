@@ -409,3 +409,64 @@ def test_route_budget_is_the_smallest_lambda_that_fits():
     assert fits and modes.tolist() == [1] and lam == pytest.approx(10.0 / (1 - 0.59375), rel=1e-9)
     fits, lam, modes = R.route_budget([100.0], [10.0], om, unit, 0.5 * unit)
     assert fits and modes.tolist() == [0] and lam == pytest.approx(90.0 / 0.09375, rel=1e-9)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# folding generated tokens into the compressed form (the optional refresh of the Method's last paragraph)
+# ---------------------------------------------------------------------------------------------------------
+def _unit_with_tail(seed, T=48, d=8, n_tail=40, bf16=False, keep=(1, 4)):
+    g = np.random.default_rng(seed)
+    mk = lambda *s: (synth.round_bf16(g.standard_normal(s).astype(np.float32)) if bf16 else g.standard_normal(s).astype(np.float32))
+    u = R.Unit(mk(T, d), mk(T, d), mk(T, d), mk(T, d), bf16, *keep)
+    rows = [(mk(d), mk(d), mk(d), mk(d)) for _ in range(n_tail)]
+    for k0, k1, v0, v1 in rows:
+        u.append(0, k0, v0)
+        u.append(1, k1, v1)
+    return u, rows
+
+
+def test_fold_leaves_exact_mode_unchanged_and_moves_rows():
+    u, rows = _unit_with_tail(21)
+    q = np.random.default_rng(1).standard_normal((2, 8)).astype(np.float32)
+    before = [u.attend(R.EXACT, l, q) for l in range(2)]
+    T0 = u.T
+    u.fold(32, 1, 4)
+    assert u.T == T0 + 32 and len(u.tail[("k", 0)]) == 8 and len(u.tail[("v", 1)]) == 8
+    for l in range(2):
+        np.testing.assert_allclose(u.attend(R.EXACT, l, q), before[l], rtol=1e-12, atol=1e-12)
+    # the chunk keeps its own top-k: floor(32 * 8 / 4) entries, all inside the chunk, ascending overall
+    for name in ("k", "v"):
+        kept = u.kept[name]
+        assert kept.size == (T0 * 8) // 4 + (32 * 8) // 4
+        assert np.all(np.diff(kept) > 0)
+        assert np.all(kept[(T0 * 8) // 4:] >= T0 * 8)
+
+
+def test_fold_chunk_selection_is_the_chunks_own_top_k():
+    u, rows = _unit_with_tail(22, T=32, d=8, n_tail=16)
+    u.fold(16, 1, 4)
+    k0 = np.stack([r[0] for r in rows])
+    k1 = np.stack([r[1] for r in rows])
+    _, z1c = R.depth_split(k0, k1, False)
+    mag = np.abs(z1c.reshape(-1)).astype(np.float64)
+    order = np.lexsort((np.arange(mag.size), -mag))
+    want = np.sort(order[:(16 * 8) // 4]) + 32 * 8
+    assert np.array_equal(u.kept["k"][(32 * 8) // 4:], want)
+    # stored coefficients of the chunk are Eq. 1 of the chunk's rows
+    np.testing.assert_array_equal(u.z1["k"][32:], z1c)
+
+
+def test_fold_with_everything_kept_is_lossless_in_residual_mode():
+    u, rows = _unit_with_tail(23, keep=(1, 1))
+    q = np.random.default_rng(2).standard_normal((1, 8)).astype(np.float32)
+    ex = u.attend(R.EXACT, 1, q)
+    u.fold(40, 1, 1)
+    np.testing.assert_allclose(u.attend(R.RESIDUAL, 1, q), ex, rtol=1e-5, atol=1e-6)
+
+
+def test_fold_in_shared_mode_replaces_tail_rows_by_the_pair_mean():
+    u, rows = _unit_with_tail(24, n_tail=16)
+    u.fold(16, 1, 4)
+    got = u.rows("k", R.SHARED, 0)[48:]
+    want = np.stack([(r[0].astype(np.float64) + r[1].astype(np.float64)) / 2 for r in rows])
+    np.testing.assert_allclose(got, want, rtol=1e-6, atol=1e-7)
