@@ -63,6 +63,8 @@ typedef struct {
     int32_t keep_den;    /*   entries per (unit, K or V); 0 <= keep_num <= keep_den                    */
     int32_t residual_rule; /* fdkv_residual_rule: how the sparse high-frequency residual is chosen     */
     int32_t block_size;  /* B of Eq. 1: 2 (also when 0) or 4 layers per depth block                    */
+    int32_t max_fold;    /* generated tokens fdkv_fold_tail may move into the compressed form per       */
+                         /*   sequence (0: none); fdkv_commit reserves row and list room for them       */
 } fdkv_config;
 
 /*
@@ -187,6 +189,21 @@ fdkv_status fdkv_decode_attn_host(fdkv_ctx* ctx, int32_t layer, int32_t batch, c
 
 /* Sets the tail length of every layer of a sequence (0 empties the tails; n <= current length). */
 fdkv_status fdkv_set_tail_len(fdkv_ctx* ctx, int32_t seq, int32_t n, void* stream);
+
+/*
+ * Periodic refresh (Method, last paragraph: routing is decided once after prefill; the cache may be refreshed every
+ * fixed number of tokens).  Moves the first n generated tokens of EVERY layer of a committed sequence out of the
+ * exact tails into the compressed form, under each unit's existing mode: the chunk is transformed by Eq. 1, keeps
+ * its own k = floor(n * head_dim * keep_num / keep_den) largest-magnitude high-frequency entries per tensor (Eq. 3
+ * applied to the chunk; ties to the lowest index) and is appended behind the unit's rows and lists; exact units get
+ * the rows themselves.  The remaining tail rows move down; T of the sequence grows by n.  Modes do not change (the
+ * originals of shared / residual units no longer exist, so a committed unit cannot be re-routed upwards).
+ * Requirements: block size 2, entry residual rule; T and n multiples of 16; every layer's tail holds the same
+ * number (>= n) of tokens, i.e. call it between decode steps; the total folded per sequence stays within
+ * cfg.max_fold; no other sequence may be staged and uncommitted (the call reuses the staging area and invalidates
+ * it).  Synchronous (waits for the stream).  FDKV_ERR_ARENA_FULL when max_fold is exhausted.
+ */
+fdkv_status fdkv_fold_tail(fdkv_ctx* ctx, int32_t seq, int32_t n, void* stream);
 
 /* Introspection of the STAGED sequence (valid from fdkv_compress_prefill until the next one).  Synchronous. */
 fdkv_status fdkv_get_shared(fdkv_ctx* ctx, int32_t seq, int32_t pair, int32_t kv_head, int32_t is_v,

@@ -35,7 +35,8 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     const int G = c.n_q_heads / c.n_kv_heads;
     if (!(G == 1 || G == 2 || G == 4 || G == 8)) return false;
     if (c.head_dim != 64 && c.head_dim != 128) return false;
-    if (c.max_batch <= 0 || c.max_prefill <= 0 || c.max_tail < 0) return false;
+    if (c.max_batch <= 0 || c.max_prefill <= 0 || c.max_tail < 0 || c.max_fold < 0) return false;
+    if ((int64_t)(c.max_prefill + (int64_t)c.max_fold) * c.head_dim >= (int64_t)1 << 31) return false;
     if ((int64_t)c.max_prefill * c.head_dim >= (int64_t)1 << 31) return false;
     if (c.dtype != FDKV_F32 && c.dtype != FDKV_BF16) return false;
     if (c.keep_den <= 0 || c.keep_num < 0 || c.keep_num > c.keep_den) return false;
@@ -43,6 +44,8 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.max_batch = c.max_batch; s.Tmax = c.max_prefill; s.max_tail = c.max_tail;
     s.dtype = c.dtype; s.esize = c.dtype == FDKV_BF16 ? 2 : 4;
     s.keep_num = c.keep_num; s.keep_den = c.keep_den;
+    s.max_fold = c.max_fold;
+    s.kfold_max = (int64_t)s.max_fold * s.d * s.keep_num / s.keep_den;
     s.kmax = (int64_t)s.Tmax * s.d * s.keep_num / s.keep_den;
     s.kcap = (int64_t)align_up((size_t)(s.kmax + kListPad), 64);
     s.ntiles_max = (s.Tmax + kResTile - 1) / kResTile;
@@ -100,13 +103,14 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     a.tail_k = take(tail);
     a.tail_v = take(tail);
     a.bump = o;
-    const size_t rows_pad = align_up((size_t)((s.Tmax + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize);
+    const size_t rows_pad = align_up((size_t)((s.Tmax + s.max_fold + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize);
     const size_t exact_unit = 2 * (size_t)s.B * rows_pad;
     const size_t resid_unit = s.tok_rule
                                   ? 2 * rows_pad + 2 * align_up((size_t)s.ktok_cap * s.d * s.esize) + align_up((size_t)s.ktok_cap * 4) +
                                         align_up((size_t)(s.ntiles_max + 1) * 4)
-                                  : 2 * rows_pad + 2 * (size_t)s.NB * (align_up((size_t)s.kcap * 4) + align_up((size_t)s.kcap * s.esize)) +
-                                        2 * align_up((size_t)s.kcap * 4) + 2 * align_up((size_t)(s.ntiles_max + 1) * 4);
+                                  : 2 * rows_pad + 2 * (size_t)s.NB * (align_up((size_t)(s.kcap + s.kfold_max) * 4) + align_up((size_t)(s.kcap + s.kfold_max) * s.esize)) +
+                                        2 * align_up((size_t)(s.kcap + s.kfold_max) * 4) +
+                                        2 * align_up((size_t)(s.ntiles_max + s.max_fold / kResTile + 2) * 4);
     a.worst_total = a.bump + (size_t)s.max_batch * s.NU * (exact_unit > resid_unit ? exact_unit : resid_unit);
 }
 
@@ -214,6 +218,8 @@ fdkv_status fdkv_reset(fdkv_ctx* c) {
     for (auto& q : c->seqs) {
         q.committed = false;
         q.T = 0;
+        q.fold_used = 0;
+        q.k_entries = 0;
         q.modes.assign(c->s.NU, -1);
         q.tail_len.assign(c->s.L, 0);
         q.bytes_by_mode[0] = q.bytes_by_mode[1] = q.bytes_by_mode[2] = 0;
@@ -476,12 +482,16 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
         CU(cudaMemcpy(q.modes.data(), c->work + c->ws.modes, (size_t)s.NU * 4, cudaMemcpyDeviceToHost));
     const int T = c->staged_T;
     const size_t rows = (size_t)T * s.d * s.esize;
-    const size_t rows_pad = (size_t)((T + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize;  // zero rows up to a whole box
+    // zero rows up to a whole box, with room for the tokens fdkv_fold_tail may append later
+    const size_t rows_pad = (size_t)((T + s.max_fold + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize;
     const int64_t k = (int64_t)T * s.d * s.keep_num / s.keep_den;
     const int ntiles = (T + kResTile - 1) / kResTile;
     // list copies include the slack so that aligned over-reads of the last tile stay inside the allocation
-    const size_t idx_b = (size_t)(k + kListPad) * 4, off_b = (size_t)(ntiles + 1) * 4;
-    const size_t val_b = c->packed_lists ? 0 : (size_t)(k + kListPad) * s.esize;  // packed entries carry their value
+    // (copy_* = what the staging area holds now; the allocations add the room of the folded chunks)
+    const size_t idx_copy = (size_t)(k + kListPad) * 4, off_copy = (size_t)(ntiles + 1) * 4;
+    const size_t val_copy = c->packed_lists ? 0 : (size_t)(k + kListPad) * s.esize;  // packed entries carry their value
+    const size_t idx_b = idx_copy + (size_t)s.kfold_max * 4, off_b = off_copy + (size_t)(s.max_fold / kResTile + 1) * 4;
+    const size_t val_b = c->packed_lists ? 0 : val_copy + (size_t)s.kfold_max * s.esize;
     const int64_t k_tok = (int64_t)T * s.keep_num / s.keep_den;
     const size_t trow_b = (size_t)(k_tok + 4) * s.d * s.esize, tlist_b = (size_t)(k_tok + 32) * 4;  // token rows, token list
     size_t need = 0;
@@ -528,7 +538,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 tl = take(tlist_b);
                 to = take(off_b);
                 CU(cudaMemcpyAsync(tl, c->work + c->ws.tok_list + (size_t)u * s.ktok_cap * 4, (size_t)k_tok * 4, cudaMemcpyDeviceToDevice, st));
-                CU(cudaMemcpyAsync(to, c->work + c->ws.tok_off + (size_t)u * (s.ntiles_max + 1) * 4, off_b, cudaMemcpyDeviceToDevice, st));
+                CU(cudaMemcpyAsync(to, c->work + c->ws.tok_off + (size_t)u * (s.ntiles_max + 1) * 4, off_copy, cudaMemcpyDeviceToDevice, st));
                 by_mode[1] += (size_t)k_tok * 4;
             }
             for (int is_v = 0; is_v < 2; ++is_v) {
@@ -551,22 +561,22 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                     by_mode[1] += (size_t)k_tok * s.d * s.esize;
                 } else if (m == FDKV_MODE_RESIDUAL) {
                     char* po = take(off_b);
-                    CU(cudaMemcpyAsync(po, c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, off_b, cudaMemcpyDeviceToDevice, st));
+                    CU(cudaMemcpyAsync(po, c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, off_copy, cudaMemcpyDeviceToDevice, st));
                     char* pi_shared = nullptr;
                     if (!c->packed_lists) {
                         pi_shared = take(idx_b);
-                        CU(cudaMemcpyAsync(pi_shared, c->work + c->ws.idx + ut * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
+                        CU(cudaMemcpyAsync(pi_shared, c->work + c->ws.idx + ut * s.kcap * 4, idx_copy, cudaMemcpyDeviceToDevice, st));
                     }
                     char *pi_l[4] = {nullptr, nullptr, nullptr, nullptr}, *pv_l[4] = {nullptr, nullptr, nullptr, nullptr};
                     for (int j = 0; j < s.NB; ++j) {  // one list per stored high-frequency tensor
                         const size_t lt = ut * s.NB + j;
                         if (c->packed_lists) {
                             pi_l[j] = take(idx_b);
-                            CU(cudaMemcpyAsync(pi_l[j], c->work + c->ws.packed + lt * s.kcap * 4, idx_b, cudaMemcpyDeviceToDevice, st));
+                            CU(cudaMemcpyAsync(pi_l[j], c->work + c->ws.packed + lt * s.kcap * 4, idx_copy, cudaMemcpyDeviceToDevice, st));
                         } else {
                             pi_l[j] = pi_shared;
                             pv_l[j] = take(val_b);
-                            CU(cudaMemcpyAsync(pv_l[j], c->work + c->ws.val + lt * s.kcap * s.esize, val_b, cudaMemcpyDeviceToDevice, st));
+                            CU(cudaMemcpyAsync(pv_l[j], c->work + c->ws.val + lt * s.kcap * s.esize, val_copy, cudaMemcpyDeviceToDevice, st));
                         }
                     }
                     for (int l = 0; l < s.B; ++l) {
@@ -588,6 +598,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     c->bump = o;
     q.committed = true;
     q.T = T;
+    q.fold_used = 0;
+    q.k_entries = k;
     for (int i = 0; i < 3; ++i) q.bytes_by_mode[i] = by_mode[i];
     return FDKV_OK;
 }
@@ -673,6 +685,120 @@ fdkv_status fdkv_set_tail_len(fdkv_ctx* c, int32_t seq, int32_t n, void* stream)
     return FDKV_OK;
 }
 
+fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
+    if (!seq_ok(c, seq) || n <= 0) return FDKV_ERR_INVALID_ARG;
+    const Shape& s = c->s;
+    if (s.B != 2 || s.tok_rule) return FDKV_ERR_UNSUPPORTED;
+    SeqState& q = c->seqs[seq];
+    if (!q.committed) return FDKV_ERR_STATE;
+    if (c->staged_seq >= 0 && !c->seqs[c->staged_seq].committed) return FDKV_ERR_STATE;  // the staging area is in use
+    if ((q.T % kResTile) || (n % kResTile) || n > s.Tmax) return FDKV_ERR_INVALID_ARG;
+    for (int l = 0; l < s.L; ++l)
+        if (q.tail_len[l] != q.tail_len[0]) return FDKV_ERR_STATE;
+    if (q.tail_len[0] < n) return FDKV_ERR_INVALID_ARG;
+    if (q.fold_used + n > s.max_fold) return FDKV_ERR_ARENA_FULL;
+    cudaStream_t st = S(stream);
+    const int T0 = q.T, len = q.tail_len[0], rest = len - n;
+    const size_t row_b = (size_t)s.d * s.esize;
+    const size_t tail_head_b = (size_t)s.tail_rows * row_b;                       // one (layer, sequence, head) tail
+    auto tail_base = [&](char* base, int l) { return base + ((size_t)l * s.max_batch + seq) * s.Hkv * tail_head_b; };
+    char* tk = c->arena + c->ar.tail_k;
+    char* tv = c->arena + c->ar.tail_v;
+    // ---- Eq. 1 and the chunk's own selection, through the staging area ----
+    c->staged_seq = -1;
+    std::fill(c->pair_compressed.begin(), c->pair_compressed.end(), 0);
+    CU(cudaMemsetAsync(wsp<uint32_t>(c, c->ws.hist), 0, (size_t)s.NT * kHistBins * 4, st));
+    for (int p0 = 0; p0 < s.P; p0 += kSplitPairs) {
+        CompressArgs a;
+        a.n_pairs = s.P - p0 < kSplitPairs ? s.P - p0 : kSplitPairs;
+        for (int j = 0; j < a.n_pairs; ++j) {
+            const int p = p0 + j;
+            a.k0[j] = tail_base(tk, 2 * p); a.k1[j] = tail_base(tk, 2 * p + 1);
+            a.v0[j] = tail_base(tv, 2 * p); a.v1[j] = tail_base(tv, 2 * p + 1);
+        }
+        a.stride_t = s.d; a.stride_h = (int64_t)s.tail_rows * s.d;
+        a.T = n; a.d = s.d; a.Hkv = s.Hkv; a.tensors = 2;
+        a.ut_base = p0 * s.Hkv * 2;
+        a.unit_stride = (int64_t)s.Tmax * s.d;
+        a.z0 = c->work + c->ws.z0; a.z1 = c->work + c->ws.z1;
+        a.hist = wsp<uint32_t>(c, c->ws.hist);
+        CU(launch_split_hist(a, s.dtype, st));
+    }
+    const int64_t kc = (int64_t)n * s.d * s.keep_num / s.keep_den;
+    SelectArgs sa;
+    sa.ut_begin = 0; sa.ut_count = s.NT;
+    sa.T = n; sa.d = s.d; sa.k = kc;
+    sa.unit_stride = (int64_t)s.Tmax * s.d; sa.kcap = s.kcap; sa.ntiles_max = s.ntiles_max;
+    sa.z1 = c->work + c->ws.z1;
+    sa.hist = wsp<uint32_t>(c, c->ws.hist);
+    sa.sel = wsp<SelState>(c, c->ws.sel);
+    sa.tile_cnt = wsp<uint32_t>(c, c->ws.tile_cnt);
+    sa.tile_eq = wsp<uint32_t>(c, c->ws.tile_eq);
+    sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
+    sa.idx = wsp<int32_t>(c, c->ws.idx);
+    sa.val = c->work + c->ws.val;
+    sa.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
+    sa.z1drop = nullptr;
+    sa.status = wsp<int32_t>(c, c->ws.status);
+    CU(launch_select_and_compact(sa, s.dtype, st));
+    // ---- append behind every unit's rows and lists, under the unit's mode ----
+    const size_t unit_stride_b = (size_t)s.Tmax * s.d * s.esize, chunk_b = (size_t)n * row_b, at = (size_t)T0 * row_b;
+    const int64_t k_old = q.k_entries;
+    const int nslices = n / kResTile;
+    for (int u = 0; u < s.NU; ++u) {
+        const int m = q.modes[u], p = u / s.Hkv, h = u % s.Hkv;
+        UnitDesc* dl[2] = {&c->desc_host[((size_t)seq * s.L + 2 * p) * s.Hkv + h], &c->desc_host[((size_t)seq * s.L + 2 * p + 1) * s.Hkv + h]};
+        if (m == FDKV_MODE_EXACT) {
+            for (int l = 0; l < 2; ++l) {
+                CU(cudaMemcpyAsync((char*)dl[l]->k_rows + at, tail_base(tk, 2 * p + l) + h * tail_head_b, chunk_b, cudaMemcpyDeviceToDevice, st));
+                CU(cudaMemcpyAsync((char*)dl[l]->v_rows + at, tail_base(tv, 2 * p + l) + h * tail_head_b, chunk_b, cudaMemcpyDeviceToDevice, st));
+            }
+            q.bytes_by_mode[2] += 4 * chunk_b;
+            continue;
+        }
+        for (int is_v = 0; is_v < 2; ++is_v) {
+            const size_t ut = (size_t)u * 2 + is_v;
+            char* rows = (char*)(is_v ? dl[0]->v_rows : dl[0]->k_rows);  // both layers share the coefficient rows
+            CU(cudaMemcpyAsync(rows + at, c->work + c->ws.z0 + ut * unit_stride_b, chunk_b, cudaMemcpyDeviceToDevice, st));
+            q.bytes_by_mode[m] += chunk_b;
+            if (m != FDKV_MODE_RESIDUAL) continue;
+            int32_t* list = const_cast<int32_t*>(is_v ? dl[0]->v_idx : dl[0]->k_idx);
+            int32_t* off = const_cast<int32_t*>(is_v ? dl[0]->v_off : dl[0]->k_off);
+            if (c->packed_lists) {  // packed entries carry slice-relative positions: valid as they are (T0 is a multiple of 16)
+                CU(cudaMemcpyAsync(list + k_old, c->work + c->ws.packed + ut * s.kcap * 4, (size_t)kc * 4, cudaMemcpyDeviceToDevice, st));
+            } else {
+                char* val = (char*)const_cast<void*>(is_v ? dl[0]->v_val : dl[0]->k_val);
+                CU(launch_offset_copy(list + k_old, wsp<int32_t>(c, c->ws.idx) + ut * s.kcap, (int)kc, T0 * s.d, st));
+                CU(cudaMemcpyAsync(val + (size_t)k_old * s.esize, c->work + c->ws.val + ut * s.kcap * s.esize, (size_t)kc * s.esize, cudaMemcpyDeviceToDevice, st));
+            }
+            CU(launch_offset_copy(off + T0 / kResTile, wsp<int32_t>(c, c->ws.tile_off) + ut * (s.ntiles_max + 1), nslices + 1, (int)k_old, st));
+            q.bytes_by_mode[1] += (size_t)kc * (c->packed_lists ? 4 : 4 + s.esize);
+        }
+    }
+    // ---- the remaining tail rows move down (through the staging area: the ranges may overlap) ----
+    if (rest > 0) {
+        char* tmp = c->work + c->ws.z1;
+        const size_t w = (size_t)rest * row_b;
+        for (int l = 0; l < s.L; ++l)
+            for (char* base : {tail_base(tk, l), tail_base(tv, l)}) {
+                CU(cudaMemcpy2DAsync(tmp, w, base + (size_t)n * row_b, tail_head_b, w, s.Hkv, cudaMemcpyDeviceToDevice, st));
+                CU(cudaMemcpy2DAsync(base, tail_head_b, tmp, w, w, s.Hkv, cudaMemcpyDeviceToDevice, st));
+            }
+    }
+    CU(launch_set_tail_len(arp<int32_t>(c, c->ar.tail_len), s.L, s.max_batch, seq, rest, st));
+    q.tail_len.assign(s.L, rest);
+    // ---- descriptors: every layer of the sequence now holds T0 + n prompt-side tokens ----
+    const size_t seq_desc = (size_t)s.L * s.Hkv;
+    for (size_t i = 0; i < seq_desc; ++i) c->desc_host[(size_t)seq * seq_desc + i].T = T0 + n;
+    CU(cudaMemcpyAsync(c->arena + c->ar.desc + (size_t)seq * seq_desc * sizeof(UnitDesc), &c->desc_host[(size_t)seq * seq_desc],
+                       seq_desc * sizeof(UnitDesc), cudaMemcpyHostToDevice, st));
+    CU(cudaStreamSynchronize(st));
+    q.T = T0 + n;
+    q.k_entries = k_old + kc;
+    q.fold_used += n;
+    return FDKV_OK;
+}
+
 fdkv_status fdkv_get_shared(fdkv_ctx* c, int32_t seq, int32_t pair, int32_t h, int32_t is_v, void* z0_out, void* stream) {
     if (!seq_ok(c, seq) || !z0_out || pair < 0 || pair >= c->s.P || h < 0 || h >= c->s.Hkv) return FDKV_ERR_INVALID_ARG;
     if (c->staged_seq != seq || !c->pair_compressed[pair]) return FDKV_ERR_STATE;
@@ -740,7 +866,7 @@ fdkv_status fdkv_decode_bytes(fdkv_ctx* c, int32_t layer, int32_t batch, size_t*
     for (int b = 0; b < batch; ++b) {
         const SeqState& q = c->seqs[b];
         if (!q.committed) return FDKV_ERR_STATE;
-        const int64_t k = (int64_t)q.T * s.d * s.keep_num / s.keep_den;
+        const int64_t k = q.k_entries;  // prompt + folded chunks
         const int ntiles = (q.T + kResTile - 1) / kResTile;
         for (int h = 0; h < s.Hkv; ++h) {
             const int m = q.modes[(layer / s.B) * s.Hkv + h];

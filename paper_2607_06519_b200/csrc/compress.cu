@@ -472,6 +472,17 @@ cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream
     return cudaGetLastError();
 }
 
+__global__ void offset_copy_kernel(int32_t* dst, const int32_t* src, int n, int add) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = src[i] + add;
+}
+cudaError_t launch_offset_copy(int32_t* dst, const int32_t* src, int n, int add, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    offset_copy_kernel<<<(n + 255) / 256, 256, 0, st>>>(dst, src, n, add);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st) {
     if (T <= 0) return cudaSuccess;
     const int vec = esize == 2 ? 8 : 4;

@@ -70,6 +70,8 @@ struct Shape {
     int tail_rows;     // max_tail rounded up to kRowPad
     int tok_rule;      // 1: token-granular residual chosen by the probe
     int B;             // layers per depth block: 2 or 4
+    int max_fold;      // generated tokens that may be folded into the compressed form per sequence
+    int64_t kfold_max; // floor(max_fold*d*num/den): list room reserved for them
     int NB;            // staged high-frequency tensors per unit-tensor: 1 (Z1 of a pair) or 4 (the layers' deviations)
     int64_t ktok_max, ktok_cap;  // floor(Tmax*num/den) and the list capacity incl. slack
 };
@@ -90,6 +92,8 @@ struct SeqState {
     std::vector<int32_t> modes;  // [NU], -1 unknown
     size_t bytes_by_mode[3] = {0, 0, 0};
     std::vector<int32_t> tail_len;  // host mirror per layer
+    int fold_used = 0;              // tokens folded so far
+    int64_t k_entries = 0;          // entries per residual list (prompt + folded chunks)
 };
 
 }  // namespace fdkv
@@ -237,6 +241,8 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st);
 bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out);
 // Same view ([rows][128] bf16, 64-channel x box_rows boxes, 128-byte swizzle) over any 256-byte aligned region.
 bool make_rows_tensor_map(void* base, size_t bytes, int box_rows, void* tmap_out);
+// dst[i] = src[i] + add, i < n (list offsets and indices of a folded chunk)
+cudaError_t launch_offset_copy(int32_t* dst, const int32_t* src, int n, int add, cudaStream_t st);
 cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st);
 
 // ---- token-granular residual (token_rule.cu) ----
