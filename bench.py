@@ -320,13 +320,19 @@ def run_ours(args, w):
         hk = [t.cpu().pin_memory() for t in new_k]
         hv = [t.cpu().pin_memory() for t in new_v]
 
+    # one call per step: every layer's query (and new rows) in one pinned buffer each, all outputs back in one
+    hq_all = torch.stack(hq).pin_memory()                      # [L, batch, Hq, d]
+    hout_all = torch.empty(hq_all.shape, dtype=tdt).pin_memory()
+    if append:
+        hk_all = torch.stack(hk).transpose(0, 1).contiguous().pin_memory()  # [step, L, batch, Hkv, d]
+        hv_all = torch.stack(hv).transpose(0, 1).contiguous().pin_memory()
+
     def host_step():
         j = step_no[0]
-        for l in range(w.n_layers):
-            if append:
-                ctx.decode_attn_host(l, hq[l], hk[l][j], hv[l][j], hout[l], od, stream=stream)
-            else:
-                ctx.decode_attn_host(l, hq[l], None, None, hout[l], od, stream=stream)
+        if append:
+            ctx.decode_step_host(hq_all, hk_all[j], hv_all[j], hout_all, od, stream=stream)
+        else:
+            ctx.decode_step_host(hq_all, None, None, hout_all, od, stream=stream)
         step_no[0] = j + 1
 
     for _ in range(min(args.warmup, 3)):

@@ -187,6 +187,14 @@ fdkv_status fdkv_decode_attn_host(fdkv_ctx* ctx, int32_t layer, int32_t batch, c
                                   const void* k_new /*HOST*/, const void* v_new /*HOST*/, void* out /*HOST*/,
                                   int32_t out_dtype, void* stream);
 
+/* All layers of one step with HOST buffers: q and out are [n_layers][batch][n_q_heads][head_dim], k_new / v_new
+ * [n_layers][batch][n_kv_heads][head_dim] or both NULL.  One host-to-device copy per input, the n_layers layer calls
+ * of fdkv_decode_attn in layer order, one device-to-host copy of all outputs, one wait for the stream.  For callers
+ * that know every layer's query up front (attention-only benchmarks, verification of a recorded step); a model that
+ * computes layer l+1's query from layer l's output uses the per-layer calls.                                      */
+fdkv_status fdkv_decode_step_host(fdkv_ctx* ctx, int32_t batch, const void* q /*HOST*/, const void* k_new /*HOST*/,
+                                  const void* v_new /*HOST*/, void* out /*HOST*/, int32_t out_dtype, void* stream);
+
 /* Sets the tail length of every layer of a sequence (0 empties the tails; n <= current length). */
 fdkv_status fdkv_set_tail_len(fdkv_ctx* ctx, int32_t seq, int32_t n, void* stream);
 

@@ -52,6 +52,7 @@ def _load():
         "fdkv_commit": [vp, i32, vp],
         "fdkv_decode_attn": [vp, i32, i32, vp, vp, vp, vp, i32, vp],
         "fdkv_decode_attn_host": [vp, i32, i32, vp, vp, vp, vp, i32, vp],
+        "fdkv_decode_step_host": [vp, i32, vp, vp, vp, vp, i32, vp],
         "fdkv_set_tail_len": [vp, i32, i32, vp],
         "fdkv_fold_tail": [vp, i32, i32, vp],
         "fdkv_get_shared": [vp, i32, i32, i32, i32, vp, vp],
@@ -240,6 +241,13 @@ class Context:
         """Same with host (ideally pinned) tensors; synchronous."""
         _check(_lib.fdkv_decode_attn_host(self.h, layer, q.shape[0], _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
                                           out_dtype, _stream(stream)), "fdkv_decode_attn_host")
+        return out
+
+    def decode_step_host(self, q, k_new, v_new, out, out_dtype, stream=None):
+        """All layers of one step with host (ideally pinned) tensors: q, out [L, batch, Hq, d]; k_new, v_new
+        [L, batch, Hkv, d] or None.  One copy in, L layer calls, one copy out; synchronous."""
+        _check(_lib.fdkv_decode_step_host(self.h, q.shape[1], _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), out_dtype,
+                                          _stream(stream)), "fdkv_decode_step_host")
         return out
 
     def set_tail_len(self, seq, n, stream=None):

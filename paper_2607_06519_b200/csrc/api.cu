@@ -90,10 +90,10 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.modes = take((size_t)s.NU * 4);
     w.partials = take((size_t)s.max_batch * s.Hq * kMaxSplits * (s.d + 4) * 4);
     w.counters = take((size_t)s.max_batch * s.Hkv * 4);
-    w.io_q = take((size_t)s.max_batch * s.Hq * s.d * 4);
-    w.io_k = take((size_t)s.max_batch * s.Hkv * s.d * 4);
-    w.io_v = take((size_t)s.max_batch * s.Hkv * s.d * 4);
-    w.io_out = take((size_t)s.max_batch * s.Hq * s.d * 4);
+    w.io_q = take((size_t)s.L * s.max_batch * s.Hq * s.d * 4);  // host-I/O staging: room for every layer of a step
+    w.io_k = take((size_t)s.L * s.max_batch * s.Hkv * s.d * 4);
+    w.io_v = take((size_t)s.L * s.max_batch * s.Hkv * s.d * 4);
+    w.io_out = take((size_t)s.L * s.max_batch * s.Hq * s.d * 4);
     w.total = o;
 
     o = 0;
@@ -672,6 +672,31 @@ fdkv_status fdkv_decode_attn_host(fdkv_ctx* c, int32_t layer, int32_t batch, con
                                 k_new ? c->work + c->ws.io_v : nullptr, c->work + c->ws.io_out, out_dtype, st);
     if (r != FDKV_OK) return r;
     CU(cudaMemcpyAsync(out, c->work + c->ws.io_out, ob, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return FDKV_OK;
+}
+
+fdkv_status fdkv_decode_step_host(fdkv_ctx* c, int32_t batch, const void* q, const void* k_new, const void* v_new, void* out,
+                                  int32_t out_dtype, void* stream) {
+    if (!c || !q || !out) return FDKV_ERR_INVALID_ARG;
+    if (batch < 1 || batch > c->s.max_batch) return FDKV_ERR_INVALID_ARG;
+    if ((k_new == nullptr) != (v_new == nullptr)) return FDKV_ERR_INVALID_ARG;
+    if (out_dtype != FDKV_F32 && out_dtype != FDKV_BF16) return FDKV_ERR_INVALID_ARG;
+    const Shape& s = c->s;
+    cudaStream_t st = S(stream);
+    const size_t qb = (size_t)batch * s.Hq * s.d * s.esize, kb = (size_t)batch * s.Hkv * s.d * s.esize;
+    const size_t ob = (size_t)batch * s.Hq * s.d * (out_dtype == FDKV_BF16 ? 2 : 4);
+    CU(cudaMemcpyAsync(c->work + c->ws.io_q, q, qb * s.L, cudaMemcpyHostToDevice, st));
+    if (k_new) {
+        CU(cudaMemcpyAsync(c->work + c->ws.io_k, k_new, kb * s.L, cudaMemcpyHostToDevice, st));
+        CU(cudaMemcpyAsync(c->work + c->ws.io_v, v_new, kb * s.L, cudaMemcpyHostToDevice, st));
+    }
+    for (int l = 0; l < s.L; ++l) {
+        fdkv_status r = decode_impl(c, l, batch, c->work + c->ws.io_q + l * qb, k_new ? c->work + c->ws.io_k + l * kb : nullptr,
+                                    k_new ? c->work + c->ws.io_v + l * kb : nullptr, c->work + c->ws.io_out + l * ob, out_dtype, st);
+        if (r != FDKV_OK) return r;
+    }
+    CU(cudaMemcpyAsync(out, c->work + c->ws.io_out, ob * s.L, cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     return FDKV_OK;
 }

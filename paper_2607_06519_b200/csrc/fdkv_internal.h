@@ -80,7 +80,7 @@ struct WsLayout {
     size_t tok_score, tok_flag, tok_list, tok_off;
     size_t energy, eval;  // four-layer blocks: per-position high-frequency energy (float32) and the kept energies
     size_t status, z0, z1, z1drop, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
-        partials, counters, io_q, io_k, io_v, io_out, total;
+        partials, counters, io_q, io_k, io_v, io_out, total;  // io_*: host-I/O staging, [L] layers each
 };
 struct ArenaLayout {
     size_t tail_len, desc, tail_k, tail_v, bump, worst_total;

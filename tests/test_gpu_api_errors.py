@@ -99,3 +99,30 @@ def test_reset_frees_the_arena():
         assert ctx.get_modes(0).tolist() == [[2, 2]]
         ctx.reset()
     ctx.close()
+
+
+def test_step_host_call_equals_per_layer_calls():
+    """fdkv_decode_step_host (all layers of a step, host buffers) returns what the per-layer device calls return."""
+    import torch
+    from paper_2607_06519_b200 import binding as B, runner, synth
+
+    w = synth.Workload(name="step", n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=128, batch=2, T=700, dtype="bf16",
+                       keep_num=1, keep_den=16, n_needles=4, W=8, seed=5, n_steps=2, seq_seeds=(5, 6))
+    pf = runner.Prefilled(w, max_tail=4)
+    for b in range(2):
+        pf.prefill(b, modes=np.array([[0, 1], [2, 1]], dtype=np.int32))
+    qs = [pf.decode_q(l, 0) for l in range(4)]
+    rows = [pf.new_rows(l, 0) for l in range(4)]
+    want = [pf.ctx.decode_attn(l, qs[l], rows[l][0], rows[l][1]) for l in range(4)]
+    torch.cuda.synchronize()
+    for b in range(2):
+        pf.ctx.set_tail_len(b, 0)
+    hq = torch.stack(qs).cpu().pin_memory()
+    hk = torch.stack([r[0] for r in rows]).cpu().pin_memory()
+    hv = torch.stack([r[1] for r in rows]).cpu().pin_memory()
+    hout = torch.empty(hq.shape, dtype=torch.bfloat16).pin_memory()
+    pf.ctx.decode_step_host(hq, hk, hv, hout, B.BF16)
+    for l in range(4):
+        assert torch.equal(hout[l], want[l].cpu())
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
