@@ -158,3 +158,72 @@ def test_block4_benchmark_workload_sampled():
     assert sum(by_mode) < 0.5 * exact_equiv  # a shared unit stores one of four layers
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_mixed_schedule_two_contexts():
+    """The paper's mixed schedule (B = 4 in the middle, B = 2 for the first and last layers) as two contexts: a
+    12-layer stack whose layers 0-3 and 8-11 form pairs (one 8-layer context) and whose layers 4-7 form one block
+    of four (a second context).  Every layer's output matches the oracle of its own block size."""
+    from gpu_util import oracle_unit
+    runner = _runner()
+    base = dict(n_q_heads=8, n_kv_heads=2, head_dim=128, batch=1, T=900, dtype="bf16", keep_num=1, keep_den=16,
+                n_needles=4, W=8, n_steps=1)
+    w2 = synth.Workload(name="edge_pairs", n_layers=8, seed=41, **base)                 # model layers 0-3, 8-11
+    w4 = synth.Workload(name="middle_block", n_layers=4, seed=42, block_size=4, **base)  # model layers 4-7
+    pf2, pf4 = runner.Prefilled(w2, max_tail=1), runner.Prefilled(w4, max_tail=1)
+    m2 = np.array([[0, 1], [1, 2], [2, 0], [1, 1]], dtype=np.int32)
+    m4 = np.array([[1, 0]], dtype=np.int32)
+    pf2.prefill(0, modes=m2)
+    pf4.prefill(0, modes=m4)
+    u2 = {(p, h): oracle_unit(w2, 0, p, h) for p in range(4) for h in range(2)}
+    u4 = {(0, h): oracle_unit4(w4, 0, 0, h) for h in range(2)}
+    G = 4
+    worst = 0.0
+    for model_layer in range(12):
+        if 4 <= model_layer < 8:
+            pf, w, local = pf4, w4, model_layer - 4
+        else:
+            pf, w, local = pf2, w2, model_layer if model_layer < 4 else model_layer - 4
+        q = pf.decode_q(local, 0)
+        out = f32(pf.ctx.decode_attn(local, q, out_dtype=0))[0]
+        torch.cuda.synchronize()
+        for h in range(2):
+            qh = f32(q)[0][h * G:(h + 1) * G]
+            if pf is pf4:
+                ref = u4[(0, h)].attend(int(m4[0][h]), local, qh)
+            else:
+                ref = u2[(local // 2, h)].attend(int(m2[local // 2][h]), local & 1, qh)
+            worst = max(worst, float(vector_errors(out[h * G:(h + 1) * G], ref).max()))
+    assert worst <= TOL["bf16"], worst
+    for pf in (pf2, pf4):
+        assert pf.ctx.device_status() == 0
+        pf.ctx.close()
+
+
+def test_block4_two_sequences_of_different_length():
+    runner = _runner()
+    w = synth.Workload(name="b4two", n_layers=4, n_q_heads=4, n_kv_heads=2, head_dim=128, batch=2, T=640, dtype="bf16",
+                       keep_num=1, keep_den=8, n_needles=4, W=8, seed=13, n_steps=3, block_size=4, seq_seeds=(13, 14))
+    pf = runner.Prefilled(w, max_tail=3)
+    modes = np.array([[1, 2]], dtype=np.int32)
+    units = {}
+    for b in range(2):
+        pf.prefill(b, modes=modes)
+        for h in range(2):
+            units[(b, h)] = R4.Unit4(synth.block_tensor(w, b, 0, h, False), synth.block_tensor(w, b, 0, h, True), True, 1, 8)
+    G = 2
+    for step in range(3):
+        for layer in range(4):
+            q = pf.decode_q(layer, step)
+            kn, vn = pf.new_rows(layer, step)
+            for b in range(2):
+                for h in range(2):
+                    units[(b, h)].append(layer, f32(kn)[b, h], f32(vn)[b, h])
+            out = f32(pf.ctx.decode_attn(layer, q, kn, vn, out_dtype=0))
+            torch.cuda.synchronize()
+            for b in range(2):
+                for h in range(2):
+                    ref = units[(b, h)].attend(int(modes[0][h]), layer, f32(q)[b][h * G:(h + 1) * G])
+                    assert vector_errors(out[b][h * G:(h + 1) * G], ref).max() <= TOL["bf16"]
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()

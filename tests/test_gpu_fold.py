@@ -76,3 +76,45 @@ def test_fold_tail_matches_the_oracle(dtype, d, T, keep):
         pf.ctx.fold_tail(0, 32)
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_fold_one_sequence_of_a_batch():
+    """Folding sequence 1 of two leaves sequence 0 untouched; batched decode afterwards sees T and T + 32."""
+    from gpu_util import oracle_unit
+    from paper_2607_06519_b200 import runner
+
+    w = synth.Workload(name="fold2", n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=128, batch=2, T=512, dtype="bf16",
+                       keep_num=1, keep_den=16, n_needles=4, W=8, seed=33, n_steps=40, seq_seeds=(33, 34))
+    pf = runner.Prefilled(w, max_tail=48, max_fold=64)
+    modes = np.array([[1, 0]], dtype=np.int32)
+    units = {}
+    for b in range(2):
+        pf.prefill(b, modes=modes)
+        for h in range(2):
+            units[(b, h)] = oracle_unit(w, b, 0, h)
+    G = 4
+
+    def step(j, check):
+        for layer in range(2):
+            q = pf.decode_q(layer, j)
+            kn, vn = pf.new_rows(layer, j)
+            for b in range(2):
+                for h in range(2):
+                    units[(b, h)].append(layer, f32(kn)[b, h], f32(vn)[b, h])
+            out = f32(pf.ctx.decode_attn(layer, q, kn, vn, out_dtype=0))
+            if check:
+                torch.cuda.synchronize()
+                for b in range(2):
+                    for h in range(2):
+                        ref = units[(b, h)].attend(int(modes[0][h]), layer, f32(q)[b][h * G:(h + 1) * G])
+                        assert vector_errors(out[b][h * G:(h + 1) * G], ref).max() <= TOL["bf16"], (j, layer, b, h)
+
+    for j in range(34):
+        step(j, check=j == 33)
+    pf.ctx.fold_tail(1, 32)
+    for h in range(2):
+        units[(1, h)].fold(32, 1, 16)
+    for j in range(34, 38):
+        step(j, check=True)
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
