@@ -206,7 +206,8 @@ fdkv_status fdkv_set_tail_len(fdkv_ctx* ctx, int32_t seq, int32_t n, void* strea
  * applied to the chunk; ties to the lowest index) and is appended behind the unit's rows and lists; exact units get
  * the rows themselves.  The remaining tail rows move down; T of the sequence grows by n.  Modes do not change (the
  * originals of shared / residual units no longer exist, so a committed unit cannot be re-routed upwards).
- * Requirements: block size 2, entry residual rule; T and n multiples of 16; every layer's tail holds the same
+ * Requirements: entry residual rule (either block size; a block of four keeps the chunk's positions of largest
+ * high-frequency energy); T and n multiples of 16; every layer's tail holds the same
  * number (>= n) of tokens, i.e. call it between decode steps; the total folded per sequence stays within
  * cfg.max_fold; no other sequence may be staged and uncommitted (the call reuses the staging area and invalidates
  * it).  Synchronous (waits for the stream).  FDKV_ERR_ARENA_FULL when max_fold is exhausted.

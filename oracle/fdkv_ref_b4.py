@@ -134,6 +134,26 @@ class Unit4:
         self.tail[("k", layer_in_block)].append(_f32(k_row))
         self.tail[("v", layer_in_block)].append(_f32(v_row))
 
+    def fold(self, n: int, keep_num: int, keep_den: int):
+        """Periodic refresh for a block of four: the first n generated tokens of the four layers leave the exact tails
+        and join the compressed form under the unit's mode; the chunk keeps its own floor(n d num / den) positions of
+        largest high-frequency energy per tensor."""
+        for name in ("k", "v"):
+            tails = [self.tail[(name, l)] for l in range(4)]
+            assert all(len(t) >= n for t in tails)
+            xc = [np.stack(t[:n]) for t in tails]
+            z0c, devc, ec = depth_split4(xc, self.bf16)
+            keptc = R.select_entries(ec, R.keep_count(n, self.d, keep_num, keep_den))
+            self.kept[name] = np.concatenate([self.kept[name], keptc + np.int32(self.T * self.d)]).astype(np.int32)
+            self.x[name] = [np.concatenate([self.x[name][l], xc[l]]) for l in range(4)]
+            self.z0[name] = np.concatenate([self.z0[name], z0c])
+            self.dev[name] = [np.concatenate([self.dev[name][l], devc[l]]) for l in range(4)]
+            self.energy[name] = np.concatenate([self.energy[name], ec])
+            for l in range(4):
+                self.tail[(name, l)] = tails[l][n:]
+        self.T += n
+        self.k_keep = self.kept["k"].size
+
     def rows(self, name: str, mode: int, layer_in_block: int) -> np.ndarray:
         pre = reconstruct4(self.z0[name], self.dev[name][layer_in_block], self.kept[name], mode,
                            self.x[name][layer_in_block])

@@ -713,7 +713,7 @@ fdkv_status fdkv_set_tail_len(fdkv_ctx* c, int32_t seq, int32_t n, void* stream)
 fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
     if (!seq_ok(c, seq) || n <= 0) return FDKV_ERR_INVALID_ARG;
     const Shape& s = c->s;
-    if (s.B != 2 || s.tok_rule) return FDKV_ERR_UNSUPPORTED;
+    if (s.tok_rule) return FDKV_ERR_UNSUPPORTED;
     SeqState& q = c->seqs[seq];
     if (!q.committed) return FDKV_ERR_STATE;
     if (c->staged_seq >= 0 && !c->seqs[c->staged_seq].committed) return FDKV_ERR_STATE;  // the staging area is in use
@@ -733,71 +733,109 @@ fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
     c->staged_seq = -1;
     std::fill(c->pair_compressed.begin(), c->pair_compressed.end(), 0);
     CU(cudaMemsetAsync(wsp<uint32_t>(c, c->ws.hist), 0, (size_t)s.NT * kHistBins * 4, st));
-    for (int p0 = 0; p0 < s.P; p0 += kSplitPairs) {
-        CompressArgs a;
-        a.n_pairs = s.P - p0 < kSplitPairs ? s.P - p0 : kSplitPairs;
-        for (int j = 0; j < a.n_pairs; ++j) {
-            const int p = p0 + j;
-            a.k0[j] = tail_base(tk, 2 * p); a.k1[j] = tail_base(tk, 2 * p + 1);
-            a.v0[j] = tail_base(tv, 2 * p); a.v1[j] = tail_base(tv, 2 * p + 1);
-        }
-        a.stride_t = s.d; a.stride_h = (int64_t)s.tail_rows * s.d;
-        a.T = n; a.d = s.d; a.Hkv = s.Hkv; a.tensors = 2;
-        a.ut_base = p0 * s.Hkv * 2;
-        a.unit_stride = (int64_t)s.Tmax * s.d;
-        a.z0 = c->work + c->ws.z0; a.z1 = c->work + c->ws.z1;
-        a.hist = wsp<uint32_t>(c, c->ws.hist);
-        CU(launch_split_hist(a, s.dtype, st));
-    }
     const int64_t kc = (int64_t)n * s.d * s.keep_num / s.keep_den;
     SelectArgs sa;
     sa.ut_begin = 0; sa.ut_count = s.NT;
     sa.T = n; sa.d = s.d; sa.k = kc;
     sa.unit_stride = (int64_t)s.Tmax * s.d; sa.kcap = s.kcap; sa.ntiles_max = s.ntiles_max;
-    sa.z1 = c->work + c->ws.z1;
     sa.hist = wsp<uint32_t>(c, c->ws.hist);
     sa.sel = wsp<SelState>(c, c->ws.sel);
     sa.tile_cnt = wsp<uint32_t>(c, c->ws.tile_cnt);
     sa.tile_eq = wsp<uint32_t>(c, c->ws.tile_eq);
     sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
     sa.idx = wsp<int32_t>(c, c->ws.idx);
-    sa.val = c->work + c->ws.val;
-    sa.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
     sa.z1drop = nullptr;
     sa.status = wsp<int32_t>(c, c->ws.status);
-    CU(launch_select_and_compact(sa, s.dtype, st));
+    if (s.B == 4) {
+        for (int p = 0; p < s.P; ++p) {
+            Split4Args a4;
+            for (int l = 0; l < 4; ++l) { a4.k[l] = tail_base(tk, 4 * p + l); a4.v[l] = tail_base(tv, 4 * p + l); }
+            a4.stride_t = s.d; a4.stride_h = (int64_t)s.tail_rows * s.d;
+            a4.T = n; a4.d = s.d; a4.Hkv = s.Hkv;
+            a4.ut_base = p * s.Hkv * 2;
+            a4.unit_stride = (int64_t)s.Tmax * s.d;
+            a4.z0 = c->work + c->ws.z0; a4.dev = c->work + c->ws.z1;
+            a4.energy = wsp<float>(c, c->ws.energy);
+            a4.drop = nullptr;
+            a4.hist = wsp<uint32_t>(c, c->ws.hist);
+            CU(launch_split4_hist(a4, s.dtype, st));
+        }
+        sa.z1 = c->work + c->ws.energy;
+        sa.val = c->work + c->ws.eval;
+        sa.packed = nullptr;
+        CU(launch_select_and_compact(sa, FDKV_F32, st));
+        Gather4Args g;
+        g.ut_begin = 0; g.ut_count = s.NT;
+        g.k = kc; g.kcap = s.kcap; g.unit_stride = (int64_t)s.Tmax * s.d;
+        g.dev = c->work + c->ws.z1;
+        g.idx = wsp<int32_t>(c, c->ws.idx);
+        g.val = c->work + c->ws.val;
+        g.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
+        g.drop = nullptr;
+        CU(launch_gather4(g, s.dtype, st));
+    } else {
+        for (int p0 = 0; p0 < s.P; p0 += kSplitPairs) {
+            CompressArgs a;
+            a.n_pairs = s.P - p0 < kSplitPairs ? s.P - p0 : kSplitPairs;
+            for (int j = 0; j < a.n_pairs; ++j) {
+                const int p = p0 + j;
+                a.k0[j] = tail_base(tk, 2 * p); a.k1[j] = tail_base(tk, 2 * p + 1);
+                a.v0[j] = tail_base(tv, 2 * p); a.v1[j] = tail_base(tv, 2 * p + 1);
+            }
+            a.stride_t = s.d; a.stride_h = (int64_t)s.tail_rows * s.d;
+            a.T = n; a.d = s.d; a.Hkv = s.Hkv; a.tensors = 2;
+            a.ut_base = p0 * s.Hkv * 2;
+            a.unit_stride = (int64_t)s.Tmax * s.d;
+            a.z0 = c->work + c->ws.z0; a.z1 = c->work + c->ws.z1;
+            a.hist = wsp<uint32_t>(c, c->ws.hist);
+            CU(launch_split_hist(a, s.dtype, st));
+        }
+        sa.z1 = c->work + c->ws.z1;
+        sa.val = c->work + c->ws.val;
+        sa.packed = c->packed_lists ? wsp<uint32_t>(c, c->ws.packed) : nullptr;
+        CU(launch_select_and_compact(sa, s.dtype, st));
+    }
     // ---- append behind every unit's rows and lists, under the unit's mode ----
     const size_t unit_stride_b = (size_t)s.Tmax * s.d * s.esize, chunk_b = (size_t)n * row_b, at = (size_t)T0 * row_b;
     const int64_t k_old = q.k_entries;
     const int nslices = n / kResTile;
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u], p = u / s.Hkv, h = u % s.Hkv;
-        UnitDesc* dl[2] = {&c->desc_host[((size_t)seq * s.L + 2 * p) * s.Hkv + h], &c->desc_host[((size_t)seq * s.L + 2 * p + 1) * s.Hkv + h]};
+        UnitDesc* dl[4] = {nullptr, nullptr, nullptr, nullptr};
+        for (int l = 0; l < s.B; ++l) dl[l] = &c->desc_host[((size_t)seq * s.L + (size_t)s.B * p + l) * s.Hkv + h];
         if (m == FDKV_MODE_EXACT) {
-            for (int l = 0; l < 2; ++l) {
-                CU(cudaMemcpyAsync((char*)dl[l]->k_rows + at, tail_base(tk, 2 * p + l) + h * tail_head_b, chunk_b, cudaMemcpyDeviceToDevice, st));
-                CU(cudaMemcpyAsync((char*)dl[l]->v_rows + at, tail_base(tv, 2 * p + l) + h * tail_head_b, chunk_b, cudaMemcpyDeviceToDevice, st));
+            for (int l = 0; l < s.B; ++l) {
+                CU(cudaMemcpyAsync((char*)dl[l]->k_rows + at, tail_base(tk, s.B * p + l) + h * tail_head_b, chunk_b, cudaMemcpyDeviceToDevice, st));
+                CU(cudaMemcpyAsync((char*)dl[l]->v_rows + at, tail_base(tv, s.B * p + l) + h * tail_head_b, chunk_b, cudaMemcpyDeviceToDevice, st));
             }
-            q.bytes_by_mode[2] += 4 * chunk_b;
+            q.bytes_by_mode[2] += 2 * (size_t)s.B * chunk_b;
             continue;
         }
         for (int is_v = 0; is_v < 2; ++is_v) {
             const size_t ut = (size_t)u * 2 + is_v;
-            char* rows = (char*)(is_v ? dl[0]->v_rows : dl[0]->k_rows);  // both layers share the coefficient rows
+            char* rows = (char*)(is_v ? dl[0]->v_rows : dl[0]->k_rows);  // every layer of the block shares the coefficient rows
             CU(cudaMemcpyAsync(rows + at, c->work + c->ws.z0 + ut * unit_stride_b, chunk_b, cudaMemcpyDeviceToDevice, st));
             q.bytes_by_mode[m] += chunk_b;
             if (m != FDKV_MODE_RESIDUAL) continue;
-            int32_t* list = const_cast<int32_t*>(is_v ? dl[0]->v_idx : dl[0]->k_idx);
             int32_t* off = const_cast<int32_t*>(is_v ? dl[0]->v_off : dl[0]->k_off);
-            if (c->packed_lists) {  // packed entries carry slice-relative positions: valid as they are (T0 is a multiple of 16)
-                CU(cudaMemcpyAsync(list + k_old, c->work + c->ws.packed + ut * s.kcap * 4, (size_t)kc * 4, cudaMemcpyDeviceToDevice, st));
+            if (c->packed_lists) {
+                // packed entries carry slice-relative positions: valid as they are (T0 is a multiple of 16); one list per
+                // stored high-frequency tensor (a pair's two layers share theirs)
+                for (int j = 0; j < s.NB; ++j) {
+                    int32_t* list = const_cast<int32_t*>(is_v ? dl[j]->v_idx : dl[j]->k_idx);
+                    CU(cudaMemcpyAsync(list + k_old, c->work + c->ws.packed + (ut * s.NB + j) * s.kcap * 4, (size_t)kc * 4, cudaMemcpyDeviceToDevice, st));
+                }
             } else {
-                char* val = (char*)const_cast<void*>(is_v ? dl[0]->v_val : dl[0]->k_val);
+                int32_t* list = const_cast<int32_t*>(is_v ? dl[0]->v_idx : dl[0]->k_idx);  // one index list for the unit
                 CU(launch_offset_copy(list + k_old, wsp<int32_t>(c, c->ws.idx) + ut * s.kcap, (int)kc, T0 * s.d, st));
-                CU(cudaMemcpyAsync(val + (size_t)k_old * s.esize, c->work + c->ws.val + ut * s.kcap * s.esize, (size_t)kc * s.esize, cudaMemcpyDeviceToDevice, st));
+                for (int j = 0; j < s.NB; ++j) {
+                    char* val = (char*)const_cast<void*>(is_v ? dl[j]->v_val : dl[j]->k_val);
+                    CU(cudaMemcpyAsync(val + (size_t)k_old * s.esize, c->work + c->ws.val + (ut * s.NB + j) * s.kcap * s.esize, (size_t)kc * s.esize,
+                                       cudaMemcpyDeviceToDevice, st));
+                }
             }
             CU(launch_offset_copy(off + T0 / kResTile, wsp<int32_t>(c, c->ws.tile_off) + ut * (s.ntiles_max + 1), nslices + 1, (int)k_old, st));
-            q.bytes_by_mode[1] += (size_t)kc * (c->packed_lists ? 4 : 4 + s.esize);
+            q.bytes_by_mode[1] += (size_t)kc * (c->packed_lists ? (size_t)4 * s.NB : 4 + (size_t)s.NB * s.esize);
         }
     }
     // ---- the remaining tail rows move down (through the staging area: the ranges may overlap) ----

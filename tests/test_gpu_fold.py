@@ -118,3 +118,42 @@ def test_fold_one_sequence_of_a_batch():
         step(j, check=True)
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_fold_tail_block_of_four():
+    """The same refresh for depth blocks of four layers (shared kept set by energy inside the chunk)."""
+    from oracle import fdkv_ref_b4 as R4
+    from paper_2607_06519_b200 import runner
+
+    w = synth.Workload(name="fold4", n_layers=8, n_q_heads=8, n_kv_heads=2, head_dim=128, batch=1, T=1024, dtype="bf16",
+                       keep_num=1, keep_den=16, n_needles=4, W=8, seed=35, n_steps=60, block_size=4)
+    pf = runner.Prefilled(w, max_tail=64, max_fold=64)
+    modes = np.array([[1, 0], [2, 1]], dtype=np.int32)
+    pf.prefill(0, modes=modes)
+    units = {(b, h): R4.Unit4(synth.block_tensor(w, 0, b, h, False), synth.block_tensor(w, 0, b, h, True), True, 1, 16)
+             for b in range(2) for h in range(2)}
+    G = 4
+
+    def step(j, check):
+        for layer in range(8):
+            blk, lb = divmod(layer, 4)
+            q = pf.decode_q(layer, j)
+            kn, vn = pf.new_rows(layer, j)
+            for h in range(2):
+                units[(blk, h)].append(lb, f32(kn)[0, h], f32(vn)[0, h])
+            out = f32(pf.ctx.decode_attn(layer, q, kn, vn, out_dtype=0))[0]
+            if check:
+                torch.cuda.synchronize()
+                for h in range(2):
+                    ref = units[(blk, h)].attend(int(modes[blk][h]), lb, f32(q)[0][h * G:(h + 1) * G])
+                    assert vector_errors(out[h * G:(h + 1) * G], ref).max() <= TOL["bf16"], (j, layer, h)
+
+    for j in range(50):
+        step(j, check=j == 49)
+    pf.ctx.fold_tail(0, 48)
+    for u in units.values():
+        u.fold(48, 1, 16)
+    for j in range(50, 54):
+        step(j, check=True)
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()

@@ -217,3 +217,31 @@ def test_unit4_on_the_synthetic_recipe():
     rs = u.attend(R4.RESIDUAL, 1, q)
     sh = u.attend(R4.SHARED, 1, q)
     assert np.abs(rs - ex).max() <= np.abs(sh - ex).max() * 1.5 + 1e-9
+
+
+def test_fold_of_a_block_of_four():
+    g = np.random.default_rng(8)
+    T, d, n_tail = 32, 8, 24
+    mk = lambda *s: g.standard_normal(s).astype(np.float32)
+    u = R4.Unit4([mk(T, d) for _ in range(4)], [mk(T, d) for _ in range(4)], False, 1, 4)
+    rows = [[(mk(d), mk(d)) for _ in range(4)] for _ in range(n_tail)]
+    for r in rows:
+        for l in range(4):
+            u.append(l, r[l][0], r[l][1])
+    q = mk(2, d)
+    before = [u.attend(R4.EXACT, l, q) for l in range(4)]
+    u.fold(16, 1, 4)
+    assert u.T == T + 16 and all(len(u.tail[("k", l)]) == 8 for l in range(4))
+    for l in range(4):
+        np.testing.assert_allclose(u.attend(R4.EXACT, l, q), before[l], rtol=1e-12, atol=1e-12)
+    # the chunk keeps its own top-k by energy, inside the chunk, ascending overall
+    xc = [np.stack([rows[t][l][0] for t in range(16)]) for l in range(4)]
+    _, devc, ec = R4.depth_split4(xc, False)
+    e = ec.reshape(-1).astype(np.float64)
+    order = np.lexsort((np.arange(e.size), -e))
+    want = np.sort(order[:(16 * d) // 4]) + T * d
+    assert np.array_equal(u.kept["k"][(T * d) // 4:], want)
+    np.testing.assert_array_equal(u.dev["k"][2][T:], devc[2])
+    # shared mode: the folded tokens become the block mean
+    got = u.rows("k", R4.SHARED, 1)[T:T + 16]
+    np.testing.assert_allclose(got, np.mean(np.stack(xc).astype(np.float64), axis=0), rtol=1e-6, atol=1e-7)
