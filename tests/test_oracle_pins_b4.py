@@ -64,7 +64,7 @@ def test_stored_values_follow_the_stated_arithmetic(bf16):
             dv = rs(np.array([f(x[l][t, c] - f(0.5) * z)], dtype=np.float32))[0]
             assert dev[l][t, c] == dv
             e.append(f(dv * dv))
-        assert energy[t, c] == f(f(e[0] + e[1]) + f(e[2] + e[3]))
+        assert energy[t, c] == rs(np.array([f(f(e[0] + e[1]) + f(e[2] + e[3]))], dtype=np.float32))[0]
     # against float64 within the storage rounding
     x64 = np.stack([a.astype(np.float64) for a in x])
     tol = 2.0 ** -8 if bf16 else 2.0 ** -22
