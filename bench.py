@@ -112,7 +112,11 @@ def oracle_sample(w, n_units: int):
         else:
             k0, k1 = synth.unit_tensor(w, 0, p, h, False)
             v0, v1 = synth.unit_tensor(w, 0, p, h, True)
-            u = R.Unit(k0, k1, v0, v1, w.dtype == "bf16", w.keep_num, w.keep_den)
+            if w.row_format == 1:
+                from oracle import fdkv_ref_fp8 as R8
+                u = R8.UnitFp8(k0, k1, v0, v1, w.dtype == "bf16", w.keep_num, w.keep_den)
+            else:
+                u = R.Unit(k0, k1, v0, v1, w.dtype == "bf16", w.keep_num, w.keep_den)
         mode = (0, 1, 0, 2, 1, 0, 1, 0)[i % 8]  # close to the 50/35/15 benchmark mix
         units.append((p, h, mode, u))
     return units
@@ -376,7 +380,8 @@ def run_ours(args, w):
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "context": w.T, "batch": w.batch, "layers": w.n_layers, "q_heads": w.n_q_heads,
                    "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "keep": f"{w.keep_num}/{w.keep_den}",
-                   "residual_rule": "tokens" if w.residual_rule == 1 else "entries", "mode_mix_shared_residual_exact": mix, "launch": "cuda_graph" if graph is not None else "stream",
+                   "residual_rule": "tokens" if w.residual_rule == 1 else "entries", "rows": "e4m3" if w.row_format == 1 else w.dtype,
+                   "block_size": w.block_size, "mode_mix_shared_residual_exact": mix, "launch": "cuda_graph" if graph is not None else "stream",
                    "l2": "inputs larger than L2 (each step streams the whole packed cache)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,

@@ -65,7 +65,23 @@ typedef struct {
     int32_t block_size;  /* B of Eq. 1: 2 (also when 0) or 4 layers per depth block                    */
     int32_t max_fold;    /* generated tokens fdkv_fold_tail may move into the compressed form per       */
                          /*   sequence (0: none); fdkv_commit reserves row and list room for them       */
+    int32_t row_format;  /* fdkv_row_format: how fdkv_commit stores the dense row streams               */
 } fdkv_config;
+
+/*
+ * FDKV_ROWS_STORAGE (default): the committed rows (Z0 of shared / residual units, the original rows of exact units)
+ *   keep the storage type.
+ * FDKV_ROWS_E4M3: they are stored as 8-bit floats (4 exponent bits with bias 7, 3 mantissa bits, no infinities,
+ *   largest finite value 448) with one float32 scale per channel of each stored tensor -- the composition with
+ *   quantisation that the Method section mentions after Eq. 3; the paper fixes no scheme, this is the build's:
+ *       amax_c = max_t |R[t][c]|;  scale_c = amax_c / 448 (float32 division; 1 when amax_c = 0);
+ *       code = e4m3(R[t][c] / scale_c)   (float32 division, round to nearest even, saturating);
+ *       attention sees decode(code) * scale_c.
+ *   Sparse residual values and the generated-token tails keep the storage type.  Halves the bytes a decode call
+ *   streams.  bf16 storage, head_dim 128, block size 2, entry residual rule, group size <= 4; fdkv_fold_tail is
+ *   unavailable.  Compression and the probe are unchanged (they see the unquantised coefficients).
+ */
+typedef enum { FDKV_ROWS_STORAGE = 0, FDKV_ROWS_E4M3 = 1 } fdkv_row_format;
 
 /*
  * Block size 4 (Method, Eq. 1 with the orthonormal DCT-II of size 4; the paper's default for middle layers).
@@ -213,6 +229,12 @@ fdkv_status fdkv_set_tail_len(fdkv_ctx* ctx, int32_t seq, int32_t n, void* strea
  * it).  Synchronous (waits for the stream).  FDKV_ERR_ARENA_FULL when max_fold is exhausted.
  */
 fdkv_status fdkv_fold_tail(fdkv_ctx* ctx, int32_t seq, int32_t n, void* stream);
+
+/* FDKV_ROWS_E4M3 only: the 8-bit codes [T][head_dim] and the float32 scales [head_dim] of one committed row stream
+ * (layer's K or V rows of a KV head: Z0 for shared / residual units, the layer's own rows for exact ones).  Device
+ * buffers, either may be NULL.  Synchronous.                                                                      */
+fdkv_status fdkv_get_rows_e4m3(fdkv_ctx* ctx, int32_t seq, int32_t layer, int32_t kv_head, int32_t is_v,
+                               uint8_t* codes_out /*DEVICE*/, float* scale_out /*DEVICE*/, void* stream);
 
 /* Introspection of the STAGED sequence (valid from fdkv_compress_prefill until the next one).  Synchronous. */
 fdkv_status fdkv_get_shared(fdkv_ctx* ctx, int32_t seq, int32_t pair, int32_t kv_head, int32_t is_v,

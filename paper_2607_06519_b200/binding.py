@@ -31,7 +31,7 @@ class FdkvError(RuntimeError):
 
 class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "max_batch", "max_prefill",
-                                         "max_tail", "dtype", "keep_num", "keep_den", "residual_rule", "block_size", "max_fold")]
+                                         "max_tail", "dtype", "keep_num", "keep_den", "residual_rule", "block_size", "max_fold", "row_format")]
 
 
 def _load():
@@ -55,6 +55,7 @@ def _load():
         "fdkv_decode_step_host": [vp, i32, vp, vp, vp, vp, i32, vp],
         "fdkv_set_tail_len": [vp, i32, i32, vp],
         "fdkv_fold_tail": [vp, i32, i32, vp],
+        "fdkv_get_rows_e4m3": [vp, i32, i32, i32, i32, vp, vp, vp],
         "fdkv_get_shared": [vp, i32, i32, i32, i32, vp, vp],
         "fdkv_get_residual": [vp, i32, i32, i32, i32, vp, vp, P(i32), vp],
         "fdkv_get_modes": [vp, i32, P(i32)],
@@ -103,6 +104,7 @@ class Config:
     residual_rule: int = 0  # 0: largest-magnitude entries; 1: the paper's probe-scored tokens
     block_size: int = 2  # layers per depth block (B of Eq. 1): 2 or 4; "pair" arguments then index blocks
     max_fold: int = 0  # generated tokens fold_tail may move into the compressed form per sequence
+    row_format: int = 0  # 0: committed rows keep the storage type; 1: e4m3 codes with per-channel scales
 
     def c(self) -> _Config:
         return _Config(*(int(getattr(self, f[0])) for f in _Config._fields_))
@@ -256,6 +258,14 @@ class Context:
     def fold_tail(self, seq, n, stream=None):
         """Moves the first n generated tokens of every layer from the exact tails into the compressed form."""
         _check(_lib.fdkv_fold_tail(self.h, seq, n, _stream(stream)), "fdkv_fold_tail")
+
+    def get_rows_e4m3(self, seq, layer, kv_head, is_v, T, stream=None):
+        """8-bit row streams: (codes uint8 [T, d], scales float32 [d]) of a committed layer's K or V rows."""
+        codes = torch.empty((T, self.cfg.head_dim), dtype=torch.uint8, device=self.device)
+        scale = torch.empty(self.cfg.head_dim, dtype=torch.float32, device=self.device)
+        _check(_lib.fdkv_get_rows_e4m3(self.h, seq, layer, kv_head, int(is_v), _ptr(codes), _ptr(scale), _stream(stream)),
+               "fdkv_get_rows_e4m3")
+        return codes, scale
 
     def get_shared(self, seq, pair, kv_head, is_v, T, stream=None):
         out = torch.empty((T, self.cfg.head_dim), dtype=self.tdtype, device=self.device)

@@ -45,6 +45,10 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.dtype = c.dtype; s.esize = c.dtype == FDKV_BF16 ? 2 : 4;
     s.keep_num = c.keep_num; s.keep_den = c.keep_den;
     s.max_fold = c.max_fold;
+    if (c.row_format != FDKV_ROWS_STORAGE && c.row_format != FDKV_ROWS_E4M3) return false;
+    s.rows_f8 = c.row_format == FDKV_ROWS_E4M3;
+    if (s.rows_f8 && !(c.dtype == FDKV_BF16 && c.head_dim == 128 && B == 2 && G <= 4 && c.residual_rule == FDKV_RESIDUAL_ENTRIES && c.max_fold == 0))
+        return false;
     s.kfold_max = (int64_t)s.max_fold * s.d * s.keep_num / s.keep_den;
     s.kmax = (int64_t)s.Tmax * s.d * s.keep_num / s.keep_den;
     s.kcap = (int64_t)align_up((size_t)(s.kmax + kListPad), 64);
@@ -193,6 +197,7 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     if (e != cudaSuccess) { delete c; return cuda_fail(e); }
     if (s.dtype == FDKV_BF16 && s.d == 128) c->has_tmap = make_arena_tensor_map(c->arena, arena_bytes, c->tmap);
     c->packed_lists = c->has_tmap && s.max_batch * s.Hkv <= kFastMaxUnits;
+    if (s.rows_f8 && !(c->packed_lists && make_rows_tensor_map_u8(c->arena, arena_bytes, kRowPad, c->tmap_u8))) { delete c; return FDKV_ERR_UNSUPPORTED; }
     if (s.tok_rule) {
         const bool ok = c->packed_lists && make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
         if (!ok) { delete c; return FDKV_ERR_UNSUPPORTED; }
@@ -494,6 +499,9 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     const size_t val_b = c->packed_lists ? 0 : val_copy + (size_t)s.kfold_max * s.esize;
     const int64_t k_tok = (int64_t)T * s.keep_num / s.keep_den;
     const size_t trow_b = (size_t)(k_tok + 4) * s.d * s.esize, tlist_b = (size_t)(k_tok + 32) * 4;  // token rows, token list
+    // 8-bit row streams: 128 bytes per token and a 1 KiB slot for the channel scales (and their maxima) per stored tensor
+    const size_t rows8 = (size_t)T * 128, rows8_pad = (size_t)((T + kRowPad - 1) / kRowPad * kRowPad) * 128, scale_slot = 1024;
+    const size_t stream_b = s.rows_f8 ? align_up(rows8_pad) + scale_slot : align_up(rows_pad);  // one committed row stream
     size_t need = 0;
     // residual lists of one tensor: packed layout = one entry list per stored high-frequency tensor (one for a pair,
     // four for a block of four layers); portable layout = one index list and one value list per such tensor
@@ -501,9 +509,9 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u];
         if (m < 0 || m > 2) return FDKV_ERR_STATE;
-        if (m == FDKV_MODE_EXACT) need += 2 * (size_t)s.B * align_up(rows_pad);
+        if (m == FDKV_MODE_EXACT) need += 2 * (size_t)s.B * stream_b;
         else if (s.tok_rule) need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * align_up(trow_b) + align_up(tlist_b) + align_up(off_b) : 0);
-        else need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * (lists_b + align_up(off_b)) : 0);
+        else need += 2 * stream_b + (m == FDKV_MODE_RESIDUAL ? 2 * (lists_b + align_up(off_b)) : 0);
     }
     if (c->bump + need > c->arena_bytes) return FDKV_ERR_ARENA_FULL;
     size_t o = c->bump;
@@ -525,13 +533,23 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
             for (int l = 0; l < s.B; ++l)
                 for (int is_v = 0; is_v < 2; ++is_v) {
                     const void* src = is_v ? c->v_layers[s.B * p + l] : c->k_layers[s.B * p + l];
+                    const char* sp = (const char*)src + (size_t)h * c->stride_h * s.esize;
+                    if (s.rows_f8) {
+                        char* dst = take(rows8_pad);
+                        float* sc = reinterpret_cast<float*>(take(scale_slot));
+                        if (rows8_pad > rows8) CU(cudaMemsetAsync(dst + rows8, 0, rows8_pad - rows8, st));
+                        CU(launch_quantise_rows(sp, c->stride_t, T, reinterpret_cast<uint8_t*>(dst), sc, st));
+                        (is_v ? dl[l]->v_rows : dl[l]->k_rows) = dst;
+                        (is_v ? dl[l]->v_scale : dl[l]->k_scale) = sc;
+                        dl[l]->rows_f8 = 1;
+                        continue;
+                    }
                     char* dst = take(rows_pad);
                     if (rows_pad > rows) CU(cudaMemsetAsync(dst + rows, 0, rows_pad - rows, st));
-                    const char* sp = (const char*)src + (size_t)h * c->stride_h * s.esize;
                     CU(launch_strided_copy(sp, c->stride_t, dst, T, s.d, s.esize, st));
                     (is_v ? dl[l]->v_rows : dl[l]->k_rows) = dst;
                 }
-            by_mode[2] += 2 * (size_t)s.B * rows;
+            by_mode[2] += 2 * (size_t)s.B * (s.rows_f8 ? rows8 + 512 : rows);
         } else {
             char *tl = nullptr, *to = nullptr;
             if (s.tok_rule && m == FDKV_MODE_RESIDUAL) {  // one token list and one offset table serve K and V
@@ -543,11 +561,21 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
             }
             for (int is_v = 0; is_v < 2; ++is_v) {
                 const size_t ut = (size_t)u * 2 + is_v;
-                char* z0 = take(rows_pad);
-                if (rows_pad > rows) CU(cudaMemsetAsync(z0 + rows, 0, rows_pad - rows, st));
-                CU(cudaMemcpyAsync(z0, c->work + c->ws.z0 + ut * unit_stride_b, rows, cudaMemcpyDeviceToDevice, st));
+                float* sc8 = nullptr;
+                char* z0;
+                if (s.rows_f8) {
+                    z0 = take(rows8_pad);
+                    sc8 = reinterpret_cast<float*>(take(scale_slot));
+                    if (rows8_pad > rows8) CU(cudaMemsetAsync(z0 + rows8, 0, rows8_pad - rows8, st));
+                    CU(launch_quantise_rows(c->work + c->ws.z0 + ut * unit_stride_b, s.d, T, reinterpret_cast<uint8_t*>(z0), sc8, st));
+                    for (int l = 0; l < s.B; ++l) { (is_v ? dl[l]->v_scale : dl[l]->k_scale) = sc8; dl[l]->rows_f8 = 1; }
+                } else {
+                    z0 = take(rows_pad);
+                    if (rows_pad > rows) CU(cudaMemsetAsync(z0 + rows, 0, rows_pad - rows, st));
+                    CU(cudaMemcpyAsync(z0, c->work + c->ws.z0 + ut * unit_stride_b, rows, cudaMemcpyDeviceToDevice, st));
+                }
                 for (int l = 0; l < s.B; ++l) (is_v ? dl[l]->v_rows : dl[l]->k_rows) = z0;
-                by_mode[m] += rows;
+                by_mode[m] += s.rows_f8 ? rows8 + 512 : rows;
                 if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
                     char* rows_res = take(trow_b);
                     CU(launch_token_gather(c->work + c->ws.z1 + ut * unit_stride_b, (const int32_t*)tl, k_tok, rows_res, st));
@@ -572,7 +600,11 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                         const size_t lt = ut * s.NB + j;
                         if (c->packed_lists) {
                             pi_l[j] = take(idx_b);
-                            CU(cudaMemcpyAsync(pi_l[j], c->work + c->ws.packed + lt * s.kcap * 4, idx_copy, cudaMemcpyDeviceToDevice, st));
+                            if (s.rows_f8)  // values relative to the channel scales, positions in the converted fragments' order
+                                CU(launch_repack_entries_f8(reinterpret_cast<uint32_t*>(pi_l[j]), wsp<uint32_t>(c, c->ws.packed) + lt * s.kcap, k,
+                                                            sc8, is_v, st));
+                            else
+                                CU(cudaMemcpyAsync(pi_l[j], c->work + c->ws.packed + lt * s.kcap * 4, idx_copy, cudaMemcpyDeviceToDevice, st));
                         } else {
                             pi_l[j] = pi_shared;
                             pv_l[j] = take(val_b);
@@ -613,6 +645,7 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
         Tmax = c->seqs[b].T > Tmax ? c->seqs[b].T : Tmax;
     }
     if (k_new) {
+        if (s.rows_f8) return FDKV_ERR_UNSUPPORTED;  // 8-bit row streams: decode over the prompt only, for now
         for (int b = 0; b < batch; ++b)
             if (c->seqs[b].tail_len[layer] >= s.max_tail) return FDKV_ERR_STATE;
         for (int b = 0; b < batch; ++b) c->seqs[b].tail_len[layer]++;
@@ -626,6 +659,8 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
     a.tail_rows = s.tail_rows;
     a.host_T = host_T.data(); a.host_modes = host_modes.data();
     a.tmap = c->has_tmap ? c->tmap : nullptr;
+    a.tmap_u8 = s.rows_f8 ? c->tmap_u8 : nullptr;
+    a.rows_f8 = s.rows_f8;
     a.arena_base = c->arena;
     a.keep_num = s.keep_num; a.keep_den = s.keep_den;
     a.packed_lists = c->packed_lists ? 1 : 0;
@@ -713,7 +748,7 @@ fdkv_status fdkv_set_tail_len(fdkv_ctx* c, int32_t seq, int32_t n, void* stream)
 fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
     if (!seq_ok(c, seq) || n <= 0) return FDKV_ERR_INVALID_ARG;
     const Shape& s = c->s;
-    if (s.tok_rule) return FDKV_ERR_UNSUPPORTED;
+    if (s.tok_rule || s.rows_f8) return FDKV_ERR_UNSUPPORTED;
     SeqState& q = c->seqs[seq];
     if (!q.committed) return FDKV_ERR_STATE;
     if (c->staged_seq >= 0 && !c->seqs[c->staged_seq].committed) return FDKV_ERR_STATE;  // the staging area is in use
@@ -862,6 +897,18 @@ fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
     return FDKV_OK;
 }
 
+fdkv_status fdkv_get_rows_e4m3(fdkv_ctx* c, int32_t seq, int32_t layer, int32_t h, int32_t is_v, uint8_t* codes_out, float* scale_out,
+                               void* stream) {
+    if (!seq_ok(c, seq) || layer < 0 || layer >= c->s.L || h < 0 || h >= c->s.Hkv) return FDKV_ERR_INVALID_ARG;
+    if (!c->s.rows_f8) return FDKV_ERR_UNSUPPORTED;
+    if (!c->seqs[seq].committed) return FDKV_ERR_STATE;
+    const UnitDesc& d = c->desc_host[((size_t)seq * c->s.L + layer) * c->s.Hkv + h];
+    if (codes_out) CU(cudaMemcpyAsync(codes_out, is_v ? d.v_rows : d.k_rows, (size_t)d.T * 128, cudaMemcpyDeviceToDevice, S(stream)));
+    if (scale_out) CU(cudaMemcpyAsync(scale_out, is_v ? d.v_scale : d.k_scale, 512, cudaMemcpyDeviceToDevice, S(stream)));
+    CU(cudaStreamSynchronize(S(stream)));
+    return FDKV_OK;
+}
+
 fdkv_status fdkv_get_shared(fdkv_ctx* c, int32_t seq, int32_t pair, int32_t h, int32_t is_v, void* z0_out, void* stream) {
     if (!seq_ok(c, seq) || !z0_out || pair < 0 || pair >= c->s.P || h < 0 || h >= c->s.Hkv) return FDKV_ERR_INVALID_ARG;
     if (c->staged_seq != seq || !c->pair_compressed[pair]) return FDKV_ERR_STATE;
@@ -933,7 +980,8 @@ fdkv_status fdkv_decode_bytes(fdkv_ctx* c, int32_t layer, int32_t batch, size_t*
         const int ntiles = (q.T + kResTile - 1) / kResTile;
         for (int h = 0; h < s.Hkv; ++h) {
             const int m = q.modes[(layer / s.B) * s.Hkv + h];
-            tot += 2 * (size_t)(q.T + q.tail_len[layer]) * s.d * s.esize;
+            tot += s.rows_f8 ? 2 * ((size_t)q.T * s.d + 512) + 2 * (size_t)q.tail_len[layer] * s.d * s.esize
+                             : 2 * (size_t)(q.T + q.tail_len[layer]) * s.d * s.esize;
             if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
                 const size_t kt = (size_t)((int64_t)q.T * s.keep_num / s.keep_den);
                 tot += 2 * kt * s.d * s.esize + kt * 4 + (size_t)(ntiles + 1) * 4;

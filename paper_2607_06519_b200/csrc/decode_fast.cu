@@ -21,6 +21,7 @@
 // finish one unit and start the next; each (CTA, unit) segment writes one split-K partial and the CTA that takes
 // the unit's last ticket combines them.
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include <algorithm>
 #include <cstdio>
@@ -116,6 +117,29 @@ __device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {  // transpose an 8
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
 }
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// the two e4m3 bytes in the low half of x -> two f16 values (exact).  (An integer form - byte permute, shift, mask, with a
+// factor 2^-8 folded into the scales - was measured: 15 % slower alone, 9 % slower when sharing the work half and half.)
+__device__ __forceinline__ uint32_t cvt_e4m3x2(uint32_t x) {
+    uint32_t d;
+    asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, t;\n\t}" : "=r"(d) : "r"(x));
+    return d;
+}
+__device__ __forceinline__ uint32_t prmt1(uint32_t a, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(d) : "r"(a), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -165,8 +189,14 @@ __device__ unsigned g_phase[kMaxCtas][12];
 #define TADD(i, v)
 #endif
 
+// F8: the packed rows are e4m3 codes (one 128-byte row per token, per-channel float32 scales): the codes are converted
+// to f16 in registers after ldmatrix, both products run as f16 mma with the K scales folded into q and the V scales
+// applied to the output; the residual scratch tile then holds f16 values relative to the scales, in the converted
+// fragments' channel order (the commit step writes the lists that way).  No tails in this form.
+template <bool F8>
 __global__ void __launch_bounds__(kThreads, 1)
-decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastSched sch, PartCount pc) {
+decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap8, DecodeArgs a, FastSched sch,
+                   PartCount pc) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
 #ifdef FDKV_TIMING
     long long t_acc[2] = {0, 0};
@@ -221,11 +251,17 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
         const int s = it % kStages;
         const uint32_t full = smem0 + kOffFull + 8 * s;
         const uint32_t dst = stage0 + s * kStageBytes;
-        mbar_expect_tx(full, kStageBytes);
-        tma_load_2d(dst, &tmap, 0, kr, full);
-        tma_load_2d(dst + kHalfBytes, &tmap, 64, kr, full);
-        tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
-        tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
+        if constexpr (F8) {  // one 128-token x 128-byte box per tensor, in the first half of the K and of the V slot
+            mbar_expect_tx(full, 2 * kHalfBytes);
+            tma_load_2d(dst, &tmap8, 0, kr, full);
+            tma_load_2d(dst + 2 * kHalfBytes, &tmap8, 0, vr, full);
+        } else {
+            mbar_expect_tx(full, kStageBytes);
+            tma_load_2d(dst, &tmap, 0, kr, full);
+            tma_load_2d(dst + kHalfBytes, &tmap, 64, kr, full);
+            tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
+            tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
+        }
     };
     // a warp is done reading stage s (tile it): the last of the eight refills it
     auto release_stage = [&](int s, int it) {
@@ -251,8 +287,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             if (te <= tb) continue;
             if (n == kMaxSeg) { atomicMax(a.status, (int32_t)kFlagCountMismatch); break; }  // cannot happen: see the launcher
             Seg g;
-            g.krow = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> 8);
-            g.vrow = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> 8);
+            g.krow = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> (F8 ? 7 : 8));  // rows of 128 or 256 bytes
+            g.vrow = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> (F8 ? 7 : 8));
             g.tkrow = g.tvrow = 0;
             g.tb = tb;
             g.npre = te - tb;
@@ -281,7 +317,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
         for (int i = 0; i < seg_info[0]; ++i) {
             Seg g = segs[i];
             g.it0 = it0;
-            if (g.tail_b >= 0) {
+            if (!F8 && g.tail_b >= 0) {
                 const int n = min(a.tail_len[a.layer * a.max_batch + g.tail_b], a.max_tail);
                 const int64_t o = (((int64_t)a.layer * a.max_batch + g.tail_b) * a.Hkv + g.tail_h) * a.tail_rows;
                 g.tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
@@ -317,7 +353,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
             const int te = u == u_last ? t_last : ntiles;
             if (te <= tb) continue;
             int ntail = 0, n_tail_rows = 0;
-            if (te == ntiles) {
+            if (!F8 && te == ntiles) {
                 n_tail_rows = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
                 ntail = (n_tail_rows + kTT - 1) / kTT;
             }
@@ -335,8 +371,19 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.Hq + h * a.G + qcol) * 128;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    qb[kk][0] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 2 * tig) : 0u;
-                    qb[kk][1] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 8 + 2 * tig) : 0u;
+                    if constexpr (F8) {
+                        // a converted register holds channels 4 tig .. 4 tig + 3 of the 16-channel step: its low pair is the
+                        // first k-slot pair, its high pair the second; q carries the K scales, as f16
+                        const int c0 = 16 * kk + 4 * tig;
+                        float qv[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) qv[i] = qcol < a.G ? __bfloat162float(qh[c0 + i]) * ud.k_scale[c0 + i] : 0.f;
+                        qb[kk][0] = pack_f16(qv[0], qv[1]);
+                        qb[kk][1] = pack_f16(qv[2], qv[3]);
+                    } else {
+                        qb[kk][0] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 2 * tig) : 0u;
+                        qb[kk][1] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 8 + 2 * tig) : 0u;
+                    }
                 }
             }
             // O^T[channel][column]: eight 16-channel m-tiles; this thread holds columns 2 tig, 2 tig + 1
@@ -514,7 +561,38 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 {
                     const int mi = lane >> 3, rr = lane & 7;
                     const int row = r0 + (mi & 1) * 8 + rr;  // ldmatrix: matrices = (tokens 0-7 | 8-15) x (chunk | chunk + 1)
-                    if (with_res && cr[1] > cr[0]) {
+                    if constexpr (F8) {
+                        // one ldmatrix.x4 covers 32 channels of the slice's 16 tokens: (tokens 0-7 | 8-15) x two 16-byte chunks
+                        const bool res_k = with_res && cr[1] > cr[0];
+                        float racc[4] = {0.f, 0.f, 0.f, 0.f};
+                        const int srow = (mi & 1) * 8 + rr;
+#pragma unroll
+                        for (int k2 = 0; k2 < 4; ++k2) {
+                            uint32_t x0, x1, x2, x3;
+                            ldsm_x4(kb + swz(row, 2 * k2 + (mi >> 1)), x0, x1, x2, x3);
+                            // a register = channels 4 tig .. 4 tig + 3 of a token: bytes (0, 1) feed the first k-slot pair, (2, 3) the second
+                            mma_f16(sacc[0], cvt_e4m3x2(x0), cvt_e4m3x2(x1), cvt_e4m3x2(x0 >> 16), cvt_e4m3x2(x1 >> 16), qb[2 * k2][0],
+                                    qb[2 * k2][1]);
+                            mma_f16(sacc[1], cvt_e4m3x2(x2), cvt_e4m3x2(x3), cvt_e4m3x2(x2 >> 16), cvt_e4m3x2(x3 >> 16), qb[2 * k2 + 1][0],
+                                    qb[2 * k2 + 1][1]);
+                            if (res_k) {
+#pragma unroll
+                                for (int kk = 2 * k2; kk < 2 * k2 + 2; ++kk) {
+                                    const int c = 2 * kk + (mi >> 1);
+                                    uint32_t e0, e1, e2, e3;
+                                    ldsm_x4(scratch + (c >> 3) * 2048 + swz(srow, c), e0, e1, e2, e3);
+                                    mma_f16(racc, e0, e1, e2, e3, qb[kk][0] ^ sgn, qb[kk][1] ^ sgn);
+                                }
+                            }
+                        }
+                        if (res_k) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) sacc[0][i] += racc[i];
+                            __syncwarp();
+                            zero_scratch();
+                            __syncwarp();
+                        }
+                    } else if (with_res && cr[1] > cr[0]) {
                         float racc[4] = {0.f, 0.f, 0.f, 0.f};  // the residual's own chain, interleaved with the two main ones
                         const int srow = (mi & 1) * 8 + rr;
 #pragma unroll
@@ -603,10 +681,10 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             const float pv_ = p[hh][e] * vscale;
-                            const float hi = __bfloat162float(__float2bfloat16_rn(pv_));
+                            const float hi = F8 ? __half2float(__float2half_rn(pv_)) : __bfloat162float(__float2bfloat16_rn(pv_));
                             v[e] = lo_part ? pv_ - hi : hi;
                         }
-                        pb[hh] = movmatrix_t(pack_bf16(v[0], v[1]));
+                        pb[hh] = movmatrix_t(F8 ? pack_f16(v[0], v[1]) : pack_bf16(v[0], v[1]));
                     }
                 }
                 TPH(5);
@@ -614,13 +692,28 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                 {
                     const int mi = lane >> 3, rr = lane & 7;
                     const int row = r0 + (mi >> 1) * 8 + rr;  // ldmatrix.trans: matrices = (chunk | chunk + 1) x (tokens 0-7 | 8-15)
-                    if (sch.experiment != 2)  // (timing experiment 2 skips this product)
+                    if constexpr (F8) {
+                        // A transposed 8 x 8 tile of 2-byte units gives this thread channels (2 gid, 2 gid + 1) of tokens
+                        // (2 tig, 2 tig + 1) as bytes (c0 t0, c1 t0, c0 t1, c1 t1): a byte permute puts one channel's token pair
+                        // in each half; the two channels become rows gid and gid + 8 of the m-tile (the merge writes them back
+                        // to their channels).
+                        const int row8 = r0 + (mi & 1) * 8 + rr;  // matrices = (tokens 0-7 | 8-15) x two 16-byte chunks
 #pragma unroll
-                    for (int jm = 0; jm < 8; ++jm) {
-                        const int c = 2 * jm + (mi & 1);
-                        uint32_t a0, a1, a2, a3;
-                        ldsm_x4_t(vb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
-                        mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0], pb[1]);
+                        for (int p2 = 0; p2 < 4; ++p2) {
+                            uint32_t x0, x1, x2, x3;
+                            ldsm_x4_t(vb + swz(row8, 2 * p2 + (mi >> 1)), x0, x1, x2, x3);
+                            x0 = prmt1(x0, 0x3120u); x1 = prmt1(x1, 0x3120u); x2 = prmt1(x2, 0x3120u); x3 = prmt1(x3, 0x3120u);
+                            mma_f16(oacc[2 * p2], cvt_e4m3x2(x0), cvt_e4m3x2(x0 >> 16), cvt_e4m3x2(x1), cvt_e4m3x2(x1 >> 16), pb[0], pb[1]);
+                            mma_f16(oacc[2 * p2 + 1], cvt_e4m3x2(x2), cvt_e4m3x2(x2 >> 16), cvt_e4m3x2(x3), cvt_e4m3x2(x3 >> 16), pb[0], pb[1]);
+                        }
+                    } else if (sch.experiment != 2) {  // (timing experiment 2 skips this product)
+#pragma unroll
+                        for (int jm = 0; jm < 8; ++jm) {
+                            const int c = 2 * jm + (mi & 1);
+                            uint32_t a0, a1, a2, a3;
+                            ldsm_x4_t(vb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
+                            mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0], pb[1]);
+                        }
                     }
                     TPH(6);
                     if (with_res && cr[3] > cr[2]) {
@@ -630,7 +723,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                             const int c = 2 * jm + (mi & 1);
                             uint32_t a0, a1, a2, a3;
                             ldsm_x4_t(scratch + (c >> 3) * 2048 + swz(srow, c), a0, a1, a2, a3);
-                            mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0] ^ sgn, pb[1] ^ sgn);
+                            if constexpr (F8) mma_f16(oacc[jm], a0, a1, a2, a3, pb[0] ^ sgn, pb[1] ^ sgn);
+                            else mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0] ^ sgn, pb[1] ^ sgn);
                         }
                         __syncwarp();
                         zero_scratch();
@@ -679,11 +773,14 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, DecodeArgs a, FastS
                         if (split) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
                     }
                     if (!split || tig < 2) {
-                        const int ch = 16 * jm + gid, col = 2 * tig;
-                        scratch_f[col * 128 + ch] = v[0];
-                        scratch_f[(col + 1) * 128 + ch] = v[1];
-                        scratch_f[col * 128 + ch + 8] = v[2];
-                        scratch_f[(col + 1) * 128 + ch + 8] = v[3];
+                        // rows gid / gid + 8 of the m-tile: channels gid and gid + 8, or (8-bit rows) 2 gid and 2 gid + 1,
+                        // whose codes are still to be multiplied by the channel's V scale
+                        const int ch_a = F8 ? 16 * jm + 2 * gid : 16 * jm + gid, ch_b = F8 ? ch_a + 1 : ch_a + 8, col = 2 * tig;
+                        const float sa = F8 ? ud.v_scale[ch_a] : 1.f, sb = F8 ? ud.v_scale[ch_b] : 1.f;
+                        scratch_f[col * 128 + ch_a] = v[0] * sa;
+                        scratch_f[(col + 1) * 128 + ch_a] = v[1] * sa;
+                        scratch_f[col * 128 + ch_b] = v[2] * sb;
+                        scratch_f[(col + 1) * 128 + ch_b] = v[3] * sb;
                     }
                 }
                 __syncthreads();
@@ -832,6 +929,30 @@ bool make_rows_tensor_map(void* base, size_t bytes, int box_rows, void* tmap_out
     return r == CUDA_SUCCESS;
 }
 
+// The same region viewed as rows of 128 bytes (8-bit row streams): one 128-byte x box_rows box per copy, 128-byte swizzle.
+bool make_rows_tensor_map_u8(void* base, size_t bytes, int box_rows, void* tmap_out) {
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    const cuuint64_t rows = bytes / 128;
+    if (rows == 0 || rows > 0x7FFFFFFFull || box_rows < 1 || box_rows > 256) return false;
+    const cuuint64_t gdim[2] = {128, rows};
+    const cuuint64_t gstride[1] = {128};
+    const cuuint32_t box[2] = {128, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<encode_fn>(fn)(reinterpret_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, gdim,
+                                                 gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
     return make_rows_tensor_map(arena, arena_bytes, kTT, tmap_out);
 }
@@ -840,13 +961,15 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     *handled = false;
     const int units = a.batch * a.Hkv;
     if (!a.tmap || !a.packed_lists || a.d != 128 || units > kMaxUnits || units < 1) return cudaSuccess;
+    if (a.rows_f8 && !a.tmap_u8) return cudaSuccess;
     static int sm_count = 0;
     static bool attr_done = false;
     if (!attr_done) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -968,7 +1091,10 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = use_pdl ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_fast_kernel, *reinterpret_cast<const CUtensorMap*>(a.tmap), a, sch, cs);
+    const CUtensorMap& m16 = *reinterpret_cast<const CUtensorMap*>(a.tmap);
+    const CUtensorMap& m8 = *reinterpret_cast<const CUtensorMap*>(a.rows_f8 ? a.tmap_u8 : a.tmap);
+    cudaError_t e = a.rows_f8 ? cudaLaunchKernelEx(&cfg, decode_fast_kernel<true>, m16, m8, a, sch, cs)
+                              : cudaLaunchKernelEx(&cfg, decode_fast_kernel<false>, m16, m8, a, sch, cs);
     if (e != cudaSuccess) return e;
     count_launch(1);
     *handled = true;

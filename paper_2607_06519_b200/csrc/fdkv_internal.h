@@ -47,7 +47,9 @@ struct UnitDesc {
                  // 2 for a layer of a four-layer block (rows scaled by 1/2, deviations by 1)
     int32_t res_kind;  // residual layout: 0 packed entries (k_idx / v_idx), 1 token rows (k_idx = token list, k_val / v_val = rows, k_off = per-slice counts)
     float scale;       // what the stored rows are multiplied by: 1/sqrt 2 (pair coefficients), 1/2 (block of four), 1 (exact)
-    int32_t pad_;
+    int32_t rows_f8;   // 1: k_rows / v_rows hold e4m3 codes (128 bytes per token) with per-channel scales below
+    const float* k_scale;  // [d] float32, rows_f8 only
+    const float* v_scale;
 };
 
 struct SelState {
@@ -71,6 +73,7 @@ struct Shape {
     int tok_rule;      // 1: token-granular residual chosen by the probe
     int B;             // layers per depth block: 2 or 4
     int max_fold;      // generated tokens that may be folded into the compressed form per sequence
+    int rows_f8;       // committed row streams are e4m3 codes with per-channel scales
     int64_t kfold_max; // floor(max_fold*d*num/den): list room reserved for them
     int NB;            // staged high-frequency tensors per unit-tensor: 1 (Z1 of a pair) or 4 (the layers' deviations)
     int64_t ktok_max, ktok_cap;  // floor(Tmax*num/den) and the list capacity incl. slack
@@ -123,6 +126,7 @@ struct fdkv_ctx {
     alignas(64) unsigned char tmap_z1_128[128];  // staged Z1 with 128-token boxes (token-score kernel)
     std::vector<uint8_t> pair_scored;            // token rule: the probe has chosen this pair's token sets
     bool packed_lists = false;              // decode runs the bf16 / head_dim 128 kernel on packed residual entries
+    alignas(64) unsigned char tmap_u8[128]; // CUtensorMap of the arena as 128-byte rows (8-bit row streams)
 };
 
 namespace fdkv {
@@ -227,6 +231,8 @@ struct DecodeArgs {
     const int32_t* host_T;      // [batch]
     const int32_t* host_modes;  // [batch][Hkv] modes of this layer's pair
     const void* tmap;           // CUtensorMap over the arena as rows of 256 bytes, or null
+    const void* tmap_u8;        // the same arena as rows of 128 bytes (8-bit row streams), or null
+    int rows_f8;
     const void* arena_base;
     int keep_num, keep_den;
     int packed_lists;
@@ -241,6 +247,14 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st);
 bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out);
 // Same view ([rows][128] bf16, 64-channel x box_rows boxes, 128-byte swizzle) over any 256-byte aligned region.
 bool make_rows_tensor_map(void* base, size_t bytes, int box_rows, void* tmap_out);
+// ---- 8-bit row streams (rows_fp8.cu) ----
+// codes[t][c] = e4m3(src[t*stride_t + c] / scale[c]), scale[c] = max_t |src| / 448 (1 if zero); src bf16, d = 128
+cudaError_t launch_quantise_rows(const void* src, int64_t stride_t, int T, uint8_t* codes, float* scale, cudaStream_t st);
+// packed residual entries for a unit whose rows are 8-bit: value -> f16(value / scale[channel]), position permuted inside
+// its 16-channel group to the order the kernel's converted fragments use (K and V differ)
+cudaError_t launch_repack_entries_f8(uint32_t* dst, const uint32_t* src, int64_t n, const float* scale, int is_v, cudaStream_t st);
+bool make_rows_tensor_map_u8(void* base, size_t bytes, int box_rows, void* tmap_out);
+
 // dst[i] = src[i] + add, i < n (list offsets and indices of a folded chunk)
 cudaError_t launch_offset_copy(int32_t* dst, const int32_t* src, int n, int add, cudaStream_t st);
 cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, int T, int d, int esize, cudaStream_t st);

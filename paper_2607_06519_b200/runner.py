@@ -18,10 +18,10 @@ def to_device(x: np.ndarray, dtype: str, device) -> torch.Tensor:
 
 
 def make_context(w: synth.Workload, max_tail: int | None = None, arena_bytes: int | None = None,
-                 device="cuda:0", max_fold: int = 0) -> B.Context:
+                 device="cuda:0", max_fold: int = 0, row_format: int = 0) -> B.Context:
     cfg = B.Config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, w.T,
                    max_tail if max_tail is not None else max(w.n_steps, 1), B.BF16 if w.dtype == "bf16" else B.F32,
-                   w.keep_num, w.keep_den, w.residual_rule, w.block_size, max_fold)
+                   w.keep_num, w.keep_den, w.residual_rule, w.block_size, max_fold, row_format or w.row_format)
     return B.Context(cfg, device=device, arena_bytes=arena_bytes)
 
 
@@ -29,10 +29,10 @@ class Prefilled:
     """One workload with every sequence compressed, routed and committed."""
 
     def __init__(self, w: synth.Workload, ctx: B.Context | None = None, max_tail: int | None = None,
-                 arena_bytes: int | None = None, device="cuda:0", max_fold: int = 0):
+                 arena_bytes: int | None = None, device="cuda:0", max_fold: int = 0, row_format: int = 0):
         self.w = w
         self.device = torch.device(device)
-        self.ctx = ctx or make_context(w, max_tail, arena_bytes, device, max_fold)
+        self.ctx = ctx or make_context(w, max_tail, arena_bytes, device, max_fold, row_format)
         self.scores = {}
         self.probe_modes = {}
         self._inputs = {}  # the library reads exact-mode rows at commit: keep the uploads alive until then

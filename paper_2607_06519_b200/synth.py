@@ -49,6 +49,7 @@ class Workload:
     seq_seeds: tuple | None = None  # per-sequence seed override (batched workload)
     residual_rule: int = 0  # 0: largest-magnitude entries; 1: probe-scored tokens (the paper's rule)
     block_size: int = 2  # layers per depth block (2 or 4)
+    row_format: int = 0  # 0: committed rows in the storage type; 1: 8-bit rows with per-channel scales
 
     @property
     def n_pairs(self) -> int:
@@ -106,6 +107,10 @@ WORKLOADS["decode128k_4l"] = WORKLOADS["decode128k"].scaled(n_layers=4, name="de
 WORKLOADS["decode32k_tok"] = WORKLOADS["decode32k"].scaled(residual_rule=1, name="decode32k_tok")
 WORKLOADS["decode32k_tok_4l"] = WORKLOADS["decode32k_tok"].scaled(n_layers=4, name="decode32k_tok_4l")
 # depth blocks of four layers (the paper's default block size): tiny correctness case and the 32k shape
+# the 32k workload with the committed rows stored as 8-bit floats
+WORKLOADS["decode32k_fp8"] = WORKLOADS["decode32k"].scaled(row_format=1, name="decode32k_fp8")
+WORKLOADS["decode32k_fp8_4l"] = WORKLOADS["decode32k_fp8"].scaled(n_layers=4, name="decode32k_fp8_4l")
+WORKLOADS["decode128k_fp8"] = WORKLOADS["decode128k"].scaled(row_format=1, name="decode128k_fp8")
 WORKLOADS["tiny_b4"] = WORKLOADS["tiny"].scaled(n_layers=4, block_size=4, name="tiny_b4")
 WORKLOADS["decode32k_b4"] = WORKLOADS["decode32k"].scaled(block_size=4, name="decode32k_b4")
 WORKLOADS["decode32k_b4_8l"] = WORKLOADS["decode32k"].scaled(n_layers=8, block_size=4, name="decode32k_b4_8l")

@@ -1,0 +1,92 @@
+"""GPU parity for 8-bit row streams (row_format = e4m3): the committed codes and per-channel scales are bit-exact against
+the oracle's quantiser; decode attention over them (f16 tensor-core products on converted fragments, scales folded
+into q and applied to the output) matches the oracle's attention over the dequantised rows within the bf16 tolerance."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import TOL, f32, vector_errors
+from oracle import fdkv_ref_fp8 as R8
+from paper_2607_06519_b200 import binding as B
+from paper_2607_06519_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _unit8(w, p, h):
+    k0, k1 = synth.unit_tensor(w, 0, p, h, False)
+    v0, v1 = synth.unit_tensor(w, 0, p, h, True)
+    return R8.UnitFp8(k0, k1, v0, v1, True, w.keep_num, w.keep_den)
+
+
+@pytest.mark.parametrize("T,Hq,Hkv,keep", [(1300, 8, 2, (1, 16)), (2100, 4, 1, (1, 32)), (300, 2, 2, (1, 8))])
+def test_rows_e4m3_parity(T, Hq, Hkv, keep):
+    from paper_2607_06519_b200 import runner
+
+    w = synth.Workload(name="f8", n_layers=4, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=128, batch=1, T=T, dtype="bf16",
+                       keep_num=keep[0], keep_den=keep[1], n_needles=4, W=8, seed=51, n_steps=1, row_format=1)
+    pf = runner.Prefilled(w, max_tail=1)
+    modes = np.array([[(p + h) % 3 for h in range(Hkv)] for p in range(2)], dtype=np.int32)
+    pf.prefill(0, modes=modes)
+    units = {(p, h): _unit8(w, p, h) for p in range(2) for h in range(Hkv)}
+    # stored codes and scales
+    for (p, h), u in units.items():
+        for layer in (2 * p, 2 * p + 1):
+            for is_v, name in ((0, "k"), (1, "v")):
+                codes, scale = pf.ctx.get_rows_e4m3(0, layer, h, is_v, T)
+                want_c, want_s = u.q_x[name][layer & 1] if modes[p][h] == 2 else u.q_z0[name]
+                assert np.array_equal(scale.cpu().numpy(), want_s), (p, h, layer, name)
+                assert np.array_equal(codes.cpu().numpy(), want_c), (p, h, layer, name)
+    # decode
+    G = w.group
+    worst = 0.0
+    for layer in range(4):
+        q = pf.decode_q(layer, 0)
+        out = f32(pf.ctx.decode_attn(layer, q, out_dtype=0))[0]
+        torch.cuda.synchronize()
+        for h in range(Hkv):
+            ref = units[(layer // 2, h)].attend(int(modes[layer // 2][h]), layer & 1, f32(q)[0][h * G:(h + 1) * G])
+            worst = max(worst, float(vector_errors(out[h * G:(h + 1) * G], ref).max()))
+    assert worst <= TOL["bf16"], worst
+    # appends are closed for this format
+    kn, vn = pf.new_rows(0, 0)
+    with pytest.raises(B.FdkvError):
+        pf.ctx.decode_attn(0, pf.decode_q(0, 0), kn, vn)
+    by_mode, exact_equiv = pf.ctx.footprint(0)
+    assert pf.ctx.decode_bytes(0, 1) < 0.62 * sum(2 * T * 128 * 2 for _ in range(Hkv)) + 64 * 1024 * Hkv
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
+
+
+def test_rows_e4m3_benchmark_workload_sampled():
+    """decode32k_fp8 (the 32k workload with 8-bit rows, quota mode mix) through the calls bench.py times: sampled units'
+    codes and scales bit-exact, one decode step of all layers within tolerance on those units."""
+    from paper_2607_06519_b200 import runner
+
+    w = synth.WORKLOADS["decode32k_fp8"]
+    sample = [(0, 1), (9, 4), (15, 7)]
+    pf = runner.Prefilled(w, max_tail=1)
+    modes = pf.prefill(0)
+    units = {(p, h): _unit8(w, p, h) for (p, h) in sample}
+    for (p, h), u in units.items():
+        codes, scale = pf.ctx.get_rows_e4m3(0, 2 * p + 1, h, 0, w.T)
+        want_c, want_s = u.q_x["k"][1] if modes[p][h] == 2 else u.q_z0["k"]
+        assert np.array_equal(scale.cpu().numpy(), want_s) and np.array_equal(codes.cpu().numpy(), want_c)
+    torch.cuda.empty_cache()
+    G = w.group
+    worst = 0.0
+    for layer in range(w.n_layers):
+        q = pf.decode_q(layer, 0)
+        out = pf.ctx.decode_attn(layer, q)
+        torch.cuda.synchronize()
+        assert torch.isfinite(out.float()).all()
+        for (p, h), u in units.items():
+            if p != layer // 2:
+                continue
+            ref = u.attend(int(modes[p][h]), layer & 1, f32(q)[0][h * G:(h + 1) * G])
+            worst = max(worst, float(vector_errors(f32(out)[0][h * G:(h + 1) * G], ref).max()))
+    assert worst <= TOL["bf16"], worst
+    by_mode, exact_equiv = pf.ctx.footprint(0)
+    assert pf.ctx.decode_bytes(0, 1) < 0.56 * 8 * 2 * w.T * 128 * 2
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
