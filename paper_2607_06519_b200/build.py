@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfdkv.so")
 SOURCES = ["api.cu", "compress.cu", "block4.cu", "rows_fp8.cu", "probe.cu", "probe_tc.cu", "token_rule.cu", "decode.cu", "decode_fast.cu"]
-HEADERS = ["fdkv_internal.h", os.path.join("..", "..", "include", "fdkv.h")]
+HEADERS = ["fdkv_internal.h", "decode_fast_tile.inc", os.path.join("..", "..", "include", "fdkv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false", "-Xptxas", "-v"]
 

@@ -645,7 +645,6 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
         Tmax = c->seqs[b].T > Tmax ? c->seqs[b].T : Tmax;
     }
     if (k_new) {
-        if (s.rows_f8) return FDKV_ERR_UNSUPPORTED;  // 8-bit row streams: decode over the prompt only, for now
         for (int b = 0; b < batch; ++b)
             if (c->seqs[b].tail_len[layer] >= s.max_tail) return FDKV_ERR_STATE;
         for (int b = 0; b < batch; ++b) c->seqs[b].tail_len[layer]++;

@@ -192,7 +192,9 @@ __device__ unsigned g_phase[kMaxCtas][12];
 // F8: the packed rows are e4m3 codes (one 128-byte row per token, per-channel float32 scales): the codes are converted
 // to f16 in registers after ldmatrix, both products run as f16 mma with the K scales folded into q and the V scales
 // applied to the output; the residual scratch tile then holds f16 values relative to the scales, in the converted
-// fragments' channel order (the commit step writes the lists that way).  No tails in this form.
+// fragments' channel order (the commit step writes the lists that way).  The generated-token tails stay bf16: when a
+// segment reaches them the warp stashes the softmax state of its 8-bit tiles, runs the tails with the plain bf16 code
+// on a fresh state and joins the two at the merge.
 template <bool F8>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap8, DecodeArgs a, FastSched sch,
@@ -251,7 +253,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         const int s = it % kStages;
         const uint32_t full = smem0 + kOffFull + 8 * s;
         const uint32_t dst = stage0 + s * kStageBytes;
-        if constexpr (F8) {  // one 128-token x 128-byte box per tensor, in the first half of the K and of the V slot
+        if (F8 && j < g.npre) {  // one 128-token x 128-byte box per tensor, in the first half of the K and of the V slot
             mbar_expect_tx(full, 2 * kHalfBytes);
             tma_load_2d(dst, &tmap8, 0, kr, full);
             tma_load_2d(dst + 2 * kHalfBytes, &tmap8, 0, vr, full);
@@ -317,7 +319,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         for (int i = 0; i < seg_info[0]; ++i) {
             Seg g = segs[i];
             g.it0 = it0;
-            if (!F8 && g.tail_b >= 0) {
+            if (g.tail_b >= 0) {
                 const int n = min(a.tail_len[a.layer * a.max_batch + g.tail_b], a.max_tail);
                 const int64_t o = (((int64_t)a.layer * a.max_batch + g.tail_b) * a.Hkv + g.tail_h) * a.tail_rows;
                 g.tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
@@ -353,7 +355,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             const int te = u == u_last ? t_last : ntiles;
             if (te <= tb) continue;
             int ntail = 0, n_tail_rows = 0;
-            if (!F8 && te == ntiles) {
+            if (te == ntiles) {
                 n_tail_rows = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
                 ntail = (n_tail_rows + kTT - 1) / kTT;
             }
@@ -367,11 +369,11 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             const bool split = a.G <= 4;
             const int qcol = split ? (gid & 3) : gid;
             uint32_t qb[8][2];
-            {
+            auto load_q = [&](bool f8) {
                 const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.Hq + h * a.G + qcol) * 128;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    if constexpr (F8) {
+                    if (F8 && f8) {
                         // a converted register holds channels 4 tig .. 4 tig + 3 of the 16-channel step: its low pair is the
                         // first k-slot pair, its high pair the second; q carries the K scales, as f16
                         const int c0 = 16 * kk + 4 * tig;
@@ -385,12 +387,15 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                         qb[kk][1] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 8 + 2 * tig) : 0u;
                     }
                 }
-            }
+            };
+            load_q(true);
             // O^T[channel][column]: eight 16-channel m-tiles; this thread holds columns 2 tig, 2 tig + 1
             float oacc[8][4];
 #pragma unroll
             for (int j = 0; j < 8; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
             float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};  // per held column; l is this thread's share
+            float m_st[2] = {-INFINITY, -INFINITY}, l_st[2] = {0.f, 0.f};     // 8-bit rows: the state stashed before the bf16 tails
+            bool stashed = false;
             // split-K part slot of this segment = number of CTAs with tiles of this unit before this one
             int slot = 0;
             for (int c2 = cta - 1; c2 >= 0; --c2) {
@@ -516,237 +521,42 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                 }
             }
 
-            for (int j = 0; j < nseg; ++j) {
-                const int itj = it + j;
-                const int s = itj % kStages;
-                const uint32_t ph = (uint32_t)(itj / kStages) & 1u;
-                const bool is_tail = j >= npre;
-                const int tile = is_tail ? j - npre : (rev ? tb + npre - 1 - j : tb + j);
-                const int rows_valid = is_tail ? n_tail_rows - tile * kTT : T - tile * kTT;  // may exceed the stage
-                const bool with_res = resid && !is_tail;
-                const float kscale = ((coef && !is_tail) ? ud.scale : 1.f) * inv_sqrt_d * kLog2e;
-                const float vscale = (coef && !is_tail) ? ud.scale : 1.f;
-#ifdef FDKV_TIMING
-                t_mark = (unsigned)clock();
-#endif
-
-                if (with_res && cr[1] > cr[0]) {
-                    if (tokmode) scatter_tok(t_krows, cr[0], cr[1], pke, ptk);
-                    else scatter(k_ent, cr[0], cr[1], pke);
-                    __syncwarp();
-                }
-                if (tokmode) prefetch_tok(t_krows, nr[0], nr[1], pke, ptk);
-                else if (resid) prefetch(k_ent, nr[0], nr[1], pke);
-
-                TPH(0);
-#ifdef FDKV_TIMING
-                const long long tw0 = clock64();
-#endif
-                wait_bar(smem0 + kOffFull + 8 * s, ph, abort_flag, a.status);
-                TPH(1);
-#ifdef FDKV_TIMING
-                TADD(4, clock64() - tw0);
-                TADD(5, 1);
-#endif
-                const uint32_t kb = stage0 + s * kStageBytes, vb = kb + 2 * kHalfBytes;
-                if (sch.experiment == 1) {  // timing experiment only: stream the tiles, compute nothing
-                    release_stage(s, itj);
-                    continue;
-                }
-
-                // ---- S[token][column] = k . q over 128 channels: one 16 x 8 tile, two accumulator chains ----
-                float sacc[2][4];
+            // O[head][channel] into the warp's float scratch: column g plus (G <= 4) its remainder column g + 4, held by the
+            // lane two over.  Rows gid / gid + 8 of an m-tile are channels gid and gid + 8, or (8-bit tiles) 2 gid and
+            // 2 gid + 1, whose code sums are still to be multiplied by the channel's V scale.
+            auto store_o = [&](bool f8_layout, bool accumulate, float f0, float f1) {
 #pragma unroll
-                for (int i = 0; i < 2; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
-                {
-                    const int mi = lane >> 3, rr = lane & 7;
-                    const int row = r0 + (mi & 1) * 8 + rr;  // ldmatrix: matrices = (tokens 0-7 | 8-15) x (chunk | chunk + 1)
-                    if constexpr (F8) {
-                        // one ldmatrix.x4 covers 32 channels of the slice's 16 tokens: (tokens 0-7 | 8-15) x two 16-byte chunks
-                        const bool res_k = with_res && cr[1] > cr[0];
-                        float racc[4] = {0.f, 0.f, 0.f, 0.f};
-                        const int srow = (mi & 1) * 8 + rr;
+                for (int jm = 0; jm < 8; ++jm) {
+                    float v[4];
 #pragma unroll
-                        for (int k2 = 0; k2 < 4; ++k2) {
-                            uint32_t x0, x1, x2, x3;
-                            ldsm_x4(kb + swz(row, 2 * k2 + (mi >> 1)), x0, x1, x2, x3);
-                            // a register = channels 4 tig .. 4 tig + 3 of a token: bytes (0, 1) feed the first k-slot pair, (2, 3) the second
-                            mma_f16(sacc[0], cvt_e4m3x2(x0), cvt_e4m3x2(x1), cvt_e4m3x2(x0 >> 16), cvt_e4m3x2(x1 >> 16), qb[2 * k2][0],
-                                    qb[2 * k2][1]);
-                            mma_f16(sacc[1], cvt_e4m3x2(x2), cvt_e4m3x2(x3), cvt_e4m3x2(x2 >> 16), cvt_e4m3x2(x3 >> 16), qb[2 * k2 + 1][0],
-                                    qb[2 * k2 + 1][1]);
-                            if (res_k) {
-#pragma unroll
-                                for (int kk = 2 * k2; kk < 2 * k2 + 2; ++kk) {
-                                    const int c = 2 * kk + (mi >> 1);
-                                    uint32_t e0, e1, e2, e3;
-                                    ldsm_x4(scratch + (c >> 3) * 2048 + swz(srow, c), e0, e1, e2, e3);
-                                    mma_f16(racc, e0, e1, e2, e3, qb[kk][0] ^ sgn, qb[kk][1] ^ sgn);
-                                }
-                            }
-                        }
-                        if (res_k) {
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) sacc[0][i] += racc[i];
-                            __syncwarp();
-                            zero_scratch();
-                            __syncwarp();
-                        }
-                    } else if (with_res && cr[1] > cr[0]) {
-                        float racc[4] = {0.f, 0.f, 0.f, 0.f};  // the residual's own chain, interleaved with the two main ones
-                        const int srow = (mi & 1) * 8 + rr;
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const int c = 2 * kk + (mi >> 1);
-                            uint32_t a0, a1, a2, a3, e0, e1, e2, e3;
-                            ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
-                            ldsm_x4(scratch + (c >> 3) * 2048 + swz(srow, c), e0, e1, e2, e3);
-                            mma_bf16(sacc[kk & 1], a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
-                            mma_bf16(racc, e0, e1, e2, e3, qb[kk][0] ^ sgn, qb[kk][1] ^ sgn);
-                        }
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) sacc[0][i] += racc[i];
-                        __syncwarp();
-                        zero_scratch();
-                        __syncwarp();
-                    } else if (sch.experiment != 3) {  // (timing experiment 3 skips this product)
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const int c = 2 * kk + (mi >> 1);
-                            uint32_t a0, a1, a2, a3;
-                            ldsm_x4(kb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
-                            mma_bf16(sacc[kk & 1], a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
+                    for (int i = 0; i < 4; ++i) {
+                        v[i] = oacc[jm][i];
+                        if (split) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
+                    }
+                    if (!split || tig < 2) {
+                        const int ch_a = f8_layout ? 16 * jm + 2 * gid : 16 * jm + gid, ch_b = f8_layout ? ch_a + 1 : ch_a + 8;
+                        const float sa = f8_layout ? ud.v_scale[ch_a] : 1.f, sb = f8_layout ? ud.v_scale[ch_b] : 1.f;
+                        float* p0 = scratch_f + 2 * tig * 128;
+                        float* p1 = p0 + 128;
+                        if (accumulate) {
+                            p0[ch_a] += v[0] * sa * f0; p1[ch_a] += v[1] * sa * f1; p0[ch_b] += v[2] * sb * f0; p1[ch_b] += v[3] * sb * f1;
+                        } else {
+                            p0[ch_a] = v[0] * sa; p1[ch_a] = v[1] * sa; p0[ch_b] = v[2] * sb; p1[ch_b] = v[3] * sb;
                         }
                     }
-                    TPH(2);
                 }
-                TPH(3);
-                if (with_res && cr[3] > cr[2]) {
-                    if (tokmode) scatter_tok(t_vrows, cr[2], cr[3], pve, ptv);
-                    else scatter(v_ent, cr[2], cr[3], pve);
-                    __syncwarp();
-                }
-                if (tokmode) prefetch_tok(t_vrows, nr[2], nr[3], pve, ptv);
-                else if (resid) prefetch(v_ent, nr[2], nr[3], pve);
-
-                TPH(4);
-                // ---- online softmax per column over this slice's 16 tokens (this thread: tokens gid, gid + 8) ----
-                float p[2][2];  // [token half][column 2 tig + e]
-                float mt[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const bool valid = r0 + gid + 8 * hh < rows_valid;
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const float sv = valid ? (sacc[0][2 * hh + e] + sacc[1][2 * hh + e]) * kscale : -INFINITY;
-                        p[hh][e] = sv;
-                        mt[e] = fmaxf(mt[e], sv);
-                    }
-                }
-#pragma unroll
-                for (int o = 4; o < 32; o <<= 1) {
-                    mt[0] = fmaxf(mt[0], __shfl_xor_sync(0xFFFFFFFFu, mt[0], o));
-                    mt[1] = fmaxf(mt[1], __shfl_xor_sync(0xFFFFFFFFu, mt[1], o));
-                }
-                float alpha[2];
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const float m_new = fmaxf(m_run[e], mt[e]);
-                    if (m_new == -INFINITY) {
-                        alpha[e] = 1.f;
-                        p[0][e] = p[1][e] = 0.f;
-                    } else {
-                        alpha[e] = ex2(m_run[e] - m_new);
-                        p[0][e] = ex2(p[0][e] - m_new);
-                        p[1][e] = ex2(p[1][e] - m_new);
-                    }
-                    l_run[e] = l_run[e] * alpha[e] + (p[0][e] + p[1][e]);
-                    m_run[e] = m_new;
-                }
-                if (__any_sync(0xFFFFFFFFu, alpha[0] != 1.f || alpha[1] != 1.f)) {
-#pragma unroll
-                    for (int jm = 0; jm < 8; ++jm) {
-                        oacc[jm][0] *= alpha[0]; oacc[jm][1] *= alpha[1]; oacc[jm][2] *= alpha[0]; oacc[jm][3] *= alpha[1];
-                    }
-                }
-                // B operand of the second product, P^T[token][column]: columns 0-3 carry the bf16 rounding of P and
-                // (G <= 4) columns 4-7 its remainder; an 8 x 8 register transpose turns the accumulator layout
-                // (token row, column pair) into the operand layout (column, token pair).
-                uint32_t pb[2];
-                {
-                    const bool lo_part = split && tig >= 2;
-#pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        float v[2];
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const float pv_ = p[hh][e] * vscale;
-                            const float hi = F8 ? __half2float(__float2half_rn(pv_)) : __bfloat162float(__float2bfloat16_rn(pv_));
-                            v[e] = lo_part ? pv_ - hi : hi;
-                        }
-                        pb[hh] = movmatrix_t(F8 ? pack_f16(v[0], v[1]) : pack_bf16(v[0], v[1]));
-                    }
-                }
-                TPH(5);
-                // ---- O^T[channel][column] += V^T . P^T : eight m-tiles of 16 channels, k = this slice's 16 tokens ----
-                {
-                    const int mi = lane >> 3, rr = lane & 7;
-                    const int row = r0 + (mi >> 1) * 8 + rr;  // ldmatrix.trans: matrices = (chunk | chunk + 1) x (tokens 0-7 | 8-15)
-                    if constexpr (F8) {
-                        // A transposed 8 x 8 tile of 2-byte units gives this thread channels (2 gid, 2 gid + 1) of tokens
-                        // (2 tig, 2 tig + 1) as bytes (c0 t0, c1 t0, c0 t1, c1 t1): a byte permute puts one channel's token pair
-                        // in each half; the two channels become rows gid and gid + 8 of the m-tile (the merge writes them back
-                        // to their channels).
-                        const int row8 = r0 + (mi & 1) * 8 + rr;  // matrices = (tokens 0-7 | 8-15) x two 16-byte chunks
-#pragma unroll
-                        for (int p2 = 0; p2 < 4; ++p2) {
-                            uint32_t x0, x1, x2, x3;
-                            ldsm_x4_t(vb + swz(row8, 2 * p2 + (mi >> 1)), x0, x1, x2, x3);
-                            x0 = prmt1(x0, 0x3120u); x1 = prmt1(x1, 0x3120u); x2 = prmt1(x2, 0x3120u); x3 = prmt1(x3, 0x3120u);
-                            mma_f16(oacc[2 * p2], cvt_e4m3x2(x0), cvt_e4m3x2(x0 >> 16), cvt_e4m3x2(x1), cvt_e4m3x2(x1 >> 16), pb[0], pb[1]);
-                            mma_f16(oacc[2 * p2 + 1], cvt_e4m3x2(x2), cvt_e4m3x2(x2 >> 16), cvt_e4m3x2(x3), cvt_e4m3x2(x3 >> 16), pb[0], pb[1]);
-                        }
-                    } else if (sch.experiment != 2) {  // (timing experiment 2 skips this product)
-#pragma unroll
-                        for (int jm = 0; jm < 8; ++jm) {
-                            const int c = 2 * jm + (mi & 1);
-                            uint32_t a0, a1, a2, a3;
-                            ldsm_x4_t(vb + (c >> 3) * kHalfBytes + swz(row, c), a0, a1, a2, a3);
-                            mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0], pb[1]);
-                        }
-                    }
-                    TPH(6);
-                    if (with_res && cr[3] > cr[2]) {
-                        const int srow = (mi >> 1) * 8 + rr;
-#pragma unroll
-                        for (int jm = 0; jm < 8; ++jm) {
-                            const int c = 2 * jm + (mi & 1);
-                            uint32_t a0, a1, a2, a3;
-                            ldsm_x4_t(scratch + (c >> 3) * 2048 + swz(srow, c), a0, a1, a2, a3);
-                            if constexpr (F8) mma_f16(oacc[jm], a0, a1, a2, a3, pb[0] ^ sgn, pb[1] ^ sgn);
-                            else mma_bf16(oacc[jm], a0, a1, a2, a3, pb[0] ^ sgn, pb[1] ^ sgn);
-                        }
-                        __syncwarp();
-                        zero_scratch();
-                    }
-                }
-                TPH(7);
-                release_stage(s, itj);
-                TPH(8);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) cr[i] = nr[i];
-                if (resid) {
-                    if (j + 1 - rb == 32) {  // the next tile opens a new batch
-                        rk[0] = rk_n[0]; rk[1] = rk_n[1]; rv[0] = rv_n[0]; rv[1] = rv_n[1];
-                        rb += 32;
-                        load_batch(rb + 32, rk_n, rv_n);
-                    }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) nr[i] = fr[i];
-                    get_ranges(j + 3, fr);
-                    l2_prefetch(fr);
-                }
-                TPH(9);
+            };
+            // (the tile body lives in decode_fast_tile.inc so that it can be instantiated per tile kind without a lambda:
+            // as a generic lambda it cost the bf16 kernel 6 %)
+#define FDKV_TAIL_TILE false
+            for (int j = 0; j < (F8 ? npre : nseg); ++j)
+#include "decode_fast_tile.inc"
+#undef FDKV_TAIL_TILE
+            if constexpr (F8) {
+#define FDKV_TAIL_TILE true
+                for (int j = npre; j < nseg; ++j)
+#include "decode_fast_tile.inc"
+#undef FDKV_TAIL_TILE
             }
             it += nseg;
             TGLOBAL(2);
@@ -759,29 +569,32 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     lq[0] += __shfl_xor_sync(0xFFFFFFFFu, lq[0], o);
                     lq[1] += __shfl_xor_sync(0xFFFFFFFFu, lq[1], o);
                 }
+                if (F8 && stashed) {
+                    // join the stashed state of the 8-bit tiles (already in the scratch) with the tails' state
+                    float f_st[2], f_tl[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float M = fmaxf(m_st[e], m_run[e]);
+                        f_st[e] = m_st[e] == -INFINITY ? 0.f : ex2(m_st[e] - M);
+                        f_tl[e] = m_run[e] == -INFINITY ? 0.f : ex2(m_run[e] - M);
+                        lq[e] = l_st[e] * f_st[e] + lq[e] * f_tl[e];
+                        m_run[e] = M;
+                    }
+                    if (!split || tig < 2) {  // the positions this lane wrote at the stash
+#pragma unroll
+                        for (int jm = 0; jm < 8; ++jm) {
+                            float* p0 = scratch_f + 2 * tig * 128 + 16 * jm + 2 * gid;
+                            p0[0] *= f_st[0]; p0[1] *= f_st[0]; p0[128] *= f_st[1]; p0[129] *= f_st[1];
+                        }
+                    }
+                    __syncwarp();
+                    store_o(false, true, f_tl[0], f_tl[1]);
+                } else {
+                    store_o(F8, false, 1.f, 1.f);
+                }
                 if (gid == 0) {
 #pragma unroll
                     for (int e = 0; e < 2; ++e) { sm_m[warp * 8 + 2 * tig + e] = m_run[e]; sm_l[warp * 8 + 2 * tig + e] = lq[e]; }
-                }
-                // O[head][channel]: column g plus (G <= 4) its remainder column g + 4, held by the lane two over
-#pragma unroll
-                for (int jm = 0; jm < 8; ++jm) {
-                    float v[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        v[i] = oacc[jm][i];
-                        if (split) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
-                    }
-                    if (!split || tig < 2) {
-                        // rows gid / gid + 8 of the m-tile: channels gid and gid + 8, or (8-bit rows) 2 gid and 2 gid + 1,
-                        // whose codes are still to be multiplied by the channel's V scale
-                        const int ch_a = F8 ? 16 * jm + 2 * gid : 16 * jm + gid, ch_b = F8 ? ch_a + 1 : ch_a + 8, col = 2 * tig;
-                        const float sa = F8 ? ud.v_scale[ch_a] : 1.f, sb = F8 ? ud.v_scale[ch_b] : 1.f;
-                        scratch_f[col * 128 + ch_a] = v[0] * sa;
-                        scratch_f[(col + 1) * 128 + ch_a] = v[1] * sa;
-                        scratch_f[col * 128 + ch_b] = v[2] * sb;
-                        scratch_f[(col + 1) * 128 + ch_b] = v[3] * sb;
-                    }
                 }
                 __syncthreads();
                 TGLOBAL(0);

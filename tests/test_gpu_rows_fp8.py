@@ -1,6 +1,6 @@
 """GPU parity for 8-bit row streams (row_format = e4m3): the committed codes and per-channel scales are bit-exact against
 the oracle's quantiser; decode attention over them (f16 tensor-core products on converted fragments, scales folded
-into q and applied to the output) matches the oracle's attention over the dequantised rows within the bf16 tolerance."""
+into q and applied to the output) matches the oracle's attention over the dequantised rows within the bf16 tolerance, with generated tokens appended to the bf16 tails."""
 import numpy as np
 import pytest
 import torch
@@ -19,13 +19,13 @@ def _unit8(w, p, h):
     return R8.UnitFp8(k0, k1, v0, v1, True, w.keep_num, w.keep_den)
 
 
-@pytest.mark.parametrize("T,Hq,Hkv,keep", [(1300, 8, 2, (1, 16)), (2100, 4, 1, (1, 32)), (300, 2, 2, (1, 8))])
-def test_rows_e4m3_parity(T, Hq, Hkv, keep):
+@pytest.mark.parametrize("T,Hq,Hkv,keep,n_steps", [(1300, 8, 2, (1, 16), 3), (2100, 4, 1, (1, 32), 131), (300, 2, 2, (1, 8), 2)])
+def test_rows_e4m3_parity(T, Hq, Hkv, keep, n_steps):
     from paper_2607_06519_b200 import runner
 
     w = synth.Workload(name="f8", n_layers=4, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=128, batch=1, T=T, dtype="bf16",
-                       keep_num=keep[0], keep_den=keep[1], n_needles=4, W=8, seed=51, n_steps=1, row_format=1)
-    pf = runner.Prefilled(w, max_tail=1)
+                       keep_num=keep[0], keep_den=keep[1], n_needles=4, W=8, seed=51, n_steps=n_steps, row_format=1)
+    pf = runner.Prefilled(w, max_tail=n_steps)
     modes = np.array([[(p + h) % 3 for h in range(Hkv)] for p in range(2)], dtype=np.int32)
     pf.prefill(0, modes=modes)
     units = {(p, h): _unit8(w, p, h) for p in range(2) for h in range(Hkv)}
@@ -37,21 +37,23 @@ def test_rows_e4m3_parity(T, Hq, Hkv, keep):
                 want_c, want_s = u.q_x[name][layer & 1] if modes[p][h] == 2 else u.q_z0[name]
                 assert np.array_equal(scale.cpu().numpy(), want_s), (p, h, layer, name)
                 assert np.array_equal(codes.cpu().numpy(), want_c), (p, h, layer, name)
-    # decode
+    # decode, appending generated tokens to the (bf16) tails: the 8-bit tiles and the tails join at the merge
     G = w.group
-    worst = 0.0
-    for layer in range(4):
-        q = pf.decode_q(layer, 0)
-        out = f32(pf.ctx.decode_attn(layer, q, out_dtype=0))[0]
-        torch.cuda.synchronize()
-        for h in range(Hkv):
-            ref = units[(layer // 2, h)].attend(int(modes[layer // 2][h]), layer & 1, f32(q)[0][h * G:(h + 1) * G])
-            worst = max(worst, float(vector_errors(out[h * G:(h + 1) * G], ref).max()))
-    assert worst <= TOL["bf16"], worst
-    # appends are closed for this format
-    kn, vn = pf.new_rows(0, 0)
-    with pytest.raises(B.FdkvError):
-        pf.ctx.decode_attn(0, pf.decode_q(0, 0), kn, vn)
+    for step in range(n_steps):
+        worst = 0.0
+        for layer in range(4):
+            q = pf.decode_q(layer, step)
+            kn, vn = pf.new_rows(layer, step)
+            for h in range(Hkv):
+                units[(layer // 2, h)].append(layer & 1, f32(kn)[0, h], f32(vn)[0, h])
+            out = f32(pf.ctx.decode_attn(layer, q, kn, vn, out_dtype=0))[0]
+            torch.cuda.synchronize()
+            for h in range(Hkv):
+                ref = units[(layer // 2, h)].attend(int(modes[layer // 2][h]), layer & 1, f32(q)[0][h * G:(h + 1) * G])
+                worst = max(worst, float(vector_errors(out[h * G:(h + 1) * G], ref).max()))
+        assert worst <= TOL["bf16"], (step, worst)
+    for b in range(1):
+        pf.ctx.set_tail_len(b, 0)
     by_mode, exact_equiv = pf.ctx.footprint(0)
     assert pf.ctx.decode_bytes(0, 1) < 0.62 * sum(2 * T * 128 * 2 for _ in range(Hkv)) + 64 * 1024 * Hkv
     assert pf.ctx.device_status() == 0
