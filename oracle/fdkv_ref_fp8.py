@@ -96,3 +96,35 @@ class UnitFp8(R.Unit):
         if tail:
             pre = np.concatenate([pre, np.stack(tail).astype(np.float64)], axis=0)
         return pre
+
+
+class Unit4Fp8:
+    """A block-of-four unit (see fdkv_ref_b4.Unit4) whose committed row streams are 8-bit."""
+
+    def __init__(self, k_layers, v_layers, bf16: bool, keep_num: int, keep_den: int):
+        from . import fdkv_ref_b4 as R4
+        self.u = R4.Unit4(k_layers, v_layers, bf16, keep_num, keep_den)
+        self.q_z0 = {n: quantise_rows(self.u.z0[n]) for n in ("k", "v")}
+        self.q_x = {n: [quantise_rows(self.u.x[n][l]) for l in range(4)] for n in ("k", "v")}
+
+    def append(self, layer_in_block: int, k_row, v_row):
+        self.u.append(layer_in_block, k_row, v_row)
+
+    def rows(self, name: str, mode: int, layer_in_block: int) -> np.ndarray:
+        u = self.u
+        if mode == R.EXACT:
+            pre = dequantise_rows(*self.q_x[name][layer_in_block])
+        else:
+            pre = 0.5 * dequantise_rows(*self.q_z0[name])
+            if mode == R.RESIDUAL and u.kept[name].size:
+                idx = u.kept[name].astype(np.int64)
+                pre.reshape(-1)[idx] += u.dev[name][layer_in_block].reshape(-1)[idx].astype(np.float64)
+        tail = u.tail[(name, layer_in_block)]
+        if tail:
+            pre = np.concatenate([pre, np.stack(tail).astype(np.float64)], axis=0)
+        return pre
+
+    def attend(self, mode: int, layer_in_block: int, q_heads) -> np.ndarray:
+        kh = self.rows("k", mode, layer_in_block)
+        vh = self.rows("v", mode, layer_in_block)
+        return np.stack([R.attention(kh, vh, q) for q in np.ascontiguousarray(q_heads, dtype=np.float32)])

@@ -47,7 +47,7 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.max_fold = c.max_fold;
     if (c.row_format != FDKV_ROWS_STORAGE && c.row_format != FDKV_ROWS_E4M3) return false;
     s.rows_f8 = c.row_format == FDKV_ROWS_E4M3;
-    if (s.rows_f8 && !(c.dtype == FDKV_BF16 && c.head_dim == 128 && B == 2 && G <= 4 && c.residual_rule == FDKV_RESIDUAL_ENTRIES && c.max_fold == 0))
+    if (s.rows_f8 && !(c.dtype == FDKV_BF16 && c.head_dim == 128 && G <= 4 && c.residual_rule == FDKV_RESIDUAL_ENTRIES && c.max_fold == 0))
         return false;
     s.kfold_max = (int64_t)s.max_fold * s.d * s.keep_num / s.keep_den;
     s.kmax = (int64_t)s.Tmax * s.d * s.keep_num / s.keep_den;

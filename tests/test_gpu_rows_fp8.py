@@ -92,3 +92,36 @@ def test_rows_e4m3_benchmark_workload_sampled():
     assert pf.ctx.decode_bytes(0, 1) < 0.56 * 8 * 2 * w.T * 128 * 2
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_rows_e4m3_with_blocks_of_four():
+    """8-bit rows combined with depth blocks of four layers: codes of the shared rows bit-exact, decode with appends."""
+    from paper_2607_06519_b200 import runner
+
+    w = synth.Workload(name="f8b4", n_layers=8, n_q_heads=8, n_kv_heads=2, head_dim=128, batch=1, T=900, dtype="bf16",
+                       keep_num=1, keep_den=16, n_needles=4, W=8, seed=53, n_steps=2, row_format=1, block_size=4)
+    pf = runner.Prefilled(w, max_tail=2)
+    modes = np.array([[1, 0], [2, 1]], dtype=np.int32)
+    pf.prefill(0, modes=modes)
+    units = {(b, h): R8.Unit4Fp8(synth.block_tensor(w, 0, b, h, False), synth.block_tensor(w, 0, b, h, True), True, 1, 16)
+             for b in range(2) for h in range(2)}
+    for (b, h), u in units.items():
+        for lb in range(4):
+            codes, scale = pf.ctx.get_rows_e4m3(0, 4 * b + lb, h, 1, w.T)
+            want_c, want_s = u.q_x["v"][lb] if modes[b][h] == 2 else u.q_z0["v"]
+            assert np.array_equal(scale.cpu().numpy(), want_s) and np.array_equal(codes.cpu().numpy(), want_c)
+    G = 4
+    for step in range(2):
+        for layer in range(8):
+            blk, lb = divmod(layer, 4)
+            q = pf.decode_q(layer, step)
+            kn, vn = pf.new_rows(layer, step)
+            for h in range(2):
+                units[(blk, h)].append(lb, f32(kn)[0, h], f32(vn)[0, h])
+            out = f32(pf.ctx.decode_attn(layer, q, kn, vn, out_dtype=0))[0]
+            torch.cuda.synchronize()
+            for h in range(2):
+                ref = units[(blk, h)].attend(int(modes[blk][h]), lb, f32(q)[0][h * G:(h + 1) * G])
+                assert vector_errors(out[h * G:(h + 1) * G], ref).max() <= TOL["bf16"], (step, layer, h)
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
