@@ -98,6 +98,8 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.io_k = take((size_t)s.L * s.max_batch * s.Hkv * s.d * 4);
     w.io_v = take((size_t)s.L * s.max_batch * s.Hkv * s.d * 4);
     w.io_out = take((size_t)s.L * s.max_batch * s.Hq * s.d * 4);
+    // job tables of the 8-bit commit: one quantise job per stored tensor, one repack job per residual list
+    w.jobs = take(s.rows_f8 ? (size_t)s.NU * 2 * s.B * (sizeof(QuantJob) + sizeof(RepackJob)) : 0);
     w.total = o;
 
     o = 0;
@@ -518,6 +520,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return c->arena + r; };
     size_t by_mode[3] = {0, 0, 0};
     const size_t unit_stride_b = (size_t)s.Tmax * s.d * s.esize;
+    std::vector<QuantJob> qjobs;   // 8-bit rows: every stored tensor is quantised by one batched pass after this loop
+    std::vector<RepackJob> rjobs;  // ... and every residual list repacked relative to its tensor's scales
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u], p = u / s.Hkv, h = u % s.Hkv;
         UnitDesc* dl[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -538,7 +542,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                         char* dst = take(rows8_pad);
                         float* sc = reinterpret_cast<float*>(take(scale_slot));
                         if (rows8_pad > rows8) CU(cudaMemsetAsync(dst + rows8, 0, rows8_pad - rows8, st));
-                        CU(launch_quantise_rows(sp, c->stride_t, T, reinterpret_cast<uint8_t*>(dst), sc, st));
+                        qjobs.push_back(QuantJob{sp, c->stride_t, T, 0, reinterpret_cast<uint8_t*>(dst), sc});
                         (is_v ? dl[l]->v_rows : dl[l]->k_rows) = dst;
                         (is_v ? dl[l]->v_scale : dl[l]->k_scale) = sc;
                         dl[l]->rows_f8 = 1;
@@ -567,7 +571,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                     z0 = take(rows8_pad);
                     sc8 = reinterpret_cast<float*>(take(scale_slot));
                     if (rows8_pad > rows8) CU(cudaMemsetAsync(z0 + rows8, 0, rows8_pad - rows8, st));
-                    CU(launch_quantise_rows(c->work + c->ws.z0 + ut * unit_stride_b, s.d, T, reinterpret_cast<uint8_t*>(z0), sc8, st));
+                    qjobs.push_back(QuantJob{c->work + c->ws.z0 + ut * unit_stride_b, s.d, T, 0, reinterpret_cast<uint8_t*>(z0), sc8});
                     for (int l = 0; l < s.B; ++l) { (is_v ? dl[l]->v_scale : dl[l]->k_scale) = sc8; dl[l]->rows_f8 = 1; }
                 } else {
                     z0 = take(rows_pad);
@@ -601,8 +605,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                         if (c->packed_lists) {
                             pi_l[j] = take(idx_b);
                             if (s.rows_f8)  // values relative to the channel scales, positions in the converted fragments' order
-                                CU(launch_repack_entries_f8(reinterpret_cast<uint32_t*>(pi_l[j]), wsp<uint32_t>(c, c->ws.packed) + lt * s.kcap, k,
-                                                            sc8, is_v, st));
+                                rjobs.push_back(RepackJob{reinterpret_cast<uint32_t*>(pi_l[j]), wsp<uint32_t>(c, c->ws.packed) + lt * s.kcap, k, sc8, is_v, 0});
                             else
                                 CU(cudaMemcpyAsync(pi_l[j], c->work + c->ws.packed + lt * s.kcap * 4, idx_copy, cudaMemcpyDeviceToDevice, st));
                         } else {
@@ -621,6 +624,16 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                     by_mode[1] += (size_t)k * (c->packed_lists ? (size_t)4 * s.NB : 4 + (size_t)s.NB * s.esize);
                 }
             }
+        }
+    }
+    if (!qjobs.empty()) {
+        QuantJob* qd = reinterpret_cast<QuantJob*>(c->work + c->ws.jobs);
+        RepackJob* rd = reinterpret_cast<RepackJob*>(qd + (size_t)s.NU * 2 * s.B);
+        CU(cudaMemcpyAsync(qd, qjobs.data(), qjobs.size() * sizeof(QuantJob), cudaMemcpyHostToDevice, st));
+        CU(launch_quantise_jobs(qd, (int)qjobs.size(), T, st));
+        if (!rjobs.empty()) {
+            CU(cudaMemcpyAsync(rd, rjobs.data(), rjobs.size() * sizeof(RepackJob), cudaMemcpyHostToDevice, st));
+            CU(launch_repack_jobs(rd, (int)rjobs.size(), k, st));
         }
     }
     const size_t seq_desc = (size_t)s.L * s.Hkv;

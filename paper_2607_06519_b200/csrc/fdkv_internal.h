@@ -83,7 +83,7 @@ struct WsLayout {
     size_t tok_score, tok_flag, tok_list, tok_off;
     size_t energy, eval;  // four-layer blocks: per-position high-frequency energy (float32) and the kept energies
     size_t status, z0, z1, z1drop, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
-        partials, counters, io_q, io_k, io_v, io_out, total;  // io_*: host-I/O staging, [L] layers each
+        partials, counters, io_q, io_k, io_v, io_out, jobs, total;  // io_*: host-I/O staging, [L] layers each
 };
 struct ArenaLayout {
     size_t tail_len, desc, tail_k, tail_v, bump, worst_total;
@@ -248,11 +248,26 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out);
 // Same view ([rows][128] bf16, 64-channel x box_rows boxes, 128-byte swizzle) over any 256-byte aligned region.
 bool make_rows_tensor_map(void* base, size_t bytes, int box_rows, void* tmap_out);
 // ---- 8-bit row streams (rows_fp8.cu) ----
-// codes[t][c] = e4m3(src[t*stride_t + c] / scale[c]), scale[c] = max_t |src| / 448 (1 if zero); src bf16, d = 128
-cudaError_t launch_quantise_rows(const void* src, int64_t stride_t, int T, uint8_t* codes, float* scale, cudaStream_t st);
-// packed residual entries for a unit whose rows are 8-bit: value -> f16(value / scale[channel]), position permuted inside
-// its 16-channel group to the order the kernel's converted fragments use (K and V differ)
-cudaError_t launch_repack_entries_f8(uint32_t* dst, const uint32_t* src, int64_t n, const float* scale, int is_v, cudaStream_t st);
+// One stored tensor: codes[t][c] = e4m3(src[t*stride_t + c] / scale[c]), scale[c] = max_t |src| / 448 (1 if zero); src bf16,
+// d = 128; scale points at a 1 KiB slot whose second half holds the channel maxima while the job runs.
+struct QuantJob {
+    const void* src;
+    int64_t stride_t;
+    int32_t T, pad_;
+    uint8_t* codes;
+    float* scale;
+};
+// One residual list of a unit whose rows are 8-bit: value -> f16(value / scale[channel]), position permuted inside its
+// 16-channel group to the order the kernel's converted fragments use (K and V differ).
+struct RepackJob {
+    uint32_t* dst;
+    const uint32_t* src;
+    int64_t n;
+    const float* scale;
+    int32_t is_v, pad_;
+};
+cudaError_t launch_quantise_jobs(const QuantJob* jobs_dev, int njobs, int T_max, cudaStream_t st);
+cudaError_t launch_repack_jobs(const RepackJob* jobs_dev, int njobs, int64_t n_max, cudaStream_t st);
 bool make_rows_tensor_map_u8(void* base, size_t bytes, int box_rows, void* tmap_out);
 
 // dst[i] = src[i] + add, i < n (list offsets and indices of a folded chunk)

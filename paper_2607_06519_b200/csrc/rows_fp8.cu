@@ -15,30 +15,38 @@ namespace {
 
 constexpr int kD = 128;
 
-// grid (token chunks): per-channel maximum of |x| over the chunk, merged with atomicMax on the bit patterns
-// (non-negative floats order like their bits).  amax must start at zero.
-__global__ void __launch_bounds__(256) absmax_kernel(const __nv_bfloat16* src, int64_t stride_t, int T, int rows_per_cta,
-                                                     uint32_t* amax_bits) {
+// All row streams of a commit are quantised by three launches over a job table (one job per stored tensor).
+// grid (token chunks, jobs): per-channel maximum of |x| over the chunk, merged with atomicMax on the bit patterns
+// (non-negative floats order like their bits); the maxima live in the second half of the job's 1 KiB scale slot.
+__global__ void __launch_bounds__(128) zero_amax_kernel(const QuantJob* jobs) {
+    reinterpret_cast<uint32_t*>(jobs[blockIdx.x].scale)[kD + threadIdx.x] = 0u;
+}
+__global__ void __launch_bounds__(256) absmax_kernel(const QuantJob* jobs, int rows_per_cta) {
     __shared__ uint32_t s_max[2][kD];
+    const QuantJob jb = jobs[blockIdx.y];
+    const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(jb.src);
     const int c = threadIdx.x & (kD - 1), half = threadIdx.x >> 7;
-    const int t0 = blockIdx.x * rows_per_cta, t1 = min(T, t0 + rows_per_cta);
+    const int t0 = blockIdx.x * rows_per_cta, t1 = min(jb.T, t0 + rows_per_cta);
+    if (t0 >= jb.T) return;
     uint32_t m = 0;
     for (int t = t0 + half; t < t1; t += 2) {
-        const uint32_t b = (uint32_t)__bfloat16_as_ushort(src[(int64_t)t * stride_t + c]) << 16;
+        const uint32_t b = (uint32_t)__bfloat16_as_ushort(src[(int64_t)t * jb.stride_t + c]) << 16;
         m = max(m, b & 0x7FFFFFFFu);
     }
     s_max[half][c] = m;
     __syncthreads();
-    if (half == 0) atomicMax(&amax_bits[c], max(s_max[0][c], s_max[1][c]));
+    if (half == 0) atomicMax(reinterpret_cast<uint32_t*>(jb.scale) + kD + c, max(s_max[0][c], s_max[1][c]));
 }
 
-// one thread per 8 channels of a token: scale from the maxima, codes out (8 bytes per store)
-__global__ void __launch_bounds__(256) quantise_kernel(const __nv_bfloat16* src, int64_t stride_t, int T, const uint32_t* amax_bits,
-                                                       uint8_t* codes, float* scale_out) {
+// grid (ceil(T * 16 / 256), jobs): one thread per 8 channels of a token: scale from the maxima, codes out (8 bytes)
+__global__ void __launch_bounds__(256) quantise_kernel(const QuantJob* jobs) {
+    const QuantJob jb = jobs[blockIdx.y];
+    const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(jb.src);
+    const uint32_t* amax_bits = reinterpret_cast<const uint32_t*>(jb.scale) + kD;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int t = (int)(i >> 4), c8 = (int)(i & 15) * 8;
-    if (t >= T) return;
-    const uint4 raw = *reinterpret_cast<const uint4*>(src + (int64_t)t * stride_t + c8);
+    if (t >= jb.T) return;
+    const uint4 raw = *reinterpret_cast<const uint4*>(src + (int64_t)t * jb.stride_t + c8);
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
     uint32_t out[2] = {0u, 0u};
 #pragma unroll
@@ -48,9 +56,9 @@ __global__ void __launch_bounds__(256) quantise_kernel(const __nv_bfloat16* src,
         const float x = __uint_as_float((j & 1) ? (w[j >> 1] & 0xFFFF0000u) : (w[j >> 1] << 16));
         const uint32_t code = (uint32_t)__nv_cvt_float_to_fp8(__fdiv_rn(x, sc), __NV_SATFINITE, __NV_E4M3);
         out[j >> 2] |= code << (8 * (j & 3));
-        if (t == 0) scale_out[c8 + j] = sc;
+        if (t == 0) jb.scale[c8 + j] = sc;
     }
-    *reinterpret_cast<uint2*>(codes + (int64_t)t * kD + c8) = make_uint2(out[0], out[1]);
+    *reinterpret_cast<uint2*>(jb.codes + (int64_t)t * kD + c8) = make_uint2(out[0], out[1]);
 }
 
 // Position of channel c inside its 16-channel group as the decode kernel's converted fragments see it.
@@ -60,42 +68,38 @@ __global__ void __launch_bounds__(256) quantise_kernel(const __nv_bfloat16* src,
 __device__ __forceinline__ int slot_k(int c) { return 2 * (c >> 2) + (c & 1) + 8 * ((c >> 1) & 1); }
 __device__ __forceinline__ int slot_v(int c) { return (c >> 1) + 8 * (c & 1); }
 
-__global__ void __launch_bounds__(256) repack_entries_f8_kernel(uint32_t* dst, const uint32_t* src, int64_t n, const float* scale,
-                                                                int is_v) {
+// grid (ceil(n / 256), jobs)
+__global__ void __launch_bounds__(256) repack_entries_f8_kernel(const RepackJob* jobs) {
+    const RepackJob jb = jobs[blockIdx.y];
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    const uint32_t w = src[i];
+    if (i >= jb.n) return;
+    const uint32_t w = jb.src[i];
     // undo the pair-path offset: byte offset / 2 = half << 10 | row << 6 | (chunk ^ row) << 3 | ch & 7
     const uint32_t off2 = w >> 16;
     const int row = (off2 >> 6) & 15, half = off2 >> 10, chunk = ((off2 >> 3) ^ (off2 >> 6)) & 7, ch = half * 64 + chunk * 8 + (off2 & 7);
-    const int g = ch & ~15, cs = g + (is_v ? slot_v(ch & 15) : slot_k(ch & 15));
+    const int g = ch & ~15, cs = g + (jb.is_v ? slot_v(ch & 15) : slot_k(ch & 15));
     const uint32_t off = (uint32_t)((cs >> 6) * 2048 + row * 128 + ((((cs >> 3) & 7) ^ (row & 7)) << 4) + (cs & 7) * 2);
     const float v = __uint_as_float((w & 0xFFFFu) << 16);
-    const __half hv = __float2half_rn(__fdiv_rn(v, scale[ch]));
-    dst[i] = (uint32_t)__half_as_ushort(hv) | ((off >> 1) << 16);
+    const __half hv = __float2half_rn(__fdiv_rn(v, jb.scale[ch]));
+    jb.dst[i] = (uint32_t)__half_as_ushort(hv) | ((off >> 1) << 16);
 }
 
 }  // namespace
 
-cudaError_t launch_quantise_rows(const void* src, int64_t stride_t, int T, uint8_t* codes, float* scale, cudaStream_t st) {
-    if (T <= 0) return cudaSuccess;
-    // the caller's scale slot is 1 KiB: [0, 512) the float32 scales, [512, 1024) the channel maxima (bit patterns)
-    uint32_t* amax = reinterpret_cast<uint32_t*>(scale) + kD;
-    cudaError_t e = cudaMemsetAsync(amax, 0, kD * sizeof(uint32_t), st);
-    if (e != cudaSuccess) return e;
-    const int rows_per_cta = 256;
-    absmax_kernel<<<(T + rows_per_cta - 1) / rows_per_cta, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(src), stride_t, T,
-                                                                         rows_per_cta, amax);
-    const int64_t threads = (int64_t)T * 16;
-    quantise_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(src), stride_t, T, amax,
-                                                                        codes, scale);
-    count_launch(2);
+cudaError_t launch_quantise_jobs(const QuantJob* jobs_dev, int njobs, int T_max, cudaStream_t st) {
+    if (njobs <= 0 || T_max <= 0) return cudaSuccess;
+    const int rows_per_cta = 1024;
+    zero_amax_kernel<<<njobs, kD, 0, st>>>(jobs_dev);
+    absmax_kernel<<<dim3((T_max + rows_per_cta - 1) / rows_per_cta, njobs), 256, 0, st>>>(jobs_dev, rows_per_cta);
+    const int64_t threads = (int64_t)T_max * 16;
+    quantise_kernel<<<dim3((unsigned)((threads + 255) / 256), njobs), 256, 0, st>>>(jobs_dev);
+    count_launch(3);
     return cudaGetLastError();
 }
 
-cudaError_t launch_repack_entries_f8(uint32_t* dst, const uint32_t* src, int64_t n, const float* scale, int is_v, cudaStream_t st) {
-    if (n <= 0) return cudaSuccess;
-    repack_entries_f8_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dst, src, n, scale, is_v);
+cudaError_t launch_repack_jobs(const RepackJob* jobs_dev, int njobs, int64_t n_max, cudaStream_t st) {
+    if (njobs <= 0 || n_max <= 0) return cudaSuccess;
+    repack_entries_f8_kernel<<<dim3((unsigned)((n_max + 255) / 256), njobs), 256, 0, st>>>(jobs_dev);
     count_launch(1);
     return cudaGetLastError();
 }
