@@ -126,3 +126,41 @@ def test_step_host_call_equals_per_layer_calls():
         assert torch.equal(hout[l], want[l].cpu())
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_unsupported_combinations_and_reset_reuse():
+    """Configurations the build has no kernels for are refused at creation; a context is reusable after reset."""
+    from paper_2607_06519_b200 import binding as B, runner, synth
+
+    base = dict(n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=128, max_batch=1, max_prefill=512, max_tail=4, dtype=B.BF16,
+                keep_num=1, keep_den=16)
+    for bad in (dict(block_size=3), dict(block_size=4, residual_rule=1), dict(row_format=1, head_dim=64),
+                dict(row_format=1, dtype=B.F32), dict(row_format=1, max_fold=16), dict(row_format=1, n_q_heads=16),
+                dict(row_format=2), dict(max_fold=-1), dict(n_layers=6, block_size=4)):
+        cfg = dict(base)
+        cfg.update(bad)
+        with pytest.raises(B.FdkvError) as e:
+            B.sizes(B.Config(**cfg))
+        assert e.value.code == 2, bad
+    # fold_tail is refused for the token rule and for 8-bit rows, get_rows_e4m3 without them
+    w = synth.Workload(name="reuse", n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=128, batch=1, T=512, dtype="bf16",
+                       keep_num=1, keep_den=16, n_needles=4, W=8, seed=61, n_steps=1, block_size=4)
+    pf = runner.Prefilled(w, max_tail=2)
+    modes = np.array([[1, 2]], dtype=np.int32)
+    pf.prefill(0, modes=modes)
+    with pytest.raises(B.FdkvError) as e:
+        pf.ctx.get_rows_e4m3(0, 0, 0, 0, 512)
+    assert e.value.code == 2
+    with pytest.raises(B.FdkvError) as e:
+        pf.ctx.fold_tail(0, 16)  # max_fold is 0
+    assert e.value.code in (1, 3)
+    q = pf.decode_q(1, 0)
+    first = pf.ctx.decode_attn(1, q).clone()
+    # reset and run the same prompt again through the same context: identical output
+    pf.ctx.reset()
+    pf.prefill(0, modes=modes)
+    again = pf.ctx.decode_attn(1, q)
+    torch.cuda.synchronize()
+    assert torch.equal(first, again)
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
