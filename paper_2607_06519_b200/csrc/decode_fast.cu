@@ -787,6 +787,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         attr_done = true;
     }
     static double res_cost = -1.0;
+    static bool res_cost_env = false;
     static bool use_pdl = true;
     // tiles copied to shared memory before the dependency wait (measured: filling every stage is best; prefetching
     // further tiles to L2 as well takes bandwidth from the CTAs of the previous kernel that are still streaming)
@@ -796,6 +797,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     if (res_cost < 0) {
         const char* ev = getenv("FDKV_RES_COST");  // tuning knobs for benchmark sweeps
         res_cost = ev ? atof(ev) : 1.7;
+        res_cost_env = ev != nullptr;
         if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 1.7;
         const char* pv = getenv("FDKV_NO_PDL");
         use_pdl = !(pv && pv[0] == '1');
@@ -822,7 +824,9 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         wt[u] = 2 * kTT * 256 / 512;
         if (a.host_modes[u] == FDKV_MODE_RESIDUAL) {
             const int64_t res_bytes = a.tok_rule ? 2 * ((int64_t)T * a.keep_num / a.keep_den) * 260 : 2 * k * 4;  // rows + index, or packed entries
-            wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * res_cost);
+            // (measured best: 1.7 when every unit gets whole CTAs, 1.5 in the flat cut of a batch)
+            const double rc = res_cost_env ? res_cost : (units <= sm_count ? 1.7 : 1.5);
+            wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * rc);
         }
         wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
         total_tiles += nt[u];
