@@ -818,19 +818,24 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         const int T = a.host_T[u / a.Hkv];
         nt[u] = (T + kTT - 1) / kTT;
         if (nt[u] >= (1 << 20)) return cudaErrorInvalidValue;  // cannot happen: T * 128 < 2^31
-        const int64_t k = (int64_t)T * 128 * a.keep_num / a.keep_den;
-        // cost per tile: bytes in units of 512 B (the K and V boxes, plus the lists' share for residual units),
-        // residual tiles scaled by the measured ratio of their compute time to a plain tile's
-        wt[u] = 2 * kTT * 256 / 512;
-        if (a.host_modes[u] == FDKV_MODE_RESIDUAL) {
-            const int64_t res_bytes = a.tok_rule ? 2 * ((int64_t)T * a.keep_num / a.keep_den) * 260 : 2 * k * 4;  // rows + index, or packed entries
-            // (measured best: 1.7 when every unit gets whole CTAs, 1.5 in the flat cut of a batch)
-            const double rc = res_cost_env ? res_cost : (units <= sm_count ? 1.7 : 1.5);
-            wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * rc);
-        }
-        wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
         total_tiles += nt[u];
     }
+    // cost per tile: bytes in units of 512 B (the K and V boxes, plus the lists' share for residual units), residual
+    // tiles scaled by the measured ratio of their compute time to a plain tile's (rc)
+    auto weigh = [&](double rc) {
+        for (int u = 0; u < units; ++u) {
+            const int T = a.host_T[u / a.Hkv];
+            const int64_t k = (int64_t)T * 128 * a.keep_num / a.keep_den;
+            wt[u] = 2 * kTT * 256 / 512;
+            if (a.host_modes[u] == FDKV_MODE_RESIDUAL) {
+                const int64_t res_bytes = a.tok_rule ? 2 * ((int64_t)T * a.keep_num / a.keep_den) * 260 : 2 * k * 4;  // rows + index, or packed entries
+                wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * rc);
+            }
+            wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
+        }
+    };
+    // (measured best: 1.7 when every unit gets whole CTAs, 1.5 in the flat cut of a batch)
+    weigh(res_cost_env ? res_cost : 1.7);
     const int ncta = (int)std::min<int64_t>(std::min(std::min(sm_count, kMaxCtas), kMaxSplits), total_tiles);
     static unsigned g_launch_no = 0;
     ++g_launch_no;
@@ -874,6 +879,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
             for (int j = 0; j < nc[u]; ++j) sch.start[c++] = ((uint32_t)u << 20) | (uint32_t)((int64_t)nt[u] * j / nc[u]);
         sch.start[ncta] = (uint32_t)units << 20;
     } else {
+        if (!res_cost_env) weigh(1.5);
         int u = 0;
         for (int c = 0; c < ncta; ++c) {
             const int64_t target = wp[units] * c / ncta;
