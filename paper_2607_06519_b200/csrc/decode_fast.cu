@@ -175,7 +175,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 #ifdef FDKV_TIMING
-__device__ long long g_timing[64][kMaxCtas][8];
+__device__ long long g_timing[64][kMaxCtas][12];
 #define TSTAMP(i) do { if (threadIdx.x == 32) g_timing[sch.tslot][blockIdx.x][i] = clock64(); } while (0)
 #define TADD(i, v) do { t_acc[i - 4] += (v); } while (0)
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
@@ -662,6 +662,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                         float* const wts = red + kCW * 128 + warp * kMaxSplits;
 #pragma unroll
                         for (int i = 0; i < kMaxSplits / 32; ++i) wts[lane + 32 * i] = mreg[i];
+                        TGLOBAL(8);
                         __syncwarp();
                         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                         for (int base = pgi; base < nparts; base += 8 * npg) {
@@ -681,6 +682,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                                 }
                             }
                         }
+                        TGLOBAL(9);
                         reinterpret_cast<float4*>(red + warp * 128)[lane] = acc;
                         if (lane == 0) sm_l[warp] = ls;
                     }
@@ -697,6 +699,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                         else
                             reinterpret_cast<float*>(a.out)[o] = r;
                     }
+                    TGLOBAL(10);
                     if (threadIdx.x == 0) a.counters[u] = 0;  // ready for the next launch
                     __syncthreads();
                 }
@@ -923,7 +926,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     *handled = true;
 #ifdef FDKV_TIMING
     if (getenv("FDKV_TIMING_DUMP") && (g_launch_no % 64) == 63) {
-        static long long h[64][kMaxCtas][8];
+        static long long h[64][kMaxCtas][12];
         cudaStreamSynchronize(st);
         cudaMemcpyFromSymbol(h, g_timing, sizeof(h));
         long long base = h[0][0][6];
@@ -949,9 +952,9 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
             }
             if (l == 45)
                 for (int c = 0; c < ncta; ++c)
-                    fprintf(stderr, "cta %3d unit %2u mode %d tiles %2lld start %6lld waited %6lld loop_end %6lld end %6lld wait_full_cyc %6lld merged %6lld ticket %6lld\n", c,
+                    fprintf(stderr, "cta %3d unit %2u mode %d tiles %2lld start %6lld waited %6lld loop_end %6lld end %6lld wait_full_cyc %6lld merged %6lld ticket %6lld weights %6lld rows %6lld written %6lld\n", c,
                             sch.start[c] >> 20, a.host_modes[sch.start[c] >> 20], h[l][c][5], h[l][c][6] - g0, h[l][c][1] - g0, h[l][c][2] - g0,
-                            h[l][c][7] - g0, h[l][c][4], h[l][c][0] - g0, h[l][c][3] - g0);
+                            h[l][c][7] - g0, h[l][c][4], h[l][c][0] - g0, h[l][c][3] - g0, h[l][c][8] - g0, h[l][c][9] - g0, h[l][c][10] - g0);
         }
     }
 #endif
