@@ -82,3 +82,67 @@ def test_random_workload(case):
                 assert err.max() <= TOL[dtype], (step, layer, b, float(err.max()))
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def _cases_new():
+    rng = np.random.default_rng(4242)
+    out = []
+    for i in range(12):
+        bs = 4 if i % 2 else 2
+        f8 = int(i % 3 != 0)
+        if not f8 and bs == 2:
+            bs = 4
+        hkv = int(rng.choice([1, 2, 3]))
+        g = int(rng.choice([1, 2, 4]))
+        T = int(rng.choice([1, 15, 16, 17, 127, 128, 129, 255, 640, 1000, 1537]))
+        keep = [(1, 16), (1, 8), (3, 7), (0, 1), (1, 1), (1, 33)][int(rng.integers(0, 6))]
+        tail = int(rng.choice([0, 1, 3, 130]))
+        out.append((i, bs, f8, hkv, g, T, keep, tail))
+    return out
+
+
+@pytest.mark.parametrize("case", _cases_new(), ids=lambda c: f"{c[0]}-B{c[1]}-f8{c[2]}-h{c[3]}-g{c[4]}-T{c[5]}-k{c[6][0]}of{c[6][1]}-t{c[7]}")
+def test_random_block4_and_8bit_rows(case):
+    """The same sweep over the newer storage forms: blocks of four layers and / or 8-bit row streams (bf16, d = 128)."""
+    from oracle import fdkv_ref_b4 as R4
+    from oracle import fdkv_ref_fp8 as R8
+    from paper_2607_06519_b200 import runner
+
+    i, bs, f8, hkv, g, T, keep, tail = case
+    w = synth.Workload(name=f"rn{i}", n_layers=2 * bs, n_q_heads=hkv * g, n_kv_heads=hkv, head_dim=128, batch=1, T=T, dtype="bf16",
+                       keep_num=keep[0], keep_den=keep[1], n_needles=min(3, T), W=min(4, T), seed=300 + i, n_steps=max(tail, 1),
+                       block_size=bs, row_format=f8)
+    pf = runner.Prefilled(w, max_tail=max(tail, 1))
+    rng = np.random.default_rng(i)
+    modes = rng.integers(0, 3, (w.n_blocks, hkv)).astype(np.int32)
+    pf.prefill(0, modes=modes)
+    units = {}
+    for b in range(w.n_blocks):
+        for h in range(hkv):
+            if bs == 4:
+                ks, vs = synth.block_tensor(w, 0, b, h, False), synth.block_tensor(w, 0, b, h, True)
+                units[(b, h)] = R8.Unit4Fp8(ks, vs, True, *keep) if f8 else R4.Unit4(ks, vs, True, *keep)
+            else:
+                k0, k1 = synth.unit_tensor(w, 0, b, h, False)
+                v0, v1 = synth.unit_tensor(w, 0, b, h, True)
+                units[(b, h)] = R8.UnitFp8(k0, k1, v0, v1, True, *keep)
+    steps = [0] if tail == 0 else list(range(tail))
+    check_at = {0, 1, 2, tail - 1}
+    for step in steps:
+        for layer in range(w.n_layers):
+            b, lb = divmod(layer, bs)
+            q = pf.decode_q(layer, step)
+            kn = vn = None
+            if tail:
+                kn, vn = pf.new_rows(layer, step)
+                for h in range(hkv):
+                    units[(b, h)].append(lb, f32(kn)[0, h], f32(vn)[0, h])
+            out = pf.ctx.decode_attn(layer, q, kn, vn, out_dtype=0)
+            if step in check_at:
+                torch.cuda.synchronize()
+                for h in range(hkv):
+                    ref = units[(b, h)].attend(int(modes[b][h]), lb, f32(q)[0][h * g:(h + 1) * g])
+                    err = vector_errors(f32(out)[0][h * g:(h + 1) * g], ref).max()
+                    assert err <= TOL["bf16"], (step, layer, h, float(err))
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
