@@ -388,7 +388,16 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     }
                 }
             };
-            load_q(true);
+            if constexpr (F8) {
+                load_q(true);
+            } else {  // (kept inline for the bf16 kernel: routing it through the lambda cost 0.5 %)
+                const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.Hq + h * a.G + qcol) * 128;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    qb[kk][0] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 2 * tig) : 0u;
+                    qb[kk][1] = qcol < a.G ? *reinterpret_cast<const uint32_t*>(qh + 16 * kk + 8 + 2 * tig) : 0u;
+                }
+            }
             // O^T[channel][column]: eight 16-channel m-tiles; this thread holds columns 2 tig, 2 tig + 1
             float oacc[8][4];
 #pragma unroll
@@ -590,7 +599,26 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     __syncwarp();
                     store_o(false, true, f_tl[0], f_tl[1]);
                 } else {
-                    store_o(F8, false, 1.f, 1.f);
+                    if constexpr (F8) {
+                        store_o(true, false, 1.f, 1.f);
+                    } else {
+#pragma unroll
+                        for (int jm = 0; jm < 8; ++jm) {
+                            float v[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                v[i] = oacc[jm][i];
+                                if (split) v[i] += __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
+                            }
+                            if (!split || tig < 2) {
+                                const int ch = 16 * jm + gid, col = 2 * tig;
+                                scratch_f[col * 128 + ch] = v[0];
+                                scratch_f[(col + 1) * 128 + ch] = v[1];
+                                scratch_f[col * 128 + ch + 8] = v[2];
+                                scratch_f[(col + 1) * 128 + ch + 8] = v[3];
+                            }
+                        }
+                    }
                 }
                 if (gid == 0) {
 #pragma unroll
