@@ -158,6 +158,7 @@ __device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
 // Bounded wait on an mbarrier phase.  Gives up after kSpinCap polls (or as soon as another thread gave up):
 // raises the CTA abort flag and the device status word, after which every wait returns at once.
 __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return;  // the common case: one poll, no look at the abort flag
     if (*abort_flag) return;
     for (uint32_t i = 0; i < kSpinCap; ++i) {
         if (mbar_try_wait(bar, parity)) return;
