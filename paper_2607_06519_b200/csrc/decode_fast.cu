@@ -243,18 +243,11 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     Seg* const segs = reinterpret_cast<Seg*>(smem_raw + kOffSeg);
     int* const seg_info = reinterpret_cast<int*>(smem_raw + kOffSegInfo);  // [0] segments, [1] tiles in total
     int* const stage_cnt = reinterpret_cast<int*>(smem_raw + kOffCnt);
-    auto issue_tile = [&](int it) {
-        int si = 0;
-        while (si + 1 < seg_info[0] && it >= segs[si + 1].it0) ++si;
-        const Seg g = segs[si];
-        const int j = it - g.it0;
-        const int tile = rev ? g.tb + g.npre - 1 - j : g.tb + j;
-        const int kr = j < g.npre ? g.krow + tile * kTT : g.tkrow + (j - g.npre) * kTT;
-        const int vr = j < g.npre ? g.vrow + tile * kTT : g.tvrow + (j - g.npre) * kTT;
+    auto issue_rows = [&](int it, int kr, int vr, bool f8_box) {
         const int s = it % kStages;
         const uint32_t full = smem0 + kOffFull + 8 * s;
         const uint32_t dst = stage0 + s * kStageBytes;
-        if (F8 && j < g.npre) {  // one 128-token x 128-byte box per tensor, in the first half of the K and of the V slot
+        if (F8 && f8_box) {  // one 128-token x 128-byte box per tensor, in the first half of the K and of the V slot
             mbar_expect_tx(full, 2 * kHalfBytes);
             tma_load_2d(dst, &tmap8, 0, kr, full);
             tma_load_2d(dst + 2 * kHalfBytes, &tmap8, 0, vr, full);
@@ -265,6 +258,16 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             tma_load_2d(dst + 2 * kHalfBytes, &tmap, 0, vr, full);
             tma_load_2d(dst + 3 * kHalfBytes, &tmap, 64, vr, full);
         }
+    };
+    auto issue_tile = [&](int it) {
+        int si = 0;
+        while (si + 1 < seg_info[0] && it >= segs[si + 1].it0) ++si;
+        const Seg g = segs[si];
+        const int j = it - g.it0;
+        const int tile = rev ? g.tb + g.npre - 1 - j : g.tb + j;
+        const int kr = j < g.npre ? g.krow + tile * kTT : g.tkrow + (j - g.npre) * kTT;
+        const int vr = j < g.npre ? g.vrow + tile * kTT : g.tvrow + (j - g.npre) * kTT;
+        issue_rows(it, kr, vr, j < g.npre);
     };
     // a warp is done reading stage s (tile it): the last of the eight refills it
     auto release_stage = [&](int s, int it) {
@@ -531,6 +534,27 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                 }
             }
 
+            // A warp is done reading stage s (tile j of this segment): the last of the eight refills it.  Three tiles ahead
+            // is usually still a packed tile of this segment, whose rows follow from registers; only across a segment
+            // boundary (or into the tails) the segment table is walked.  The refill sits on the critical path of the ring.
+            const int unit_kr = (int)((reinterpret_cast<uint64_t>(ud.k_rows) - arena) >> (F8 ? 7 : 8));
+            const int unit_vr = (int)((reinterpret_cast<uint64_t>(ud.v_rows) - arena) >> (F8 ? 7 : 8));
+            auto release_here = [&](int s, int j) {
+                __syncwarp();
+                if (lane == 0) {
+                    const int old = atomicAdd(stage_cnt + s, 1);
+                    if (old == kCW - 1) {
+                        stage_cnt[s] = 0;
+                        const int jn = j + kStages;
+                        if (jn < npre) {
+                            const int tn = rev ? tb + npre - 1 - jn : tb + jn;
+                            issue_rows(it + jn, unit_kr + tn * kTT, unit_vr + tn * kTT, true);
+                        } else if (it + jn < seg_info[1]) {
+                            issue_tile(it + jn);
+                        }
+                    }
+                }
+            };
             // O[head][channel] into the warp's float scratch: column g plus (G <= 4) its remainder column g + 4, held by the
             // lane two over.  Rows gid / gid + 8 of an m-tile are channels gid and gid + 8, or (8-bit tiles) 2 gid and
             // 2 gid + 1, whose code sums are still to be multiplied by the channel's V scale.
