@@ -243,8 +243,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     Seg* const segs = reinterpret_cast<Seg*>(smem_raw + kOffSeg);
     int* const seg_info = reinterpret_cast<int*>(smem_raw + kOffSegInfo);  // [0] segments, [1] tiles in total
     int* const stage_cnt = reinterpret_cast<int*>(smem_raw + kOffCnt);
-    auto issue_rows = [&](int it, int kr, int vr, bool f8_box) {
-        const int s = it % kStages;
+    auto issue_rows = [&](int s, int kr, int vr, bool f8_box) {  // s = the tile's stage (its index in the CTA's sequence mod kStages)
         const uint32_t full = smem0 + kOffFull + 8 * s;
         const uint32_t dst = stage0 + s * kStageBytes;
         if (F8 && f8_box) {  // one 128-token x 128-byte box per tensor, in the first half of the K and of the V slot
@@ -267,7 +266,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         const int tile = rev ? g.tb + g.npre - 1 - j : g.tb + j;
         const int kr = j < g.npre ? g.krow + tile * kTT : g.tkrow + (j - g.npre) * kTT;
         const int vr = j < g.npre ? g.vrow + tile * kTT : g.tvrow + (j - g.npre) * kTT;
-        issue_rows(it, kr, vr, j < g.npre);
+        issue_rows(it % kStages, kr, vr, j < g.npre);
     };
     // a warp is done reading stage s (tile it): the last of the eight refills it
     auto release_stage = [&](int s, int it) {
@@ -542,13 +541,13 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             auto release_here = [&](int s, int j) {
                 __syncwarp();
                 if (lane == 0) {
-                    const int old = atomicAdd(stage_cnt + s, 1);
+                    // (atomicInc wraps the counter back to zero at the eighth arrival; tile j + kStages reuses stage s)
+                    const unsigned old = atomicInc(reinterpret_cast<unsigned*>(stage_cnt) + s, kCW - 1);
                     if (old == kCW - 1) {
-                        stage_cnt[s] = 0;
                         const int jn = j + kStages;
                         if (jn < npre) {
                             const int tn = rev ? tb + npre - 1 - jn : tb + jn;
-                            issue_rows(it + jn, unit_kr + tn * kTT, unit_vr + tn * kTT, true);
+                            issue_rows(s, unit_kr + tn * kTT, unit_vr + tn * kTT, true);
                         } else if (it + jn < seg_info[1]) {
                             issue_tile(it + jn);
                         }
