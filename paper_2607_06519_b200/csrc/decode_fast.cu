@@ -52,8 +52,9 @@ static_assert(kTT == kRowPad, "row blocks are padded to whole stages");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct FastSched {
-    uint32_t start[kMaxCtas + 1];  // unit << 20 | first 64-token tile of CTA c; start[ncta] = units << 20
+    uint32_t start[kMaxCtas + 1];  // unit << 20 | first 16-token slice of CTA c; start[ncta] = units << 20
     int ncta, units, tslot, prologue_tiles, reverse_odd, experiment;
+    int any_tail;  // some sequence of the batch holds generated tokens in this layer's tail (host mirror)
 };
 struct PartCount {
     uint8_t n[kMaxUnits];  // split-K parts per unit (at most kMaxSplits)
@@ -66,7 +67,9 @@ constexpr int kOffFull = 0, kOffAbort = 128, kOffTicket = 132, kOffM = 256, kOff
 // one (unit, tile range) segment of a CTA: arena rows of its K / V boxes and tail, first tile, prefill tiles, first
 // index in the CTA's tile sequence, and the sequence / head whose tail it also streams (or -1)
 struct Seg {
-    int krow, vrow, tkrow, tvrow, tb, npre, it0, tail_b, tail_h;
+    int krow, vrow, tkrow, tvrow;
+    int tb, rows16, npre;  // first token of the range, its tokens rounded up to 16, its 128-token tiles (the last may be partial)
+    int it0, tail_u;       // first tile in the CTA's sequence; the unit whose tail follows the range, or -1
 };
 static_assert(kMaxSeg * sizeof(Seg) <= 896, "segment table fits its header slot");
 
@@ -263,9 +266,11 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         while (si + 1 < seg_info[0] && it >= segs[si + 1].it0) ++si;
         const Seg g = segs[si];
         const int j = it - g.it0;
-        const int tile = rev ? g.tb + g.npre - 1 - j : g.tb + j;
-        const int kr = j < g.npre ? g.krow + tile * kTT : g.tkrow + (j - g.npre) * kTT;
-        const int vr = j < g.npre ? g.vrow + tile * kTT : g.tvrow + (j - g.npre) * kTT;
+        // ranges start on any 16-token slice and their tiles count from there; the box of the partial tile that ends a
+        // range is moved back over rows the CTA has read already (masked when used), so that no copy passes the range's end
+        const int tok = max(0, g.tb + min((rev ? g.npre - 1 - j : j) * kTT, g.rows16 - kTT));
+        const int kr = j < g.npre ? g.krow + tok : g.tkrow + (j - g.npre) * kTT;
+        const int vr = j < g.npre ? g.vrow + tok : g.tvrow + (j - g.npre) * kTT;
         issue_rows(it % kStages, kr, vr, j < g.npre);
     };
     // a warp is done reading stage s (tile it): the last of the eight refills it
@@ -286,20 +291,20 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         for (int u = u_first; u <= u_last && u < sch.units; ++u) {
             const int b = u / a.Hkv, h = u % a.Hkv;
             const UnitDesc* ud = a.desc + ((int64_t)b * a.L + a.layer) * a.Hkv + h;
-            const int ntiles = (ud->T + kTT - 1) / kTT;
-            const int tb = u == u_first ? t_first : 0;
-            const int te = u == u_last ? t_last : ntiles;
-            if (te <= tb) continue;
+            const int nsl = (ud->T + kResTile - 1) / kResTile;
+            const int sb = u == u_first ? t_first : 0;
+            const int se = u == u_last ? t_last : nsl;
+            if (se <= sb) continue;
             if (n == kMaxSeg) { atomicMax(a.status, (int32_t)kFlagCountMismatch); break; }  // cannot happen: see the launcher
             Seg g;
             g.krow = (int)((reinterpret_cast<uint64_t>(ud->k_rows) - arena) >> (F8 ? 7 : 8));  // rows of 128 or 256 bytes
             g.vrow = (int)((reinterpret_cast<uint64_t>(ud->v_rows) - arena) >> (F8 ? 7 : 8));
             g.tkrow = g.tvrow = 0;
-            g.tb = tb;
-            g.npre = te - tb;
+            g.tb = sb * kResTile;
+            g.rows16 = (min(se, nsl) - sb) * kResTile;
+            g.npre = (g.rows16 + kTT - 1) / kTT;
             g.it0 = it0;
-            g.tail_b = te == ntiles ? b : -1;  // this CTA also streams the unit's tail (length known after the wait)
-            g.tail_h = h;
+            g.tail_u = se == nsl ? u : -1;  // this CTA also streams the unit's tail (length known after the wait)
             segs[n++] = g;
             it0 += g.npre;
         }
@@ -313,18 +318,25 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     // per-warp scratch starts zeroed
     for (int i = threadIdx.x; i < kCW * kScratchBytes / 16; i += kThreads)
         st_shared_zero16(smem0 + kHeaderBytes + kStages * kStageBytes + i * 16);
+    __syncthreads();  // barriers initialised, static table built (still inside the previous kernel's shadow)
     // everything below may depend on the kernels launched before this one (q, appended tail rows, partial slots)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     TGLOBAL(1);
+    if (!sch.any_tail) {
+        // no tails anywhere: the static table is final; a short first segment may have left stages to fill
+        if (is_producer)
+            for (int it = prologue_issued; it < kStages && it < seg_info[1]; ++it) issue_tile(it);
+    } else {
     if (is_producer) {
         // tails: rows and lengths may have been written by the kernel right before this one
         int it0 = 0;
         for (int i = 0; i < seg_info[0]; ++i) {
             Seg g = segs[i];
             g.it0 = it0;
-            if (g.tail_b >= 0) {
-                const int n = min(a.tail_len[a.layer * a.max_batch + g.tail_b], a.max_tail);
-                const int64_t o = (((int64_t)a.layer * a.max_batch + g.tail_b) * a.Hkv + g.tail_h) * a.tail_rows;
+            if (g.tail_u >= 0) {
+                const int tail_b = g.tail_u / a.Hkv, tail_h = g.tail_u % a.Hkv;
+                const int n = min(a.tail_len[a.layer * a.max_batch + tail_b], a.max_tail);
+                const int64_t o = (((int64_t)a.layer * a.max_batch + tail_b) * a.Hkv + tail_h) * a.tail_rows;
                 g.tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
                 g.tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
                 it0 += (n + kTT - 1) / kTT;
@@ -336,6 +348,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         for (int it = prologue_issued; it < kStages && it < it0; ++it) issue_tile(it);  // nobody computes yet: fill every stage
     }
     __syncthreads();
+    }
 
     // ================= compute: every warp takes 16 tokens of every stage =================
     {
@@ -353,19 +366,20 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             const int b = u / a.Hkv, h = u % a.Hkv;
             const UnitDesc ud = a.desc[((int64_t)b * a.L + a.layer) * a.Hkv + h];
             const int T = ud.T;
-            const int ntiles = (T + kTT - 1) / kTT;
-            const int tb = u == u_first ? t_first : 0;
-            const int te = u == u_last ? t_last : ntiles;
-            if (te <= tb) continue;
+            const int nres = (T + kResTile - 1) / kResTile;
+            const int sb = u == u_first ? t_first : 0;
+            const int se = u == u_last ? t_last : nres;
+            if (se <= sb) continue;
+            // this CTA's tokens of the unit: [tok_b, tok_e), cut on 16-token slices; 128-token tiles count from tok_b
+            const int tok_b = sb * kResTile, tok_e = min(se * kResTile, T), rows16 = (se - sb) * kResTile;
             int ntail = 0, n_tail_rows = 0;
-            if (te == ntiles) {
+            if (sch.any_tail && se == nres) {
                 n_tail_rows = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
                 ntail = (n_tail_rows + kTT - 1) / kTT;
             }
-            const int npre = te - tb, nseg = npre + ntail;
+            const int npre = (rows16 + kTT - 1) / kTT, nseg = npre + ntail;
             const bool coef = ud.mode != FDKV_MODE_EXACT, resid = ud.mode == FDKV_MODE_RESIDUAL && sch.experiment != 5;  // (experiment 5: no residual work)
             const uint32_t sgn = ud.sign < 0.f ? 0x80008000u : 0u;
-            const int nres = (T + kResTile - 1) / kResTile;
 
             // q fragments: B operand columns = the G query heads of this KV head.  With G <= 4 columns 4-7 repeat
             // them: in the second product those columns carry the bf16 rounding remainder of P, so P acts in ~16 bits.
@@ -435,8 +449,10 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                 const int jj = jb + lane;
                 k[0] = k[1] = v[0] = v[1] = 0;
                 if (resid && jj < npre) {
-                    const int o = (rev ? tb + npre - 1 - jj : tb + jj) * (kTT / kResTile) + warp;
-                    const int o0 = min(o, nres), o1 = min(o + 1, nres);
+                    // the tile's slices not yet read: [first, se); the box may start before them (see issue_tile)
+                    const int first = sb + (rev ? npre - 1 - jj : jj) * (kTT / kResTile);
+                    const int o = max(0, min(first, se - kTT / kResTile)) + warp;
+                    const int o0 = min(max(o, first), se), o1 = min(max(o + 1, first), se);
                     k[0] = ud.k_off[o0]; k[1] = ud.k_off[o1];
                     if (tokmode) { v[0] = k[0]; v[1] = k[1]; }
                     else { v[0] = ud.v_off[o0]; v[1] = ud.v_off[o1]; }
@@ -546,8 +562,8 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     if (old == kCW - 1) {
                         const int jn = j + kStages;
                         if (jn < npre) {
-                            const int tn = rev ? tb + npre - 1 - jn : tb + jn;
-                            issue_rows(s, unit_kr + tn * kTT, unit_vr + tn * kTT, true);
+                            const int tok = max(0, tok_b + min((rev ? npre - 1 - jn : jn) * kTT, rows16 - kTT));
+                            issue_rows(s, unit_kr + tok, unit_vr + tok, true);
                         } else if (it + jn < seg_info[1]) {
                             issue_tile(it + jn);
                         }
@@ -867,16 +883,33 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     FastSched sch;
     PartCount cs;
     std::vector<int64_t> wp(units + 1, 0);
-    std::vector<int> nt(units), wt(units);
+    // ranges are cut on 16-token slices (the granularity of the residual lists), so that the CTAs of a unit differ by
+    // at most one slice; each range is streamed as 128-token tiles from its first slice, the last one partial
+    std::vector<int> nt(units), ns(units), wt(units);  // 128-token tiles, 16-token slices, cost per tile
     int64_t total_tiles = 0;
     for (int u = 0; u < units; ++u) {
         const int T = a.host_T[u / a.Hkv];
         nt[u] = (T + kTT - 1) / kTT;
-        if (nt[u] >= (1 << 20)) return cudaErrorInvalidValue;  // cannot happen: T * 128 < 2^31
+        ns[u] = (T + kResTile - 1) / kResTile;
+        if (ns[u] >= (1 << 20)) return cudaErrorInvalidValue;  // cannot happen: T * 128 < 2^31
         total_tiles += nt[u];
     }
     // cost per tile: bytes in units of 512 B (the K and V boxes, plus the lists' share for residual units), residual
     // tiles scaled by the measured ratio of their compute time to a plain tile's (rc)
+    // With whole CTAs per unit (latency-bound regime) a residual tile of the entry form costs a fixed part (the scratch
+    // tile and the second products) plus a part per list entry: measured 2.0 plain tiles at 1024 entries per tile and
+    // tensor (keep 1/16), 1.65 at 512 (keep 1/32); with 8-bit rows (a dearer plain tile) about 1.7 at either density.
+    static double res_a_env = -1.0, res_b_env = -1.0;
+    static bool res_ab_read = false;
+    if (!res_ab_read) {
+        const char* ea = getenv("FDKV_RES_A");  // tuning knobs for benchmark sweeps
+        const char* eb = getenv("FDKV_RES_B");
+        if (ea) res_a_env = atof(ea);
+        if (eb) res_b_env = atof(eb);
+        res_ab_read = true;
+    }
+    const double res_a = res_a_env >= 0 ? res_a_env : a.rows_f8 ? 1.55 : 1.25;
+    const double res_b = res_b_env >= 0 ? res_b_env : a.rows_f8 ? 0.15 : 0.87;
     auto weigh = [&](double rc) {
         for (int u = 0; u < units; ++u) {
             const int T = a.host_T[u / a.Hkv];
@@ -884,13 +917,14 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
             wt[u] = 2 * kTT * 256 / 512;
             if (a.host_modes[u] == FDKV_MODE_RESIDUAL) {
                 const int64_t res_bytes = a.tok_rule ? 2 * ((int64_t)T * a.keep_num / a.keep_den) * 260 : 2 * k * 4;  // rows + index, or packed entries
-                wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * rc);
+                if (rc == 0.0) wt[u] = (int)(wt[u] * (res_a + res_b * (double)k / nt[u] / 1024.0));
+                else wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * rc);
             }
-            wp[u + 1] = wp[u] + (int64_t)nt[u] * wt[u];
+            wp[u + 1] = wp[u] + (int64_t)ns[u] * wt[u];  // (in eighths of the tile cost)
         }
     };
     // (measured best: 1.7 when every unit gets whole CTAs, 1.5 in the flat cut of a batch)
-    weigh(res_cost_env ? res_cost : 1.7);
+    weigh(res_cost_env ? res_cost : a.tok_rule ? 1.7 : 0.0);
     const int ncta = (int)std::min<int64_t>(std::min(std::min(sm_count, kMaxCtas), kMaxSplits), total_tiles);
     static unsigned g_launch_no = 0;
     ++g_launch_no;
@@ -898,6 +932,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     sch.ncta = ncta;
     sch.prologue_tiles = prologue_tiles;
     sch.reverse_odd = reverse_odd ? 1 : 0;
+    sch.any_tail = a.any_tail;
     { const char* ex = getenv("FDKV_DECODE_EXPERIMENT"); sch.experiment = ex ? atoi(ex) : 0; }
     sch.units = units;
     bool whole = whole_ctas && units <= ncta;
@@ -931,7 +966,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     if (whole) {
         int c = 0;
         for (int u = 0; u < units; ++u)
-            for (int j = 0; j < nc[u]; ++j) sch.start[c++] = ((uint32_t)u << 20) | (uint32_t)((int64_t)nt[u] * j / nc[u]);
+            for (int j = 0; j < nc[u]; ++j) sch.start[c++] = ((uint32_t)u << 20) | (uint32_t)((int64_t)ns[u] * j / nc[u]);
         sch.start[ncta] = (uint32_t)units << 20;
     } else {
         if (!res_cost_env) weigh(1.5);
@@ -939,8 +974,8 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         for (int c = 0; c < ncta; ++c) {
             const int64_t target = wp[units] * c / ncta;
             while (u + 1 < units && wp[u + 1] <= target) ++u;
-            const int tile = (int)((target - wp[u]) / wt[u]);
-            sch.start[c] = ((uint32_t)u << 20) | (uint32_t)tile;
+            const int slice = (int)((target - wp[u]) / wt[u]);
+            sch.start[c] = ((uint32_t)u << 20) | (uint32_t)slice;
         }
         sch.start[ncta] = (uint32_t)units << 20;
     }
@@ -951,7 +986,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         const int ub = (int)(sch.start[c + 1] >> 20), tb = (int)(sch.start[c + 1] & 0xFFFFFu);
         int nseg_cta = 0;
         for (int u = ua; u <= ub && u < units; ++u) {
-            const int b0 = u == ua ? ta : 0, b1 = u == ub ? tb : nt[u];
+            const int b0 = u == ua ? ta : 0, b1 = u == ub ? tb : ns[u];
             if (b1 > b0) ++nseg_cta;
             if (b1 > b0 && cs.n[u] < 255) cs.n[u]++;
         }

@@ -83,6 +83,8 @@ def test_tiny_compress_probe_decode(dtype):
     ("f32", 96, 128, 8, 1, (0, 1), 1),      # keep nothing: residual == shared
     ("bf16", 100, 64, 8, 1, (1, 1), 0),     # keep everything, G = 8
     ("bf16", 2100, 128, 4, 1, (1, 32), 40), # several splits, tail longer than a tile
+    ("bf16", 5003, 128, 8, 2, (1, 16), 2),  # CTA ranges cut on 16-token slices: partial last tiles, T not a multiple of 16
+    ("bf16", 9000, 128, 12, 3, (1, 8), 3),  # three units, ranges of a few slices over one tile, dense lists
 ])
 def test_shapes_and_edges(dtype, T, d, Hq, Hkv, keep, tail):
     runner = _runner()
