@@ -99,7 +99,10 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.io_v = take((size_t)s.L * s.max_batch * s.Hkv * s.d * 4);
     w.io_out = take((size_t)s.L * s.max_batch * s.Hq * s.d * 4);
     // job tables of the 8-bit commit: one quantise job per stored tensor, one repack job per residual list
-    w.jobs = take(s.rows_f8 ? (size_t)s.NU * 2 * s.B * (sizeof(QuantJob) + sizeof(RepackJob)) : 0);
+    // job tables of a commit: quantise / repack jobs (8-bit rows), then the copy jobs (at most 2 B row copies, or 2 row
+    // copies, 2 offset tables and 2 NB lists, per unit)
+    w.jobs = take((s.rows_f8 ? (size_t)s.NU * 2 * s.B * (sizeof(QuantJob) + sizeof(RepackJob)) : 0) +
+                  (size_t)s.NU * (2 * s.B + 4 + 2 * s.NB) * sizeof(CopyJob));
     w.total = o;
 
     o = 0;
@@ -522,6 +525,12 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
     const size_t unit_stride_b = (size_t)s.Tmax * s.d * s.esize;
     std::vector<QuantJob> qjobs;   // 8-bit rows: every stored tensor is quantised by one batched pass after this loop
     std::vector<RepackJob> rjobs;  // ... and every residual list repacked relative to its tensor's scales
+    std::vector<CopyJob> cjobs;    // device-to-device copies into the arena: one launch over this table after the loop
+    int64_t copy_max = 0;
+    auto copy_job = [&](const void* src, void* dst, size_t bytes, int64_t src_pitch, int row_bytes) {
+        cjobs.push_back(CopyJob{(const char*)src, (char*)dst, (int64_t)bytes, src_pitch, row_bytes, 0});
+        copy_max = std::max<int64_t>(copy_max, (int64_t)bytes);
+    };
     for (int u = 0; u < s.NU; ++u) {
         const int m = q.modes[u], p = u / s.Hkv, h = u % s.Hkv;
         UnitDesc* dl[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -550,7 +559,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                     }
                     char* dst = take(rows_pad);
                     if (rows_pad > rows) CU(cudaMemsetAsync(dst + rows, 0, rows_pad - rows, st));
-                    CU(launch_strided_copy(sp, c->stride_t, dst, T, s.d, s.esize, st));
+                    copy_job(sp, dst, rows, (int64_t)c->stride_t * s.esize, s.d * s.esize);
                     (is_v ? dl[l]->v_rows : dl[l]->k_rows) = dst;
                 }
             by_mode[2] += 2 * (size_t)s.B * (s.rows_f8 ? rows8 + 512 : rows);
@@ -576,7 +585,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 } else {
                     z0 = take(rows_pad);
                     if (rows_pad > rows) CU(cudaMemsetAsync(z0 + rows, 0, rows_pad - rows, st));
-                    CU(cudaMemcpyAsync(z0, c->work + c->ws.z0 + ut * unit_stride_b, rows, cudaMemcpyDeviceToDevice, st));
+                    copy_job(c->work + c->ws.z0 + ut * unit_stride_b, z0, rows, 16, 16);
                 }
                 for (int l = 0; l < s.B; ++l) (is_v ? dl[l]->v_rows : dl[l]->k_rows) = z0;
                 by_mode[m] += s.rows_f8 ? rows8 + 512 : rows;
@@ -593,7 +602,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                     by_mode[1] += (size_t)k_tok * s.d * s.esize;
                 } else if (m == FDKV_MODE_RESIDUAL) {
                     char* po = take(off_b);
-                    CU(cudaMemcpyAsync(po, c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, off_copy, cudaMemcpyDeviceToDevice, st));
+                    copy_job(c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, po, off_copy, 16, 16);
                     char* pi_shared = nullptr;
                     if (!c->packed_lists) {
                         pi_shared = take(idx_b);
@@ -607,7 +616,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                             if (s.rows_f8)  // values relative to the channel scales, positions in the converted fragments' order
                                 rjobs.push_back(RepackJob{reinterpret_cast<uint32_t*>(pi_l[j]), wsp<uint32_t>(c, c->ws.packed) + lt * s.kcap, k, sc8, is_v, 0});
                             else
-                                CU(cudaMemcpyAsync(pi_l[j], c->work + c->ws.packed + lt * s.kcap * 4, idx_copy, cudaMemcpyDeviceToDevice, st));
+                                copy_job(c->work + c->ws.packed + lt * s.kcap * 4, pi_l[j], idx_copy, 16, 16);
                         } else {
                             pi_l[j] = pi_shared;
                             pv_l[j] = take(val_b);
@@ -625,6 +634,11 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 }
             }
         }
+    }
+    if (!cjobs.empty()) {
+        CopyJob* cd = reinterpret_cast<CopyJob*>(c->work + c->ws.jobs + (s.rows_f8 ? (size_t)s.NU * 2 * s.B * (sizeof(QuantJob) + sizeof(RepackJob)) : 0));
+        CU(cudaMemcpyAsync(cd, cjobs.data(), cjobs.size() * sizeof(CopyJob), cudaMemcpyHostToDevice, st));
+        CU(launch_copy_jobs(cd, (int)cjobs.size(), copy_max, st));
     }
     if (!qjobs.empty()) {
         QuantJob* qd = reinterpret_cast<QuantJob*>(c->work + c->ws.jobs);

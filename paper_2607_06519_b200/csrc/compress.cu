@@ -356,7 +356,7 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
             // rank of this lane's first tie among the unit-tensor's ties
             uint32_t keep = is_gt;
             const uint32_t any_eq = __ballot_sync(0xFFFFFFFFu, is_eq != 0);
-            if (any_eq) {
+            if (any_eq && eq_rank < need) {  // (ties are kept in index order: once `need` of them lie before this point, none is)
                 const uint32_t n_eq = __popc(is_eq);
                 uint32_t incl = n_eq;
 #pragma unroll
@@ -469,6 +469,36 @@ cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream
             tile_write_kernel<float><<<grid, 256, 0, st>>>(a);
         count_launch(3);
     }
+    return cudaGetLastError();
+}
+
+// grid (chunks of 32 KiB, jobs): the device-to-device copies of a commit (row streams, strided source rows of exact
+// units, residual lists, offset tables) as one launch instead of several hundred copy calls
+constexpr int kCopyChunk = 32 * 1024;
+__global__ void __launch_bounds__(256) copy_jobs_kernel(const CopyJob* jobs) {
+    const CopyJob jb = jobs[blockIdx.y];
+    const int64_t c0 = (int64_t)blockIdx.x * kCopyChunk;
+    if (c0 >= jb.bytes) return;
+    const int64_t c1 = min(jb.bytes, c0 + kCopyChunk);
+    const bool plain = jb.src_pitch == jb.row_bytes;
+    auto src_of = [&](int64_t o) {
+        if (plain) return o;
+        const int64_t r = o / jb.row_bytes;
+        return r * jb.src_pitch + (o - r * jb.row_bytes);
+    };
+    // 16-byte vectors when both sides allow it (offset tables of later unit-tensors start on 4-byte boundaries only)
+    const bool vec_ok = (((uintptr_t)jb.src | (uintptr_t)jb.dst) & 15) == 0;
+    const int64_t v1 = vec_ok ? (c1 & ~(int64_t)15) : c0;
+#pragma unroll 4
+    for (int64_t o = c0 + threadIdx.x * 16; o < v1; o += 256 * 16)
+        *reinterpret_cast<uint4*>(jb.dst + o) = *reinterpret_cast<const uint4*>(jb.src + src_of(o));
+    for (int64_t o = v1 + threadIdx.x * 4; o < c1; o += 256 * 4)
+        *reinterpret_cast<uint32_t*>(jb.dst + o) = *reinterpret_cast<const uint32_t*>(jb.src + src_of(o));
+}
+cudaError_t launch_copy_jobs(const CopyJob* jobs_dev, int njobs, int64_t bytes_max, cudaStream_t st) {
+    if (njobs <= 0 || bytes_max <= 0) return cudaSuccess;
+    copy_jobs_kernel<<<dim3((unsigned)((bytes_max + kCopyChunk - 1) / kCopyChunk), njobs), 256, 0, st>>>(jobs_dev);
+    count_launch(1);
     return cudaGetLastError();
 }
 

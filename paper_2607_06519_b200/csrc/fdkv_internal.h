@@ -267,6 +267,17 @@ struct RepackJob {
     const float* scale;
     int32_t is_v, pad_;
 };
+// One copy of the commit step: dst[0, bytes) = consecutive rows of row_bytes taken every src_pitch bytes from src
+// (row_bytes == src_pitch: a plain copy).  Pointers 16-byte aligned, row_bytes and src_pitch multiples of 16, bytes a
+// multiple of 4.  All copies of a commit run as one launch over a job table.
+struct CopyJob {
+    const char* src;
+    char* dst;
+    int64_t bytes;
+    int64_t src_pitch;
+    int32_t row_bytes, pad_;
+};
+cudaError_t launch_copy_jobs(const CopyJob* jobs_dev, int njobs, int64_t bytes_max, cudaStream_t st);
 cudaError_t launch_quantise_jobs(const QuantJob* jobs_dev, int njobs, int T_max, cudaStream_t st);
 cudaError_t launch_repack_jobs(const RepackJob* jobs_dev, int njobs, int64_t n_max, cudaStream_t st);
 bool make_rows_tensor_map_u8(void* base, size_t bytes, int box_rows, void* tmap_out);
