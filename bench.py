@@ -32,10 +32,10 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES = {
-    # profiles/decode_fast_kernel_decode32k.md: 138.56 MB read + ~4.4 MB written per launch, captured on the 4-layer cut
+    # profiles/decode_fast_kernel_decode32k.md: 138.55 MB read + ~3.9 MB written per launch, captured on the 4-layer cut
     # (same 8 units and bytes per launch as the 32-layer workload)
-    "decode32k": 143.0e6,
-    "decode32k_4l": 143.0e6,
+    "decode32k": 142.4e6,
+    "decode32k_4l": 142.4e6,
 }
 
 
