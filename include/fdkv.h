@@ -251,6 +251,18 @@ fdkv_status fdkv_get_modes(fdkv_ctx* ctx, int32_t seq, int32_t* modes_host /*HOS
 /* Bytes a committed sequence holds in the arena per mode, and what the uncompressed cache would take. */
 fdkv_status fdkv_footprint(fdkv_ctx* ctx, int32_t seq, size_t* bytes_by_mode_host /*HOST [3]*/,
                            size_t* exact_equiv_bytes_host /*HOST*/);
+/* Host-only planning call (no GPU is touched; usable without a device): how a decode launch of the tensor-core kernel
+ * (bf16 storage, head_dim 128) would cut its work over `n_ctas` thread blocks.  The work list is every (sequence, KV
+ * head) unit's prefill tokens in 16-token slices, unit-major; a residual unit's slices weigh more (Method, the
+ * paragraph after Eq. 3: decode reconstructs per head mode, so the modes set the cost).  Inputs (HOST): T[batch] prefill
+ * lengths, modes[batch * n_kv_heads] of the layer's units.  Outputs (HOST): start_out[n_ctas + 1], block c handles the
+ * range [start_out[c], start_out[c+1]) where an entry is unit << 20 | slice and the last one is units << 20;
+ * *n_ctas_out <= n_ctas blocks are used; parts_out[batch * n_kv_heads] = split-K parts per unit (blocks whose range
+ * holds at least one of its slices).  Errors: FDKV_ERR_INVALID_ARG for null pointers, sizes out of range or more units
+ * than the kernel takes (1024).                                                                                      */
+fdkv_status fdkv_plan_decode(int32_t batch, int32_t n_kv_heads, const int32_t* T_host, const int32_t* modes_host,
+                             int32_t keep_num, int32_t keep_den, int32_t residual_rule, int32_t row_format, int32_t n_ctas,
+                             uint32_t* start_out, int32_t* n_ctas_out, int32_t* parts_out);
 /* Bytes the decode kernels read from the packed cache for one call of `layer` over `batch` sequences
  * (coefficient or exact rows, residual lists and their tile offsets, tails): the roofline numerator.      */
 fdkv_status fdkv_decode_bytes(fdkv_ctx* ctx, int32_t layer, int32_t batch, size_t* bytes_host /*HOST*/);

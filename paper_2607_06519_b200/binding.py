@@ -62,6 +62,7 @@ def _load():
         "fdkv_get_token_set": [vp, i32, i32, i32, vp, vp, P(i32), vp],
         "fdkv_footprint": [vp, i32, P(sz), P(sz)],
         "fdkv_decode_bytes": [vp, i32, i32, P(sz)],
+        "fdkv_plan_decode": [i32, i32, P(i32), P(i32), i32, i32, i32, i32, i32, P(C.c_uint32), P(i32), P(i32)],
         "fdkv_device_status": [vp],
         "fdkv_compress_unit_noalloc": [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, P(i32), vp],
     }
@@ -130,6 +131,25 @@ def _stream(stream) -> int:
 
 def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def plan_decode(T, modes, n_kv_heads: int, keep_num: int, keep_den: int, n_ctas: int, residual_rule: int = 0, row_format: int = 0):
+    """fdkv_plan_decode (host only): T = prefill length per sequence, modes = [batch][n_kv_heads] of the layer's units.
+    Returns (ranges, parts): ranges[c] = ((unit, slice) begin, (unit, slice) end) of thread block c, parts[u] = split-K
+    parts of unit u."""
+    batch = len(T)
+    t_arr = (C.c_int32 * batch)(*[int(t) for t in T])
+    flat = [int(m) for row in modes for m in row]
+    if len(flat) != batch * n_kv_heads:
+        raise ValueError("modes must be [batch][n_kv_heads]")
+    m_arr = (C.c_int32 * len(flat))(*flat)
+    start = (C.c_uint32 * (n_ctas + 1))()
+    used = C.c_int32(0)
+    parts = (C.c_int32 * len(flat))()
+    _check(_lib.fdkv_plan_decode(batch, n_kv_heads, t_arr, m_arr, keep_num, keep_den, residual_rule, row_format, n_ctas, start,
+                                 C.byref(used), parts), "fdkv_plan_decode")
+    pts = [(int(v) >> 20, int(v) & 0xFFFFF) for v in start[:used.value + 1]]
+    return [(pts[c], pts[c + 1]) for c in range(used.value)], list(parts)
 
 
 def compress_unit_noalloc(x0, x1, keep_num: int, keep_den: int, z0_out, idx_out, val_out, stream=None) -> int:

@@ -997,6 +997,26 @@ fdkv_status fdkv_footprint(fdkv_ctx* c, int32_t seq, size_t* bytes_by_mode_host,
     return FDKV_OK;
 }
 
+fdkv_status fdkv_plan_decode(int32_t batch, int32_t n_kv_heads, const int32_t* T_host, const int32_t* modes_host,
+                             int32_t keep_num, int32_t keep_den, int32_t residual_rule, int32_t row_format, int32_t n_ctas,
+                             uint32_t* start_out, int32_t* n_ctas_out, int32_t* parts_out) {
+    if (!T_host || !modes_host || !start_out || !n_ctas_out || !parts_out) return FDKV_ERR_INVALID_ARG;
+    if (batch < 1 || n_kv_heads < 1 || (int64_t)batch * n_kv_heads > kFastMaxUnits || n_ctas < 1 || n_ctas > 160) return FDKV_ERR_INVALID_ARG;
+    if (keep_num < 0 || keep_den < 1 || keep_num > keep_den) return FDKV_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b)
+        if (T_host[b] < 1 || (int64_t)T_host[b] * 128 >= ((int64_t)1 << 31)) return FDKV_ERR_INVALID_ARG;
+    for (int i = 0; i < batch * n_kv_heads; ++i)
+        if (modes_host[i] < 0 || modes_host[i] > 2) return FDKV_ERR_INVALID_ARG;
+    DecodeArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.batch = batch; a.Hkv = n_kv_heads; a.d = 128;
+    a.host_T = T_host; a.host_modes = modes_host;
+    a.keep_num = keep_num; a.keep_den = keep_den;
+    a.tok_rule = residual_rule == FDKV_RESIDUAL_TOKENS ? 1 : 0;
+    a.rows_f8 = row_format != 0 ? 1 : 0;
+    return plan_decode_host(a, n_ctas, start_out, n_ctas_out, parts_out) == cudaSuccess ? FDKV_OK : FDKV_ERR_INVALID_ARG;
+}
+
 fdkv_status fdkv_decode_bytes(fdkv_ctx* c, int32_t layer, int32_t batch, size_t* bytes_host) {
     if (!c || !bytes_host || layer < 0 || layer >= c->s.L || batch < 1 || batch > c->s.max_batch) return FDKV_ERR_INVALID_ARG;
     const Shape& s = c->s;

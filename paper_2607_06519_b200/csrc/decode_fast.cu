@@ -842,22 +842,9 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
     return make_rows_tensor_map(arena, arena_bytes, kTT, tmap_out);
 }
 
-cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handled) {
-    *handled = false;
-    const int units = a.batch * a.Hkv;
-    if (!a.tmap || !a.packed_lists || a.d != 128 || units > kMaxUnits || units < 1) return cudaSuccess;
-    if (a.rows_f8 && !a.tmap_u8) return cudaSuccess;
-    static int sm_count = 0;
-    static bool attr_done = false;
-    if (!attr_done) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+// Host side of a launch: the cost-weighted cut of the batch's (unit, 16-token slice) list into one range per CTA and the
+// split-K part count of every unit.  Uses only the host views in `a` (lengths, modes, shape); no device access.
+static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_count, FastSched& sch, PartCount& cs, bool& use_pdl_out) {
     static double res_cost = -1.0;
     static bool res_cost_env = false;
     static bool use_pdl = true;
@@ -881,8 +868,6 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
         prologue_tiles = pt ? std::max(0, std::min(kStages, atoi(pt))) : kStages;
     }
     // ---- cost-weighted schedule: whole CTAs per unit when there are enough CTAs, else a flat cut of the (unit, tile) list ----
-    FastSched sch;
-    PartCount cs;
     std::vector<int64_t> wp(units + 1, 0);
     // ranges are cut on 16-token slices (the granularity of the residual lists), so that the CTAs of a unit differ by
     // at most one slice; each range is streamed as 128-token tiles from its first slice, the last one partial
@@ -979,6 +964,21 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
             sch.start[c] = ((uint32_t)u << 20) | (uint32_t)slice;
         }
         sch.start[ncta] = (uint32_t)units << 20;
+        // A CTA's segment table holds kMaxSeg units: where the cost cut gives one CTA a longer run of very short units
+        // (a batch of one long and many one-token sequences), move whole units to its neighbours: first towards the
+        // front, then towards the back.  Ranges stay ordered; a CTA may end up without work.
+        auto nseg = [&](uint32_t s0, uint32_t s1) {
+            const int ua = (int)(s0 >> 20), ta = (int)(s0 & 0xFFFFFu), ub = (int)(s1 >> 20), tb = (int)(s1 & 0xFFFFFu);
+            int n = 0;
+            for (int u2 = ua; u2 <= ub && u2 < units; ++u2)
+                if ((u2 == ub ? tb : ns[u2]) > (u2 == ua ? ta : 0)) ++n;
+            return n;
+        };
+        for (int c = ncta - 1; c >= 1; --c)
+            while (nseg(sch.start[c], sch.start[c + 1]) > kMaxSeg) sch.start[c] = ((sch.start[c] >> 20) + 1) << 20;
+        for (int c = 0; c + 1 < ncta; ++c)
+            while (nseg(sch.start[c], sch.start[c + 1]) > kMaxSeg)
+                sch.start[c + 1] = (sch.start[c + 1] & 0xFFFFFu) ? (sch.start[c + 1] >> 20) << 20 : ((sch.start[c + 1] >> 20) - 1) << 20;
     }
     // parts per unit = CTAs whose range contains at least one of its tiles
     for (int u = 0; u < kMaxUnits; ++u) cs.n[u] = 0;
@@ -991,10 +991,53 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
             if (b1 > b0) ++nseg_cta;
             if (b1 > b0 && cs.n[u] < 255) cs.n[u]++;
         }
-        if (nseg_cta > kMaxSeg) return cudaErrorInvalidValue;  // more one-tile units per CTA than the segment table holds
+        if (nseg_cta > kMaxSeg) return cudaErrorInvalidValue;  // only when units > kMaxSeg * CTAs (see the pass above)
     }
     for (int u = 0; u < units; ++u)
         if (cs.n[u] > kMaxSplits) return cudaErrorInvalidValue;  // cannot happen: ncta <= kMaxSplits
+    use_pdl_out = use_pdl;
+    return cudaSuccess;
+}
+
+// The plan alone, for a given number of CTAs (fdkv_plan_decode: host only, no device is touched).
+cudaError_t plan_decode_host(const DecodeArgs& a, int n_ctas, uint32_t* start_out, int32_t* ncta_out, int32_t* parts_out) {
+    const int units = a.batch * a.Hkv;
+    if (units < 1 || units > kMaxUnits || n_ctas < 1) return cudaErrorInvalidValue;
+    FastSched sch;
+    PartCount cs;
+    bool pdl = true;
+    const cudaError_t e = plan_decode_schedule(a, units, n_ctas, sch, cs, pdl);
+    if (e != cudaSuccess) return e;
+    for (int c = 0; c <= sch.ncta; ++c) start_out[c] = sch.start[c];
+    for (int u = 0; u < units; ++u) parts_out[u] = cs.n[u];
+    *ncta_out = sch.ncta;
+    return cudaSuccess;
+}
+
+cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handled) {
+    *handled = false;
+    const int units = a.batch * a.Hkv;
+    if (!a.tmap || !a.packed_lists || a.d != 128 || units > kMaxUnits || units < 1) return cudaSuccess;
+    if (a.rows_f8 && !a.tmap_u8) return cudaSuccess;
+    static int sm_count = 0;
+    static bool attr_done = false;
+    if (!attr_done) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    FastSched sch;
+    PartCount cs;
+    bool use_pdl = true;
+    {
+        const cudaError_t pe = plan_decode_schedule(a, units, sm_count, sch, cs, use_pdl);
+        if (pe != cudaSuccess) return pe;
+    }
+    const int ncta = sch.ncta;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ncta);
     cfg.blockDim = dim3(kThreads);

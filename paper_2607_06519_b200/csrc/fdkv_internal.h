@@ -277,6 +277,7 @@ struct CopyJob {
     int64_t src_pitch;
     int32_t row_bytes, pad_;
 };
+cudaError_t plan_decode_host(const DecodeArgs& a, int n_ctas, uint32_t* start_out, int32_t* ncta_out, int32_t* parts_out);
 cudaError_t launch_copy_jobs(const CopyJob* jobs_dev, int njobs, int64_t bytes_max, cudaStream_t st);
 cudaError_t launch_quantise_jobs(const QuantJob* jobs_dev, int njobs, int T_max, cudaStream_t st);
 cudaError_t launch_repack_jobs(const RepackJob* jobs_dev, int njobs, int64_t n_max, cudaStream_t st);
