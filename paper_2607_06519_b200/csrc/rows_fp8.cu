@@ -15,48 +15,67 @@ namespace {
 
 constexpr int kD = 128;
 
-// All row streams of a commit are quantised by three launches over a job table (one job per stored tensor).
+// All row streams of a commit are quantised by four launches over a job table (one job per stored tensor).
 // grid (token chunks, jobs): per-channel maximum of |x| over the chunk, merged with atomicMax on the bit patterns
 // (non-negative floats order like their bits); the maxima live in the second half of the job's 1 KiB scale slot.
 __global__ void __launch_bounds__(128) zero_amax_kernel(const QuantJob* jobs) {
     reinterpret_cast<uint32_t*>(jobs[blockIdx.x].scale)[kD + threadIdx.x] = 0u;
 }
 __global__ void __launch_bounds__(256) absmax_kernel(const QuantJob* jobs, int rows_per_cta) {
-    __shared__ uint32_t s_max[2][kD];
+    __shared__ uint32_t s_max[16][kD];
     const QuantJob jb = jobs[blockIdx.y];
     const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(jb.src);
-    const int c = threadIdx.x & (kD - 1), half = threadIdx.x >> 7;
+    // a thread takes 8 channels (16 bytes) of every 16th row of the chunk
+    const int c8 = (threadIdx.x & 15) * 8, rg = threadIdx.x >> 4;
     const int t0 = blockIdx.x * rows_per_cta, t1 = min(jb.T, t0 + rows_per_cta);
     if (t0 >= jb.T) return;
-    uint32_t m = 0;
-    for (int t = t0 + half; t < t1; t += 2) {
-        const uint32_t b = (uint32_t)__bfloat16_as_ushort(src[(int64_t)t * jb.stride_t + c]) << 16;
-        m = max(m, b & 0x7FFFFFFFu);
+    uint32_t m[4] = {0u, 0u, 0u, 0u};  // two 15-bit magnitudes per word
+    for (int t = t0 + rg; t < t1; t += 16) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(src + (int64_t)t * jb.stride_t + c8);
+        m[0] = __vmaxu2(m[0], raw.x & 0x7FFF7FFFu);
+        m[1] = __vmaxu2(m[1], raw.y & 0x7FFF7FFFu);
+        m[2] = __vmaxu2(m[2], raw.z & 0x7FFF7FFFu);
+        m[3] = __vmaxu2(m[3], raw.w & 0x7FFF7FFFu);
     }
-    s_max[half][c] = m;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        s_max[rg][c8 + 2 * j] = (m[j] & 0xFFFFu) << 16;  // as float32 bit patterns
+        s_max[rg][c8 + 2 * j + 1] = m[j] & 0xFFFF0000u;
+    }
     __syncthreads();
-    if (half == 0) atomicMax(reinterpret_cast<uint32_t*>(jb.scale) + kD + c, max(s_max[0][c], s_max[1][c]));
+    if (threadIdx.x < kD) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int r = 0; r < 16; ++r) v = max(v, s_max[r][threadIdx.x]);
+        atomicMax(reinterpret_cast<uint32_t*>(jb.scale) + kD + threadIdx.x, v);
+    }
 }
 
-// grid (ceil(T * 16 / 256), jobs): one thread per 8 channels of a token: scale from the maxima, codes out (8 bytes)
+// one CTA per job: the channel scales from the maxima
+__global__ void __launch_bounds__(128) scale_kernel(const QuantJob* jobs) {
+    const QuantJob jb = jobs[blockIdx.x];
+    const float amax = __uint_as_float(reinterpret_cast<const uint32_t*>(jb.scale)[kD + threadIdx.x]);
+    jb.scale[threadIdx.x] = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+}
+
+// grid (ceil(T * 16 / 256), jobs): one thread per 8 channels of a token: codes out (8 bytes)
 __global__ void __launch_bounds__(256) quantise_kernel(const QuantJob* jobs) {
     const QuantJob jb = jobs[blockIdx.y];
     const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(jb.src);
-    const uint32_t* amax_bits = reinterpret_cast<const uint32_t*>(jb.scale) + kD;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int t = (int)(i >> 4), c8 = (int)(i & 15) * 8;
     if (t >= jb.T) return;
     const uint4 raw = *reinterpret_cast<const uint4*>(src + (int64_t)t * jb.stride_t + c8);
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    const float4 s0 = *reinterpret_cast<const float4*>(jb.scale + c8), s1 = *reinterpret_cast<const float4*>(jb.scale + c8 + 4);
+    const float scv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
     uint32_t out[2] = {0u, 0u};
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const float amax = __uint_as_float(amax_bits[c8 + j]);
-        const float sc = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+        const float sc = scv[j];
         const float x = __uint_as_float((j & 1) ? (w[j >> 1] & 0xFFFF0000u) : (w[j >> 1] << 16));
         const uint32_t code = (uint32_t)__nv_cvt_float_to_fp8(__fdiv_rn(x, sc), __NV_SATFINITE, __NV_E4M3);
         out[j >> 2] |= code << (8 * (j & 3));
-        if (t == 0) jb.scale[c8 + j] = sc;
     }
     *reinterpret_cast<uint2*>(jb.codes + (int64_t)t * kD + c8) = make_uint2(out[0], out[1]);
 }
@@ -91,9 +110,10 @@ cudaError_t launch_quantise_jobs(const QuantJob* jobs_dev, int njobs, int T_max,
     const int rows_per_cta = 1024;
     zero_amax_kernel<<<njobs, kD, 0, st>>>(jobs_dev);
     absmax_kernel<<<dim3((T_max + rows_per_cta - 1) / rows_per_cta, njobs), 256, 0, st>>>(jobs_dev, rows_per_cta);
+    scale_kernel<<<njobs, kD, 0, st>>>(jobs_dev);
     const int64_t threads = (int64_t)T_max * 16;
     quantise_kernel<<<dim3((unsigned)((threads + 255) / 256), njobs), 256, 0, st>>>(jobs_dev);
-    count_launch(3);
+    count_launch(4);
     return cudaGetLastError();
 }
 
