@@ -568,8 +568,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
             if (s.tok_rule && m == FDKV_MODE_RESIDUAL) {  // one token list and one offset table serve K and V
                 tl = take(tlist_b);
                 to = take(off_b);
-                CU(cudaMemcpyAsync(tl, c->work + c->ws.tok_list + (size_t)u * s.ktok_cap * 4, (size_t)k_tok * 4, cudaMemcpyDeviceToDevice, st));
-                CU(cudaMemcpyAsync(to, c->work + c->ws.tok_off + (size_t)u * (s.ntiles_max + 1) * 4, off_copy, cudaMemcpyDeviceToDevice, st));
+                copy_job(c->work + c->ws.tok_list + (size_t)u * s.ktok_cap * 4, tl, (size_t)k_tok * 4, 16, 16);
+                copy_job(c->work + c->ws.tok_off + (size_t)u * (s.ntiles_max + 1) * 4, to, off_copy, 16, 16);
                 by_mode[1] += (size_t)k_tok * 4;
             }
             for (int is_v = 0; is_v < 2; ++is_v) {
@@ -591,7 +591,8 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 by_mode[m] += s.rows_f8 ? rows8 + 512 : rows;
                 if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
                     char* rows_res = take(trow_b);
-                    CU(launch_token_gather(c->work + c->ws.z1 + ut * unit_stride_b, (const int32_t*)tl, k_tok, rows_res, st));
+                    // (the list is read where the probe left it: its copy into the arena runs with the other copies after this loop)
+                    CU(launch_token_gather(c->work + c->ws.z1 + ut * unit_stride_b, wsp<int32_t>(c, c->ws.tok_list) + (size_t)u * s.ktok_cap, k_tok, rows_res, st));
                     for (int l = 0; l < s.B; ++l) {
                         UnitDesc* d = dl[l];
                         d->res_kind = 1;
