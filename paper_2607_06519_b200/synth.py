@@ -104,6 +104,8 @@ WORKLOADS = {
 WORKLOADS["decode32k_4l"] = WORKLOADS["decode32k"].scaled(n_layers=4, name="decode32k_4l")
 WORKLOADS["decode128k_4l"] = WORKLOADS["decode128k"].scaled(n_layers=4, name="decode128k_4l")
 # the same 32k workload with the paper's token-granular residual (probe-scored tokens keep whole rows)
+# the 32k workload while it generates: every step appends one token to every layer's exact tail (stream launches)
+WORKLOADS["decode32k_gen"] = WORKLOADS["decode32k"].scaled(n_steps=64, name="decode32k_gen")
 WORKLOADS["decode32k_tok"] = WORKLOADS["decode32k"].scaled(residual_rule=1, name="decode32k_tok")
 WORKLOADS["decode32k_tok_4l"] = WORKLOADS["decode32k_tok"].scaled(n_layers=4, name="decode32k_tok_4l")
 # depth blocks of four layers (the paper's default block size): tiny correctness case and the 32k shape
