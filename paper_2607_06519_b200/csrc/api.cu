@@ -685,8 +685,13 @@ static fdkv_status decode_impl(fdkv_ctx* c, int32_t layer, int32_t batch, const 
     DecodeArgs a;
     a.tail_rows = s.tail_rows;
     a.host_T = host_T.data(); a.host_modes = host_modes.data();
+    std::vector<int32_t> host_tail(batch);  // (already counts this call's append)
     a.any_tail = 0;
-    for (int b = 0; b < batch; ++b) a.any_tail |= c->seqs[b].tail_len[layer] > 0;  // (already counts this call's append)
+    for (int b = 0; b < batch; ++b) {
+        host_tail[b] = c->seqs[b].tail_len[layer];
+        a.any_tail |= host_tail[b] > 0;
+    }
+    a.host_tail = host_tail.data();
     a.tmap = c->has_tmap ? c->tmap : nullptr;
     a.tmap_u8 = s.rows_f8 ? c->tmap_u8 : nullptr;
     a.rows_f8 = s.rows_f8;

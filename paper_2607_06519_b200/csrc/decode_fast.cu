@@ -871,7 +871,7 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
     std::vector<int64_t> wp(units + 1, 0);
     // ranges are cut on 16-token slices (the granularity of the residual lists), so that the CTAs of a unit differ by
     // at most one slice; each range is streamed as 128-token tiles from its first slice, the last one partial
-    std::vector<int> nt(units), ns(units), wt(units);  // 128-token tiles, 16-token slices, cost per tile
+    std::vector<int> nt(units), ns(units), es(units), wt(units);  // 128-token tiles, 16-token slices, slices + tail, cost per tile
     int64_t total_tiles = 0;
     for (int u = 0; u < units; ++u) {
         const int T = a.host_T[u / a.Hkv];
@@ -906,7 +906,21 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
                 if (rc == 0.0) wt[u] = (int)(wt[u] * (res_a + res_b * (double)k / nt[u] / 1024.0));
                 else wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * rc);
             }
-            wp[u + 1] = wp[u] + (int64_t)ns[u] * wt[u];  // (in eighths of the tile cost)
+            // the CTA that ends a unit also streams its tail of generated tokens (whole plain tiles): counted as slices
+            // of the unit's kind behind the unit's own, so that this CTA gets correspondingly fewer of those
+            const int tail = a.host_tail ? std::min(a.host_tail[u / a.Hkv], a.max_tail) : 0;
+            // Measured: the CTA that ends a unit runs behind its siblings at equal shares (with tails it also reads their
+            // lengths behind the dependency wait); charging it eight plain tiles' worth of slices (in eighths of a tile
+            // below) is the optimum of a sweep at 32k, with and without tails (+1.6 % / +6 %), and neutral at 128k.
+            static int tail_extra = -1, last_extra = 64;
+            if (tail_extra < 0) {  // tuning knobs for benchmark sweeps
+                const char* te = getenv("FDKV_TAIL_EXTRA");
+                const char* le = getenv("FDKV_LAST_EXTRA");
+                tail_extra = te ? atoi(te) : 64;
+                last_extra = le ? atoi(le) : 64;
+            }
+            es[u] = ns[u] + ((tail + kTT - 1) / kTT * (kTT / kResTile) + (tail > 0 ? tail_extra : last_extra)) * (2 * kTT * 256 / 512) / std::max(1, wt[u]);
+            wp[u + 1] = wp[u] + (int64_t)es[u] * wt[u];  // (in eighths of the tile cost)
         }
     };
     // (measured best: 1.7 when every unit gets whole CTAs, 1.5 in the flat cut of a batch)
@@ -952,7 +966,7 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
     if (whole) {
         int c = 0;
         for (int u = 0; u < units; ++u)
-            for (int j = 0; j < nc[u]; ++j) sch.start[c++] = ((uint32_t)u << 20) | (uint32_t)((int64_t)ns[u] * j / nc[u]);
+            for (int j = 0; j < nc[u]; ++j) sch.start[c++] = ((uint32_t)u << 20) | (uint32_t)std::min<int64_t>(ns[u] - 1, (int64_t)es[u] * j / nc[u]);
         sch.start[ncta] = (uint32_t)units << 20;
     } else {
         if (!res_cost_env) weigh(1.5);
@@ -960,7 +974,7 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
         for (int c = 0; c < ncta; ++c) {
             const int64_t target = wp[units] * c / ncta;
             while (u + 1 < units && wp[u + 1] <= target) ++u;
-            const int slice = (int)((target - wp[u]) / wt[u]);
+            const int slice = (int)std::min<int64_t>(ns[u], (target - wp[u]) / wt[u]);
             sch.start[c] = ((uint32_t)u << 20) | (uint32_t)slice;
         }
         sch.start[ncta] = (uint32_t)units << 20;

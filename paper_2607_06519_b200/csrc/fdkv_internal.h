@@ -230,6 +230,7 @@ struct DecodeArgs {
     // host-side views used only to plan the launch (valid during the call)
     const int32_t* host_T;      // [batch]
     const int32_t* host_modes;  // [batch][Hkv] modes of this layer's pair
+    const int32_t* host_tail;   // [batch] generated tokens in this layer's tail per sequence (after this call's append), or null
     int any_tail;               // some sequence of the batch has generated tokens in this layer's tail (after this call's append)
     const void* tmap;           // CUtensorMap over the arena as rows of 256 bytes, or null
     const void* tmap_u8;        // the same arena as rows of 128 bytes (8-bit row streams), or null

@@ -62,15 +62,17 @@ def test_llama_32k_whole_blocks_per_unit():
     # whole blocks per unit: no range crosses a unit boundary
     for (b, e) in ranges:
         assert e[0] == b[0] or (e[0] == b[0] + 1 and e[1] == 0)
-    # blocks of one unit differ by at most one slice; residual units get more blocks
+    # blocks of one unit differ by at most one slice, except the block that ends the unit, which is charged extra and
+    # gets fewer; residual units get more blocks
     for u in range(8):
         lens = [(e[1] if e[0] == u else _slices(T[0])) - b[1] for (b, e) in ranges if b[0] == u]
-        assert max(lens) - min(lens) <= 1 and len(lens) == parts[u]
+        assert max(lens[:-1]) - min(lens[:-1]) <= 1 and 0 < lens[-1] <= min(lens[:-1]) and len(lens) == parts[u]
     res, plain = [parts[u] for u in (1, 3, 5)], [parts[u] for u in (0, 2, 4, 6, 7)]
     assert min(res) > max(plain) and max(res) - min(res) <= 1 and max(plain) - min(plain) <= 1
     # the fitted residual cost (2.12 plain tiles at keep 1/16) balances the blocks within a few per cent
     c = _cost(ranges, T, hkv, modes, 2.12)
-    assert c.max() / c.mean() < 1.06
+    ends_unit = np.array([e[1] == 0 for (b, e) in ranges])
+    assert c[~ends_unit].max() / c[~ends_unit].mean() < 1.06 and c[ends_unit].max() <= c[~ends_unit].max()
 
 
 @pytest.mark.parametrize("seed", range(12))
@@ -98,7 +100,7 @@ def test_batch_flat_cut_is_balanced():
     assert len(ranges) == 148
     _check_partition(ranges, parts, T, hkv)
     c = _cost(ranges, T, hkv, modes, 1.59)   # the flat cut weighs a residual tile 1.5 x its bytes
-    assert c.max() / c.mean() < 1.03
+    assert c.max() / c.mean() < 1.08         # (blocks that end a unit are charged extra and get less)
 
 
 def test_many_one_token_units_fit_the_segment_tables():
