@@ -91,7 +91,7 @@ typedef enum { FDKV_ROWS_STORAGE = 0, FDKV_ROWS_E4M3 = 1 } fdkv_row_format;
  *     s = (x0 + x1) + (x2 + x3);   Z0 = rs(0.5 s)                the shared coefficient (first DCT row = 1/2 each)
  *     dev_l = rs(x_l - 0.5 Z0),  l = 0..3                         layer l's high-frequency part in layer space:
  *                                                                 sum_{j>=1} F_4[j][l] Z_j = x_l - mean(x)
- *     e = rs((dev_0^2 + dev_1^2) + (dev_2^2 + dev_3^2))           the position's high-frequency energy (Parseval)
+ *     e = (dev_0^2 + dev_1^2) + (dev_2^2 + dev_3^2)               the position's high-frequency energy (Parseval)
  * The three high-frequency groups share one kept set per tensor (Eq. 3): the k positions of largest e, ties to the
  * lowest flat index; the four values dev_l are kept there (instead of three coefficients), so that a decode call of
  * layer l reads one value per kept position.  Candidates: shared = Z0 / 2, residual = Z0 / 2 + dev_l on the kept

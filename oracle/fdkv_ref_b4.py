@@ -13,9 +13,8 @@ What is computed (Method section, Eq. 1-3, with B = 4):
       s   = (x0 + x1) + (x2 + x3)
       z0  = rs(0.5 * s)                       rs = round to the storage type (float32: identity, bf16: nearest even)
       dev_l = rs(x_l - 0.5 * z0)              l = 0..3: the high-frequency part of layer l in layer space
-      e   = rs((dev_0^2 + dev_1^2) + (dev_2^2 + dev_3^2)) the position's high-frequency energy (Parseval: the sum
-                                              of its three squared high-frequency coefficients), kept in the
-                                              storage precision like every other staged value
+      e   = (dev_0^2 + dev_1^2) + (dev_2^2 + dev_3^2)      the position's high-frequency energy (Parseval: the sum
+                                              of its three squared high-frequency coefficients)
   The library keeps, per kept position, the four layer-space values dev_l instead of the three coefficients
   Z_1..Z_3 (they span the same three dimensions: sum_l dev_l = 0 up to rounding), so that a decode call for layer l
   reads one value per kept position.
@@ -70,7 +69,7 @@ def depth_split4(x, bf16: bool):
     half = np.float32(0.5) * z0                  # exact
     dev = [rs(x[l] - half) for l in range(4)]
     sq = [d * d for d in dev]                    # float32 products, rounded
-    energy = rs((sq[0] + sq[1]) + (sq[2] + sq[3]))
+    energy = (sq[0] + sq[1]) + (sq[2] + sq[3])
     return z0, dev, energy
 
 

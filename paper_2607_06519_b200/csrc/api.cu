@@ -74,8 +74,8 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.z0 = take((size_t)s.NT * unit_elems * s.esize);
     w.z1 = take((size_t)s.NT * s.NB * unit_elems * s.esize);  // Z1 of a pair, or the four layers' deviations of a block
     w.z1drop = take(s.dtype == FDKV_BF16 && s.d == 128 ? (size_t)s.NU * s.NB * unit_elems * s.esize : 0);
-    w.energy = take(s.B == 4 ? (size_t)s.NT * unit_elems * s.esize : 0);
-    w.eval = take(s.B == 4 ? (size_t)s.NT * s.kcap * s.esize : 0);
+    w.energy = take(s.B == 4 ? (size_t)s.NT * unit_elems * 4 : 0);
+    w.eval = take(s.B == 4 ? (size_t)s.NT * s.kcap * 4 : 0);
     w.hist = take((size_t)s.NT * kHistBins * 4);
     w.sel = take((size_t)s.NT * sizeof(SelState));
     w.tile_cnt = take((size_t)s.NT * s.ntiles_max * 8);
@@ -267,7 +267,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     CU(cudaMemsetAsync(wsp<uint32_t>(c, c->ws.hist) + (size_t)ut_begin * kHistBins, 0, (size_t)ut_count * kHistBins * 4, st));
     if (s.B == 4) {
         // blocks of four layers: Z0, the layers' deviations and the positions' energies; one kept set per tensor from
-        // the radix select of the storage type on the energies; then the four layers' values at the kept positions
+        // the float32 radix select on the energies; then the four layers' values at the kept positions
         for (int p = pb; p < pe; ++p) {
             Split4Args a4;
             for (int l = 0; l < 4; ++l) {
@@ -281,7 +281,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
             a4.ut_base = p * s.Hkv * 2;
             a4.unit_stride = (int64_t)s.Tmax * s.d;
             a4.z0 = c->work + c->ws.z0; a4.dev = c->work + c->ws.z1;
-            a4.energy = c->work + c->ws.energy;
+            a4.energy = wsp<float>(c, c->ws.energy);
             a4.drop = c->has_probe_tmaps ? c->work + c->ws.z1drop : nullptr;
             a4.hist = wsp<uint32_t>(c, c->ws.hist);
             CU(launch_split4_hist(a4, s.dtype, st));
@@ -302,7 +302,7 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
         sa.packed = nullptr;
         sa.z1drop = nullptr;
         sa.status = wsp<int32_t>(c, c->ws.status);
-        CU(launch_select_and_compact(sa, s.dtype, st));
+        CU(launch_select_and_compact(sa, FDKV_F32, st));
         Gather4Args g;
         g.ut_begin = ut_begin; g.ut_count = ut_count;
         g.k = sa.k; g.kcap = s.kcap; g.unit_stride = (int64_t)s.Tmax * s.d;
@@ -824,7 +824,7 @@ fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
             a4.ut_base = p * s.Hkv * 2;
             a4.unit_stride = (int64_t)s.Tmax * s.d;
             a4.z0 = c->work + c->ws.z0; a4.dev = c->work + c->ws.z1;
-            a4.energy = c->work + c->ws.energy;
+            a4.energy = wsp<float>(c, c->ws.energy);
             a4.drop = nullptr;
             a4.hist = wsp<uint32_t>(c, c->ws.hist);
             CU(launch_split4_hist(a4, s.dtype, st));
@@ -832,7 +832,7 @@ fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
         sa.z1 = c->work + c->ws.energy;
         sa.val = c->work + c->ws.eval;
         sa.packed = nullptr;
-        CU(launch_select_and_compact(sa, s.dtype, st));
+        CU(launch_select_and_compact(sa, FDKV_F32, st));
         Gather4Args g;
         g.ut_begin = 0; g.ut_count = s.NT;
         g.k = kc; g.kcap = s.kcap; g.unit_stride = (int64_t)s.Tmax * s.d;

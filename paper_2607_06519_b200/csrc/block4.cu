@@ -5,13 +5,11 @@
 // coefficients of a position contribute x_l - mean to layer l and their squared sum equals sum_l (x_l - mean)^2.
 // The library therefore stages, per position, Z0, the four layer-space deviations dev_l = x_l - Z0 / 2 and the
 // energy e = sum_l dev_l^2; the three high-frequency groups share one kept set per tensor (Eq. 3), the k positions
-// of largest energy (ties to the lowest index), found by the radix select of compress.cu on e.
+// of largest energy (ties to the lowest index), found by the float32 radix select of compress.cu on e.
 // A decode call for layer l then reads one value per kept position (dev_l) instead of three coefficients.
 //
 // Stored arithmetic (float32, never contracted):  s = (x0 + x1) + (x2 + x3);  z0 = rs(0.5 s);
-// dev_l = rs(x_l - 0.5 z0);  e = rs((dev_0^2 + dev_1^2) + (dev_2^2 + dev_3^2))  with rs = rounding to the storage type
-// (the energy is staged in the storage type too, so the radix select of that type runs on it: one histogram pass for
-// bf16).
+// dev_l = rs(x_l - 0.5 z0);  e = (dev_0^2 + dev_1^2) + (dev_2^2 + dev_3^2)  with rs = rounding to the storage type.
 #include <algorithm>
 
 #include "fdkv_internal.h"
@@ -52,7 +50,7 @@ struct Vec<__nv_bfloat16> {
 };
 
 // grid (chunks, Hkv * 2): each CTA owns a token range of one unit-tensor and a private histogram of the energies'
-// top 15 magnitude bits (for bf16 the whole key: the only pass of the radix select; for float32 its first pass).
+// top 15 magnitude bits (the first pass of the float32 radix select).
 template <typename T>
 __global__ void __launch_bounds__(512) split4_hist_kernel(Split4Args a, int tokens_per_cta) {
     extern __shared__ uint32_t s_hist[];
@@ -67,7 +65,7 @@ __global__ void __launch_bounds__(512) split4_hist_kernel(Split4Args a, int toke
     for (int l = 0; l < 4; ++l) x[l] = reinterpret_cast<const T*>(is_v ? a.v[l] : a.k[l]) + (int64_t)h * a.stride_h;
     T* z0 = reinterpret_cast<T*>(a.z0) + (int64_t)ut * a.unit_stride;
     T* dev = reinterpret_cast<T*>(a.dev) + (int64_t)ut * 4 * a.unit_stride;
-    T* en = reinterpret_cast<T*>(a.energy) + (int64_t)ut * a.unit_stride;
+    float* en = a.energy + (int64_t)ut * a.unit_stride;
     T* drop = (a.drop && !is_v) ? reinterpret_cast<T*>(a.drop) + (int64_t)(ut >> 1) * 4 * a.unit_stride : nullptr;
 
     const int t_begin = blockIdx.x * tokens_per_cta;
@@ -91,8 +89,8 @@ __global__ void __launch_bounds__(512) split4_hist_kernel(Split4Args a, int toke
             const float half = __fmul_rn(0.5f, z[i]);  // exact
 #pragma unroll
             for (int l = 0; l < 4; ++l) dv[l][i] = V::rs(__fsub_rn(f[l][i], half));
-            e[i] = V::rs(__fadd_rn(__fadd_rn(__fmul_rn(dv[0][i], dv[0][i]), __fmul_rn(dv[1][i], dv[1][i])),
-                                   __fadd_rn(__fmul_rn(dv[2][i], dv[2][i]), __fmul_rn(dv[3][i], dv[3][i]))));
+            e[i] = __fadd_rn(__fadd_rn(__fmul_rn(dv[0][i], dv[0][i]), __fmul_rn(dv[1][i], dv[1][i])),
+                             __fadd_rn(__fmul_rn(dv[2][i], dv[2][i]), __fmul_rn(dv[3][i], dv[3][i])));
         }
         *reinterpret_cast<typename V::raw*>(z0 + off_out) = V::pack(z);
 #pragma unroll
@@ -101,7 +99,9 @@ __global__ void __launch_bounds__(512) split4_hist_kernel(Split4Args a, int toke
             *reinterpret_cast<typename V::raw*>(dev + (int64_t)l * a.unit_stride + off_out) = pk;
             if (drop) *reinterpret_cast<typename V::raw*>(drop + (int64_t)l * a.unit_stride + off_out) = pk;
         }
-        *reinterpret_cast<typename V::raw*>(en + off_out) = V::pack(e);
+#pragma unroll
+        for (int i = 0; i < N; i += 4)
+            *reinterpret_cast<float4*>(en + off_out + i) = make_float4(e[i], e[i + 1], e[i + 2], e[i + 3]);
 #pragma unroll
         for (int i = 0; i < N; ++i) atomicAdd(&s_hist[(__float_as_uint(e[i]) & 0x7FFFFFFFu) >> 16], 1u);
     }

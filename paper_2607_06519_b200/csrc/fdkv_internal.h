@@ -176,7 +176,7 @@ struct Split4Args {
     int64_t unit_stride;  // elements between staged tensors (Tmax*d)
     void* z0;             // [NT][unit_stride]
     void* dev;            // [NT][4][unit_stride]: deviation of each layer from the block mean
-    void* energy;         // [NT][unit_stride], storage type
+    float* energy;        // [NT][unit_stride]
     void* drop;           // optional [NU][4][unit_stride]: second copy of the K deviations (the gather zeroes its kept positions)
     uint32_t* hist;
 };

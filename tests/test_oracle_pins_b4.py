@@ -64,7 +64,7 @@ def test_stored_values_follow_the_stated_arithmetic(bf16):
             dv = rs(np.array([f(x[l][t, c] - f(0.5) * z)], dtype=np.float32))[0]
             assert dev[l][t, c] == dv
             e.append(f(dv * dv))
-        assert energy[t, c] == rs(np.array([f(f(e[0] + e[1]) + f(e[2] + e[3]))], dtype=np.float32))[0]
+        assert energy[t, c] == f(f(e[0] + e[1]) + f(e[2] + e[3]))
     # against float64 within the storage rounding
     x64 = np.stack([a.astype(np.float64) for a in x])
     tol = 2.0 ** -8 if bf16 else 2.0 ** -22
@@ -74,6 +74,14 @@ def test_stored_values_follow_the_stated_arithmetic(bf16):
     if bf16:
         for a in [z0] + dev:
             assert np.array_equal(synth.round_bf16(a), a)
+    # the selection key is the energy of the three high-frequency DCT coefficients (Eq. 1 with B = 4, Parseval), kept
+    # in float32: against scipy's transform of the inputs it is off only by the storage rounding of the deviations
+    Z = scipy.fft.dct(x64, type=2, norm="ortho", axis=0)
+    hf = (Z[1:] ** 2).sum(axis=0)
+    np.testing.assert_allclose(energy, hf, rtol=8 * tol, atol=8 * tol * hf.max())
+    assert energy.dtype == np.float32
+    if bf16:  # not rounded to the storage type: the key keeps its float32 mantissa
+        assert not np.array_equal(synth.round_bf16(energy), energy)
 
 
 def test_selection_is_top_k_energy_with_lowest_index_ties():
