@@ -83,16 +83,23 @@ def attention(khat, vhat, q):
     return (p @ vhat) / p.sum()
 
 
-def token_scores(z1k, q_pair, group: int, h: int, pos):
-    """s_t = max over probe queries that can see t of |Q (K_t - Khat_t^shared)^T| = |Q . c z1k_t|."""
-    c = np.sqrt(0.5)
+def token_scores(z0k, z1k, q_pair, group: int, h: int, pos):
+    """The unnumbered token score between Eq. 2 and Eq. 3, literally: s_t = max over the probe queries that can see t
+    (and over the block's layers and the group's heads) of |Q (K_t - Khat_t^shared)^T|, with K = F^T [Z0; Z1] the key
+    rows the stored coefficients stand for and Khat^shared = F^T [Z0; 0] the shared-depth candidate of Eq. 3 (S empty).
+    No 1/sqrt(d): the printed score has none."""
+    F = dct_matrix(2)
+    Z = np.stack([z0k, z1k]).astype(np.float64)
+    Z_shared = np.stack([z0k.astype(np.float64), np.zeros_like(z1k, dtype=np.float64)])
+    K = np.einsum("kl,ktc->ltc", F, Z)                # F^T Z: [layer, T, d]
+    K_shared = np.einsum("kl,ktc->ltc", F, Z_shared)
     T = z1k.shape[0]
     best = np.zeros(T)
-    visible = np.arange(T)[None, :] <= np.asarray(pos)[:, None]
+    visible = np.arange(T)[None, :] <= np.asarray(pos)[:, None]  # [W, T]
     for layer in range(2):
         for g in range(group):
             Q = q_pair[layer][:, h * group + g, :].astype(np.float64)
-            s = np.abs(Q @ (c * z1k.astype(np.float64)).T)
+            s = np.abs(Q @ (K[layer] - K_shared[layer]).T)      # [W, T]
             s = np.where(visible, s, 0.0)
             best = np.maximum(best, s.max(axis=0))
     return best

@@ -57,7 +57,7 @@ def test_bruteforce_reproduces_golden(dtype):
                 ref = rec["decode"][f"l{layer}_{mname}"]
                 np.testing.assert_allclose(o[:, :3], ref["first3"], rtol=1e-9, atol=1e-12)
                 assert float(np.abs(o).max()) == pytest.approx(ref["max_abs"], rel=1e-9)
-        s = bf.token_scores(z1k, pq, w.group, h, pos)
+        s = bf.token_scores(z0k, z1k, pq, w.group, h, pos)
         order = np.lexsort((np.arange(w.T), -s))
         tok = np.sort(order[: w.T // 8])
         assert tok[:8].tolist() == rec["token_rule"]["tok_head"]

@@ -328,13 +328,33 @@ def test_token_rule_vs_bruteforce_and_needles():
     q = (synth.probe_q(w, 0, 0), synth.probe_q(w, 0, 1))
     for h in range(w.n_kv_heads):
         k0, k1 = synth.unit_tensor(w, 0, 0, h, False)
-        _, z1 = R.depth_split(k0, k1, bf16=False)
+        z0, z1 = R.depth_split(k0, k1, bf16=False)
         s = R.token_scores(z1, q[0], q[1], w.group, h, pos)
-        np.testing.assert_allclose(s, bf.token_scores(z1, q, w.group, h, pos), rtol=1e-12)
+        # literal form: |Q (K_t - Khat_t^shared)^T| with both key matrices rebuilt through the DCT matrix; the
+        # difference of two O(|z0|) reconstructions costs a few ulps of |Q| |z0|, hence the absolute term
+        lit = bf.token_scores(z0, z1, q, w.group, h, pos)
+        np.testing.assert_allclose(s, lit, rtol=1e-12, atol=1e-12 * float(np.abs(z0).max()) * w.head_dim)
         tok = R.select_tokens(s, w.T // 8)
         order = np.lexsort((np.arange(w.T), -s))
         assert np.array_equal(tok, np.sort(order[: w.T // 8]))
         assert set(synth.needle_positions(w, 0, 0, h).tolist()) <= set(tok.tolist())
+
+
+def test_token_score_closed_form_single_entry():
+    # one non-zero high-frequency coefficient a at (t0, c0): K_t - Khat_t^shared = +-a/sqrt(2) e_c0 in the two layers,
+    # so s_t0 = max_q |Q[q][c0]| * |a| / sqrt(2) over the queries at positions >= t0, and every other token scores 0
+    T, d, G, Hq, W = 10, 4, 2, 2, 3
+    z1 = np.zeros((T, d), dtype=np.float32)
+    t0, c0, a = 6, 2, -3.0
+    z1[t0, c0] = a
+    g = np.random.default_rng(11)
+    q0 = g.standard_normal((W, Hq, d)).astype(np.float32)
+    q1 = g.standard_normal((W, Hq, d)).astype(np.float32)
+    pos = np.array([2, 6, 9], dtype=np.int32)   # the query at position 2 cannot see token 6
+    s = R.token_scores(z1, q0, q1, G, 0, pos)
+    want = max(abs(float(q[w_, g_, c0])) for q in (q0, q1) for g_ in range(G) for w_ in (1, 2)) * abs(a) * np.sqrt(0.5)
+    assert s[t0] == pytest.approx(want, rel=1e-12)
+    assert np.count_nonzero(s) == 1
 
 
 # ---------------------------------------------------------------- token-granular residual (the paper's own rule)
