@@ -298,44 +298,38 @@ int64_t fdkv_ref_select_tokens(const double* s, int64_t T, int64_t k_tok, int32_
     return k_tok;
 }
 
-/* ---- budgeted routing (Method: "the memory budget is enforced by increasing lambda until the estimated peak KV
- * footprint satisfies the requested budget") ------------------------------------------------------------------
- * Footprint(lambda) = sum over units of Omega(mode_u(lambda)) * bytes_exact_unit, with the mode rule above; it can only
- * change where two of a unit's three loss lines cross, so the smallest lambda that fits is 0 or (just above) one of
- * those crossings.  Candidates are visited in ascending order; each is tried at lambda = crossing * (1 + 2^-40) so
- * that the unit that crosses there has already taken its cheaper mode.  Returns 1 and the first lambda that fits
- * (with its modes), or 0 with lambda = +inf and every unit shared when even that does not fit.                   */
-static int cmp_f64(const void* a, const void* b) {
-    double x = *(const double*)a, y = *(const double*)b;
-    return (x > y) - (x < y);
-}
+/* ---- budgeted routing (Method: the memory budget is enforced by increasing lambda until the estimated peak KV
+ * footprint satisfies the requested budget) ------------------------------------------------------------------------
+ * Footprint(lambda) = sum over units of Omega(mode_u(lambda)) * bytes_exact_unit, with the mode rule above.  The plain
+ * procedure: try lambda = 0, then lambda = lam_lo, lam_lo * ratio, lam_lo * ratio^2, ... (an ascending grid, ratio > 1)
+ * and stop at the first value whose routing fits.  Returns 1 with that lambda, its modes and the grid value tried just
+ * before it (which did not fit; -1 when lambda = 0 already fits).  The footprint cannot fall below the all-shared one,
+ * so the scan gives up -- returns 0, lambda = +inf, every unit shared -- once a grid value routes every unit to shared
+ * and still does not fit, or after max_steps values.                                                               */
 int fdkv_ref_route_budget(const double* e_shared, const double* e_residual, int64_t n_units, const double* omega,
-                          double bytes_exact_unit, double budget_bytes, double* lambda_out, int32_t* modes_out) {
-    int64_t n_cand = 3 * n_units + 1;
-    double* cand = (double*)malloc((size_t)n_cand * sizeof(double));
-    cand[0] = 0.0;
-    for (int64_t u = 0; u < n_units; ++u) {
-        cand[1 + 3 * u] = (e_shared[u] - e_residual[u]) / (omega[1] - omega[0]); /* shared <-> residual */
-        cand[2 + 3 * u] = e_residual[u] / (omega[2] - omega[1]);                 /* residual <-> exact  */
-        cand[3 + 3 * u] = e_shared[u] / (omega[2] - omega[0]);                   /* shared <-> exact    */
-    }
-    qsort(cand, (size_t)n_cand, sizeof(double), cmp_f64);
-    int fits = 0;
-    for (int64_t i = 0; i < n_cand && !fits; ++i) {
-        if (!(cand[i] >= 0.0) || isinf(cand[i])) continue;
-        double lam = cand[i] * (1.0 + ldexp(1.0, -40));
+                          double bytes_exact_unit, double budget_bytes, double lam_lo, double ratio, int64_t max_steps,
+                          double* lambda_out, double* lambda_prev_out, int32_t* modes_out) {
+    double lam = 0.0, prev = -1.0;
+    for (int64_t step = 0; step <= max_steps; ++step) {
         double total = 0.0;
+        int all_shared = 1;
         for (int64_t u = 0; u < n_units; ++u) {
             int m = fdkv_ref_mode(e_shared[u], e_residual[u], omega, lam, NULL, NULL);
             modes_out[u] = m;
             total += omega[m] * bytes_exact_unit;
+            if (m != 0) all_shared = 0;
         }
-        if (total <= budget_bytes) { fits = 1; *lambda_out = lam; }
+        if (total <= budget_bytes) {
+            *lambda_out = lam;
+            *lambda_prev_out = prev;
+            return 1;
+        }
+        if (all_shared) break;
+        prev = lam;
+        lam = step == 0 ? lam_lo : lam * ratio;
     }
-    if (!fits) {
-        *lambda_out = INFINITY;
-        for (int64_t u = 0; u < n_units; ++u) modes_out[u] = 0;
-    }
-    free(cand);
-    return fits;
+    *lambda_out = INFINITY;
+    *lambda_prev_out = prev;
+    for (int64_t u = 0; u < n_units; ++u) modes_out[u] = 0;
+    return 0;
 }

@@ -31,7 +31,8 @@ _lib.fdkv_ref_omega.argtypes = [_i64, _i64, _i64, _i64, _f64p]
 _lib.fdkv_ref_omega_tokens.argtypes = [_i64, _i64, _i64, _i64, _f64p]
 _lib.fdkv_ref_mode.argtypes = [C.c_double, C.c_double, _f64p, C.c_double, _f64p, C.POINTER(C.c_double)]
 _lib.fdkv_ref_mode.restype = C.c_int
-_lib.fdkv_ref_route_budget.argtypes = [_f64p, _f64p, _i64, _f64p, C.c_double, C.c_double, C.POINTER(C.c_double), _i32p]
+_lib.fdkv_ref_route_budget.argtypes = [_f64p, _f64p, _i64, _f64p, C.c_double, C.c_double, C.c_double, C.c_double, _i64,
+                                          C.POINTER(C.c_double), C.POINTER(C.c_double), _i32p]
 _lib.fdkv_ref_route_budget.restype = C.c_int
 _lib.fdkv_ref_attention.argtypes = [_f64p, _f64p, _i64, _i64, _f32p, _f64p]
 _lib.fdkv_ref_token_scores.argtypes = [_f32p, _i64, _i64, _f32p, _f32p, _i64, _i64, _i64, _i32p, _i64, _f64p]
@@ -132,15 +133,18 @@ def mode_rule(e_shared: float, e_residual: float, om, lam: float):
     return int(m), loss, float(margin.value)
 
 
-def route_budget(e_shared, e_residual, om, bytes_exact_unit: float, budget_bytes: float):
-    """Smallest lambda whose routing fits the budget: (fits, lambda, modes)."""
+def route_budget(e_shared, e_residual, om, bytes_exact_unit: float, budget_bytes: float, lam_lo: float = 1e-9,
+                 ratio: float = 1.0 + 2.0 ** -12, max_steps: int = 400000):
+    """Plain scan: lambda = 0, lam_lo, lam_lo * ratio, ... until the routing fits the budget.
+    Returns (fits, lambda, modes, previous grid value): the true threshold lies in (previous, lambda]."""
     e_sh = np.ascontiguousarray(e_shared, dtype=np.float64).ravel()
     e_rs = np.ascontiguousarray(e_residual, dtype=np.float64).ravel()
     modes = np.zeros(e_sh.size, dtype=np.int32)
-    lam = C.c_double(0.0)
+    lam, prev = C.c_double(0.0), C.c_double(0.0)
     fits = _lib.fdkv_ref_route_budget(e_sh, e_rs, e_sh.size, np.ascontiguousarray(om, dtype=np.float64), float(bytes_exact_unit),
-                                      float(budget_bytes), C.byref(lam), modes)
-    return bool(fits), float(lam.value), modes
+                                      float(budget_bytes), float(lam_lo), float(ratio), int(max_steps), C.byref(lam),
+                                      C.byref(prev), modes)
+    return bool(fits), float(lam.value), modes, float(prev.value)
 
 
 def attention(khat, vhat, q) -> np.ndarray:

@@ -395,7 +395,7 @@ def test_token_rule_candidates_probe_and_attention_vs_bruteforce():
 
 
 # ---------------------------------------------------------------- budgeted routing
-def test_route_budget_is_the_smallest_lambda_that_fits():
+def test_route_budget_scan_brackets_the_smallest_lambda_that_fits():
     rng = np.random.default_rng(90)
     n = 40
     e_sh = rng.lognormal(3.0, 1.0, n)
@@ -410,25 +410,28 @@ def test_route_budget_is_the_smallest_lambda_that_fits():
     grid = np.concatenate([[0.0], np.geomspace(1e-3, 1e6, 400)])
     fp = np.array([footprint(l) for l in grid])
     assert np.all(np.diff(fp) <= 1e-6)
+    # the analytic threshold: the footprint only changes where two loss lines of a unit cross
+    cross = np.concatenate([(e_sh - e_rs) / (om[1] - om[0]), e_rs / (om[2] - om[1]), e_sh / (om[2] - om[0])])
     for frac in (1.0, 0.9, 0.7, 0.6, 0.55, 0.5):
         budget = frac * n * unit
-        fits, lam, modes = R.route_budget(e_sh, e_rs, om, unit, budget)
+        fits, lam, modes, prev = R.route_budget(e_sh, e_rs, om, unit, budget)
         assert fits
         assert footprint(lam) <= budget
         assert [R.mode_rule(a, b, om, lam)[0] for a, b in zip(e_sh, e_rs)] == modes.tolist()
         if lam > 0:
-            assert footprint(lam * (1 - 1e-9)) > budget            # minimal: anything smaller does not fit
-            assert not np.any((grid < lam * (1 - 1e-9)) & (fp <= budget))
+            assert footprint(prev) > budget and prev < lam <= max(prev * (1 + 2.0 ** -11), 1e-9)
+            assert not np.any((grid <= prev) & (fp <= budget))
+            assert np.any((cross > prev) & (cross <= lam))         # a crossing inside the bracket explains the step
         else:
-            assert np.all(modes == R.EXACT)
+            assert np.all(modes == R.EXACT) and prev == -1.0
     # below the all-shared footprint nothing fits
-    fits, lam, modes = R.route_budget(e_sh, e_rs, om, unit, 0.49 * n * unit)
+    fits, lam, modes, _ = R.route_budget(e_sh, e_rs, om, unit, 0.49 * n * unit)
     assert not fits and np.isinf(lam) and np.all(modes == 0)
     # one unit, by hand: shared<->residual crossing at (100-10)/(0.59375-0.5) = 960, residual<->exact at 10/0.40625
-    fits, lam, modes = R.route_budget([100.0], [10.0], om, unit, 0.6 * unit)
-    assert fits and modes.tolist() == [1] and lam == pytest.approx(10.0 / (1 - 0.59375), rel=1e-9)
-    fits, lam, modes = R.route_budget([100.0], [10.0], om, unit, 0.5 * unit)
-    assert fits and modes.tolist() == [0] and lam == pytest.approx(90.0 / 0.09375, rel=1e-9)
+    fits, lam, modes, prev = R.route_budget([100.0], [10.0], om, unit, 0.6 * unit)
+    assert fits and modes.tolist() == [1] and prev < 10.0 / (1 - 0.59375) <= lam
+    fits, lam, modes, prev = R.route_budget([100.0], [10.0], om, unit, 0.5 * unit)
+    assert fits and modes.tolist() == [0] and prev < 90.0 / 0.09375 <= lam and lam / prev < 1.001
 
 
 # ---------------------------------------------------------------------------------------------------------
