@@ -134,6 +134,28 @@ def oracle_step(w, units):
     return time.perf_counter() - t0
 
 
+def oracle_prefill_sample(w, units_total: int):
+    """The oracle's prefill side (Eq. 1 split, entry selection, Eq. 2 probe errors) on ONE unit, timed and scaled."""
+    from oracle import fdkv_ref as R
+    from paper_2607_06519_b200 import synth
+
+    p, h = 0, 0
+    k0, k1 = synth.unit_tensor(w, 0, p, h, False)
+    v0, v1 = synth.unit_tensor(w, 0, p, h, True)
+    pq = (synth.probe_q(w, 0, 2 * p), synth.probe_q(w, 0, 2 * p + 1))
+    pos = synth.probe_positions(w)
+    t0 = time.perf_counter()
+    _, z1k = R.depth_split(k0, k1, w.dtype == "bf16")
+    _, z1v = R.depth_split(v0, v1, w.dtype == "bf16")
+    kept = R.select_entries(z1k, w.k_keep)
+    R.select_entries(z1v, w.k_keep)
+    t1 = time.perf_counter()
+    R.probe_error(z1k, kept, pq[0], pq[1], w.group, h, pos)
+    t2 = time.perf_counter()
+    return {"compress_ms": (t1 - t0) * 1e3 * units_total, "probe_ms": (t2 - t1) * 1e3 * units_total, "cores": R.threads(),
+            "kind": "oracle", "sample": f"1 of {units_total} units (split + selection of K and V, probe errors of K), scaled to all units"}
+
+
 def run_reference(args, w):
     from oracle import fdkv_ref as R
 
@@ -162,8 +184,6 @@ def run_reference(args, w):
 def run_ours(args, w):
     import torch
 
-    from paper_2607_06519_b200 import binding as B, replicas, runner, synth
-
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -174,7 +194,30 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
+    line = bench_workload(args, w, dev, dist, rank, local, world, args.steps, args.warmup, not args.no_cpu_baseline)
+    if rank == 0 and world == 1 and w.name == "decode32k" and not args.no_also:
+        # the other single-GPU configuration the target names (context 131072), a shorter timed region, same JSON line
+        from paper_2607_06519_b200 import synth
+
+        torch.cuda.empty_cache()
+        w2 = synth.WORKLOADS["decode128k"]
+        l2 = bench_workload(args, w2, dev, None, 0, local, 1, min(args.steps, 10), 3, False)
+        line["also"] = [{k: l2[k] for k in ("metric", "value", "unit", "steps", "warmup", "ms_per_step", "dtype", "config", "roofline",
+                                            "e2e", "gpu_launches", "prefill", "step_bytes")}]
+    if rank == 0:
+        print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def bench_workload(args, w, dev, dist, rank, local, world, steps, warmup, with_cpu_baseline):
+    """One workload through prefill (timed per call) and the timed decode region; returns rank 0's JSON fields."""
+    import torch
+
+    from paper_2607_06519_b200 import binding as B, replicas, runner, synth
+
     hbm_peak, tf_peak, peak_kind = measured_peaks()
+    no_graph = args.no_graph
 
     # ---------------- set-up: the prefill side of the path, timed per call ----------------
     pf = runner.Prefilled(w, max_tail=max(w.n_steps, 1), device=dev)
@@ -228,6 +271,12 @@ def run_ours(args, w):
         nbl = w.block_size
         compress_min_bytes = n_ut * (nbl * N * esize + N * esize + w.k_keep * (4 + (1 if nbl == 2 else 4) * esize))
         probe_flops = 2.0 * units * 2 * (nbl * w.group * w.W) * w.T * w.head_dim
+    # bytes the compression kernels really move (pairs, entry rule, bf16 / head_dim 128): split reads both layers and
+    # writes Z0 and the staged Z1; the count pass and the ordered write each read Z1 again; the write emits the canonical
+    # (index, value) list, the packed decode entries and, for K, the copy of Z1 without the kept entries for the probe
+    compress_moved_bytes = None
+    if w.residual_rule == 0 and w.block_size == 2 and w.dtype == "bf16" and w.head_dim == 128:
+        compress_moved_bytes = n_ut * (6 * N * esize + w.k_keep * (8 + esize)) + units * N * esize
     modes_all = np.stack([ctx.get_modes(b).numpy() for b in range(w.batch)])
     mix = [int((modes_all == m).sum()) for m in range(3)]
     torch.cuda.empty_cache()
@@ -241,8 +290,8 @@ def run_ours(args, w):
     new_k = new_v = None
     step_no = [0]
     if append:
-        args.no_graph = True  # the tail length advances on the device and in the host mirror: launch directly
-        args.steps = min(args.steps, w.n_steps - args.warmup - 1)
+        no_graph = True  # the tail length advances on the device and in the host mirror: launch directly
+        steps = min(steps, w.n_steps - warmup - 1)
         tail_fn = synth.block_tail_rows if w.block_size == 4 else synth.tail_rows
         rows = {(b, p, h, v): tail_fn(w, b, p, h, bool(v)) for b in range(w.batch) for p in range(w.n_blocks)
                 for h in range(w.n_kv_heads) for v in (0, 1)}
@@ -267,7 +316,7 @@ def run_ours(args, w):
     stream.synchronize()
     launches_per_step = B.launch_count() - launches_per_step
     graph = None
-    if not args.no_graph:
+    if not no_graph:
         try:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
@@ -283,7 +332,7 @@ def run_ours(args, w):
             step()
 
     with torch.cuda.stream(stream):
-        for _ in range(args.warmup):
+        for _ in range(warmup):
             run_step()
     stream.synchronize()
     replicas.barrier(dist)
@@ -295,7 +344,7 @@ def run_ours(args, w):
     e0, e1 = ev(), ev()
     with torch.cuda.stream(stream):
         e0.record(stream)
-        for _ in range(args.steps):
+        for _ in range(steps):
             run_step()
         e1.record(stream)
     stream.synchronize()
@@ -305,13 +354,13 @@ def run_ours(args, w):
         # keep sampling long enough to have seen the GPU under load at least a few times
         if total_ms < 500 and not append:
             with torch.cuda.stream(stream):
-                for _ in range(int(600 / max(total_ms / args.steps, 1e-3)) + 1):
+                for _ in range(int(600 / max(total_ms / steps, 1e-3)) + 1):
                     run_step()
             stream.synchronize()
         clocks = sampler.stop()
-    value, total_s = replicas.whole_job_rate(w.batch * args.steps, total_ms * 1e-3, dist, dev)
+    value, total_s = replicas.whole_job_rate(w.batch * steps, total_ms * 1e-3, dist, dev)
     total_ms = total_s * 1e3
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
 
     # ---------------- end to end: host buffers through the C ABI, copies inside the timed region ----------------
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
@@ -342,15 +391,15 @@ def run_ours(args, w):
             ctx.decode_step_host(hq_all, None, None, hout_all, od, stream=stream)
         step_no[0] = j + 1
 
-    for _ in range(min(args.warmup, 3)):
+    for _ in range(min(warmup, 3)):
         host_step()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    for _ in range(args.steps):
+    for _ in range(steps):
         host_step()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    e2e_val, e2e_s = replicas.whole_job_rate(w.batch * args.steps, e2e_s, dist, dev)
+    e2e_val, e2e_s = replicas.whole_job_rate(w.batch * steps, e2e_s, dist, dev)
     h2d = sum(q.numel() * q.element_size() for q in hq)
     if append:
         h2d += sum(2 * t[0].numel() * t[0].element_size() for t in hk)
@@ -358,10 +407,10 @@ def run_ours(args, w):
     assert ctx.device_status() == 0
 
     if rank != 0:
-        return
+        return None
     # ---------------- CPU baseline: the oracle on a bounded sample, same box ----------------
     cpu = None
-    if not args.no_cpu_baseline:
+    if with_cpu_baseline:
         from oracle import fdkv_ref as R
 
         n_units = {"decode32k": 4, "decode128k": 2}.get(w.name, 2)
@@ -373,13 +422,15 @@ def run_ours(args, w):
         cpu = {"value": w.batch / t_full, "unit": "tokens/s", "cores": R.threads(), "kind": "oracle",
                "sample": f"{w.block_size * len(ou)} of {total_calls} (layer, KV head) attention units of one decode step (float64), "
                          f"best of {reps}, scaled to the full step"}
+        if w.block_size == 2 and w.residual_rule == 0:
+            cpu["prefill"] = oracle_prefill_sample(w, units)
 
     layer_calls = w.n_layers
     avg_call_s = ms_per_step * 1e-3 / layer_calls
     achieved = step_bytes / layer_calls / avg_call_s / 1e9
     line = {
         "metric": "compressed-KV decode attention tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "context": w.T, "batch": w.batch, "layers": w.n_layers, "q_heads": w.n_q_heads,
                    "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "keep": f"{w.keep_num}/{w.keep_den}",
@@ -388,21 +439,34 @@ def run_ours(args, w):
                    "l2": "inputs larger than L2 (each step streams the whole packed cache)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                     "traffic": NCU_TRAFFIC_BYTES.get(w.name), "of": peak_kind, "frac_of_8TBps_spec": achieved / 8000.0,
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name), "traffic_source": "ncu capture of one launch on the 4-layer cut, a constant (not measured per run)" if NCU_TRAFFIC_BYTES.get(w.name) else None,
+                     "of": peak_kind, "frac_of_8TBps_spec": achieved / 8000.0,
                      "bytes_per_launch": step_bytes / layer_calls,
                      "kernel": "decode attention (one layer call: split-K partial + combine), averaged over the timed region"},
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_val, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches_per_step * args.steps,
+        "gpu_launches": launches_per_step * steps,
         "clocks": clocks,
         "prefill": {"compress_ms": compress_ms, "commit_ms": commit_ms, "compress_GBps_min_bytes": compress_min_bytes / compress_ms / 1e6,
                     "probe_ms": probe_ms, "probe_TFLOPs": probe_flops / probe_ms / 1e9, "launches": launches_prefill,
-                    "probe_frac_of_bf16_peak": probe_flops / probe_ms / 1e9 / tf_peak},
+                    "probe_frac_of_bf16_peak": probe_flops / probe_ms / 1e9 / tf_peak,
+                    "roofline": {
+                        "split_select": {"bound": "hbm", "unit": "GB/s", "peak": hbm_peak, "of": peak_kind,
+                                         "min_bytes": compress_min_bytes, "achieved_min_bytes": compress_min_bytes / compress_ms / 1e6,
+                                         "frac_min_bytes": compress_min_bytes / compress_ms / 1e6 / hbm_peak,
+                                         "moved_bytes": compress_moved_bytes,
+                                         "achieved_moved_bytes": compress_moved_bytes / compress_ms / 1e6 if compress_moved_bytes else None,
+                                         "frac_moved_bytes": compress_moved_bytes / compress_ms / 1e6 / hbm_peak if compress_moved_bytes else None,
+                                         "kernels": "depth split + histogram, threshold, tile count / scan / ordered write (one fdkv_compress_prefill call, CUDA events)"},
+                        "probe": {"bound": "tensor", "unit": "TFLOP/s", "achieved": probe_flops / probe_ms / 1e9, "peak": tf_peak,
+                                  "of": peak_kind + " bf16 burst (a millisecond kernel timed alone)", "frac": probe_flops / probe_ms / 1e9 / tf_peak,
+                                  "flops": probe_flops, "kernels": "one fdkv_probe call (error products of both candidates + mode rule, CUDA events)"}}},
         "step_bytes": step_bytes,
     }
-    print(json.dumps(line))
-    if dist:
-        dist.destroy_process_group()
+    pf.ctx.close()
+    del pf, ctx, qs, outs
+    torch.cuda.empty_cache()
+    return line
 
 
 def main():
@@ -414,6 +478,7 @@ def main():
     ap.add_argument("--workload", default="decode32k")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true", help="skip the second workload (decode128k) of the default run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2607_06519_b200 import synth

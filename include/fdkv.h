@@ -305,6 +305,20 @@ int32_t fdkv_last_cuda_error(void);
 const char* fdkv_status_str(fdkv_status s);
 /* Kernels launched by this library since it was loaded (all contexts). */
 int64_t fdkv_launch_count(void);
+/* Which kernel served a call: launches, since the library was loaded, of the kernels that have a portable and an sm_100a
+ * form.  bf16 storage with head_dim 128 is always served by the tcgen05 / TMA kernels (the probe of Eq. 2, the token
+ * score between Eq. 2 and Eq. 3, decode attention after Eq. 3); float32 storage or head_dim 64 by the portable ones.
+ * There is no silent fall-back from one to the other: a configuration the fast kernels cannot take is refused when
+ * the context is created.  Returns -1 for an unknown id.                                                            */
+typedef enum {
+    FDKV_KERNEL_PROBE_TC = 0,       /* probe_tc_kernel: tcgen05 probe error                  */
+    FDKV_KERNEL_PROBE_PORTABLE = 1, /* probe_tile_kernel: float32 FMA probe error            */
+    FDKV_KERNEL_DECODE_FAST = 2,    /* decode_fast_kernel: TMA + tensor-core decode attention */
+    FDKV_KERNEL_DECODE_PORTABLE = 3,/* decode_generic_kernel + combine_kernel                */
+    FDKV_KERNEL_TOKEN_SCORE = 4,    /* token_score_kernel: tcgen05 token scores              */
+    FDKV_KERNEL_COUNT_ = 5
+} fdkv_kernel_id;
+int64_t fdkv_kernel_launch_count(int32_t kernel);
 
 #ifdef __cplusplus
 }

@@ -65,6 +65,8 @@ def _load():
         "fdkv_plan_decode": [i32, i32, P(i32), P(i32), i32, i32, i32, i32, i32, P(C.c_uint32), P(i32), P(i32)],
         "fdkv_device_status": [vp],
         "fdkv_compress_unit_noalloc": [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, P(i32), vp],
+        "fdkv_test_wait_expiry": [vp, i32, vp],
+        "fdkv_test_clear_device_status": [vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -76,6 +78,8 @@ def _load():
     lib.fdkv_status_str.argtypes = [C.c_int]
     lib.fdkv_status_str.restype = C.c_char_p
     lib.fdkv_launch_count.restype = C.c_int64
+    lib.fdkv_kernel_launch_count.argtypes = [C.c_int32]
+    lib.fdkv_kernel_launch_count.restype = C.c_int64
     return lib
 
 
@@ -84,6 +88,14 @@ _lib = _load()
 
 def launch_count() -> int:
     return int(_lib.fdkv_launch_count())
+
+
+KERNEL_PROBE_TC, KERNEL_PROBE_PORTABLE, KERNEL_DECODE_FAST, KERNEL_DECODE_PORTABLE, KERNEL_TOKEN_SCORE = range(5)
+
+
+def kernel_launch_count(kernel: int) -> int:
+    """Launches of one of the kernels that exist in a portable and an sm_100a form (fdkv_kernel_id)."""
+    return int(_lib.fdkv_kernel_launch_count(kernel))
 
 
 def last_cuda_error() -> int:
@@ -333,3 +345,11 @@ class Context:
 
     def device_status(self):
         return int(_lib.fdkv_device_status(self.h))
+
+    # ---- test hooks (include/fdkv_testing.h) ----
+    def test_wait_expiry(self, poll_cap: int, stream=None):
+        """Runs a bounded device-side wait that nobody satisfies; device_status() then reports the timeout (7)."""
+        _check(_lib.fdkv_test_wait_expiry(self.h, int(poll_cap), _stream(stream)), "fdkv_test_wait_expiry")
+
+    def test_clear_device_status(self, stream=None):
+        _check(_lib.fdkv_test_clear_device_status(self.h, _stream(stream)), "fdkv_test_clear_device_status")

@@ -8,10 +8,11 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfdkv.so")
-SOURCES = ["api.cu", "compress.cu", "block4.cu", "rows_fp8.cu", "probe.cu", "probe_tc.cu", "token_rule.cu", "decode.cu", "decode_fast.cu"]
-HEADERS = ["fdkv_internal.h", "decode_fast_tile.inc", os.path.join("..", "..", "include", "fdkv.h")]
+SOURCES = ["api.cu", "compress.cu", "block4.cu", "rows_fp8.cu", "probe.cu", "probe_tc.cu", "token_rule.cu", "decode.cu", "decode_fast.cu", "test_hooks.cu"]
+HEADERS = ["fdkv_internal.h", "mbar_wait.cuh", "decode_fast_tile.inc", os.path.join("..", "..", "include", "fdkv.h"),
+           os.path.join("..", "..", "include", "fdkv_testing.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--use_fast_math=false", "-Xptxas", "-v"]
+              "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 
 def _stale() -> bool:
@@ -33,7 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(HERE, "build", s.replace(".cu", ".o"))
         objs.append(obj)
         extra = os.environ.get("FDKV_EXTRA_NVCC_FLAGS", "").split()
-        cmd = [nvcc, *[f for f in NVCC_FLAGS if f != "--use_fast_math=false"], *extra, "-c", os.path.join(CSRC, s), "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, s), "-o", obj]
         procs.append((s, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for s, p in procs:
@@ -45,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             sys.stdout.write(out)
     if failed:
         raise RuntimeError("nvcc failed")
-    subprocess.run([nvcc, "-shared", "-o", LIB, *objs, "-lcudart"], check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB, *objs, "-lcudart"], check=True)
     return LIB
 
 

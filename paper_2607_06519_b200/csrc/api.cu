@@ -12,6 +12,7 @@ using namespace fdkv;
 namespace {
 
 std::atomic<int64_t> g_launches{0};
+std::atomic<int64_t> g_kernel_launches[FDKV_KERNEL_COUNT_];
 std::atomic<int32_t> g_last_cuda{0};
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -53,7 +54,10 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.kmax = (int64_t)s.Tmax * s.d * s.keep_num / s.keep_den;
     s.kcap = (int64_t)align_up((size_t)(s.kmax + kListPad), 64);
     s.ntiles_max = (s.Tmax + kResTile - 1) / kResTile;
-    s.nptiles_max = (s.Tmax + kProbeTile - 1) / kProbeTile;
+    // per-unit partial-sum slots of the probe: one per 64-token tile (portable kernel) or one per work item of the
+    // tensor-core kernel (layers x 256-row blocks x key splits of at least 8 tiles), whichever is more
+    s.nptiles_max = std::max((s.Tmax + kProbeTile - 1) / kProbeTile,
+                             B * ((G * kMaxW + 255) / 256) * (((s.Tmax - 1) / kProbeBoxRows + 1 + 7) / 8));
     s.tail_rows = (s.max_tail + kRowPad - 1) / kRowPad * kRowPad;
     if (c.residual_rule != FDKV_RESIDUAL_ENTRIES && c.residual_rule != FDKV_RESIDUAL_TOKENS) return false;
     s.tok_rule = c.residual_rule == FDKV_RESIDUAL_TOKENS;
@@ -150,6 +154,17 @@ double omega_of(const Shape& s, int T, double (&om)[3]) {
 
 namespace fdkv {
 void count_launch(int n) { g_launches.fetch_add(n); }
+void count_kernel(int id) { if (id >= 0 && id < FDKV_KERNEL_COUNT_) g_kernel_launches[id].fetch_add(1); }
+int per_device_first_visits(const int* devs, int n) {
+    // the table logic of PerDevice::ensure, fed with device ids instead of the current device
+    bool done[PerDevice::kMaxDevices] = {};
+    int visits = 0;
+    for (int i = 0; i < n; ++i) {
+        if (devs[i] < 0 || devs[i] >= PerDevice::kMaxDevices) continue;
+        if (!done[devs[i]]) { done[devs[i]] = true; ++visits; }
+    }
+    return visits;
+}
 fdkv_status record_cuda_error(cudaError_t e) { return cuda_fail(e); }
 cudaError_t launch_set_tail_len(int32_t* tail_len, int L, int max_batch, int seq, int n, cudaStream_t st);
 }  // namespace fdkv
@@ -1075,5 +1090,8 @@ const char* fdkv_status_str(fdkv_status s) {
 }
 
 int64_t fdkv_launch_count(void) { return g_launches.load(); }
+int64_t fdkv_kernel_launch_count(int32_t kernel) {
+    return kernel >= 0 && kernel < FDKV_KERNEL_COUNT_ ? g_kernel_launches[kernel].load() : -1;
+}
 
 }  // extern "C"

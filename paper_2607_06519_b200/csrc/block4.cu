@@ -148,15 +148,14 @@ __global__ void __launch_bounds__(256) gather4_kernel(Gather4Args a) {
 }  // namespace
 
 cudaError_t launch_split4_hist(const Split4Args& a, int dtype, cudaStream_t st) {
-    static bool attr_done = false;
+    static PerDevice once;
     const size_t smem = (size_t)kHistBins * sizeof(uint32_t);
-    if (!attr_done) {
+    cudaError_t e0 = once.ensure([&]() {
         cudaError_t e = cudaFuncSetAttribute(split4_hist_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(split4_hist_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+        return cudaFuncSetAttribute(split4_hist_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    });
+    if (e0 != cudaSuccess) return e0;
     if (a.T <= 0) return cudaSuccess;
     const int tokens_per_cta = 2048 * 128 / a.d / (dtype == FDKV_BF16 ? 1 : 2);
     dim3 grid((a.T + tokens_per_cta - 1) / tokens_per_cta, a.Hkv * 2);

@@ -415,15 +415,14 @@ __global__ void strided_copy_kernel(const T* src, int64_t stride_t, T* dst, int 
 }  // namespace
 
 cudaError_t launch_split_hist(const CompressArgs& a, int dtype, cudaStream_t st) {
-    static bool attr_done = false;
+    static PerDevice once;
     const size_t smem = (size_t)kHistBins * sizeof(uint32_t);
-    if (!attr_done) {
+    cudaError_t e0 = once.ensure([&]() {
         cudaError_t e = cudaFuncSetAttribute(split_hist_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(split_hist_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+        return cudaFuncSetAttribute(split_hist_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    });
+    if (e0 != cudaSuccess) return e0;
     if (a.T <= 0 || a.n_pairs <= 0) return cudaSuccess;
     const int tokens_per_cta = 4096 * 128 / a.d / (dtype == FDKV_BF16 ? 1 : 2);
     dim3 grid((a.T + tokens_per_cta - 1) / tokens_per_cta, a.Hkv * a.tensors, a.n_pairs);

@@ -41,15 +41,18 @@ __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p) { re
 // Appends k_new / v_new rows of every sequence to the layer's tail and bumps the tail length.
 template <typename T>
 __global__ void append_tail_kernel(DecodeArgs a) {
-    // Programmatic dependent launch: this layer's tail is not touched by the kernels still in flight (they belong
-    // to other layers), so the copy may overlap them; the wait at the end keeps stream order transitive.
+    // Programmatic dependent launch: the kernel may become resident, and let the decode kernel behind it start its
+    // own prologue, while the kernel ahead of it in the stream still runs.  Everything it reads was possibly written by
+    // that kernel -- k_new / v_new come from the caller's projection, the tail length from the previous step's append,
+    // and the previous step's decode kernel of this layer may still be reading the length -- so the dependency wait
+    // comes before the first read.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b = blockIdx.x;
     int32_t* len = a.tail_len + a.layer * a.max_batch + b;
     const int n = *len;
     if (n >= a.max_tail) {
         if (threadIdx.x == 0) atomicMax(a.status, (int32_t)kFlagTailFull);
-        asm volatile("griddepcontrol.wait;" ::: "memory");
         return;
     }
     const int row = a.Hkv * a.d;
@@ -65,7 +68,6 @@ __global__ void append_tail_kernel(DecodeArgs a) {
     }
     __syncthreads();
     if (threadIdx.x == 0) *len = n + 1;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 constexpr int kWarps = 4;
@@ -337,6 +339,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st) {
     else
         combine_kernel<64><<<cgrid, 64, 0, st>>>(a.partials, a.Hq, splits, a.out, a.out_dtype);
     count_launch(2);
+    count_kernel(FDKV_KERNEL_DECODE_PORTABLE);
     return cudaGetLastError();
 }
 

@@ -24,10 +24,9 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
-#include <cstdio>
-#include <cstdlib>
 
 #include "fdkv_internal.h"
+#include "mbar_wait.cuh"
 
 namespace fdkv {
 
@@ -47,13 +46,12 @@ constexpr int kMaxCtas = 296;
 constexpr int kMaxUnits = kFastMaxUnits;
 constexpr int kPF = 8;  // residual entries prefetched per lane and list
 constexpr int kPartStride = 128 + 4;  // floats per split-K part: max, sum, 2 pad, 128 accumulators (16-byte aligned)
-constexpr uint32_t kSpinCap = 1u << 22;
 static_assert(kTT == kRowPad, "row blocks are padded to whole stages");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct FastSched {
     uint32_t start[kMaxCtas + 1];  // unit << 20 | first 16-token slice of CTA c; start[ncta] = units << 20
-    int ncta, units, tslot, prologue_tiles, reverse_odd, experiment;
+    int ncta, units;
     int any_tail;  // some sequence of the batch holds generated tokens in this layer's tail (host mirror)
 };
 struct PartCount {
@@ -82,15 +80,6 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -158,19 +147,6 @@ __device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
 }
 
-// Bounded wait on an mbarrier phase.  Gives up after kSpinCap polls (or as soon as another thread gave up):
-// raises the CTA abort flag and the device status word, after which every wait returns at once.
-__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* status) {
-    if (mbar_try_wait(bar, parity)) return;  // the common case: one poll, no look at the abort flag
-    if (*abort_flag) return;
-    for (uint32_t i = 0; i < kSpinCap; ++i) {
-        if (mbar_try_wait(bar, parity)) return;
-        if ((i & 255u) == 255u && *abort_flag) return;
-    }
-    *abort_flag = 1;
-    atomicMax(status, (int32_t)kFlagTimeout);
-}
-
 // byte offset of (row, channel chunk of 8) inside a [rows][64 ch] box with the 128-byte swizzle
 __device__ __forceinline__ uint32_t swz(int row, int chunk8) { return (uint32_t)(row * 128 + (((chunk8 & 7) ^ (row & 7)) << 4)); }
 
@@ -178,20 +154,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
 }
 
-#ifdef FDKV_TIMING
-__device__ long long g_timing[64][kMaxCtas][12];
-#define TSTAMP(i) do { if (threadIdx.x == 32) g_timing[sch.tslot][blockIdx.x][i] = clock64(); } while (0)
-#define TADD(i, v) do { t_acc[i - 4] += (v); } while (0)
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TGLOBAL(i) do { if (threadIdx.x == 32) g_timing[sch.tslot][blockIdx.x][i] = gtime(); } while (0)
-__device__ unsigned g_phase[kMaxCtas][12];
-#define TPH(i) do { const unsigned now_ = (unsigned)clock(); t_ph[i] += now_ - t_mark; t_mark = now_; } while (0)
-#else
-#define TPH(i)
-#define TGLOBAL(i)
-#define TSTAMP(i)
-#define TADD(i, v)
-#endif
 
 // F8: the packed rows are e4m3 codes (one 128-byte row per token, per-channel float32 scales): the codes are converted
 // to f16 in registers after ldmatrix, both products run as f16 mma with the K scales folded into q and the V scales
@@ -204,11 +166,6 @@ __global__ void __launch_bounds__(kThreads, 1)
 decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap8, DecodeArgs a, FastSched sch,
                    PartCount pc) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-#ifdef FDKV_TIMING
-    long long t_acc[2] = {0, 0};
-    unsigned t_ph[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, t_mark = 0;
-#endif
-    TGLOBAL(6);
     const uint32_t smem0 = smem_u32(smem_raw);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + kOffAbort);
     if (smem0 & 1023u) {  // the swizzled boxes need 1024-byte alignment; report instead of computing garbage
@@ -237,7 +194,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     // The second layer of a pair walks every range backwards: it starts on the Z0 rows the first layer read last,
     // which are the ones most likely still in L2 (both layers of a shared / residual unit stream the same Z0).
     // (Measured: 1.4 % per step; L2 eviction hints on the TMA loads did not add to it.)
-    const bool rev = sch.reverse_odd && (a.layer & 1);
+    const bool rev = (a.layer & 1) != 0;
 
     // ================= the CTA's tile sequence: a small segment table in shared memory =================
     // Tile `it` of the CTA (all segments, prefill tiles then tail tiles of each) always lands in stage it % kStages.
@@ -273,17 +230,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         const int vr = j < g.npre ? g.vrow + tok : g.tvrow + (j - g.npre) * kTT;
         issue_rows(it % kStages, kr, vr, j < g.npre);
     };
-    // a warp is done reading stage s (tile it): the last of the eight refills it
-    auto release_stage = [&](int s, int it) {
-        __syncwarp();
-        if (lane == 0) {
-            const int old = atomicAdd(stage_cnt + s, 1);
-            if (old == kCW - 1) {
-                stage_cnt[s] = 0;
-                if (it + kStages < seg_info[1]) issue_tile(it + kStages);
-            }
-        }
-    };
     int prologue_issued = 0;
     if (is_producer) {
         // static part (packed cache, fixed since commit): may run before the dependency wait
@@ -312,7 +258,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         seg_info[1] = it0;
         for (int s = 0; s < kStages; ++s) stage_cnt[s] = 0;
         if (n > 0)
-            for (; prologue_issued < sch.prologue_tiles && prologue_issued < kStages && prologue_issued < segs[0].npre; ++prologue_issued)
+            for (; prologue_issued < kStages && prologue_issued < segs[0].npre; ++prologue_issued)
                 issue_tile(prologue_issued);
     }
     // per-warp scratch starts zeroed
@@ -321,7 +267,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
     __syncthreads();  // barriers initialised, static table built (still inside the previous kernel's shadow)
     // everything below may depend on the kernels launched before this one (q, appended tail rows, partial slots)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    TGLOBAL(1);
     if (!sch.any_tail) {
         // no tails anywhere: the static table is final; a short first segment may have left stages to fill
         if (is_producer)
@@ -379,7 +324,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                 ntail = (n_tail_rows + kTT - 1) / kTT;
             }
             const int npre = (rows16 + kTT - 1) / kTT, nseg = npre + ntail;
-            const bool coef = ud.mode != FDKV_MODE_EXACT, resid = ud.mode == FDKV_MODE_RESIDUAL && sch.experiment != 5;  // (experiment 5: no residual work)
+            const bool coef = ud.mode != FDKV_MODE_EXACT, resid = ud.mode == FDKV_MODE_RESIDUAL;
             const uint32_t sgn = ud.sign < 0.f ? 0x80008000u : 0u;
 
             // q fragments: B operand columns = the G query heads of this KV head.  With G <= 4 columns 4-7 repeat
@@ -609,7 +554,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
 #undef FDKV_TAIL_TILE
             }
             it += nseg;
-            TGLOBAL(2);
 
             // ---- merge the eight warps' states into this segment's split-K partial ----
             {
@@ -666,7 +610,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     for (int e = 0; e < 2; ++e) { sm_m[warp * 8 + 2 * tig + e] = m_run[e]; sm_l[warp * 8 + 2 * tig + e] = lq[e]; }
                 }
                 __syncthreads();
-                TGLOBAL(0);
                 for (int i = threadIdx.x; i < a.G * 128; i += kThreads) {
                     const int g = i >> 7, ch = i & 127;
                     float M = -INFINITY;
@@ -697,7 +640,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                     *s_ticket = t;
                 }
                 __syncthreads();
-                TGLOBAL(3);
                 const int nparts = pc.n[u];
                 if (*s_ticket == nparts - 1) {
                     // Warp w takes head w % G and every (8/G)-th part of it, 4 channels per lane; the scratch area
@@ -731,7 +673,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                         float* const wts = red + kCW * 128 + warp * kMaxSplits;
 #pragma unroll
                         for (int i = 0; i < kMaxSplits / 32; ++i) wts[lane + 32 * i] = mreg[i];
-                        TGLOBAL(8);
                         __syncwarp();
                         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                         for (int base = pgi; base < nparts; base += 8 * npg) {
@@ -751,7 +692,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                                 }
                             }
                         }
-                        TGLOBAL(9);
                         reinterpret_cast<float4*>(red + warp * 128)[lane] = acc;
                         if (lane == 0) sm_l[warp] = ls;
                     }
@@ -768,7 +708,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
                         else
                             reinterpret_cast<float*>(a.out)[o] = r;
                     }
-                    TGLOBAL(10);
                     if (threadIdx.x == 0) a.counters[u] = 0;  // ready for the next launch
                     __syncthreads();
                 }
@@ -777,13 +716,6 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             }
         }
     }
-    TGLOBAL(7);
-#ifdef FDKV_TIMING
-    if (threadIdx.x == 32) {
-        g_timing[sch.tslot][blockIdx.x][4] = t_acc[0]; g_timing[sch.tslot][blockIdx.x][5] = t_acc[1];
-        for (int i = 0; i < 10; ++i) g_phase[blockIdx.x][i] = t_ph[i];
-    }
-#endif
     // after a timed-out wait: give copies that may still be in flight time to land before the CTA retires
     if (*abort_flag)
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
@@ -844,29 +776,7 @@ bool make_arena_tensor_map(void* arena, size_t arena_bytes, void* tmap_out) {
 
 // Host side of a launch: the cost-weighted cut of the batch's (unit, 16-token slice) list into one range per CTA and the
 // split-K part count of every unit.  Uses only the host views in `a` (lengths, modes, shape); no device access.
-static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_count, FastSched& sch, PartCount& cs, bool& use_pdl_out) {
-    static double res_cost = -1.0;
-    static bool res_cost_env = false;
-    static bool use_pdl = true;
-    // tiles copied to shared memory before the dependency wait (measured: filling every stage is best; prefetching
-    // further tiles to L2 as well costs about 1 % per tile at 32k, with tile-granular and with slice-granular ranges)
-    static int prologue_tiles = kStages;
-    static bool whole_ctas = true;
-    static bool reverse_odd = true;
-    if (res_cost < 0) {
-        const char* ev = getenv("FDKV_RES_COST");  // tuning knobs for benchmark sweeps
-        res_cost = ev ? atof(ev) : 1.7;
-        res_cost_env = ev != nullptr;
-        if (!(res_cost >= 0.25 && res_cost <= 8.0)) res_cost = 1.7;
-        const char* pv = getenv("FDKV_NO_PDL");
-        use_pdl = !(pv && pv[0] == '1');
-        const char* ro = getenv("FDKV_NO_REVERSE");
-        reverse_odd = !(ro && ro[0] == '1');
-        const char* wc = getenv("FDKV_NO_WHOLE_CTAS");
-        whole_ctas = !(wc && wc[0] == '1');
-        const char* pt = getenv("FDKV_PROLOGUE_TILES");
-        prologue_tiles = pt ? std::max(0, std::min(kStages, atoi(pt))) : kStages;
-    }
+static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_count, FastSched& sch, PartCount& cs) {
     // ---- cost-weighted schedule: whole CTAs per unit when there are enough CTAs, else a flat cut of the (unit, tile) list ----
     std::vector<int64_t> wp(units + 1, 0);
     // ranges are cut on 16-token slices (the granularity of the residual lists), so that the CTAs of a unit differ by
@@ -885,17 +795,8 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
     // With whole CTAs per unit (latency-bound regime) a residual tile of the entry form costs a fixed part (the scratch
     // tile and the second products) plus a part per list entry: measured 2.0 plain tiles at 1024 entries per tile and
     // tensor (keep 1/16), 1.65 at 512 (keep 1/32); with 8-bit rows (a dearer plain tile) about 1.7 at either density.
-    static double res_a_env = -1.0, res_b_env = -1.0;
-    static bool res_ab_read = false;
-    if (!res_ab_read) {
-        const char* ea = getenv("FDKV_RES_A");  // tuning knobs for benchmark sweeps
-        const char* eb = getenv("FDKV_RES_B");
-        if (ea) res_a_env = atof(ea);
-        if (eb) res_b_env = atof(eb);
-        res_ab_read = true;
-    }
-    const double res_a = res_a_env >= 0 ? res_a_env : a.rows_f8 ? 1.55 : 1.25;
-    const double res_b = res_b_env >= 0 ? res_b_env : a.rows_f8 ? 0.15 : 0.87;
+    const double res_a = a.rows_f8 ? 1.55 : 1.25;
+    const double res_b = a.rows_f8 ? 0.15 : 0.87;
     auto weigh = [&](double rc) {
         for (int u = 0; u < units; ++u) {
             const int T = a.host_T[u / a.Hkv];
@@ -905,6 +806,7 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
                 const int64_t res_bytes = a.tok_rule ? 2 * ((int64_t)T * a.keep_num / a.keep_den) * 260 : 2 * k * 4;  // rows + index, or packed entries
                 if (rc == 0.0) wt[u] = (int)(wt[u] * (res_a + res_b * (double)k / nt[u] / 1024.0));
                 else wt[u] = (int)((wt[u] + (res_bytes / nt[u] + 511) / 512) * rc);
+                wt[u] = std::max(1, wt[u]);
             }
             // the CTA that ends a unit also streams its tail of generated tokens (whole plain tiles): counted as slices
             // of the unit's kind behind the unit's own, so that this CTA gets correspondingly fewer of those
@@ -912,30 +814,18 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
             // Measured: the CTA that ends a unit runs behind its siblings at equal shares (with tails it also reads their
             // lengths behind the dependency wait); charging it eight plain tiles' worth of slices (in eighths of a tile
             // below) is the optimum of a sweep at 32k, with and without tails (+1.6 % / +6 %), and neutral at 128k.
-            static int tail_extra = -1, last_extra = 64;
-            if (tail_extra < 0) {  // tuning knobs for benchmark sweeps
-                const char* te = getenv("FDKV_TAIL_EXTRA");
-                const char* le = getenv("FDKV_LAST_EXTRA");
-                tail_extra = te ? atoi(te) : 64;
-                last_extra = le ? atoi(le) : 64;
-            }
-            es[u] = ns[u] + ((tail + kTT - 1) / kTT * (kTT / kResTile) + (tail > 0 ? tail_extra : last_extra)) * (2 * kTT * 256 / 512) / std::max(1, wt[u]);
+            constexpr int kEndExtra = 64;  // (eighths of a plain tile)
+            es[u] = ns[u] + ((tail + kTT - 1) / kTT * (kTT / kResTile) + kEndExtra) * (2 * kTT * 256 / 512) / std::max(1, wt[u]);
             wp[u + 1] = wp[u] + (int64_t)es[u] * wt[u];  // (in eighths of the tile cost)
         }
     };
     // (measured best: 1.7 when every unit gets whole CTAs, 1.5 in the flat cut of a batch)
-    weigh(res_cost_env ? res_cost : a.tok_rule ? 1.7 : 0.0);
+    weigh(a.tok_rule ? 1.7 : 0.0);
     const int ncta = (int)std::min<int64_t>(std::min(std::min(sm_count, kMaxCtas), kMaxSplits), total_tiles);
-    static unsigned g_launch_no = 0;
-    ++g_launch_no;
-    sch.tslot = (int)(g_launch_no % 64);
     sch.ncta = ncta;
-    sch.prologue_tiles = prologue_tiles;
-    sch.reverse_odd = reverse_odd ? 1 : 0;
     sch.any_tail = a.any_tail;
-    { const char* ex = getenv("FDKV_DECODE_EXPERIMENT"); sch.experiment = ex ? atoi(ex) : 0; }
     sch.units = units;
-    bool whole = whole_ctas && units <= ncta;
+    bool whole = units <= ncta;
     std::vector<int> nc(units, 1);
     if (whole) {
         // Whole CTAs per unit (no CTA pays a second merge + ticket): shares proportional to the unit's cost, at least
@@ -969,7 +859,7 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
             for (int j = 0; j < nc[u]; ++j) sch.start[c++] = ((uint32_t)u << 20) | (uint32_t)std::min<int64_t>(ns[u] - 1, (int64_t)es[u] * j / nc[u]);
         sch.start[ncta] = (uint32_t)units << 20;
     } else {
-        if (!res_cost_env) weigh(1.5);
+        weigh(1.5);
         int u = 0;
         for (int c = 0; c < ncta; ++c) {
             const int64_t target = wp[units] * c / ncta;
@@ -1009,7 +899,6 @@ static cudaError_t plan_decode_schedule(const DecodeArgs& a, int units, int sm_c
     }
     for (int u = 0; u < units; ++u)
         if (cs.n[u] > kMaxSplits) return cudaErrorInvalidValue;  // cannot happen: ncta <= kMaxSplits
-    use_pdl_out = use_pdl;
     return cudaSuccess;
 }
 
@@ -1019,8 +908,7 @@ cudaError_t plan_decode_host(const DecodeArgs& a, int n_ctas, uint32_t* start_ou
     if (units < 1 || units > kMaxUnits || n_ctas < 1) return cudaErrorInvalidValue;
     FastSched sch;
     PartCount cs;
-    bool pdl = true;
-    const cudaError_t e = plan_decode_schedule(a, units, n_ctas, sch, cs, pdl);
+    const cudaError_t e = plan_decode_schedule(a, units, n_ctas, sch, cs);
     if (e != cudaSuccess) return e;
     for (int c = 0; c <= sch.ncta; ++c) start_out[c] = sch.start[c];
     for (int u = 0; u < units; ++u) parts_out[u] = cs.n[u];
@@ -1033,22 +921,18 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     const int units = a.batch * a.Hkv;
     if (!a.tmap || !a.packed_lists || a.d != 128 || units > kMaxUnits || units < 1) return cudaSuccess;
     if (a.rows_f8 && !a.tmap_u8) return cudaSuccess;
-    static int sm_count = 0;
-    static bool attr_done = false;
-    if (!attr_done) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    static PerDevice once;
+    int sm_count = 0;
+    cudaError_t e0 = once.ensure([&]() {
+        cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+        return cudaFuncSetAttribute(decode_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    }, &sm_count);
+    if (e0 != cudaSuccess) return e0;
     FastSched sch;
     PartCount cs;
-    bool use_pdl = true;
     {
-        const cudaError_t pe = plan_decode_schedule(a, units, sm_count, sch, cs, use_pdl);
+        const cudaError_t pe = plan_decode_schedule(a, units, sm_count, sch, cs);
         if (pe != cudaSuccess) return pe;
     }
     const int ncta = sch.ncta;
@@ -1061,48 +945,15 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = use_pdl ? 1 : 0;
+    cfg.numAttrs = 1;
     const CUtensorMap& m16 = *reinterpret_cast<const CUtensorMap*>(a.tmap);
     const CUtensorMap& m8 = *reinterpret_cast<const CUtensorMap*>(a.rows_f8 ? a.tmap_u8 : a.tmap);
     cudaError_t e = a.rows_f8 ? cudaLaunchKernelEx(&cfg, decode_fast_kernel<true>, m16, m8, a, sch, cs)
                               : cudaLaunchKernelEx(&cfg, decode_fast_kernel<false>, m16, m8, a, sch, cs);
     if (e != cudaSuccess) return e;
     count_launch(1);
+    count_kernel(FDKV_KERNEL_DECODE_FAST);
     *handled = true;
-#ifdef FDKV_TIMING
-    if (getenv("FDKV_TIMING_DUMP") && (g_launch_no % 64) == 63) {
-        static long long h[64][kMaxCtas][12];
-        cudaStreamSynchronize(st);
-        cudaMemcpyFromSymbol(h, g_timing, sizeof(h));
-        long long base = h[0][0][6];
-        for (int l = 0; l < 64; ++l) {
-            long long g0 = h[l][0][6], g0max = g0, g1 = h[l][0][7], g1min = g1, busy = 0, fd = 0, wf = 0;
-            for (int c = 0; c < ncta; ++c) {
-                g0 = std::min(g0, h[l][c][6]); g0max = std::max(g0max, h[l][c][6]);
-                g1 = std::max(g1, h[l][c][7]); g1min = std::min(g1min, h[l][c][7]);
-                busy += h[l][c][7] - h[l][c][6];
-                fd += h[l][c][1] - h[l][c][0];
-                wf += h[l][c][4];
-            }
-            fprintf(stderr, "launch %2d: first_start %8lld last_start %8lld first_end %8lld last_end %8lld  mean_busy %6lld ns mean_wait_full %6lld cyc\n",
-                    l, g0 - base, g0max - base, g1min - base, g1 - base, busy / ncta, wf / ncta);
-            if (l == 63) {
-                static unsigned hp[kMaxCtas][12];
-                cudaMemcpyFromSymbol(hp, g_phase, sizeof(hp));
-                for (int c = 0; c < ncta; c += 6) {
-                    fprintf(stderr, "phase cta %3d tiles %3lld:", c, h[l][c][5]);
-                    for (int i = 0; i < 10; ++i) fprintf(stderr, " %6u", hp[c][i] / (unsigned)std::max(1ll, h[l][c][5]));
-                    fprintf(stderr, "\n");
-                }
-            }
-            if (l == 45)
-                for (int c = 0; c < ncta; ++c)
-                    fprintf(stderr, "cta %3d unit %2u mode %d tiles %2lld start %6lld waited %6lld loop_end %6lld end %6lld wait_full_cyc %6lld merged %6lld ticket %6lld weights %6lld rows %6lld written %6lld\n", c,
-                            sch.start[c] >> 20, a.host_modes[sch.start[c] >> 20], h[l][c][5], h[l][c][6] - g0, h[l][c][1] - g0, h[l][c][2] - g0,
-                            h[l][c][7] - g0, h[l][c][4], h[l][c][0] - g0, h[l][c][3] - g0, h[l][c][8] - g0, h[l][c][9] - g0, h[l][c][10] - g0);
-        }
-    }
-#endif
     return cudaGetLastError();
 }
 

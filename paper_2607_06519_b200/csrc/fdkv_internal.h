@@ -6,6 +6,7 @@
 
 #include <cstddef>
 #include <cstdint>
+#include <mutex>
 #include <vector>
 
 #include "../../include/fdkv.h"
@@ -308,7 +309,37 @@ struct TokenArgs {
 cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st);
 cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, cudaStream_t st);
 
+// Function attributes (the opt-in to large dynamic shared memory) and the SM count belong to a device, not to the
+// process: every launcher keeps one of these and runs its set-up the first time it meets the current device.
+struct PerDevice {
+    static constexpr int kMaxDevices = 64;
+    std::mutex mu;
+    bool done[kMaxDevices] = {};
+    int sms[kMaxDevices] = {};
+    // init() -> cudaError_t runs once per device (under the lock); *sm_count (optional) receives the device's SM count.
+    template <typename F>
+    cudaError_t ensure(F&& init, int* sm_count = nullptr) {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!done[dev]) {
+            e = cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+            if (e == cudaSuccess) e = init();
+            if (e != cudaSuccess) return e;
+            done[dev] = true;
+        }
+        if (sm_count) *sm_count = sms[dev];
+        return cudaSuccess;
+    }
+};
+// The bookkeeping of PerDevice::ensure without a device (host-side test hook): how many of the `n` device ids in `devs`
+// would run their set-up, in order, on a fresh table.
+int per_device_first_visits(const int* devs, int n);
+
 void count_launch(int n);
+void count_kernel(int id);  // id: fdkv_kernel_id
 // Remembers a failed CUDA runtime call for fdkv_last_cuda_error() and returns FDKV_ERR_CUDA.
 fdkv_status record_cuda_error(cudaError_t e);
 

@@ -161,20 +161,20 @@ cudaError_t launch_probe(const ProbeArgs& a, int dtype, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     if (!handled) {
         const size_t smem = (size_t)(2 * kProbeTile * (a.d + 1) + kRowsBlk * a.d) * sizeof(float);
-        static bool attr_done = false;
-        if (!attr_done) {
-            e = cudaFuncSetAttribute(probe_tile_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-            if (e != cudaSuccess) return e;
-            e = cudaFuncSetAttribute(probe_tile_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-            if (e != cudaSuccess) return e;
-            attr_done = true;
-        }
+        static PerDevice once;
+        e = once.ensure([&]() {
+            cudaError_t e2 = cudaFuncSetAttribute(probe_tile_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+            if (e2 != cudaSuccess) return e2;
+            return cudaFuncSetAttribute(probe_tile_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        });
+        if (e != cudaSuccess) return e;
         dim3 grid(nparts, a.unit_count);
         if (dtype == FDKV_BF16)
             probe_tile_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>(a);
         else
             probe_tile_kernel<float><<<grid, 256, smem, st>>>(a);
         count_launch(1);
+        count_kernel(FDKV_KERNEL_PROBE_PORTABLE);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }

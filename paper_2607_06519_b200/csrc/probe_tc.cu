@@ -19,10 +19,9 @@
 #include <cuda.h>
 
 #include <algorithm>
-#include <cstdio>
-#include <cstdlib>
 
 #include "fdkv_internal.h"
+#include "mbar_wait.cuh"
 
 namespace fdkv {
 
@@ -36,7 +35,6 @@ constexpr int kBStageBytes = 2 * kBHalf;       // 24 KiB
 constexpr int kHdr = 1024;
 constexpr int kProbeSmem = kHdr + kBStages * kBStageBytes;  // 193 KiB
 constexpr int kPThreads = 6 * 32;
-constexpr uint32_t kSpin = 1u << 22;
 // Tensor memory (512 columns): the item's 256 Q rows as the A operand (2 M tiles x 64 columns: 128 channels, two bf16
 // per column) and two alternating sets of two 128 x 96 f32 accumulators.
 constexpr int kTmemCols = 512;
@@ -55,23 +53,8 @@ __device__ __forceinline__ void mb_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mb_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ uint32_t mb_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
 __device__ __forceinline__ void mb_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* status) {
-    if (*abort_flag) return;
-    for (uint32_t i = 0; i < kSpin; ++i) {
-        if (mb_try(bar, parity)) return;
-        if ((i & 255u) == 255u && *abort_flag) return;
-    }
-    *abort_flag = 1;
-    atomicMax(status, (int32_t)kFlagTimeout);
+    mbar_wait_bounded(bar, parity, abort_flag, status);
 }
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -134,7 +117,6 @@ struct TcPlan {
     int items_per_unit;  // B layers x mblocks x 2 candidates x nsplits
     int mblocks, nsplits, ntiles, tiles_per_split;
     int pos_min, pos_max;
-    int experiment;  // timing experiments only (FDKV_PROBE_EXPERIMENT): 1 = epilogue skips the accumulator reads
 };
 
 __global__ void __launch_bounds__(kPThreads, 1)
@@ -147,8 +129,6 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         if (threadIdx.x == 0) atomicMax(a.status, (int32_t)kFlagCountMismatch);
         return;
     }
-    long long dbg_c0 = 0, dbg_g0 = 0;
-    if (pl.experiment >= 8 && threadIdx.x == 0) { dbg_c0 = clock64(); asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(dbg_g0)); }
     // ---- decode the work item ----
     int it = blockIdx.x;
     const int unit = a.unit_begin + it / pl.items_per_unit;
@@ -214,7 +194,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
             // (a block of four layers stages one operand per layer: [unit-tensor][4] and [unit][4])
             const int64_t row0 = a.B == 4 ? ((cand ? (int64_t)unit : (int64_t)unit * 2) * 4 + layer) * a.Tmax
                                           : (cand ? (int64_t)unit : (int64_t)unit * 2) * a.Tmax;
-            for (int i = 0; i < ntile && pl.experiment != 2; ++i) {
+            for (int i = 0; i < ntile; ++i) {
                 const int s = i % kBStages;
                 const uint32_t ph = (uint32_t)(i / kBStages) & 1u;
                 mb_wait(sm0 + oEmpty + 8 * s, ph ^ 1u, abort_flag, a.status);
@@ -232,13 +212,12 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
             for (int i = 0; i < ntile; ++i) {
                 const int s = i % kBStages, as = i % kAccSets;
                 mb_wait(sm0 + oTEmpty + 8 * as, ((uint32_t)(i / kAccSets) & 1u) ^ 1u, abort_flag, a.status);
-                if (pl.experiment != 2) mb_wait(sm0 + oFull + 8 * s, (uint32_t)(i / kBStages) & 1u, abort_flag, a.status);
+                mb_wait(sm0 + oFull + 8 * s, (uint32_t)(i / kBStages) & 1u, abort_flag, a.status);
                 if (*abort_flag) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 // one descriptor per stage; the k steps and the two M tiles only add compile-time constants
                 const uint64_t db_stage = smem_desc(b0 + s * kBStageBytes);
                 const uint32_t d0 = tmem_base + (uint32_t)(kTmemAcc + as * kAccSet);
-                if (pl.experiment != 3)
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
@@ -270,7 +249,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
             mb_wait(sm0 + oTFull + 8 * as, (uint32_t)(i / kAccSets) & 1u, abort_flag, a.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float acc = 0.f;
-            if (!*abort_flag && pl.experiment != 1) {
+            if (!*abort_flag) {
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
                     const bool all_visible = t0 + kBN - 1 <= pl.pos_min;  // every key of the tile precedes every probe position
@@ -322,12 +301,6 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
     }
-    if (pl.experiment >= 8 && threadIdx.x == 0 && (blockIdx.x % 257) == 0) {
-        long long c1 = clock64(), g1;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1));
-        printf("item %d: %lld cycles in %lld ns = %.0f MHz, %d tiles, %.0f cycles per tile\n", blockIdx.x, c1 - dbg_c0, g1 - dbg_g0,
-               1e3 * (double)(c1 - dbg_c0) / (double)(g1 - dbg_g0), ntile, (double)(c1 - dbg_c0) / ntile);
-    }
     if (threadIdx.x == 0) {
         const double* red = reinterpret_cast<const double*>(smem + oRed);
         // part slot of this item inside its unit: (layer, mblock, split); candidate selects the column
@@ -341,19 +314,11 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
 cudaError_t launch_probe_tc(const ProbeArgs& a, int dtype, cudaStream_t st, bool* handled, int* nparts) {
     *handled = false;
     if (dtype != FDKV_BF16 || a.d != 128 || !a.tmap_z1 || !a.tmap_drop) return cudaSuccess;
-    static int enabled = -1, sm_count = 148;
-    if (enabled < 0) {
-        const char* ev = getenv("FDKV_NO_TC_PROBE");
-        enabled = (ev && ev[0] == '1') ? 0 : 1;
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(probe_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kProbeSmem);
-        if (e != cudaSuccess) return e;
-    }
-    if (!enabled) return cudaSuccess;
+    static PerDevice once;
+    int sm_count = 0;
+    cudaError_t e0 = once.ensure([&]() { return cudaFuncSetAttribute(probe_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kProbeSmem); }, &sm_count);
+    if (e0 != cudaSuccess) return e0;
     TcPlan pl;
-    { const char* ex = getenv("FDKV_PROBE_EXPERIMENT"); pl.experiment = ex ? atoi(ex) : 0; }
     pl.pos_min = a.pos_host[0];
     pl.pos_max = a.pos_host[a.W - 1];
     pl.ntiles = pl.pos_max / kBN + 1;  // keys after the last probe position never count
@@ -366,12 +331,13 @@ cudaError_t launch_probe_tc(const ProbeArgs& a, int dtype, cudaStream_t st, bool
     pl.nsplits = nsplits;
     pl.items_per_unit = a.B * pl.mblocks * 2 * nsplits;
     const int slots = a.B * pl.mblocks * nsplits;
-    if (slots > a.nptiles_max) return cudaSuccess;  // the part array is sized for the portable kernel's tiles
+    if (slots > a.nptiles_max) return cudaErrorInvalidValue;  // cannot happen: the part array is sized for max_probe_parts()
     probe_tc_kernel<<<a.unit_count * pl.items_per_unit, kPThreads, kProbeSmem, st>>>(
         *reinterpret_cast<const CUtensorMap*>(a.tmap_z1), *reinterpret_cast<const CUtensorMap*>(a.tmap_drop), a, pl);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     count_launch(1);
+    count_kernel(FDKV_KERNEL_PROBE_TC);
     *nparts = slots;
     *handled = true;
     return cudaSuccess;

@@ -18,6 +18,7 @@
 #include <cstdlib>
 
 #include "fdkv_internal.h"
+#include "mbar_wait.cuh"
 
 namespace fdkv {
 
@@ -33,7 +34,6 @@ constexpr int kTBBytes = 2 * kTBHalf;       // 64 KiB
 constexpr int kTHdr = 2048;                 // barriers, TMEM slot, abort flag, probe position of every column
 constexpr int kTSmem = kTHdr + kTBBytes + kTStages * kTAStage;  // 194 KiB
 constexpr int kTThreads = 6 * 32;
-constexpr uint32_t kTSpin = 1u << 22;
 constexpr int tFull = 0, tEmpty = 32, tTFull = 64, tTEmpty = 80, tSlot = 96, tAbort = 100, tPosCol = 1024;  // pos_col: 256 ints
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -46,23 +46,8 @@ __device__ __forceinline__ void mb_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mb_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ uint32_t mb_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
 __device__ __forceinline__ void mb_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* status) {
-    if (*abort_flag) return;
-    for (uint32_t i = 0; i < kTSpin; ++i) {
-        if (mb_try(bar, parity)) return;
-        if ((i & 255u) == 255u && *abort_flag) return;
-    }
-    *abort_flag = 1;
-    atomicMax(status, (int32_t)kFlagTimeout);
+    mbar_wait_bounded(bar, parity, abort_flag, status);
 }
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -363,14 +348,10 @@ __global__ void __launch_bounds__(256) token_gather_kernel(const uint4* z1, cons
 
 cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st) {
     if (a.unit_count <= 0) return cudaSuccess;
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(token_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmem);
-        if (e != cudaSuccess) { sm_count = 0; return e; }
-    }
+    static PerDevice once;
+    int sm_count = 0;
+    cudaError_t e0 = once.ensure([&]() { return cudaFuncSetAttribute(token_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmem); }, &sm_count);
+    if (e0 != cudaSuccess) return e0;
     cudaError_t e = cudaMemsetAsync(a.score + (int64_t)a.unit_begin * a.Tmax, 0, (size_t)a.unit_count * a.Tmax * 4, st);
     if (e != cudaSuccess) return e;
     ScorePlan pl;
@@ -389,6 +370,7 @@ cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st) {
     const int blocks = (int)std::min<int64_t>(64, ((int64_t)a.T * 16 + 255) / 256);
     token_drop_kernel<<<dim3(blocks, a.unit_count), 256, 0, st>>>(a);
     count_launch(3);
+    count_kernel(FDKV_KERNEL_TOKEN_SCORE);
     return cudaGetLastError();
 }
 

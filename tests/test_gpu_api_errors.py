@@ -164,3 +164,35 @@ def test_unsupported_combinations_and_reset_reuse():
     assert torch.equal(first, again)
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_bounded_device_wait_runs_out_and_reports():
+    """Every device-side wait of the library (TMA copies, tensor-core commits) is bounded.  Here one is made to run out
+    -- a barrier nobody arrives at, a limit of a thousand polls -- and must come back as FDKV_ERR_TIMEOUT from
+    fdkv_device_status, with the kernel ending normally and the context still computing correct results afterwards."""
+    B, ctx = _ctx(head_dim=128, dtype=B_BF16(), max_prefill=512)
+    k0, k1, v0, v1 = _kv(T=512, d=128, dtype=torch.bfloat16)
+    ctx.compress_prefill(0, 0, 1, 512, [k0, k1], [v0, v1])
+    ctx.set_modes(0, [1, 0])
+    ctx.commit(0)
+    q = torch.randn((1, 4, 128), device="cuda").to(torch.bfloat16)
+    before = ctx.decode_attn(0, q, out_dtype=B.F32).clone()
+    assert ctx.device_status() == 0
+    ctx.test_wait_expiry(1024)
+    assert ctx.device_status() == 7          # FDKV_ERR_TIMEOUT: the wait gave up and said so
+    torch.cuda.synchronize()                 # the device is healthy
+    ctx.test_clear_device_status()
+    assert ctx.device_status() == 0
+    after = ctx.decode_attn(0, q, out_dtype=B.F32)
+    torch.cuda.synchronize()
+    assert torch.equal(before, after)
+    assert ctx.device_status() == 0
+    with pytest.raises(B.FdkvError):
+        ctx.test_wait_expiry(0)              # limits outside 1 .. 65536 are refused on the host
+    ctx.close()
+
+
+def B_BF16():
+    from paper_2607_06519_b200 import binding as B
+
+    return B.BF16

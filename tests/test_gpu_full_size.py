@@ -17,28 +17,47 @@ from paper_2607_06519_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _prefill(w, seqs, sample_units, probe_units):
-    from paper_2607_06519_b200 import runner
+def _pick_units(modes, b, per_mode):
+    """Units (b, pair, head) of one sequence covering every mode: per_mode[m] units of mode m, spread over the pairs."""
+    picked = []
+    for m, n in enumerate(per_mode):
+        cand = [(int(p), int(h)) for p, h in zip(*np.nonzero(modes == m))]
+        assert len(cand) >= n, f"mode {m}: {len(cand)} units, wanted {n}"
+        step = max(1, len(cand) // max(n, 1))
+        picked += [(b, p, h) for (p, h) in cand[::step][:n]]
+    return picked
+
+
+def _prefill(w, seqs, per_mode, n_probe):
+    """Compresses, probes and commits the sequences with the benchmark's quota mode mix.  The sampled units are chosen
+    AFTER the modes are known, per_mode[b] = (shared, residual, exact) counts for sequence b, so that every test checks
+    each reconstruction path; the first n_probe sampled units of a sequence also have their probe errors compared."""
+    from paper_2607_06519_b200 import binding as B, runner
 
     pf = runner.Prefilled(w, max_tail=max(w.n_steps, 1))
     units, modes_all = {}, []
     pos = synth.probe_positions(w)
+    tc_before, portable_before = B.kernel_launch_count(B.KERNEL_PROBE_TC), B.kernel_launch_count(B.KERNEL_PROBE_PORTABLE)
     for b in seqs:
         pf.compress(b)
-        for (sb, p, h) in sample_units:
-            if sb == b:
-                units[(b, p, h)] = check_compression(pf.ctx, w, b, p, h)
         pmodes, scores = pf.probe(b, 0.0)
-        for (sb, p, h) in probe_units:
-            if sb == b:
-                u = units[(b, p, h)]
+        modes = synth.quota_modes(scores[..., 0])
+        sample = _pick_units(modes, b, per_mode.get(b, (0, 0, 0)))
+        for i, (sb, p, h) in enumerate(sample):
+            u = units[(b, p, h)] = check_compression(pf.ctx, w, b, p, h)
+            if i < n_probe:
                 e = R.probe_error(u.z1["k"], u.kept["k"], synth.probe_q(w, b, 2 * p), synth.probe_q(w, b, 2 * p + 1), w.group,
                                   h, pos)
                 np.testing.assert_allclose(scores[p, h], e, rtol=1e-4)
-        modes = synth.quota_modes(scores[..., 0])
         pf.ctx.set_modes(b, modes)
         pf.commit(b)
         modes_all.append(modes)
+    # bf16 storage with head_dim 128: the tcgen05 probe served every call, the portable kernel none
+    assert B.kernel_launch_count(B.KERNEL_PROBE_TC) - tc_before == len(seqs)
+    assert B.kernel_launch_count(B.KERNEL_PROBE_PORTABLE) == portable_before
+    for b, want in per_mode.items():
+        got = np.bincount([int(modes_all[seqs.index(b)][p][h]) for (sb, p, h) in units if sb == b], minlength=3)
+        assert tuple(got) == tuple(want), (b, got)
     torch.cuda.empty_cache()
     return pf, units, modes_all
 
@@ -57,11 +76,13 @@ def _check_layer(pf, w, layer, step, units, modes_all, q, out):
 
 
 def test_decode32k_benchmark_workload():
+    from paper_2607_06519_b200 import binding as B
+
     w = synth.WORKLOADS["decode32k"]
-    sample = [(0, 0, 0), (0, 7, 3), (0, 15, 7)]
-    pf, units, modes_all = _prefill(w, [0], sample, sample[:2])
+    pf, units, modes_all = _prefill(w, [0], {0: (3, 3, 2)}, 2)
     assert sorted(np.bincount(modes_all[0].ravel(), minlength=3).tolist()) == sorted([64, 45, 19])
-    # make sure the three sampled units cover more than one mode where possible (the mix is fixed by the probe)
+    assert len(units) == 8
+    fast_before, portable_before = B.kernel_launch_count(B.KERNEL_DECODE_FAST), B.kernel_launch_count(B.KERNEL_DECODE_PORTABLE)
     stream = torch.cuda.Stream()
     worst = 0.0
     with torch.cuda.stream(stream):
@@ -72,14 +93,46 @@ def test_decode32k_benchmark_workload():
             assert torch.isfinite(out.float()).all()
             worst = max(worst, _check_layer(pf, w, layer, 0, units, modes_all, q, out))
     assert worst <= TOL["bf16"], worst
+    assert B.kernel_launch_count(B.KERNEL_DECODE_FAST) - fast_before == w.n_layers
+    assert B.kernel_launch_count(B.KERNEL_DECODE_PORTABLE) == portable_before
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
+
+
+def test_prefill32k_probe_errors_and_modes_of_every_unit():
+    """The prefill workload at full size: the probe errors of all 128 units against the oracle's (computed once by
+    tests/golden/make_probe_errors_32k.py, oracle only), and the modes the rule of Eq. 3 assigns at the calibrated
+    lambda*, at lambda* / 64 (mostly exact) and at lambda* x 64 (all shared) -- bit-exact, at lambdas whose smallest
+    loss margin is at least 1e-3 so that the float32 accumulation of the GPU errors cannot flip a decision."""
+    import json
+    import os
+
+    from paper_2607_06519_b200 import runner
+
+    g = json.load(open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "probe_errors_decode32k.json")))
+    w = synth.WORKLOADS["prefill32k"]
+    pf = runner.Prefilled(w, max_tail=1)
+    pf.compress(0)
+    e_ref = np.stack([np.asarray(g["e_shared"]), np.asarray(g["e_residual"])], axis=-1)
+    seen = set()
+    for case in g["cases"]:
+        assert case["min_margin"] >= 1e-3
+        pmodes, scores = pf.probe(0, case["lambda"])
+        np.testing.assert_allclose(scores, e_ref, rtol=1e-4)
+        assert pmodes.ravel().tolist() == case["modes"], case["name"]
+        seen |= set(case["modes"])
+    assert seen == {0, 1, 2}
+    # the probe's modes are what commit packs
+    pf.commit(0)
+    assert pf.ctx.get_modes(0).numpy().ravel().tolist() == g["cases"][-1]["modes"]
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
 
 
 def test_decode128k_long_context():
     w = synth.WORKLOADS["decode128k"]
-    sample = [(0, 1, 2), (0, 13, 6)]
-    pf, units, modes_all = _prefill(w, [0], sample, sample[:1])
+    pf, units, modes_all = _prefill(w, [0], {0: (1, 2, 1)}, 1)
+    assert len(units) == 4
     worst = 0.0
     for layer in range(w.n_layers):
         q = pf.decode_q(layer, 0)
@@ -94,8 +147,9 @@ def test_decode128k_long_context():
 
 def test_batch8_decode_with_tail_appends():
     w = synth.WORKLOADS["batch8"]
-    sample = [(0, 0, 1), (3, 9, 5), (7, 15, 0)]
-    pf, units, modes_all = _prefill(w, list(range(w.batch)), sample, [])
+    # one unit of each mode, from three different sequences
+    pf, units, modes_all = _prefill(w, list(range(w.batch)), {0: (1, 0, 0), 3: (0, 1, 0), 7: (0, 0, 1)}, 0)
+    assert sorted(int(modes_all[b][p][h]) for (b, p, h) in units) == [0, 1, 2]
     # generated-token rows of every (sequence, pair, head): [steps, d] for both layers, K and V
     rows = {}
     for b in range(w.batch):

@@ -188,10 +188,15 @@ def test_budgeted_routing_matches_oracle():
         fits, lam, modes = pf.ctx.route_budget(0, budget)
         rf, rl, rm, rprev = R.route_budget(e[..., 0], e[..., 1], om, unit_bytes, budget)
         assert fits and rf
-        # the library's lambda routes, under the oracle's rule and errors, exactly as the library says and fits ...
-        at_lam = [R.mode_rule(a, b, om, lam)[0] for a, b in e.reshape(-1, 2)]
-        assert modes.numpy().ravel().tolist() == at_lam, frac
-        assert sum(om[m] for m in at_lam) * unit_bytes <= budget
+        # the library's lambda routes, under the oracle's rule and errors, as the library says and fits.  The library
+        # stops a hair past one unit's crossing computed from ITS errors (float32 accumulation, 1e-6 off the oracle's),
+        # so that unit's decision is compared a relative 1e-4 to either side of lambda.
+        got = modes.numpy().ravel().tolist()
+        lo = [R.mode_rule(a, b, om, lam * (1 - 1e-4))[0] for a, b in e.reshape(-1, 2)]
+        hi = [R.mode_rule(a, b, om, lam * (1 + 1e-4))[0] for a, b in e.reshape(-1, 2)]
+        assert all(g in (l, h) for g, l, h in zip(got, lo, hi)), frac
+        assert sum(l != h for l, h in zip(lo, hi)) <= 2
+        assert sum(om[m] for m in got) * unit_bytes <= budget
         # ... and is the smallest such: it lies in the bracket of the oracle's upward scan (previous grid value does not
         # fit, the next does), up to the float32 accumulation of the library's probe errors
         assert (rprev if rprev > 0 else 0.0) * (1 - 1e-4) <= lam <= rl * (1 + 1e-4) + 1e-12, (frac, rprev, lam, rl)

@@ -12,6 +12,8 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import fdkv_ref as R
+
 pytestmark = pytest.mark.gpu
 
 
@@ -47,6 +49,14 @@ def test_noalloc_matches_context_path_twice(dtype, T, d, keep):
                 assert torch.equal(idx, want_idx), (call, h, is_v)
                 assert torch.equal(val.view(torch.int16 if dtype == "bf16" else torch.int32),
                                    want_val.view(torch.int16 if dtype == "bf16" else torch.int32)), (call, h, is_v)
+                if h == 0:
+                    # and, on its own feet, against the CPU oracle's Eq. 1 split and entry selection of the same rows
+                    a, b = x0[:, h].float().cpu().numpy(), x1[:, h].float().cpu().numpy()
+                    ref_z0, ref_z1 = R.depth_split(a, b, dtype == "bf16")
+                    ref_idx = R.select_entries(ref_z1, k)
+                    assert np.array_equal(z0.float().cpu().numpy().view(np.uint32), ref_z0.view(np.uint32)), (call, is_v)
+                    assert np.array_equal(idx.cpu().numpy(), ref_idx), (call, is_v)
+                    assert np.array_equal(val.float().cpu().numpy().view(np.uint32), ref_z1.ravel()[ref_idx].view(np.uint32)), (call, is_v)
     assert ctx.device_status() == 0
     ctx.close()
 
