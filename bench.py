@@ -264,8 +264,9 @@ def bench_workload(args, w, dev, dist, rank, local, world, steps, warmup, with_c
     if w.residual_rule == 1:
         # token rule: compression is the depth split alone (the probe selects); the probe runs three products
         # (token scores, then the two candidates' errors)
-        compress_min_bytes = n_ut * (2 * N * esize + N * esize) + units * (2 * w.k_tok * w.head_dim * esize + 4 * w.k_tok)
-        probe_flops = 2.0 * units * 3 * (2 * w.group * w.W) * w.T * w.head_dim
+        nbl, nhf = w.block_size, (1 if w.block_size == 2 else 4)  # layers per block; stored high-frequency rows per kept token and tensor
+        compress_min_bytes = n_ut * (nbl * N * esize + N * esize) + units * (2 * nhf * w.k_tok * w.head_dim * esize + 4 * w.k_tok)
+        probe_flops = 2.0 * units * 3 * (nbl * w.group * w.W) * w.T * w.head_dim
     else:
         # read the block's layers, write the shared coefficient, the index and the kept values
         nbl = w.block_size

@@ -97,7 +97,10 @@ typedef enum { FDKV_ROWS_STORAGE = 0, FDKV_ROWS_E4M3 = 1 } fdkv_row_format;
  * layer l reads one value per kept position.  Candidates: shared = Z0 / 2, residual = Z0 / 2 + dev_l on the kept
  * positions, exact = x_l.  Eq. 2 averages over the block's four layers; Omega(residual) counts four values and one
  * int32 index per kept position, Omega(exact) four layers.  The mixed schedule of the paper (B = 4 in the middle,
- * B = 2 for the first and last layers) is two contexts, one per block size.  Entry residual rule only.
+ * B = 2 for the first and last layers) is two contexts, one per block size.  Under FDKV_RESIDUAL_TOKENS (the paper's
+ * default pairing: blocks of four with probe-scored tokens) a token's score is the maximum over the block's four layers of
+ * | Q_l . dev_l[t,:] |, one token set serves K and V and all four layers, and the kept tokens store the four layers'
+ * deviation rows (Omega(residual) counts 2 * 4 * k_tok * d * e + 4 * k_tok bytes).
  */
 
 /*
@@ -108,7 +111,8 @@ typedef enum { FDKV_ROWS_STORAGE = 0, FDKV_ROWS_E4M3 = 1 } fdkv_row_format;
  *   probe_pos[q] >= t of | Q . (c * Z1K[t,:]) |; the k_tok = floor(T * keep_num / keep_den) tokens with the
  *   largest score (ties: lowest t) keep ALL head_dim high-frequency coefficients of K and of V.  The scores
  *   need the probe queries, so the set is chosen inside fdkv_probe (which is then mandatory before commit, even
- *   when modes are overridden); Omega(residual) counts 2*k_tok*d*e + 4*k_tok bytes.  bf16, head_dim 128 only.
+ *   when modes are overridden); Omega(residual) counts 2*k_tok*d*e + 4*k_tok bytes.  bf16, head_dim 128 only; either
+ *   block size (see the note on block size 4 above for the score and the stored rows there).
  */
 typedef enum { FDKV_RESIDUAL_ENTRIES = 0, FDKV_RESIDUAL_TOKENS = 1 } fdkv_residual_rule;
 

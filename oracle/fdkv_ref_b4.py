@@ -108,6 +108,33 @@ def probe_error4(dev_k, kept_idx, q, group: int, h: int, pos):
     return float(tot[0]), float(tot[1])
 
 
+def token_scores4(dev_k, q, group: int, h: int, pos) -> np.ndarray:
+    """The token score between Eq. 2 and Eq. 3 for a block of four: s_t = max over the block's layers l, the group's
+    query heads and the probe queries that can see token t of |Q_l . (K_l[t] - Khat_l^shared[t])|, where the shared-depth
+    candidate misses exactly layer l's deviation from the block mean: K_l - Khat_l^shared = dev_l.  No 1/sqrt(d): the
+    printed score has none.  dev_k: the four layers' stored key deviations [T, d]; q: their probe queries [W, Hq, d]."""
+    T = dev_k[0].shape[0]
+    pos = np.asarray(pos, dtype=np.int64)
+    visible = np.arange(T)[None, :] <= pos[:, None]                   # [W, T]
+    best = np.zeros(T, dtype=np.float64)
+    for l in range(4):
+        miss = np.asarray(dev_k[l], dtype=np.float64)
+        for g in range(group):
+            ql = np.asarray(q[l], dtype=np.float64)[:, h * group + g, :]
+            s = np.abs(ql @ miss.T)                                     # [W, T]
+            best = np.maximum(best, np.where(visible, s, 0.0).max(axis=0))
+    return best
+
+
+def omega4_tokens(T: int, d: int, e_bytes: int, k_tok: int) -> np.ndarray:
+    """Normalised memory cost under the token rule: a kept token stores the four layers' deviation rows of K and of V
+    and one int32 token index."""
+    shared = 2.0 * T * d * e_bytes
+    residual = shared + 2.0 * 4.0 * k_tok * d * e_bytes + 4.0 * k_tok
+    exact = 2.0 * 4.0 * T * d * e_bytes
+    return np.array([shared / exact, residual / exact, 1.0], dtype=np.float64)
+
+
 def omega4(T: int, d: int, e_bytes: int, k: int) -> np.ndarray:
     """Normalised memory cost of the three modes for one (block, KV head), K and V together."""
     shared = 2.0 * T * d * e_bytes
@@ -119,16 +146,25 @@ def omega4(T: int, d: int, e_bytes: int, k: int) -> np.ndarray:
 class Unit4:
     """Compressed state of one (block of four layers, KV head): shared coefficient, deviations, kept sets, tails."""
 
-    def __init__(self, k_layers, v_layers, bf16: bool, keep_num: int, keep_den: int):
+    def __init__(self, k_layers, v_layers, bf16: bool, keep_num: int, keep_den: int, select: bool = True):
         self.x = {"k": [_f32(a) for a in k_layers], "v": [_f32(a) for a in v_layers]}
         self.T, self.d = self.x["k"][0].shape
         self.bf16 = bf16
         self.k_keep = R.keep_count(self.T, self.d, keep_num, keep_den)
+        self.k_tok = (self.T * keep_num) // keep_den
         self.z0, self.dev, self.energy, self.kept = {}, {}, {}, {}
         for name in ("k", "v"):
             self.z0[name], self.dev[name], self.energy[name] = depth_split4(self.x[name], bf16)
-            self.kept[name] = R.select_entries(self.energy[name], self.k_keep)
+            if select:  # entry form: the positions of largest high-frequency energy, K and V independently
+                self.kept[name] = R.select_entries(self.energy[name], self.k_keep)
         self.tail = {(n, l): [] for n in ("k", "v") for l in range(4)}
+
+    def use_tokens(self, tokens):
+        """Token rule (Eq. 3 with one indicator per token): the listed tokens keep every high-frequency value of K and of
+        V, in all four layers."""
+        self.tokens = np.asarray(tokens, dtype=np.int32)
+        ent = R.token_entries(self.tokens, self.d)
+        self.kept = {"k": ent, "v": ent}
 
     def append(self, layer_in_block: int, k_row, v_row):
         self.tail[("k", layer_in_block)].append(_f32(k_row))

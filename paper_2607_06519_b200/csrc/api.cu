@@ -62,7 +62,6 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     if (c.residual_rule != FDKV_RESIDUAL_ENTRIES && c.residual_rule != FDKV_RESIDUAL_TOKENS) return false;
     s.tok_rule = c.residual_rule == FDKV_RESIDUAL_TOKENS;
     if (s.tok_rule && !(c.dtype == FDKV_BF16 && c.head_dim == 128)) return false;  // tensor-core kernels only
-    if (s.tok_rule && B != 2) return false;
     s.ktok_max = (int64_t)s.Tmax * s.keep_num / s.keep_den;
     s.ktok_cap = (int64_t)align_up((size_t)(s.ktok_max + 32), 64);
     s.NU = s.P * s.Hkv;
@@ -119,7 +118,7 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     const size_t rows_pad = align_up((size_t)((s.Tmax + s.max_fold + kRowPad - 1) / kRowPad * kRowPad) * s.d * s.esize);
     const size_t exact_unit = 2 * (size_t)s.B * rows_pad;
     const size_t resid_unit = s.tok_rule
-                                  ? 2 * rows_pad + 2 * align_up((size_t)s.ktok_cap * s.d * s.esize) + align_up((size_t)s.ktok_cap * 4) +
+                                  ? 2 * rows_pad + 2 * (size_t)s.NB * align_up((size_t)s.ktok_cap * s.d * s.esize) + align_up((size_t)s.ktok_cap * 4) +
                                         align_up((size_t)(s.ntiles_max + 1) * 4)
                                   : 2 * rows_pad + 2 * (size_t)s.NB * (align_up((size_t)(s.kcap + s.kfold_max) * 4) + align_up((size_t)(s.kcap + s.kfold_max) * s.esize)) +
                                         2 * align_up((size_t)(s.kcap + s.kfold_max) * 4) +
@@ -144,7 +143,7 @@ double omega_of(const Shape& s, int T, double (&om)[3]) {
     const double k_tok = (double)((int64_t)T * s.keep_num / s.keep_den);
     const double b_sh = 2.0 * Td * e, b_ex = 2.0 * s.B * Td * e;
     double b_rs;
-    if (s.tok_rule) b_rs = b_sh + 2.0 * k_tok * s.d * e + 4.0 * k_tok;
+    if (s.tok_rule) b_rs = b_sh + 2.0 * k_tok * s.d * e * s.NB + 4.0 * k_tok;
     else b_rs = b_sh + 2.0 * k * (s.NB * e + 4.0);
     om[0] = b_sh / b_ex; om[1] = b_rs / b_ex; om[2] = 1.0;
     return b_ex;
@@ -219,7 +218,7 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     c->packed_lists = c->has_tmap && s.max_batch * s.Hkv <= kFastMaxUnits;
     if (s.rows_f8 && !(c->packed_lists && make_rows_tensor_map_u8(c->arena, arena_bytes, kRowPad, c->tmap_u8))) { delete c; return FDKV_ERR_UNSUPPORTED; }
     if (s.tok_rule) {
-        const bool ok = c->packed_lists && make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
+        const bool ok = c->packed_lists && make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.NB * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
         if (!ok) { delete c; return FDKV_ERR_UNSUPPORTED; }
     }
     if (s.dtype == FDKV_BF16 && s.d == 128)
@@ -297,9 +296,13 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
             a4.unit_stride = (int64_t)s.Tmax * s.d;
             a4.z0 = c->work + c->ws.z0; a4.dev = c->work + c->ws.z1;
             a4.energy = wsp<float>(c, c->ws.energy);
-            a4.drop = c->has_probe_tmaps ? c->work + c->ws.z1drop : nullptr;
+            a4.drop = (c->has_probe_tmaps && !s.tok_rule) ? c->work + c->ws.z1drop : nullptr;  // (the token rule writes its own copy in fdkv_probe)
             a4.hist = wsp<uint32_t>(c, c->ws.hist);
             CU(launch_split4_hist(a4, s.dtype, st));
+        }
+        if (s.tok_rule) {  // the token rule selects inside fdkv_probe
+            for (int p = pb; p < pe; ++p) { c->pair_compressed[p] = 1; c->pair_probed[p] = 0; c->pair_scored[p] = 0; }
+            return FDKV_OK;
         }
         SelectArgs sa;
         sa.ut_begin = ut_begin; sa.ut_count = ut_count;
@@ -413,6 +416,7 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     a.status = wsp<int32_t>(c, c->ws.status);
     if (s.tok_rule) {
         TokenArgs t;
+        t.B = s.B;
         t.unit_begin = a.unit_begin; t.unit_count = a.unit_count;
         t.T = T; t.Tmax = s.Tmax; t.Hq = s.Hq; t.Hkv = s.Hkv; t.G = s.G; t.W = W; t.ntiles_max = s.ntiles_max;
         t.k_tok = (int64_t)T * s.keep_num / s.keep_den; t.ktok_cap = s.ktok_cap; t.unit_stride = (int64_t)s.Tmax * s.d;
@@ -530,7 +534,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
         const int m = q.modes[u];
         if (m < 0 || m > 2) return FDKV_ERR_STATE;
         if (m == FDKV_MODE_EXACT) need += 2 * (size_t)s.B * stream_b;
-        else if (s.tok_rule) need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * align_up(trow_b) + align_up(tlist_b) + align_up(off_b) : 0);
+        else if (s.tok_rule) need += 2 * align_up(rows_pad) + (m == FDKV_MODE_RESIDUAL ? 2 * (size_t)s.NB * align_up(trow_b) + align_up(tlist_b) + align_up(off_b) : 0);
         else need += 2 * stream_b + (m == FDKV_MODE_RESIDUAL ? 2 * (lists_b + align_up(off_b)) : 0);
     }
     if (c->bump + need > c->arena_bytes) return FDKV_ERR_ARENA_FULL;
@@ -605,17 +609,23 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                 for (int l = 0; l < s.B; ++l) (is_v ? dl[l]->v_rows : dl[l]->k_rows) = z0;
                 by_mode[m] += s.rows_f8 ? rows8 + 512 : rows;
                 if (m == FDKV_MODE_RESIDUAL && s.tok_rule) {
-                    char* rows_res = take(trow_b);
+                    // the selected tokens' high-frequency rows, densely packed: Z1 rows of a pair (both layers read them with
+                    // opposite signs), each layer's own deviation rows of a block of four (stored doubled: see the gather kernel)
                     // (the list is read where the probe left it: its copy into the arena runs with the other copies after this loop)
-                    CU(launch_token_gather(c->work + c->ws.z1 + ut * unit_stride_b, wsp<int32_t>(c, c->ws.tok_list) + (size_t)u * s.ktok_cap, k_tok, rows_res, st));
+                    char* rows_l[4] = {nullptr, nullptr, nullptr, nullptr};
+                    for (int j = 0; j < s.NB; ++j) {
+                        rows_l[j] = take(trow_b);
+                        CU(launch_token_gather(c->work + c->ws.z1 + (ut * s.NB + j) * unit_stride_b, wsp<int32_t>(c, c->ws.tok_list) + (size_t)u * s.ktok_cap, k_tok,
+                                               rows_l[j], s.B == 4 ? 1 : 0, st));
+                    }
                     for (int l = 0; l < s.B; ++l) {
                         UnitDesc* d = dl[l];
                         d->res_kind = 1;
                         d->k_idx = (const int32_t*)tl;
                         d->k_off = (const int32_t*)to;
-                        (is_v ? d->v_val : d->k_val) = rows_res;
+                        (is_v ? d->v_val : d->k_val) = rows_l[s.NB == 1 ? 0 : l];
                     }
-                    by_mode[1] += (size_t)k_tok * s.d * s.esize;
+                    by_mode[1] += (size_t)s.NB * k_tok * s.d * s.esize;
                 } else if (m == FDKV_MODE_RESIDUAL) {
                     char* po = take(off_b);
                     copy_job(c->work + c->ws.tile_off + ut * (s.ntiles_max + 1) * 4, po, off_copy, 16, 16);

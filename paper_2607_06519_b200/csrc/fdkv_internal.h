@@ -291,6 +291,7 @@ cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, in
 
 // ---- token-granular residual (token_rule.cu) ----
 struct TokenArgs {
+    int B;  // layers per depth block: 2 (one Z1 operand, both layers' queries) or 4 (one deviation operand per layer)
     int unit_begin, unit_count;
     int T, Tmax, Hq, Hkv, G, W, ntiles_max;
     int64_t k_tok, ktok_cap, unit_stride;
@@ -307,7 +308,7 @@ struct TokenArgs {
     int32_t* status;
 };
 cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st);
-cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, cudaStream_t st);
+cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, int twice, cudaStream_t st);
 
 // Function attributes (the opt-in to large dynamic shared memory) and the SM count belong to a device, not to the
 // process: every launcher keeps one of these and runs its set-up the first time it meets the current device.

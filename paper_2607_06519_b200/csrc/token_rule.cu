@@ -1,7 +1,9 @@
 // Token-granular sparse residual (the paper's rule, Method between Eq. 2 and Eq. 3; bf16, head_dim 128).
 //
-//   s_t = max over (layer of the pair, group query head, probe query q with pos[q] >= t) | Q . (c * Z1K[t,:]) |
-//   keep the k_tok tokens with the largest s_t (ties: lowest t); they keep all 128 coefficients of K and of V.
+//   s_t = max over (layer of the depth block, group query head, probe query q with pos[q] >= t) | Q_l . (K_l[t,:] - Khat_l^shared[t,:]) |
+//       = | Q_l . (+-c Z1K[t,:]) | for a pair, | Q_l . dev_l[t,:] | for a block of four (dev_l = layer l's deviation from the block mean);
+//   keep the k_tok tokens with the largest s_t (ties: lowest t); they keep all 128 high-frequency values of K and of V
+//   (of every layer of a block of four).
 //
 // 1. token_score_kernel (tcgen05): the transposed probe product D[token][probe row] = Z1K . Q^T, so that a thread
 //    of the epilogue owns one token (TMEM lane) and takes the maximum over its row's columns in registers.  A = 128
@@ -123,7 +125,7 @@ token_score_kernel(const __grid_constant__ CUtensorMap tmap, TokenArgs a, ScoreP
     }
     // ---- B: probe rows r = mblock*256 + i of this layer, r = g*W + qi -> Q[layer][qi][h*G+g][:]; padding rows zero ----
     {
-        const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[2 * pair + layer]);
+        const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[a.B * pair + layer]);
         for (int v = threadIdx.x; v < kTN * 16; v += kTThreads) {
             const int i = v >> 4, chunk = v & 15;
             const int r = mblock * kTN + i;
@@ -150,7 +152,8 @@ token_score_kernel(const __grid_constant__ CUtensorMap tmap, TokenArgs a, ScoreP
 
     if (warp == 0) {
         if (lane == 0) {
-            const int64_t row0 = (int64_t)unit * 2 * a.Tmax;  // K coefficients of the unit: unit-tensor 2*unit
+            // K high-frequency rows of the unit: unit-tensor 2*unit (a block of four stages one operand per layer)
+            const int64_t row0 = a.B == 4 ? ((int64_t)unit * 2 * 4 + layer) * a.Tmax : (int64_t)unit * 2 * a.Tmax;
             for (int i = 0; i < ntile; ++i) {
                 const int s = i % kTStages;
                 mb_wait(sm0 + tEmpty + 8 * s, ((uint32_t)(i / kTStages) & 1u) ^ 1u, abort_flag, a.status);
@@ -187,7 +190,7 @@ token_score_kernel(const __grid_constant__ CUtensorMap tmap, TokenArgs a, ScoreP
     } else {
         // ---- epilogue: thread = token (TMEM lane); maximum of |D| over the probe rows that can see the token ----
         const int lq = warp & 3;
-        const float c32 = __uint_as_float(0x3F3504F3u);
+        const float c32 = a.B == 4 ? 1.f : __uint_as_float(0x3F3504F3u);  // a pair's rows are Z1: K - Khat^shared = +-c Z1
         uint32_t* score = a.score + (int64_t)unit * a.Tmax;
         for (int i = 0; i < ntile; ++i) {
             const int as = i & 1;
@@ -327,8 +330,9 @@ __global__ void __launch_bounds__(1024) token_select_kernel(TokenArgs a) {
 // Z1K with the selected rows zeroed.  grid (row blocks, units), 256 threads, one 16-byte vector per thread and step.
 __global__ void __launch_bounds__(256) token_drop_kernel(TokenArgs a) {
     const int unit = a.unit_begin + blockIdx.y;
-    const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.z1) + (int64_t)unit * 2 * a.unit_stride);
-    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.z1drop) + (int64_t)unit * a.unit_stride);
+    const int nb = a.B == 4 ? 4 : 1, l = blockIdx.z;  // staged high-frequency tensors per unit-tensor
+    const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.z1) + ((int64_t)unit * 2 * nb + l) * a.unit_stride);
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.z1drop) + ((int64_t)unit * nb + l) * a.unit_stride);
     const uint8_t* flag = a.flag + (int64_t)unit * a.Tmax;
     const int64_t nvec = (int64_t)a.T * 16;
     for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * blockDim.x) {
@@ -338,10 +342,18 @@ __global__ void __launch_bounds__(256) token_drop_kernel(TokenArgs a) {
     }
 }
 
-// out[j][:] = z1[list[j]][:]
-__global__ void __launch_bounds__(256) token_gather_kernel(const uint4* z1, const int32_t* list, int64_t k_tok, uint4* out) {
-    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < k_tok * 16; v += (int64_t)gridDim.x * blockDim.x)
-        out[v] = z1[(int64_t)list[v >> 4] * 16 + (v & 15)];
+// out[j][:] = z1[list[j]][:], optionally doubled (exact in bf16): a block of four scales its rows by 1/2 at decode time and
+// its deviations by 1, so their stored rows carry the factor 2
+__global__ void __launch_bounds__(256) token_gather_kernel(const uint4* z1, const int32_t* list, int64_t k_tok, uint4* out, int twice) {
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < k_tok * 16; v += (int64_t)gridDim.x * blockDim.x) {
+        uint4 x = z1[(int64_t)list[v >> 4] * 16 + (v & 15)];
+        if (twice) {
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&x);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) h[i] = __hadd2(h[i], h[i]);
+        }
+        out[v] = x;
+    }
 }
 
 }  // namespace
@@ -358,26 +370,26 @@ cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st) {
     pl.pos_min = a.pos_host[0];
     pl.ntiles = a.pos_host[a.W - 1] / kTM + 1;  // tokens after the last probe position are seen by nobody: score 0
     pl.mblocks = (a.G * a.W + kTN - 1) / kTN;
-    const int base_items = a.unit_count * 2 * pl.mblocks;
+    const int base_items = a.unit_count * a.B * pl.mblocks;
     int nsplits = std::max(1, std::min((4 * sm_count + base_items - 1) / base_items, (pl.ntiles + 7) / 8));
     pl.tiles_per_split = (pl.ntiles + nsplits - 1) / nsplits;
     pl.nsplits = (pl.ntiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
-    pl.items_per_unit = 2 * pl.mblocks * pl.nsplits;
+    pl.items_per_unit = a.B * pl.mblocks * pl.nsplits;
     token_score_kernel<<<a.unit_count * pl.items_per_unit, kTThreads, kTSmem, st>>>(*reinterpret_cast<const CUtensorMap*>(a.tmap_z1_128), a, pl);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     token_select_kernel<<<a.unit_count, 1024, 0, st>>>(a);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const int blocks = (int)std::min<int64_t>(64, ((int64_t)a.T * 16 + 255) / 256);
-    token_drop_kernel<<<dim3(blocks, a.unit_count), 256, 0, st>>>(a);
+    token_drop_kernel<<<dim3(blocks, a.unit_count, a.B == 4 ? 4 : 1), 256, 0, st>>>(a);
     count_launch(3);
     count_kernel(FDKV_KERNEL_TOKEN_SCORE);
     return cudaGetLastError();
 }
 
-cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, cudaStream_t st) {
+cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, int twice, cudaStream_t st) {
     if (k_tok <= 0) return cudaSuccess;
     const int blocks = (int)std::min<int64_t>(256, (k_tok * 16 + 255) / 256);
-    token_gather_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(z1), list, k_tok, reinterpret_cast<uint4*>(out));
+    token_gather_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(z1), list, k_tok, reinterpret_cast<uint4*>(out), twice);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -115,6 +115,8 @@ WORKLOADS["decode32k_fp8_4l"] = WORKLOADS["decode32k_fp8"].scaled(n_layers=4, na
 WORKLOADS["decode128k_fp8"] = WORKLOADS["decode128k"].scaled(row_format=1, name="decode128k_fp8")
 WORKLOADS["tiny_b4"] = WORKLOADS["tiny"].scaled(n_layers=4, block_size=4, name="tiny_b4")
 WORKLOADS["decode32k_b4"] = WORKLOADS["decode32k"].scaled(block_size=4, name="decode32k_b4")
+# the paper's default pairing: blocks of four layers with probe-scored tokens
+WORKLOADS["decode32k_b4_tok"] = WORKLOADS["decode32k"].scaled(block_size=4, residual_rule=1, name="decode32k_b4_tok")
 WORKLOADS["decode32k_b4_8l"] = WORKLOADS["decode32k"].scaled(n_layers=8, block_size=4, name="decode32k_b4_8l")
 
 

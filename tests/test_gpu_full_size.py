@@ -223,3 +223,52 @@ def test_decode32k_token_rule():
     assert worst <= TOL["bf16"], worst
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+def test_decode32k_blocks_of_four_token_rule():
+    """The paper's default pairing at the 32k benchmark shape (blocks of four layers, probe-scored tokens): token sets by
+    score band, probe errors and one decode step of all layers on the GPU's own sets, sampled units of each mode."""
+    from oracle import fdkv_ref_b4 as R4
+    from paper_2607_06519_b200 import runner
+
+    w = synth.WORKLOADS["decode32k_b4_tok"]
+    pf = runner.Prefilled(w, max_tail=1)
+    pf.compress(0)
+    pmodes, scores = pf.probe(0, 0.0)
+    pos = synth.probe_positions(w)
+    modes = synth.quota_modes(scores[..., 0])
+    sample = _pick_units(modes, 0, (1, 2, 1))
+    units = {}
+    for (b, blk, h) in sample:
+        u = R4.Unit4(synth.block_tensor(w, 0, blk, h, False), synth.block_tensor(w, 0, blk, h, True), True, w.keep_num, w.keep_den,
+                     select=False)
+        pq = [synth.probe_q(w, 0, 4 * blk + l) for l in range(4)]
+        tok, sc = pf.ctx.get_token_set(0, blk, h, w.T)
+        tok, sc = tok.cpu().numpy(), f32(sc).astype(np.float64)
+        s_ref = R4.token_scores4(u.dev["k"], pq, w.group, h, pos)
+        np.testing.assert_allclose(sc, s_ref, rtol=1e-5, atol=1e-6 * s_ref.max())
+        kth = np.sort(s_ref)[::-1][w.k_tok - 1]
+        assert tok.size == w.k_tok and np.all(np.diff(tok) > 0)
+        assert set(np.flatnonzero(s_ref > kth * (1 + 2e-5)).tolist()) <= set(tok.tolist()) <= set(np.flatnonzero(s_ref >= kth * (1 - 2e-5)).tolist())
+        u.use_tokens(tok)
+        e = R4.probe_error4(u.dev["k"], u.kept["k"], pq, w.group, h, pos)
+        np.testing.assert_allclose(scores[blk, h], e, rtol=1e-4)
+        units[(blk, h)] = u
+    pf.ctx.set_modes(0, modes)
+    pf.commit(0)
+    torch.cuda.empty_cache()
+    G, worst = w.group, 0.0
+    for layer in range(w.n_layers):
+        blk, lb = divmod(layer, 4)
+        q = pf.decode_q(layer, 0)
+        out = pf.ctx.decode_attn(layer, q)
+        torch.cuda.synchronize()
+        assert torch.isfinite(out.float()).all()
+        for (ub, h), u in units.items():
+            if ub != blk:
+                continue
+            ref = u.attend(int(modes[blk][h]), lb, f32(q)[0][h * G:(h + 1) * G])
+            worst = max(worst, float(vector_errors(f32(out)[0][h * G:(h + 1) * G], ref).max()))
+    assert worst <= TOL["bf16"], worst
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()

@@ -79,3 +79,70 @@ def test_token_rule_against_oracle(T, keep, W, tail):
             assert err.max() <= TOL["bf16"], (step, layer, float(err.max()))
     assert pf.ctx.device_status() == 0
     pf.ctx.close()
+
+
+@pytest.mark.parametrize("T,keep,W,tail", [(2100 + 37, (1, 16), 64, 3), (517, (1, 8), 8, 0), (300, (0, 1), 16, 1)])
+def test_token_rule_on_blocks_of_four(T, keep, W, tail):
+    """The paper's default pairing -- depth blocks of four layers with probe-scored tokens: one token set per (block, KV
+    head) from max over the four layers of |Q_l . dev_l[t]|, the four layers' deviation rows kept for those tokens."""
+    from oracle import fdkv_ref_b4 as R4
+    from paper_2607_06519_b200 import runner
+
+    w = synth.WORKLOADS["decode32k"].scaled(n_layers=8, T=T, n_needles=min(16, T), n_steps=max(tail, 1), W=W, keep_num=keep[0],
+                                            keep_den=keep[1], residual_rule=1, block_size=4, name="tok_b4")
+    pf = runner.Prefilled(w, max_tail=max(tail, 1))
+    pf.compress(0)
+    lam = 20.0
+    pmodes, scores = pf.probe(0, lam)
+    pos = synth.probe_positions(w)
+    om = R4.omega4_tokens(w.T, w.head_dim, 2, w.k_tok)
+    units = {}
+    for blk in range(w.n_blocks):
+        pq = [synth.probe_q(w, 0, 4 * blk + l) for l in range(4)]
+        for h in range(w.n_kv_heads):
+            u = R4.Unit4(synth.block_tensor(w, 0, blk, h, False), synth.block_tensor(w, 0, blk, h, True), True, w.keep_num, w.keep_den,
+                         select=False)
+            tok, sc = pf.ctx.get_token_set(0, blk, h, w.T)
+            tok, sc = tok.cpu().numpy(), f32(sc).astype(np.float64)
+            s_ref = R4.token_scores4(u.dev["k"], pq, w.group, h, pos)
+            np.testing.assert_allclose(sc, s_ref, rtol=1e-5, atol=1e-6 * max(1.0, s_ref.max()))
+            assert tok.size == w.k_tok and np.all(np.diff(tok) > 0)
+            if 0 < w.k_tok < w.T:
+                kth = np.sort(s_ref)[::-1][w.k_tok - 1]
+                must = np.flatnonzero(s_ref > kth * (1 + EPS))
+                may = np.flatnonzero(s_ref >= kth * (1 - EPS))
+                assert set(must.tolist()) <= set(tok.tolist()) <= set(may.tolist())
+            u.use_tokens(tok)
+            e = R4.probe_error4(u.dev["k"], u.kept["k"], pq, w.group, h, pos)
+            np.testing.assert_allclose(scores[blk, h], e, rtol=1e-4, atol=1e-9)
+            m_ref, _, margin = R.mode_rule(e[0], e[1], om, lam)
+            if margin > 1e-3:
+                assert int(pmodes[blk, h]) == m_ref
+            units[(blk, h)] = u
+    modes = np.array([[(blk + h) % 3 for h in range(w.n_kv_heads)] for blk in range(w.n_blocks)])
+    modes[0, 0] = 1
+    pf.ctx.set_modes(0, modes)
+    pf.commit(0)
+    by_mode, exact_equiv = pf.ctx.footprint(0)
+    n_res = int((modes == 1).sum())
+    assert by_mode[1] == n_res * (2 * w.T * 128 * 2 + 2 * 4 * w.k_tok * 128 * 2 + 4 * w.k_tok)
+    assert exact_equiv == w.n_blocks * w.n_kv_heads * 2 * 4 * w.T * 128 * 2
+    G = w.group
+    for step in range(max(tail, 1)):
+        for layer in range(w.n_layers):
+            blk, lb = divmod(layer, 4)
+            q = pf.decode_q(layer, step)
+            kn = vn = None
+            if tail:
+                kn, vn = pf.new_rows(layer, step)
+                for h in range(w.n_kv_heads):
+                    units[(blk, h)].append(lb, f32(kn)[0, h], f32(vn)[0, h])
+            out = f32(pf.ctx.decode_attn(layer, q, kn, vn))[0]
+            torch.cuda.synchronize()
+            ql = f32(q)[0]
+            for h in range(w.n_kv_heads):
+                ref = units[(blk, h)].attend(int(modes[blk][h]), lb, ql[h * G:(h + 1) * G])
+                err = vector_errors(out[h * G:(h + 1) * G], ref)
+                assert err.max() <= TOL["bf16"], (step, layer, h, float(err.max()))
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()

@@ -253,3 +253,63 @@ def test_fold_of_a_block_of_four():
     # shared mode: the folded tokens become the block mean
     got = u.rows("k", R4.SHARED, 1)[T:T + 16]
     np.testing.assert_allclose(got, np.mean(np.stack(xc).astype(np.float64), axis=0), rtol=1e-6, atol=1e-7)
+
+
+# ---------------------------------------------------------------- the paper's token rule on blocks of four
+def test_token_scores_of_a_block_literally_and_by_reduction():
+    """s_t = max |Q (K_t - Khat_t^shared)^T| with K = F4^T Z and Khat^shared = F4^T [Z0; 0; 0; 0], both rebuilt through
+    scipy's orthonormal DCT-II, against the oracle's shortcut K - Khat^shared = dev_l; and a block whose layers 2, 3 repeat
+    layers 0, 1 must score like the pair oracle (dev = +-(x0 - x1) / 2 = +-c z1)."""
+    T, d, G, Hq, W = 20, 8, 2, 4, 5
+    g = np.random.default_rng(21)
+    x = [g.standard_normal((T, d)).astype(np.float32) for _ in range(4)]
+    q = [g.standard_normal((W, Hq, d)).astype(np.float32) for _ in range(4)]
+    pos = np.array([3, 7, 12, 15, 19], dtype=np.int32)
+    _, dev, _ = R4.depth_split4(x, False)
+    x64 = np.stack([a.astype(np.float64) for a in x])
+    Z = scipy.fft.dct(x64, type=2, norm="ortho", axis=0)
+    Zs = Z.copy()
+    Zs[1:] = 0.0
+    K = scipy.fft.idct(Z, type=2, norm="ortho", axis=0)
+    Ks = scipy.fft.idct(Zs, type=2, norm="ortho", axis=0)
+    for h in range(2):
+        want = np.zeros(T)
+        for l in range(4):
+            for gg in range(G):
+                s = np.abs(q[l][:, h * G + gg, :].astype(np.float64) @ (K[l] - Ks[l]).T)
+                want = np.maximum(want, np.where(np.arange(T)[None, :] <= pos[:, None], s, 0.0).max(axis=0))
+        got = R4.token_scores4(dev, q, G, h, pos)
+        np.testing.assert_allclose(got, want, rtol=2e-6, atol=2e-6 * np.abs(x64).max() * d)  # (float32 storage of dev)
+        assert np.all(got[pos[-1] + 1:] == 0)
+    # reduction to the pair oracle with integer-valued layers (every step exact)
+    x0 = g.integers(-8, 9, (T, d)).astype(np.float32) * 2
+    x1 = g.integers(-8, 9, (T, d)).astype(np.float32) * 2
+    q0 = g.integers(-3, 4, (W, Hq, d)).astype(np.float32)
+    q1 = g.integers(-3, 4, (W, Hq, d)).astype(np.float32)
+    _, dev2, _ = R4.depth_split4([x0, x1, x0, x1], False)
+    _, z1 = R.depth_split(x0, x1, False)
+    for h in range(2):
+        np.testing.assert_allclose(R4.token_scores4(dev2, [q0, q1, q0, q1], G, h, pos), R.token_scores(z1, q0, q1, G, h, pos), rtol=1e-6)
+
+
+def test_unit4_under_the_token_rule():
+    g = np.random.default_rng(22)
+    T, d = 48, 8
+    mk = lambda: g.standard_normal((T, d)).astype(np.float32)
+    u = R4.Unit4([mk() for _ in range(4)], [mk() for _ in range(4)], False, 1, 4, select=False)
+    tok = np.array([1, 5, 6, 20, 47], dtype=np.int32)
+    u.use_tokens(tok)
+    assert np.array_equal(u.kept["k"], u.kept["v"]) and u.kept["k"].size == tok.size * d
+    for l in range(4):
+        rows = u.rows("k", R4.RESIDUAL, l)
+        np.testing.assert_allclose(rows[tok], u.x["k"][l][tok], rtol=0, atol=4e-7 * np.abs(np.stack(u.x["k"])).max())  # kept tokens restored
+        other = np.setdiff1d(np.arange(T), tok)
+        np.testing.assert_array_equal(rows[other], 0.5 * u.z0["k"][other].astype(np.float64))              # the rest is the block mean
+    om = R4.omega4_tokens(1000, 128, 2, 62)
+    np.testing.assert_allclose(om, [0.25, 0.25 + (2 * 4 * 62 * 128 * 2 + 4 * 62) / (8 * 1000 * 128 * 2), 1.0])
+    # keeping every token restores every layer, keeping none is the shared cache
+    u.use_tokens(np.arange(T))
+    for l in range(4):
+        np.testing.assert_allclose(u.rows("v", R4.RESIDUAL, l), u.x["v"][l], rtol=0, atol=4e-7 * np.abs(np.stack(u.x["v"])).max())
+    u.use_tokens(np.zeros(0, np.int32))
+    assert np.array_equal(u.rows("k", R4.RESIDUAL, 2), u.rows("k", R4.SHARED, 2))
