@@ -273,11 +273,11 @@ def bench_workload(args, w, dev, dist, rank, local, world, steps, warmup, with_c
         compress_min_bytes = n_ut * (nbl * N * esize + N * esize + w.k_keep * (4 + (1 if nbl == 2 else 4) * esize))
         probe_flops = 2.0 * units * 2 * (nbl * w.group * w.W) * w.T * w.head_dim
     # bytes the compression kernels really move (pairs, entry rule, bf16 / head_dim 128): split reads both layers and
-    # writes Z0 and the staged Z1; the count pass and the ordered write each read Z1 again; the write emits the canonical
-    # (index, value) list, the packed decode entries and, for K, the copy of Z1 without the kept entries for the probe
+    # writes Z0 and the staged Z1; the one-pass select reads Z1 once more and emits the canonical (index, value) list,
+    # the packed decode entries and, for K, the copy of Z1 without the kept entries for the probe
     compress_moved_bytes = None
     if w.residual_rule == 0 and w.block_size == 2 and w.dtype == "bf16" and w.head_dim == 128:
-        compress_moved_bytes = n_ut * (6 * N * esize + w.k_keep * (8 + esize)) + units * N * esize
+        compress_moved_bytes = n_ut * (5 * N * esize + w.k_keep * (8 + esize)) + units * N * esize
     modes_all = np.stack([ctx.get_modes(b).numpy() for b in range(w.batch)])
     mix = [int((modes_all == m).sum()) for m in range(3)]
     torch.cuda.empty_cache()
@@ -458,7 +458,7 @@ def bench_workload(args, w, dev, dist, rank, local, world, steps, warmup, with_c
                                          "moved_bytes": compress_moved_bytes,
                                          "achieved_moved_bytes": compress_moved_bytes / compress_ms / 1e6 if compress_moved_bytes else None,
                                          "frac_moved_bytes": compress_moved_bytes / compress_ms / 1e6 / hbm_peak if compress_moved_bytes else None,
-                                         "kernels": "depth split + histogram, threshold, tile count / scan / ordered write (one fdkv_compress_prefill call, CUDA events)"},
+                                         "kernels": "depth split + histogram, threshold, one-pass ordered select (one fdkv_compress_prefill call, CUDA events)"},
                         "probe": {"bound": "tensor", "unit": "TFLOP/s", "achieved": probe_flops / probe_ms / 1e9, "peak": tf_peak,
                                   "of": peak_kind + " bf16 burst (a millisecond kernel timed alone)", "frac": probe_flops / probe_ms / 1e9 / tf_peak,
                                   "flops": probe_flops, "kernels": "one fdkv_probe call (error products of both candidates + mode rule, CUDA events)"}}},

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfdkv.so")
-SOURCES = ["api.cu", "compress.cu", "block4.cu", "rows_fp8.cu", "probe.cu", "probe_tc.cu", "token_rule.cu", "decode.cu", "decode_fast.cu", "test_hooks.cu"]
+SOURCES = ["api.cu", "compress.cu", "select_fused.cu", "block4.cu", "rows_fp8.cu", "probe.cu", "probe_tc.cu", "token_rule.cu", "decode.cu", "decode_fast.cu", "test_hooks.cu"]
 HEADERS = ["fdkv_internal.h", "mbar_wait.cuh", "decode_fast_tile.inc", os.path.join("..", "..", "include", "fdkv.h"),
            os.path.join("..", "..", "include", "fdkv_testing.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",

@@ -294,23 +294,11 @@ __global__ void __launch_bounds__(1024) tile_scan_kernel(SelectArgs a) {
     }
 }
 
-// Packed entry of the bf16 / head_dim 128 decode kernel: low half = value bits, high half = (byte offset / 2) of the
-// entry inside a 16-token x 128-channel scratch tile laid out as two 64-channel halves of 128-byte rows whose
-// 16-byte chunks are XOR-swizzled with the row (the layout ldmatrix reads without bank conflicts).
-template <typename T>
-__device__ __forceinline__ uint32_t packed_entry(T v, int flat);
-template <>
-__device__ __forceinline__ uint32_t packed_entry<float>(float, int) { return 0u; }
-template <>
-__device__ __forceinline__ uint32_t packed_entry<__nv_bfloat16>(__nv_bfloat16 v, int flat) {
-    const int row = (flat >> 7) & 15, ch = flat & 127;
-    const uint32_t off = (uint32_t)((ch >> 6) * 2048 + row * 128 + ((((ch >> 3) & 7) ^ (row & 7)) << 4) + (ch & 7) * 2);
-    return (uint32_t)__bfloat16_as_ushort(v) | ((off >> 1) << 16);
-}
-
 // ----- C5: ordered write ---------------------------------------------------------------------------
 // One warp per tile walks its entries in flat-index order; an entry is kept when its key is above the
 // threshold, or equal to it and among the first `need` such entries of the whole unit-tensor.
+// (C3-C5 serve float32 keys: float32 storage and the energies of four-layer blocks.  bf16 storage takes the
+// one-pass kernel of select_fused.cu.)
 template <typename T>
 __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
     using S = Store<T>;
@@ -324,7 +312,6 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
     const T* z = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride;
     int32_t* idx = a.idx + (int64_t)ut * a.kcap;
     T* val = reinterpret_cast<T*>(a.val) + (int64_t)ut * a.kcap;
-    uint32_t* pk = a.packed ? a.packed + (int64_t)ut * a.kcap : nullptr;
     T* drop = (a.z1drop && !(ut & 1)) ? reinterpret_cast<T*>(a.z1drop) + (int64_t)(ut >> 1) * a.unit_stride : nullptr;
     uint32_t pos = (uint32_t)a.tile_off[(int64_t)ut * (a.ntiles_max + 1) + tile];
     uint32_t eq_rank = a.tile_eq[(int64_t)ut * a.ntiles_max + tile];
@@ -387,7 +374,6 @@ __global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
                 const T v = S::element(vreg[c], i);
                 idx[w] = (int32_t)(e + i);
                 val[w] = v;
-                if (pk) pk[w] = packed_entry<T>(v, (int)(e + i));
                 ++w;
             }
             // K tensors only: the coefficients the residual candidate drops (Z1 with the kept entries zeroed), the
@@ -455,19 +441,13 @@ cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int ntiles = (a.T + kResTile - 1) / kResTile;
-    if (ntiles > 0) {
-        dim3 grid((ntiles + 7) / 8, a.ut_count);
-        if (dtype == FDKV_BF16)
-            tile_count_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a);
-        else
-            tile_count_kernel<float><<<grid, 256, 0, st>>>(a);
-        tile_scan_kernel<<<a.ut_count, 1024, 0, st>>>(a);
-        if (dtype == FDKV_BF16)
-            tile_write_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a);
-        else
-            tile_write_kernel<float><<<grid, 256, 0, st>>>(a);
-        count_launch(3);
-    }
+    if (ntiles <= 0) return cudaSuccess;
+    if (dtype == FDKV_BF16) return launch_select_fused_bf16(a, st);
+    dim3 grid((ntiles + 7) / 8, a.ut_count);
+    tile_count_kernel<float><<<grid, 256, 0, st>>>(a);
+    tile_scan_kernel<<<a.ut_count, 1024, 0, st>>>(a);
+    tile_write_kernel<float><<<grid, 256, 0, st>>>(a);
+    count_launch(3);
     return cudaGetLastError();
 }
 
