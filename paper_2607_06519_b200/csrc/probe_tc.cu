@@ -6,14 +6,17 @@
 // and summed without ever leaving the SM:
 //   * work item = (unit, layer of the pair, block of 256 probe rows, candidate, range of 128-token key tiles);
 //     one CTA per item, 6 warps: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner), warps 2-5 = epilogue;
-//   * A (the item's 256 Q rows) is written once into tensor memory (128 columns: lane = row, two bf16 channels per
-//     column) by the threads that own the lanes; B tiles (192 tokens x 128 channels, 128-byte-swizzled K-major)
-//     stream through a 4-stage TMA ring;
-//   * per key tile 16 tcgen05.mma (M = 128, N = 192, K = 16, kind::f16, A from TMEM, bf16 x bf16 -> f32) fill two
-//     128x192 f32 accumulators in TMEM (384 columns).  (With N = 96 two accumulator sets alternate; measured
-//     slightly slower: the tensor pipe, not the epilogue, is the limit.);
+//   * A (the item's 256 Q rows, two M tiles) is written once into shared memory by the epilogue threads, in the
+//     128-byte-swizzled K-major layout a TMA copy would give it; B tiles (128 tokens x 128 channels, same layout)
+//     stream through a 5-stage TMA ring;
+//   * per key tile 16 tcgen05.mma (M = 128, N = 128, K = 16, kind::f16, both operands from shared memory,
+//     bf16 x bf16 -> f32) fill one of two alternating sets of two 128 x 128 f32 accumulators: all 512 columns of
+//     tensor memory.  The hand-over of an accumulator set (commit -> epilogue -> release -> next MMA) is a round trip of
+//     about a microsecond; with a single set it was paid on every tile and cost as much as the arithmetic, which is
+//     why A lives in shared memory: the 128 columns it took in tensor memory buy the second set;
 //   * epilogue: tcgen05.ld (32 lanes x 32 columns per instruction), square, mask keys after the row's probe
-//     position, accumulate; one float64 sum per item, summed across items in a fixed order by the finalize kernel.
+//     position, accumulate; the set is released as soon as its last columns are in registers; one float64 sum per
+//     item, summed across items in a fixed order by the finalize kernel.
 // Every mbarrier wait is bounded; on expiry the CTA flags the device status word, stops waiting and still frees
 // its tensor memory before it retires.
 #include <cuda.h>
@@ -27,19 +30,20 @@ namespace fdkv {
 
 namespace {
 
-constexpr int kBN = kProbeBoxRows;             // key tokens per tile (N of the MMA): 96 (two accumulator sets) or 192 (one)
-constexpr int kBStages = kBN == 96 ? 8 : 4;
-constexpr int kAccSets = kBN == 96 ? 2 : 1;
-constexpr int kBHalf = kBN * 128;              // one 64-channel half of a B tile: 12 KiB
-constexpr int kBStageBytes = 2 * kBHalf;       // 24 KiB
+constexpr int kBN = kProbeBoxRows;             // key tokens per tile (N of the MMA)
+constexpr int kBStages = 5;
+constexpr int kAccSets = 2;
+constexpr int kBHalf = kBN * 128;              // one 64-channel half of a B tile: 16 KiB
+constexpr int kBStageBytes = 2 * kBHalf;       // 32 KiB
 constexpr int kHdr = 1024;
-constexpr int kProbeSmem = kHdr + kBStages * kBStageBytes;  // 193 KiB
+constexpr int kAHalf = 128 * 128;              // one 64-channel half of an A tile (128 Q rows): 16 KiB
+constexpr int kABytes = 2 * 2 * kAHalf;        // two M tiles: 64 KiB
+constexpr int kProbeSmem = kHdr + kABytes + kBStages * kBStageBytes;  // 225 KiB
 constexpr int kPThreads = 6 * 32;
-// Tensor memory (512 columns): the item's 256 Q rows as the A operand (2 M tiles x 64 columns: 128 channels, two bf16
-// per column) and two alternating sets of two 128 x 96 f32 accumulators.
+// Tensor memory (512 columns): two alternating sets of two 128 x 128 f32 accumulators (one per M tile).
 constexpr int kTmemCols = 512;
-constexpr int kTmemA = 0, kTmemAcc = 128, kAccSet = 2 * kBN;
-static_assert(kTmemAcc + kAccSets * kAccSet <= kTmemCols && kBN % 96 == 0, "tensor memory budget");
+constexpr int kAccSet = 2 * kBN;
+static_assert(kAccSets * kAccSet <= kTmemCols && kBN == 128, "tensor memory budget");
 // header: full[8] @0, empty[8] @64, tfull[2] @128, tempty[2] @144, tmem slot @160, abort @164, reduce @192 (4 doubles)
 constexpr int oFull = 0, oEmpty = 64, oTFull = 128, oTEmpty = 144, oSlot = 160, oAbort = 164, oRed = 192;
 
@@ -75,12 +79,12 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = kBN
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
-// D[tmem] (+)= A[tmem] * B[smem]^T; ACC = 0 overwrites D
+// D[tmem] (+)= A[smem] * B[smem]^T; ACC = 0 overwrites D
 template <int ACC>
-__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db) {
+__device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint64_t da, uint64_t db) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "r"(tmem_a), "l"(db), "r"(kIdesc), "n"(ACC)
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(da), "l"(db), "r"(kIdesc), "n"(ACC)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -95,22 +99,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
           "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
-}
-
-// 64 consecutive 32-bit columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_st64(uint32_t taddr, const uint32_t (&r)[64]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x64.b32 [%0], "
-        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,"
-        "%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63,%64};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
-          "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
-          "r"(r[30]), "r"(r[31]), "r"(r[32]), "r"(r[33]), "r"(r[34]), "r"(r[35]), "r"(r[36]), "r"(r[37]), "r"(r[38]), "r"(r[39]),
-          "r"(r[40]), "r"(r[41]), "r"(r[42]), "r"(r[43]), "r"(r[44]), "r"(r[45]), "r"(r[46]), "r"(r[47]), "r"(r[48]), "r"(r[49]),
-          "r"(r[50]), "r"(r[51]), "r"(r[52]), "r"(r[53]), "r"(r[54]), "r"(r[55]), "r"(r[56]), "r"(r[57]), "r"(r[58]), "r"(r[59]),
-          "r"(r[60]), "r"(r[61]), "r"(r[62]), "r"(r[63])
-        : "memory");
 }
 
 struct TcPlan {
@@ -157,34 +145,24 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + oSlot);
-    // ---- A operand: row r = mblock*256 + mt*128 + lane-row of this layer's probe block, r = g*W + qi ->
-    //      Q[layer][qi][h*G+g][:], written by the thread that owns that TMEM lane (two bf16 channels per column) ----
+    // ---- A operand: row r = mblock*256 + mt*128 + rl of this layer's probe block, r = g*W + qi -> Q[layer][qi][h*G+g][:],
+    //      row rl of M tile mt: 16 chunks of 16 bytes, chunk c of a 64-channel half stored at chunk c ^ (rl & 7) ----
     if (warp >= 2) {
-        const int lq = warp & 3, rl = lq * 32 + lane;
+        const int rl = (warp & 3) * 32 + lane;
         const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[a.B * pair + layer]);
 #pragma unroll 1
         for (int mt = 0; mt < 2; ++mt) {
             const int r = mblock * 256 + mt * 128 + rl;
-            uint32_t w[64];
-            if (r < rows_layer) {
-                const uint4* src = reinterpret_cast<const uint4*>(q + ((int64_t)(r % a.W) * a.Hq + h * a.G + r / a.W) * 128);
+            uint8_t* const arow = smem + kHdr + mt * 2 * kAHalf + rl * 128;
+            const uint4* src = reinterpret_cast<const uint4*>(q + ((int64_t)(r % a.W) * a.Hq + h * a.G + r / a.W) * 128);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const uint4 v = src[i];
-                    w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 64; ++i) w[i] = 0u;  // padding rows contribute nothing
-            }
-            tmem_st64(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(kTmemA + mt * 64), w);
+            for (int i = 0; i < 16; ++i)  // (padding rows are zero: they contribute nothing)
+                *reinterpret_cast<uint4*>(arow + (i >> 3) * kAHalf + (((i & 7) ^ (rl & 7)) << 4)) = r < rows_layer ? src[i] : make_uint4(0u, 0u, 0u, 0u);
         }
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic stores, read by the tensor core
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t b0 = sm0 + kHdr;
+    const uint32_t b0 = sm0 + kHdr + kABytes;
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -215,17 +193,18 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
                 mb_wait(sm0 + oFull + 8 * s, (uint32_t)(i / kBStages) & 1u, abort_flag, a.status);
                 if (*abort_flag) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // one descriptor per stage; the k steps and the two M tiles only add compile-time constants
+                // one descriptor per stage and for A; the k steps and the two M tiles only add compile-time constants
                 const uint64_t db_stage = smem_desc(b0 + s * kBStageBytes);
-                const uint32_t d0 = tmem_base + (uint32_t)(kTmemAcc + as * kAccSet);
+                const uint64_t da_all = smem_desc(sm0 + kHdr);
+                const uint32_t d0 = tmem_base + (uint32_t)(as * kAccSet);
 #pragma unroll
-                for (int mt = 0; mt < 2; ++mt) {
+                for (int k = 0; k < 8; ++k) {  // 8 steps of 16 channels: 32 bytes inside the swizzle atom of either operand
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {  // 8 steps of 16 channels: 8 TMEM columns of A, 32 bytes of B inside the swizzle atom
+                    for (int mt = 0; mt < 2; ++mt) {  // the two M tiles alternate: consecutive MMAs never wait for each other's accumulator
                         const uint64_t db = db_stage + (uint64_t)(((k >> 2) * kBHalf + (k & 3) * 32) >> 4);
-                        const uint32_t ta = tmem_base + (uint32_t)(kTmemA + mt * 64 + k * 8);
-                        if (k == 0) umma_ts<0>(d0 + mt * kBN, ta, db);
-                        else umma_ts<1>(d0 + mt * kBN, ta, db);
+                        const uint64_t da = da_all + (uint64_t)((mt * 2 * kAHalf + (k >> 2) * kAHalf + (k & 3) * 32) >> 4);
+                        if (k == 0) umma_ss<0>(d0 + mt * kBN, da, db);
+                        else umma_ss<1>(d0 + mt * kBN, da, db);
                     }
                 }
                 umma_commit(sm0 + oEmpty + 8 * s);    // the B stage is free once these MMAs have read it
@@ -250,44 +229,44 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float acc = 0.f;
             if (!*abort_flag) {
+                const bool all_visible = t0 + kBN - 1 <= pl.pos_min;  // every key of the tile precedes every probe position
 #pragma unroll
-                for (int mt = 0; mt < 2; ++mt) {
-                    const bool all_visible = t0 + kBN - 1 <= pl.pos_min;  // every key of the tile precedes every probe position
+                for (int round = 0; round < 4; ++round) {  // 64 accumulator columns of this lane per round, two loads in flight
+                    const int mt = round >> 1, c0 = (round & 1) * 64;
+                    uint32_t r0[32], r1[32];
+                    const uint32_t ta = tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(as * kAccSet + mt * kBN + c0);
+                    const int tc = t0 + c0;
+                    tmem_ld32(ta, r0);
+                    tmem_ld32(ta + 32, r1);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (round == 3) {  // the set's last columns are in registers: hand it back before the arithmetic
+                        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) mb_arrive(sm0 + oTEmpty + 8 * as);
+                    }
+                    if (all_visible && pos_row[mt] >= 0) {
+                        float acc1 = 0.f;
 #pragma unroll
-                    for (int cg = 0; cg < kBN / 96; ++cg) {  // 96 accumulator columns of this lane per round, three loads in flight
-                        uint32_t r0[32], r1[32], r2[32];
-                        const uint32_t ta = tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(kTmemAcc + as * kAccSet + mt * kBN + cg * 96);
-                        const int tc = t0 + cg * 96;
-                        tmem_ld32(ta, r0);
-                        tmem_ld32(ta + 32, r1);
-                        tmem_ld32(ta + 64, r2);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                        if (all_visible && pos_row[mt] >= 0) {
-                            float acc1 = 0.f, acc2 = 0.f;
+                        for (int j = 0; j < 32; ++j) {
+                            const float u = __uint_as_float(r0[j]), v = __uint_as_float(r1[j]);
+                            acc = fmaf(u, u, acc);
+                            acc1 = fmaf(v, v, acc1);
+                        }
+                        acc += acc1;
+                    } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const float u = __uint_as_float(r0[j]), v = __uint_as_float(r1[j]), w = __uint_as_float(r2[j]);
-                                acc = fmaf(u, u, acc);
-                                acc1 = fmaf(v, v, acc1);
-                                acc2 = fmaf(w, w, acc2);
-                            }
-                            acc += acc1 + acc2;
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const float u = __uint_as_float(r0[j]), v = __uint_as_float(r1[j]), w = __uint_as_float(r2[j]);
-                                if (tc + j <= pos_row[mt]) acc = fmaf(u, u, acc);
-                                if (tc + 32 + j <= pos_row[mt]) acc = fmaf(v, v, acc);
-                                if (tc + 64 + j <= pos_row[mt]) acc = fmaf(w, w, acc);
-                            }
+                        for (int j = 0; j < 32; ++j) {
+                            const float u = __uint_as_float(r0[j]), v = __uint_as_float(r1[j]);
+                            if (tc + j <= pos_row[mt]) acc = fmaf(u, u, acc);
+                            if (tc + 32 + j <= pos_row[mt]) acc = fmaf(v, v, acc);
                         }
                     }
                 }
+            } else {
+                __syncwarp();
+                if (lane == 0) mb_arrive(sm0 + oTEmpty + 8 * as);
             }
             total += (double)acc;
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mb_arrive(sm0 + oTEmpty + 8 * as);
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
