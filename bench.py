@@ -29,13 +29,12 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (None until a capture exists for that workload).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from one ncu capture (a constant, not
+# measured per run; None for workloads without a capture): 142.8 MB read + 3.8 MB written per launch on the 4-layer
+# cut of the 32k workload, which has the same 8 units and bytes per launch as the 32-layer workload
 NCU_TRAFFIC_BYTES = {
-    # profiles/decode_fast_kernel_decode32k.md: 138.55 MB read + ~3.9 MB written per launch, captured on the 4-layer cut
-    # (same 8 units and bytes per launch as the 32-layer workload)
-    "decode32k": 142.4e6,
-    "decode32k_4l": 142.4e6,
+    "decode32k": 146.6e6,
+    "decode32k_4l": 146.6e6,
 }
 
 
