@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(256) refine_hist_kernel(const float* z1, int64
     if (s_h[threadIdx.x]) atomicAdd(&hist[(int64_t)ut * kHistBins + threadIdx.x], s_h[threadIdx.x]);
 }
 
-// ----- C3: per 32-token tile, how many keys are above / equal to the threshold ------------------------
+// ----- C3: per 16-token tile, how many keys are above / equal to the threshold ------------------------
 template <typename T>
 __global__ void __launch_bounds__(256) tile_count_kernel(SelectArgs a) {
     using S = Store<T>;

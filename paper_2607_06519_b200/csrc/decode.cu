@@ -303,6 +303,9 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
 
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st) {
     cudaError_t e;
+    bool handled = false;
+    if ((e = launch_decode_fast(a, st, &handled)) != cudaSuccess) return e;  // (appends k_new / v_new itself)
+    if (handled) return cudaSuccess;
     if (a.k_new) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(a.batch);
@@ -320,9 +323,6 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         count_launch(1);
     }
-    bool handled = false;
-    if ((e = launch_decode_fast(a, st, &handled)) != cudaSuccess) return e;
-    if (handled) return cudaSuccess;
     if (a.packed_lists) return cudaErrorNotSupported;  // packed residual lists are only read by the kernel above
 
     const int ntiles = (a.Tmax_batch + kGTile - 1) / kGTile;

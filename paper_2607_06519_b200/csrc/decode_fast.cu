@@ -57,6 +57,9 @@ struct FastSched {
 struct PartCount {
     uint8_t n[kMaxUnits];  // split-K parts per unit (at most kMaxSplits)
 };
+struct TailLens {
+    uint16_t n[kMaxUnits];  // generated tokens in this layer's tail per sequence, this call's append included (host mirror)
+};
 static_assert(kMaxSplits < 256 && kMaxSplits % 32 == 0, "part counts are bytes; the combine holds one part per lane and round");
 
 // header offsets
@@ -164,7 +167,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 template <bool F8>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap8, DecodeArgs a, FastSched sch,
-                   PartCount pc) {
+                   PartCount pc, TailLens tl) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t smem0 = smem_u32(smem_raw);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + kOffAbort);
@@ -272,15 +275,34 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
         if (is_producer)
             for (int it = prologue_issued; it < kStages && it < seg_info[1]; ++it) issue_tile(it);
     } else {
+    if (warp == 0 && a.k_new) {
+        // Generated tokens of this call: the thread block that streams a unit's tail appends the unit's new K and V
+        // rows itself (16 lanes x 16 bytes each) and makes them visible to the tensor copies it issues next; a layer
+        // call stays one kernel, and k_new / v_new are read behind the dependency wait.
+        for (int i = 0; i < seg_info[0]; ++i) {
+            const int tu = segs[i].tail_u;
+            if (tu < 0) continue;
+            const int tb = tu / a.Hkv, th = tu % a.Hkv;
+            const int n = min((int)tl.n[tb], a.max_tail);
+            if (n <= 0) continue;
+            const int64_t row = (((int64_t)a.layer * a.max_batch + tb) * a.Hkv + th) * a.tail_rows + (n - 1);
+            const uint4* src = reinterpret_cast<const uint4*>(lane < 16 ? a.k_new : a.v_new) + ((int64_t)tb * a.Hkv + th) * 16 + (lane & 15);
+            uint4* dst = reinterpret_cast<uint4*>(lane < 16 ? a.tail_k : a.tail_v) + row * 16 + (lane & 15);
+            *dst = *src;
+            if (lane == 0 && th == 0) a.tail_len[a.layer * a.max_batch + tb] = n;  // the device copy of the length (other kernels read it)
+        }
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __syncwarp();
+    }
     if (is_producer) {
-        // tails: rows and lengths may have been written by the kernel right before this one
+        // tails: rows may have been written by the kernel right before this one (or just above); lengths are the host's
         int it0 = 0;
         for (int i = 0; i < seg_info[0]; ++i) {
             Seg g = segs[i];
             g.it0 = it0;
             if (g.tail_u >= 0) {
                 const int tail_b = g.tail_u / a.Hkv, tail_h = g.tail_u % a.Hkv;
-                const int n = min(a.tail_len[a.layer * a.max_batch + tail_b], a.max_tail);
+                const int n = min((int)tl.n[tail_b], a.max_tail);
                 const int64_t o = (((int64_t)a.layer * a.max_batch + tail_b) * a.Hkv + tail_h) * a.tail_rows;
                 g.tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
                 g.tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
@@ -320,7 +342,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             const int tok_b = sb * kResTile, tok_e = min(se * kResTile, T), rows16 = (se - sb) * kResTile;
             int ntail = 0, n_tail_rows = 0;
             if (sch.any_tail && se == nres) {
-                n_tail_rows = min(a.tail_len[a.layer * a.max_batch + b], a.max_tail);
+                n_tail_rows = min((int)tl.n[b], a.max_tail);
                 ntail = (n_tail_rows + kTT - 1) / kTT;
             }
             const int npre = (rows16 + kTT - 1) / kTT, nseg = npre + ntail;
@@ -948,8 +970,10 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     cfg.numAttrs = 1;
     const CUtensorMap& m16 = *reinterpret_cast<const CUtensorMap*>(a.tmap);
     const CUtensorMap& m8 = *reinterpret_cast<const CUtensorMap*>(a.rows_f8 ? a.tmap_u8 : a.tmap);
-    cudaError_t e = a.rows_f8 ? cudaLaunchKernelEx(&cfg, decode_fast_kernel<true>, m16, m8, a, sch, cs)
-                              : cudaLaunchKernelEx(&cfg, decode_fast_kernel<false>, m16, m8, a, sch, cs);
+    TailLens tl;
+    for (int b = 0; b < a.batch; ++b) tl.n[b] = (uint16_t)std::min(a.host_tail ? a.host_tail[b] : 0, 65535);
+    cudaError_t e = a.rows_f8 ? cudaLaunchKernelEx(&cfg, decode_fast_kernel<true>, m16, m8, a, sch, cs, tl)
+                              : cudaLaunchKernelEx(&cfg, decode_fast_kernel<false>, m16, m8, a, sch, cs, tl);
     if (e != cudaSuccess) return e;
     count_launch(1);
     count_kernel(FDKV_KERNEL_DECODE_FAST);
