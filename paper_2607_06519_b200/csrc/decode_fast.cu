@@ -58,7 +58,7 @@ struct PartCount {
     uint8_t n[kMaxUnits];  // split-K parts per unit (at most kMaxSplits)
 };
 struct TailLens {
-    uint16_t n[kMaxUnits];  // generated tokens in this layer's tail per sequence, this call's append included (host mirror)
+    int32_t n[kMaxUnits];  // generated tokens in this layer's tail per sequence, this call's append included (host mirror)
 };
 static_assert(kMaxSplits < 256 && kMaxSplits % 32 == 0, "part counts are bytes; the combine holds one part per lane and round");
 
@@ -283,7 +283,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             const int tu = segs[i].tail_u;
             if (tu < 0) continue;
             const int tb = tu / a.Hkv, th = tu % a.Hkv;
-            const int n = min((int)tl.n[tb], a.max_tail);
+            const int n = min(tl.n[tb], a.max_tail);
             if (n <= 0) continue;
             const int64_t row = (((int64_t)a.layer * a.max_batch + tb) * a.Hkv + th) * a.tail_rows + (n - 1);
             const uint4* src = reinterpret_cast<const uint4*>(lane < 16 ? a.k_new : a.v_new) + ((int64_t)tb * a.Hkv + th) * 16 + (lane & 15);
@@ -302,7 +302,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             g.it0 = it0;
             if (g.tail_u >= 0) {
                 const int tail_b = g.tail_u / a.Hkv, tail_h = g.tail_u % a.Hkv;
-                const int n = min((int)tl.n[tail_b], a.max_tail);
+                const int n = min(tl.n[tail_b], a.max_tail);
                 const int64_t o = (((int64_t)a.layer * a.max_batch + tail_b) * a.Hkv + tail_h) * a.tail_rows;
                 g.tkrow = (int)(((reinterpret_cast<uint64_t>(a.tail_k) - arena) >> 8) + o);
                 g.tvrow = (int)(((reinterpret_cast<uint64_t>(a.tail_v) - arena) >> 8) + o);
@@ -342,7 +342,7 @@ decode_fast_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_consta
             const int tok_b = sb * kResTile, tok_e = min(se * kResTile, T), rows16 = (se - sb) * kResTile;
             int ntail = 0, n_tail_rows = 0;
             if (sch.any_tail && se == nres) {
-                n_tail_rows = min((int)tl.n[b], a.max_tail);
+                n_tail_rows = min(tl.n[b], a.max_tail);
                 ntail = (n_tail_rows + kTT - 1) / kTT;
             }
             const int npre = (rows16 + kTT - 1) / kTT, nseg = npre + ntail;
@@ -971,7 +971,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st, bool* handl
     const CUtensorMap& m16 = *reinterpret_cast<const CUtensorMap*>(a.tmap);
     const CUtensorMap& m8 = *reinterpret_cast<const CUtensorMap*>(a.rows_f8 ? a.tmap_u8 : a.tmap);
     TailLens tl;
-    for (int b = 0; b < a.batch; ++b) tl.n[b] = (uint16_t)std::min(a.host_tail ? a.host_tail[b] : 0, 65535);
+    for (int b = 0; b < a.batch; ++b) tl.n[b] = a.host_tail ? a.host_tail[b] : 0;
     cudaError_t e = a.rows_f8 ? cudaLaunchKernelEx(&cfg, decode_fast_kernel<true>, m16, m8, a, sch, cs, tl)
                               : cudaLaunchKernelEx(&cfg, decode_fast_kernel<false>, m16, m8, a, sch, cs, tl);
     if (e != cudaSuccess) return e;
