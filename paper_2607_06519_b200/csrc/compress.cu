@@ -1,5 +1,6 @@
-// Prefill compression kernels: depth split (Eq. 1, B = 2) fused with the magnitude histogram, the
-// radix-select threshold, and the index-ordered compaction of the sparse residual (Eq. 3, entry form).
+// Prefill compression kernels: depth split (Eq. 1, B = 2) fused with the magnitude histogram and the
+// radix-select threshold of the sparse residual (Eq. 3, entry form); the index-ordered compaction that follows
+// is select_fused.cu.
 #include <algorithm>
 #include <mutex>
 
@@ -20,12 +21,6 @@ struct Store<float> {
     using vec_t = float4;
     __device__ static void unpack(const vec_t& v, float* f) { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
     __device__ static vec_t pack(const float* f) { return make_float4(f[0], f[1], f[2], f[3]); }
-    // element i of the vector (i only known at run time: select, never index, so the vector stays in registers)
-    __device__ static float element(const vec_t& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
-    // the vector with the elements whose bit is set in `mask` zeroed
-    __device__ static vec_t clear(const vec_t& v, uint32_t mask) {
-        return make_float4(mask & 1u ? 0.f : v.x, mask & 2u ? 0.f : v.y, mask & 4u ? 0.f : v.z, mask & 8u ? 0.f : v.w);
-    }
 };
 template <>
 struct Store<__nv_bfloat16> {
@@ -47,19 +42,6 @@ struct Store<__nv_bfloat16> {
             uint32_t lo = __bfloat16_as_ushort(__float2bfloat16_rn(f[2 * i]));
             uint32_t hi = __bfloat16_as_ushort(__float2bfloat16_rn(f[2 * i + 1]));
             w[i] = lo | (hi << 16);
-        }
-        return make_uint4(w[0], w[1], w[2], w[3]);
-    }
-    __device__ static __nv_bfloat16 element(const vec_t& v, int i) {
-        const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
-        return __ushort_as_bfloat16((unsigned short)((i & 1) ? (w >> 16) : (w & 0xFFFFu)));
-    }
-    __device__ static vec_t clear(const vec_t& v, uint32_t mask) {
-        uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (mask >> (2 * j) & 1u) w[j] &= 0xFFFF0000u;
-            if (mask >> (2 * j + 1) & 1u) w[j] &= 0x0000FFFFu;
         }
         return make_uint4(w[0], w[1], w[2], w[3]);
     }
@@ -214,175 +196,7 @@ __global__ void __launch_bounds__(256) refine_hist_kernel(const float* z1, int64
     if (s_h[threadIdx.x]) atomicAdd(&hist[(int64_t)ut * kHistBins + threadIdx.x], s_h[threadIdx.x]);
 }
 
-// ----- C3: per 16-token tile, how many keys are above / equal to the threshold ------------------------
-template <typename T>
-__global__ void __launch_bounds__(256) tile_count_kernel(SelectArgs a) {
-    using S = Store<T>;
-    constexpr int VEC = S::VEC;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x * 8 + warp;
-    const int ut = a.ut_begin + blockIdx.y;
-    const int ntiles = (a.T + kResTile - 1) / kResTile;
-    if (tile >= ntiles) return;
-    const uint32_t tau = a.sel[ut].tau;
-    const T* z = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride;
-    const int64_t e_begin = (int64_t)tile * kResTile * a.d;
-    const int64_t e_end = min((int64_t)a.T * a.d, e_begin + (int64_t)kResTile * a.d);
-    uint32_t gt = 0, eq = 0;
-    for (int64_t e = e_begin + lane * VEC; e < e_end; e += 32 * VEC) {
-        float f[VEC];
-        S::unpack(*reinterpret_cast<const typename S::vec_t*>(z + e), f);
-#pragma unroll
-        for (int i = 0; i < VEC; ++i) {
-            const uint32_t k = key_of(f[i]);
-            gt += k > tau;
-            eq += k == tau;
-        }
-    }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-        gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o);
-        eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o);
-    }
-    if (lane == 0) {
-        a.tile_cnt[((int64_t)ut * a.ntiles_max + tile) * 2 + 0] = gt;
-        a.tile_cnt[((int64_t)ut * a.ntiles_max + tile) * 2 + 1] = eq;
-    }
-}
-
-// ----- C4: index-ordered scan over tiles ------------------------------------------------------------
-// off[j] = (#keys > tau before tile j) + min(#keys == tau before tile j, need); eq_base[j] = #keys == tau before j.
-__global__ void __launch_bounds__(1024) tile_scan_kernel(SelectArgs a) {
-    __shared__ uint32_t s_gt[1024], s_eq[1024];
-    const int ut = a.ut_begin + blockIdx.x;
-    const int ntiles = (a.T + kResTile - 1) / kResTile;
-    const uint32_t need = a.sel[ut].need;
-    const uint32_t* cnt = a.tile_cnt + (int64_t)ut * a.ntiles_max * 2;
-    uint32_t* eqb = a.tile_eq + (int64_t)ut * a.ntiles_max;
-    int32_t* off = a.tile_off + (int64_t)ut * (a.ntiles_max + 1);
-    uint32_t carry_gt = 0, carry_eq = 0;
-    for (int base = 0; base < ntiles; base += 1024) {
-        const int j = base + threadIdx.x;
-        const uint32_t g = j < ntiles ? cnt[2 * j] : 0, e = j < ntiles ? cnt[2 * j + 1] : 0;
-        uint32_t ig = g, ie = e;
-        s_gt[threadIdx.x] = ig;
-        s_eq[threadIdx.x] = ie;
-        __syncthreads();
-        for (int o = 1; o < 1024; o <<= 1) {
-            const uint32_t ag = threadIdx.x >= o ? s_gt[threadIdx.x - o] : 0;
-            const uint32_t ae = threadIdx.x >= o ? s_eq[threadIdx.x - o] : 0;
-            __syncthreads();
-            ig += ag;
-            ie += ae;
-            s_gt[threadIdx.x] = ig;
-            s_eq[threadIdx.x] = ie;
-            __syncthreads();
-        }
-        if (j < ntiles) {
-            const uint32_t pg = carry_gt + ig - g, pe = carry_eq + ie - e;
-            off[j] = (int32_t)(pg + min(pe, need));
-            eqb[j] = pe;
-        }
-        carry_gt += s_gt[1023];
-        carry_eq += s_eq[1023];
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        const uint32_t total = carry_gt + min(carry_eq, need);
-        off[ntiles] = (int32_t)total;
-        if ((int64_t)total != a.k) atomicMax(a.status, (int32_t)kFlagCountMismatch);
-    }
-}
-
-// ----- C5: ordered write ---------------------------------------------------------------------------
-// One warp per tile walks its entries in flat-index order; an entry is kept when its key is above the
-// threshold, or equal to it and among the first `need` such entries of the whole unit-tensor.
-// (C3-C5 serve float32 keys: float32 storage and the energies of four-layer blocks.  bf16 storage takes the
-// one-pass kernel of select_fused.cu.)
-template <typename T>
-__global__ void __launch_bounds__(256) tile_write_kernel(SelectArgs a) {
-    using S = Store<T>;
-    constexpr int VEC = S::VEC;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x * 8 + warp;
-    const int ut = a.ut_begin + blockIdx.y;
-    const int ntiles = (a.T + kResTile - 1) / kResTile;
-    if (tile >= ntiles) return;
-    const uint32_t tau = a.sel[ut].tau, need = a.sel[ut].need;
-    const T* z = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride;
-    int32_t* idx = a.idx + (int64_t)ut * a.kcap;
-    T* val = reinterpret_cast<T*>(a.val) + (int64_t)ut * a.kcap;
-    T* drop = (a.z1drop && !(ut & 1)) ? reinterpret_cast<T*>(a.z1drop) + (int64_t)(ut >> 1) * a.unit_stride : nullptr;
-    uint32_t pos = (uint32_t)a.tile_off[(int64_t)ut * (a.ntiles_max + 1) + tile];
-    uint32_t eq_rank = a.tile_eq[(int64_t)ut * a.ntiles_max + tile];
-    const int64_t e_begin = (int64_t)tile * kResTile * a.d;
-    const int64_t e_end = min((int64_t)a.T * a.d, e_begin + (int64_t)kResTile * a.d);
-    constexpr int CH = 8;  // vectors in flight per lane: all loads of a round are issued before any is used
-    for (int64_t base0 = e_begin; base0 < e_end; base0 += (int64_t)CH * 32 * VEC) {
-        typename S::vec_t vreg[CH];
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const int64_t e = base0 + ((int64_t)c * 32 + lane) * VEC;
-            if (e < e_end) vreg[c] = *reinterpret_cast<const typename S::vec_t*>(z + e);
-        }
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const int64_t e = base0 + ((int64_t)c * 32 + lane) * VEC;
-            if (base0 + (int64_t)c * 32 * VEC >= e_end) break;  // warp-uniform
-            float f[VEC];
-            uint32_t is_gt = 0, is_eq = 0;
-            if (e < e_end) {
-                S::unpack(vreg[c], f);
-#pragma unroll
-                for (int i = 0; i < VEC; ++i) {
-                    const uint32_t k = key_of(f[i]);
-                    is_gt |= (uint32_t)(k > tau) << i;
-                    is_eq |= (uint32_t)(k == tau) << i;
-                }
-            }
-            // rank of this lane's first tie among the unit-tensor's ties
-            uint32_t keep = is_gt;
-            const uint32_t any_eq = __ballot_sync(0xFFFFFFFFu, is_eq != 0);
-            if (any_eq && eq_rank < need) {  // (ties are kept in index order: once `need` of them lie before this point, none is)
-                const uint32_t n_eq = __popc(is_eq);
-                uint32_t incl = n_eq;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                    if (lane >= o) incl += v;
-                }
-                uint32_t r = eq_rank + incl - n_eq;
-#pragma unroll
-                for (int i = 0; i < VEC; ++i)
-                    if (is_eq >> i & 1u) {
-                        if (r < need) keep |= 1u << i;
-                        ++r;
-                    }
-                eq_rank += __shfl_sync(0xFFFFFFFFu, incl, 31);
-            }
-            const uint32_t n_keep = __popc(keep);
-            uint32_t incl = n_keep;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            uint32_t w = pos + incl - n_keep;
-            // most lanes keep nothing, few keep more than one or two of their elements: walk the set bits
-            for (uint32_t kk = keep; kk; kk &= kk - 1) {
-                const int i = __ffs((int)kk) - 1;
-                const T v = S::element(vreg[c], i);
-                idx[w] = (int32_t)(e + i);
-                val[w] = v;
-                ++w;
-            }
-            // K tensors only: the coefficients the residual candidate drops (Z1 with the kept entries zeroed), the
-            // second B operand of the tensor-core probe
-            if (drop && e < e_end) *reinterpret_cast<typename S::vec_t*>(drop + e) = S::clear(vreg[c], keep);
-            pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
-        }
-    }
-}
+// (C3-C5, the index-ordered compaction, live in select_fused.cu.)
 
 template <typename T>
 __global__ void strided_copy_kernel(const T* src, int64_t stride_t, T* dst, int T_, int d) {
@@ -440,15 +254,8 @@ cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int ntiles = (a.T + kResTile - 1) / kResTile;
-    if (ntiles <= 0) return cudaSuccess;
-    if (dtype == FDKV_BF16) return launch_select_fused_bf16(a, st);
-    dim3 grid((ntiles + 7) / 8, a.ut_count);
-    tile_count_kernel<float><<<grid, 256, 0, st>>>(a);
-    tile_scan_kernel<<<a.ut_count, 1024, 0, st>>>(a);
-    tile_write_kernel<float><<<grid, 256, 0, st>>>(a);
-    count_launch(3);
-    return cudaGetLastError();
+    if (a.T <= 0) return cudaSuccess;
+    return launch_select_fused(a, dtype, st);
 }
 
 // grid (chunks of 32 KiB, jobs): the device-to-device copies of a commit (row streams, strided source rows of exact

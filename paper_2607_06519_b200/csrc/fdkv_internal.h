@@ -163,8 +163,8 @@ struct SelectArgs {
     int32_t* status;
 };
 cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream_t st);
-// bf16 storage: count, offsets and ordered write as one pass over Z1 (select_fused.cu); a.sel holds the thresholds
-cudaError_t launch_select_fused_bf16(const SelectArgs& a, cudaStream_t st);
+// count, offsets and ordered write as one pass over the keys (select_fused.cu); a.sel holds the thresholds
+cudaError_t launch_select_fused(const SelectArgs& a, int dtype, cudaStream_t st);
 
 // ---- four-layer blocks (block4.cu) ----
 struct Split4Args {

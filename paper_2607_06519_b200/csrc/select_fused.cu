@@ -1,4 +1,5 @@
-// Index-ordered compaction of the sparse residual (Eq. 3, entry form) for bf16 storage, as one pass over Z1.
+// Index-ordered compaction of the sparse residual (Eq. 3, entry form), as one pass over the keys (Z1 in the storage
+// type, or the float32 energies of four-layer blocks).
 //
 // Persistent thread blocks take 32 KiB chunks of the unit-tensors in ticket order (a global counter, so every chunk
 // with a lower ticket has been started by a block that is resident: the look-back below cannot wait on work that
@@ -6,8 +7,8 @@
 // are resident at one time then work on different unit-tensors, and a look-back finds a finished record a few
 // chunks back instead of walking through hundreds of chunks that are all in flight.  A chunk is copied into shared memory by one bulk TMA copy while the previous chunk is processed (two
 // buffers, one mbarrier each).  Per chunk:
-//   A  every thread compares eight 16-byte vectors with the threshold on 16-bit pairs inside 32-bit registers and
-//      writes one keep byte and one tie byte per vector into two 16 384-bit maps; K tensors also get their copy with
+//   A  every thread compares its 16-byte vectors with the threshold (bf16: on 16-bit pairs inside 32-bit registers) and
+//      writes one keep byte and one tie byte per eight elements into two bit maps; K tensors also get their copy with
 //      the kept coefficients zeroed (the second operand of the probe);
 //   B  one prefix sum over the word counts of both maps; the chunk's counts (keys above / equal to the threshold) are
 //      published, and the counts of all earlier chunks of the unit-tensor are summed by a decoupled look-back over
@@ -30,18 +31,17 @@ namespace fdkv {
 
 namespace {
 
-constexpr int kChunkElems = 16384;              // elements of a chunk: 32 KiB of bf16
-constexpr int kChunkWords = kChunkElems / 32;   // words of a chunk's bit map
+constexpr int kChunkBytes = 32768;              // a chunk: 16 384 bf16 or 8 192 float32 keys
+constexpr int kMaxChunkWords = kChunkBytes / 2 / 32;  // words of a chunk's bit map (bf16)
 constexpr int kFusedThreads = 256;
-constexpr int kWordsPerThread = kChunkWords / kFusedThreads;  // 1 or 2 consecutive words of a bit map
 constexpr uint32_t kSpinCap = 1u << 22;         // polls of a look-back before it gives up
 
 // shared memory (bytes)
 constexpr int oBuf = 0;                               // 2 x 32 KiB chunk buffers
-constexpr int oKeep = 2 * kChunkElems * 2;            // keep map
-constexpr int oTie = oKeep + kChunkWords * 4;         // tie map
-constexpr int oPre = oTie + kChunkWords * 4;          // prefix of the keep map's word counts, kChunkWords + 1 entries
-constexpr int oWarp = oPre + (kChunkWords + 8) * 4;   // per-warp sums
+constexpr int oKeep = 2 * kChunkBytes;                // keep map
+constexpr int oTie = oKeep + kMaxChunkWords * 4;      // tie map
+constexpr int oPre = oTie + kMaxChunkWords * 4;       // list position of every word's first entry
+constexpr int oWarp = oPre + (kMaxChunkWords + 8) * 4;  // per-warp sums
 constexpr int oMisc = oWarp + 128;                    // tickets [2], before_gt, before_eq, abort flag
 constexpr int oBar = oMisc + 64;                      // two mbarriers
 constexpr int kFusedSmem = oBar + 16;
@@ -96,8 +96,13 @@ __device__ __forceinline__ uint32_t block_prefix(uint32_t mine, uint32_t* warp_s
     return before + incl - mine;
 }
 
-__global__ void __launch_bounds__(kFusedThreads) select_fused_bf16_kernel(SelectArgs a, int chunks_per_ut, int nchunks,
-                                                                          uint32_t* ticket, unsigned long long* records) {
+template <typename T>
+__global__ void __launch_bounds__(kFusedThreads) select_fused_kernel(SelectArgs a, int chunks_per_ut, int nchunks, uint32_t* ticket,
+                                                                     unsigned long long* records) {
+    constexpr bool BF = sizeof(T) == 2;
+    constexpr int kChunkElems = kChunkBytes / (int)sizeof(T);
+    constexpr int kChunkWords = kChunkElems / 32;
+    constexpr int kWordsPerThread = kChunkWords / kFusedThreads;  // 2 (bf16) or 1 (float32) consecutive words of a bit map
     extern __shared__ __align__(128) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t* const keep_map = reinterpret_cast<uint32_t*>(smem + oKeep);
@@ -115,9 +120,9 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_bf16_kernel(Select
         if (t < (uint32_t)nchunks) {
             const int ut = a.ut_begin + (int)(t % (uint32_t)a.ut_count), ck = (int)(t / (uint32_t)a.ut_count);
             const int64_t e0 = (int64_t)ck * kChunkElems;
-            const uint32_t bytes = (uint32_t)min((int64_t)kChunkElems, (int64_t)a.T * a.d - e0) * 2u;
-            const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(a.z1) + (int64_t)ut * a.unit_stride + e0;
-            const uint32_t bar = bar0 + 8 * b, dst = smem_u32(smem + oBuf + b * kChunkElems * 2);
+            const uint32_t bytes = (uint32_t)min((int64_t)kChunkElems, (int64_t)a.T * a.d - e0) * (uint32_t)sizeof(T);
+            const T* src = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride + e0;
+            const uint32_t bar = bar0 + 8 * b, dst = smem_u32(smem + oBuf + b * kChunkBytes);
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                          "l"(src), "r"(bytes), "r"(bar)
@@ -142,8 +147,9 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_bf16_kernel(Select
         const uint32_t tau = a.sel[ut].tau, need = a.sel[ut].need;
         const int64_t e0 = (int64_t)ck * kChunkElems;
         const int n_e = (int)min((int64_t)kChunkElems, (int64_t)a.T * a.d - e0);  // a multiple of 8
-        const uint8_t* const buf = smem + oBuf + cur * kChunkElems * 2;
-        __nv_bfloat16* const drop = (a.z1drop && !(ut & 1))
+        const uint8_t* const buf = smem + oBuf + cur * kChunkBytes;
+        // (only bf16 storage has the copy without the kept entries: it is the tensor-core probe's operand)
+        __nv_bfloat16* const drop = (BF && a.z1drop && !(ut & 1))
                                         ? reinterpret_cast<__nv_bfloat16*>(a.z1drop) + (int64_t)(ut >> 1) * a.unit_stride + e0
                                         : nullptr;
         // a threshold above every key (nothing kept) has no 16-bit form: both addends zero leave bit 15 of every half clear
@@ -156,19 +162,31 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_bf16_kernel(Select
         // ---- A: keep and tie bytes, the dropped-coefficient copy ----
 #pragma unroll 4
         for (int q = 0; q < kChunkElems / 8 / kFusedThreads; ++q) {
-            const int vi = q * kFusedThreads + tid;  // vector of eight elements = one byte of the maps
+            const int vi = q * kFusedThreads + tid;  // eight elements = one byte of the maps
             uint32_t m8 = 0, e8 = 0;
             if (vi * 8 < n_e) {
-                const uint4 v = *reinterpret_cast<const uint4*>(buf + vi * 16);
-                const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
-                const uint32_t g0 = a0 + add_gt, g1 = a1 + add_gt, g2 = a2 + add_gt, g3 = a3 + add_gt;
-                const uint32_t x0 = g0 ^ (a0 + add_ge), x1 = g1 ^ (a1 + add_ge), x2 = g2 ^ (a2 + add_ge), x3 = g3 ^ (a3 + add_ge);
-                m8 = pair_mask8(g0, g1, g2, g3);
-                if (((x0 | x1 | x2 | x3) & 0x80008000u) && !none) e8 = pair_mask8(x0, x1, x2, x3);
-                if (drop) {
-                    // kept halves cleared: bit 15 / 31 of the compare sums widened to half masks (kept ties follow in C)
-                    auto cleared = [](uint32_t wv, uint32_t g) { return wv & ~(((g >> 15) & 0x00010001u) * 0xFFFFu); };
-                    *reinterpret_cast<uint4*>(drop + vi * 8) = make_uint4(cleared(v.x, g0), cleared(v.y, g1), cleared(v.z, g2), cleared(v.w, g3));
+                if constexpr (BF) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(buf + vi * 16);
+                    const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
+                    const uint32_t g0 = a0 + add_gt, g1 = a1 + add_gt, g2 = a2 + add_gt, g3 = a3 + add_gt;
+                    const uint32_t x0 = g0 ^ (a0 + add_ge), x1 = g1 ^ (a1 + add_ge), x2 = g2 ^ (a2 + add_ge), x3 = g3 ^ (a3 + add_ge);
+                    m8 = pair_mask8(g0, g1, g2, g3);
+                    if (((x0 | x1 | x2 | x3) & 0x80008000u) && !none) e8 = pair_mask8(x0, x1, x2, x3);
+                    if (drop) {
+                        // kept halves cleared: bit 15 / 31 of the compare sums widened to half masks (kept ties follow in C)
+                        auto cleared = [](uint32_t wv, uint32_t g) { return wv & ~(((g >> 15) & 0x00010001u) * 0xFFFFu); };
+                        *reinterpret_cast<uint4*>(drop + vi * 8) = make_uint4(cleared(v.x, g0), cleared(v.y, g1), cleared(v.z, g2), cleared(v.w, g3));
+                    }
+                } else {
+                    // float32 keys: the 31 magnitude bits (a threshold above every key compares false everywhere)
+                    const uint4 lo = *reinterpret_cast<const uint4*>(buf + vi * 32), hi = *reinterpret_cast<const uint4*>(buf + vi * 32 + 16);
+                    const uint32_t k8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t key = k8[i] & 0x7FFFFFFFu;
+                        m8 |= (uint32_t)(key > tau) << i;
+                        e8 |= (uint32_t)(key == tau) << i;
+                    }
                 }
             }
             reinterpret_cast<uint8_t*>(keep_map)[vi] = (uint8_t)m8;
@@ -264,8 +282,8 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_bf16_kernel(Select
         }
         // ---- E: entry-parallel write ----
         int32_t* const idx = a.idx + (int64_t)ut * a.kcap + base;
-        uint16_t* const val = reinterpret_cast<uint16_t*>(a.val) + (int64_t)ut * a.kcap + base;
-        uint32_t* const pk = a.packed ? a.packed + (int64_t)ut * a.kcap + base : nullptr;
+        T* const val = reinterpret_cast<T*>(a.val) + (int64_t)ut * a.kcap + base;
+        uint32_t* const pk = (BF && a.packed) ? a.packed + (int64_t)ut * a.kcap + base : nullptr;
         for (uint32_t r = tid; r < n_keep; r += kFusedThreads) {
             // the last word whose prefix does not exceed r holds entry r (empty words share their successor's prefix)
             int w = 0;
@@ -273,15 +291,17 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_bf16_kernel(Select
             for (int s = kChunkWords / 2; s; s >>= 1)
                 if (pre[w + s] <= r) w += s;
             const int flat = w * 32 + kth_set_bit(keep_map[w], r - pre[w]);
-            const uint32_t bits = reinterpret_cast<const uint16_t*>(buf)[flat];
+            const T v = reinterpret_cast<const T*>(buf)[flat];
             idx[r] = (int32_t)(e0 + flat);
-            val[r] = (uint16_t)bits;
-            if (pk) {
-                // (byte offset / 2) inside a 16-token x 128-channel tile of two 64-channel halves with 128-byte rows whose
-                // 16-byte chunks are XOR-swizzled with the row
-                const int row = (flat >> 7) & 15, ch = flat & 127;
-                const uint32_t o = (uint32_t)((ch >> 6) * 2048 + row * 128 + ((((ch >> 3) & 7) ^ (row & 7)) << 4) + (ch & 7) * 2);
-                pk[r] = bits | ((o >> 1) << 16);
+            val[r] = v;
+            if constexpr (BF) {
+                if (pk) {
+                    // (byte offset / 2) inside a 16-token x 128-channel tile of two 64-channel halves with 128-byte rows whose
+                    // 16-byte chunks are XOR-swizzled with the row
+                    const int row = (flat >> 7) & 15, ch = flat & 127;
+                    const uint32_t o = (uint32_t)((ch >> 6) * 2048 + row * 128 + ((((ch >> 3) & 7) ^ (row & 7)) << 4) + (ch & 7) * 2);
+                    pk[r] = (uint32_t)__bfloat16_as_ushort(v) | ((o >> 1) << 16);
+                }
             }
         }
         __syncthreads();  // the buffer and the maps are free again
@@ -290,18 +310,21 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_bf16_kernel(Select
 
 }  // namespace
 
-cudaError_t launch_select_fused_bf16(const SelectArgs& a, cudaStream_t st) {
+cudaError_t launch_select_fused(const SelectArgs& a, int dtype, cudaStream_t st) {
     static PerDevice once;
     cudaError_t e = once.ensure([&]() {
-        return cudaFuncSetAttribute(select_fused_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem);
+        cudaError_t e1 = cudaFuncSetAttribute(select_fused_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem);
+        if (e1 != cudaSuccess) return e1;
+        return cudaFuncSetAttribute(select_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem);
     });
     if (e != cudaSuccess) return e;
     const int64_t n = (int64_t)a.T * a.d;
-    const int chunks_per_ut = (int)((n + kChunkElems - 1) / kChunkElems);
+    const int chunk_elems = kChunkBytes / (dtype == FDKV_BF16 ? 2 : 4);
+    const int chunks_per_ut = (int)((n + chunk_elems - 1) / chunk_elems);
     const int64_t nchunks = (int64_t)chunks_per_ut * a.ut_count;
     if (nchunks <= 0) return cudaSuccess;
-    // the look-back records (one 64-bit word per chunk) and the ticket counter live in the per-tile count arrays of
-    // the general path, which this kernel does not need; both start at zero
+    // the look-back records (one 64-bit word per chunk) and the ticket counter live in two per-tile scratch arrays of
+    // the workspace (a chunk holds at least four 16-token tiles); both start at zero
     unsigned long long* records = reinterpret_cast<unsigned long long*>(a.tile_cnt) + (int64_t)a.ut_begin * a.ntiles_max;
     uint32_t* ticket = a.tile_eq + (int64_t)a.ut_begin * a.ntiles_max;
     if ((e = cudaMemsetAsync(records, 0, (size_t)nchunks * 8, st)) != cudaSuccess) return e;
@@ -310,7 +333,10 @@ cudaError_t launch_select_fused_bf16(const SelectArgs& a, cudaStream_t st) {
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const int grid = (int)std::min<int64_t>(nchunks, (int64_t)sms * 3);  // three blocks of 70 KiB per SM
-    select_fused_bf16_kernel<<<grid, kFusedThreads, kFusedSmem, st>>>(a, chunks_per_ut, (int)nchunks, ticket, records);
+    if (dtype == FDKV_BF16)
+        select_fused_kernel<__nv_bfloat16><<<grid, kFusedThreads, kFusedSmem, st>>>(a, chunks_per_ut, (int)nchunks, ticket, records);
+    else
+        select_fused_kernel<float><<<grid, kFusedThreads, kFusedSmem, st>>>(a, chunks_per_ut, (int)nchunks, ticket, records);
     count_launch(1);
     return cudaGetLastError();
 }
