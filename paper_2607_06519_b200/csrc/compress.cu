@@ -177,23 +177,74 @@ __global__ void __launch_bounds__(1024) threshold_kernel(uint32_t* hist, SelStat
 }
 
 // ----- C2b (float32 only): histogram of the next 8 key bits among entries that match the prefix ------
+// The first refinement (prefix = the 15 bits of the split's histogram) also collects the low 16 bits of every matching
+// key in the unit-tensor's index list, which nothing has written yet (`cap` entries); the histogram holds the bins in
+// words [0, 256), the candidate count in word 256 and an overflow flag in word 257.  The second refinement then reads
+// those candidates instead of the whole tensor; only if they did not fit does the full pass run again.
+constexpr int kCandCount = 256, kCandOverflow = 257;
+constexpr int kCandBlock = 2048;  // candidates a thread block of the first refinement gathers before its one reservation in the list
 __global__ void __launch_bounds__(256) refine_hist_kernel(const float* z1, int64_t unit_stride, int64_t n,
                                                           int ut_begin, const SelState* sel, uint32_t* hist,
-                                                          int shift_prefix, int shift_digit) {
+                                                          int shift_prefix, int shift_digit, int32_t* cand_all, int64_t cap,
+                                                          int only_on_overflow) {
     __shared__ uint32_t s_h[256];
+    __shared__ uint16_t s_c[kCandBlock];
+    __shared__ uint32_t s_n, s_base;
     const int ut = ut_begin + blockIdx.y;
+    uint32_t* const h = hist + (int64_t)ut * kHistBins;
+    if (only_on_overflow && !h[kCandOverflow]) return;  // (block-uniform: the candidates served this pass)
     s_h[threadIdx.x] = 0;
+    if (threadIdx.x == 0) s_n = 0;
     __syncthreads();
     const uint32_t prefix = sel[ut].prefix;
     if (prefix != 0xFFFFFFFFu) {
         const float* z = z1 + (int64_t)ut * unit_stride;
         for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
             const uint32_t key = key_of(z[i]);
-            if ((key >> shift_prefix) == prefix) atomicAdd(&s_h[(key >> shift_digit) & 0xFFu], 1u);
+            if ((key >> shift_prefix) == prefix) {
+                atomicAdd(&s_h[(key >> shift_digit) & 0xFFu], 1u);
+                if (cand_all) {
+                    const uint32_t pos = atomicAdd(&s_n, 1u);
+                    if (pos < (uint32_t)kCandBlock) s_c[pos] = (uint16_t)(key & 0xFFFFu);
+                }
+            }
         }
     }
     __syncthreads();
-    if (s_h[threadIdx.x]) atomicAdd(&hist[(int64_t)ut * kHistBins + threadIdx.x], s_h[threadIdx.x]);
+    if (s_h[threadIdx.x]) atomicAdd(&h[threadIdx.x], s_h[threadIdx.x]);
+    if (cand_all) {
+        const uint32_t mine = s_n;
+        if (threadIdx.x == 0) {
+            s_base = atomicAdd(&h[kCandCount], mine);
+            if (mine > (uint32_t)kCandBlock) h[kCandOverflow] = 1u;  // more than the block could hold: the full pass runs again
+        }
+        __syncthreads();
+        const uint32_t base = s_base;
+        for (uint32_t i = threadIdx.x; i < min(mine, (uint32_t)kCandBlock); i += blockDim.x)
+            if ((int64_t)(base + i) < cap) cand_all[(int64_t)ut * cap + base + i] = (int32_t)s_c[i];
+    }
+}
+// second refinement from the collected candidates: one thread block per unit-tensor
+__global__ void __launch_bounds__(256) refine_candidates_kernel(int ut_begin, const SelState* sel, uint32_t* hist, const int32_t* cand_all,
+                                                                int64_t cap) {
+    __shared__ uint32_t s_h[256];
+    const int ut = ut_begin + blockIdx.x;
+    uint32_t* const h = hist + (int64_t)ut * kHistBins;
+    const uint32_t count = h[kCandCount];
+    if ((int64_t)count > cap || h[kCandOverflow]) {  // they did not fit: the full pass that follows does the work
+        if (threadIdx.x == 0) h[kCandOverflow] = 1u;
+        return;
+    }
+    s_h[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t prefix = sel[ut].prefix;  // 23 bits by now: the candidates share its upper 15
+    if (prefix != 0xFFFFFFFFu)
+        for (uint32_t i = threadIdx.x; i < count; i += blockDim.x) {
+            const uint32_t c = (uint32_t)cand_all[(int64_t)ut * cap + i];
+            if ((c >> 8) == (prefix & 0xFFu)) atomicAdd(&s_h[c & 0xFFu], 1u);
+        }
+    __syncthreads();
+    if (s_h[threadIdx.x]) h[threadIdx.x] = s_h[threadIdx.x];
 }
 
 // (C3-C5, the index-ordered compaction, live in select_fused.cu.)
@@ -245,12 +296,13 @@ cudaError_t launch_select_and_compact(const SelectArgs& a, int dtype, cudaStream
         threshold_kernel<<<a.ut_count, 1024, 0, st>>>(a.hist, a.sel, a.ut_begin, kHistBins, 15, 1, 0, 0, k);
         const int chunks = (int)std::min<int64_t>(64, (n + 256 * 16 - 1) / (256 * 16));
         refine_hist_kernel<<<dim3(chunks, a.ut_count), 256, 0, st>>>(reinterpret_cast<const float*>(a.z1), a.unit_stride,
-                                                                     n, a.ut_begin, a.sel, a.hist, 16, 8);
+                                                                     n, a.ut_begin, a.sel, a.hist, 16, 8, a.idx, a.kcap, 0);
         threshold_kernel<<<a.ut_count, 256, 0, st>>>(a.hist, a.sel, a.ut_begin, 256, 8, 0, 0, 0, k);
+        refine_candidates_kernel<<<a.ut_count, 256, 0, st>>>(a.ut_begin, a.sel, a.hist, a.idx, a.kcap);
         refine_hist_kernel<<<dim3(chunks, a.ut_count), 256, 0, st>>>(reinterpret_cast<const float*>(a.z1), a.unit_stride,
-                                                                     n, a.ut_begin, a.sel, a.hist, 8, 0);
+                                                                     n, a.ut_begin, a.sel, a.hist, 8, 0, nullptr, 0, 1);
         threshold_kernel<<<a.ut_count, 256, 0, st>>>(a.hist, a.sel, a.ut_begin, 256, 8, 0, 1, 0, k);
-        count_launch(5);
+        count_launch(6);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
