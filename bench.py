@@ -35,6 +35,9 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC_BYTES = {
     "decode32k": 146.6e6,
     "decode32k_4l": 146.6e6,
+    # 554.0 MB read + 4.5 MB written per launch on the 4-layer cut of the 128k workload
+    "decode128k": 558.5e6,
+    "decode128k_4l": 558.5e6,
 }
 
 
