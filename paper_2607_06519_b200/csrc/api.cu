@@ -81,8 +81,8 @@ void make_layouts(const Shape& s, WsLayout& w, ArenaLayout& a) {
     w.eval = take(s.B == 4 ? (size_t)s.NT * s.kcap * 4 : 0);
     w.hist = take((size_t)s.NT * kHistBins * 4);
     w.sel = take((size_t)s.NT * sizeof(SelState));
-    w.tile_cnt = take((size_t)s.NT * s.ntiles_max * 8);
-    w.tile_eq = take((size_t)s.NT * s.ntiles_max * 4);
+    w.lb_records = take((size_t)s.NT * s.ntiles_max * 8);
+    w.lb_ticket = take(256);
     w.tile_off = take((size_t)s.NT * (s.ntiles_max + 1) * 4);
     w.idx = take((size_t)s.NT * s.kcap * 4);
     w.val = take((size_t)s.NT * s.NB * s.kcap * s.esize);
@@ -312,8 +312,8 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
         sa.z1 = c->work + c->ws.energy;
         sa.hist = wsp<uint32_t>(c, c->ws.hist);
         sa.sel = wsp<SelState>(c, c->ws.sel);
-        sa.tile_cnt = wsp<uint32_t>(c, c->ws.tile_cnt);
-        sa.tile_eq = wsp<uint32_t>(c, c->ws.tile_eq);
+        sa.lb_records = wsp<unsigned long long>(c, c->ws.lb_records);
+        sa.lb_ticket = wsp<uint32_t>(c, c->ws.lb_ticket);
         sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
         sa.idx = wsp<int32_t>(c, c->ws.idx);
         sa.val = c->work + c->ws.eval;
@@ -359,8 +359,8 @@ fdkv_status fdkv_compress_prefill(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t 
     sa.z1 = c->work + c->ws.z1;
     sa.hist = wsp<uint32_t>(c, c->ws.hist);
     sa.sel = wsp<SelState>(c, c->ws.sel);
-    sa.tile_cnt = wsp<uint32_t>(c, c->ws.tile_cnt);
-    sa.tile_eq = wsp<uint32_t>(c, c->ws.tile_eq);
+    sa.lb_records = wsp<unsigned long long>(c, c->ws.lb_records);
+    sa.lb_ticket = wsp<uint32_t>(c, c->ws.lb_ticket);
     sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
     sa.idx = wsp<int32_t>(c, c->ws.idx);
     sa.val = c->work + c->ws.val;
@@ -834,8 +834,8 @@ fdkv_status fdkv_fold_tail(fdkv_ctx* c, int32_t seq, int32_t n, void* stream) {
     sa.unit_stride = (int64_t)s.Tmax * s.d; sa.kcap = s.kcap; sa.ntiles_max = s.ntiles_max;
     sa.hist = wsp<uint32_t>(c, c->ws.hist);
     sa.sel = wsp<SelState>(c, c->ws.sel);
-    sa.tile_cnt = wsp<uint32_t>(c, c->ws.tile_cnt);
-    sa.tile_eq = wsp<uint32_t>(c, c->ws.tile_eq);
+    sa.lb_records = wsp<unsigned long long>(c, c->ws.lb_records);
+    sa.lb_ticket = wsp<uint32_t>(c, c->ws.lb_ticket);
     sa.tile_off = wsp<int32_t>(c, c->ws.tile_off);
     sa.idx = wsp<int32_t>(c, c->ws.idx);
     sa.z1drop = nullptr;

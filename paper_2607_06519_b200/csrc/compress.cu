@@ -371,7 +371,7 @@ cudaError_t launch_strided_copy(const void* src, int64_t stride_t, void* dst, in
 // ---------------------------------------------------------------------------------------------------------------
 // Allocation-free compression of one [T][d] tensor pair (declared in fdkv.h as fdkv_compress_unit_noalloc).
 // Same kernels as fdkv_compress_prefill; the scratch they need (the Z1 temporary, the magnitude histogram, the
-// select state and the per-tile counts / offsets) lives in the file-scope device array below instead of a
+// select state, the look-back records and the tile offsets) lives in the file-scope device array below instead of a
 // caller-provided workspace.  Every GPU that loads this library holds the array until the process exits.
 // ---------------------------------------------------------------------------------------------------------------
 namespace fdkv {
@@ -383,9 +383,9 @@ constexpr size_t kNaZ1 = 0;                                                     
 constexpr size_t kNaHist = kNaZ1 + (size_t)kNoAllocMaxElems * 4;
 constexpr size_t kNaSel = kNaHist + (size_t)fdkv::kHistBins * 4;
 constexpr size_t kNaStatus = kNaSel + 256;
-constexpr size_t kNaCnt = kNaStatus + 256;
-constexpr size_t kNaEq = kNaCnt + (size_t)kNoAllocMaxTiles * 8;
-constexpr size_t kNaOff = kNaEq + (size_t)kNoAllocMaxTiles * 4;
+constexpr size_t kNaRecords = kNaStatus + 256;
+constexpr size_t kNaTicket = kNaRecords + (size_t)kNoAllocMaxTiles * 8;
+constexpr size_t kNaOff = kNaTicket + 256;
 constexpr size_t kNaBytes = (kNaOff + (size_t)(kNoAllocMaxTiles + 1) * 4 + 255) / 256 * 256;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
@@ -457,8 +457,8 @@ extern "C" fdkv_status fdkv_compress_unit_noalloc(const void* x0, const void* x1
     sa.z1 = sc + kNaZ1;
     sa.hist = reinterpret_cast<uint32_t*>(sc + kNaHist);
     sa.sel = reinterpret_cast<SelState*>(sc + kNaSel);
-    sa.tile_cnt = reinterpret_cast<uint32_t*>(sc + kNaCnt);
-    sa.tile_eq = reinterpret_cast<uint32_t*>(sc + kNaEq);
+    sa.lb_records = reinterpret_cast<unsigned long long*>(sc + kNaRecords);
+    sa.lb_ticket = reinterpret_cast<uint32_t*>(sc + kNaTicket);
     sa.tile_off = reinterpret_cast<int32_t*>(sc + kNaOff);
     sa.idx = idx_out; sa.val = val_out; sa.packed = nullptr; sa.z1drop = nullptr;
     sa.status = reinterpret_cast<int32_t*>(sc + kNaStatus);

@@ -80,7 +80,7 @@ struct Shape {
 struct WsLayout {
     size_t tok_score, tok_flag, tok_list, tok_off;
     size_t energy, eval;  // four-layer blocks: per-position high-frequency energy (float32) and the kept energies
-    size_t status, z0, z1, z1drop, hist, sel, tile_cnt, tile_eq, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
+    size_t status, z0, z1, z1drop, hist, sel, lb_records, lb_ticket, tile_off, idx, val, packed, probe_part, probe_pos, scores, modes,
         partials, counters, io_q, io_k, io_v, io_out, jobs, total;  // io_*: host-I/O staging, [L] layers each
 };
 struct ArenaLayout {
@@ -154,7 +154,8 @@ struct SelectArgs {
     const void* z1;
     uint32_t* hist;
     SelState* sel;
-    uint32_t *tile_cnt, *tile_eq;
+    unsigned long long* lb_records;  // look-back records of the ordered select: one 64-bit word per (unit-tensor, chunk), ntiles_max per unit-tensor
+    uint32_t* lb_ticket;             // its ticket counter (one word)
     int32_t* tile_off;
     int32_t* idx;
     void* val;

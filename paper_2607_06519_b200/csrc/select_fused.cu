@@ -323,10 +323,10 @@ cudaError_t launch_select_fused(const SelectArgs& a, int dtype, cudaStream_t st)
     const int chunks_per_ut = (int)((n + chunk_elems - 1) / chunk_elems);
     const int64_t nchunks = (int64_t)chunks_per_ut * a.ut_count;
     if (nchunks <= 0) return cudaSuccess;
-    // the look-back records (one 64-bit word per chunk) and the ticket counter live in two per-tile scratch arrays of
-    // the workspace (a chunk holds at least four 16-token tiles); both start at zero
-    unsigned long long* records = reinterpret_cast<unsigned long long*>(a.tile_cnt) + (int64_t)a.ut_begin * a.ntiles_max;
-    uint32_t* ticket = a.tile_eq + (int64_t)a.ut_begin * a.ntiles_max;
+    // the look-back records (one 64-bit word per chunk; a chunk holds at least four 16-token tiles, the array one word
+    // per tile) and the ticket counter start at zero
+    unsigned long long* records = a.lb_records + (int64_t)a.ut_begin * a.ntiles_max;
+    uint32_t* ticket = a.lb_ticket;
     if ((e = cudaMemsetAsync(records, 0, (size_t)nchunks * 8, st)) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(ticket, 0, 4, st)) != cudaSuccess) return e;
     int dev = 0, sms = 0;
