@@ -197,6 +197,10 @@ fdkv_status fdkv_commit(fdkv_ctx* ctx, int32_t seq, void* stream);
  * q: [batch][n_q_heads][d].  k_new / v_new: [batch][n_kv_heads][d], appended to the layer's tail before
  * attending, or both NULL (no append).  out: [batch][n_q_heads][d] in out_dtype.
  * Sequence slots 0..batch-1 must be committed.
+ * Stream order: q, k_new and v_new are read only after every kernel enqueued earlier on `stream` has completed
+ * (the kernels start early under programmatic dependent launch, but wait before their first read of caller data),
+ * so the caller's projection kernels may be enqueued directly ahead of this call.  The tail lengths are tracked on
+ * the host: a call that would exceed max_tail returns FDKV_ERR_STATE before anything is enqueued.
  */
 fdkv_status fdkv_decode_attn(fdkv_ctx* ctx, int32_t layer, int32_t batch, const void* q, const void* k_new,
                              const void* v_new, void* out, int32_t out_dtype, void* stream);
