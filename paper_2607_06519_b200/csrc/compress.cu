@@ -128,39 +128,48 @@ __global__ void __launch_bounds__(1024) split_hist_kernel(CompressArgs a, int to
 __global__ void __launch_bounds__(1024) threshold_kernel(uint32_t* hist, SelState* sel, int ut_begin, int nbins,
                                                          int bits, int first, int last, int shift_final,
                                                          uint32_t k_init) {
-    __shared__ uint32_t s_part[1024];
+    __shared__ uint32_t s_tot[32];
     __shared__ uint32_t s_found_bin, s_found_above;
     const int ut = ut_begin + blockIdx.x;
     uint32_t* h = hist + (int64_t)ut * kHistBins;
     SelState st = sel[ut];
     if (first) { st.prefix = 0; st.k_rem = k_init; }
-    const int per = nbins / blockDim.x;  // nbins is a multiple of blockDim (32768 or 256 with 256 threads)
-    // thread i owns bins [nbins - (i+1)*per, nbins - i*per): thread 0 owns the largest keys
-    const int hi = nbins - threadIdx.x * per;
+    // Warp w owns the segment of nbins / nwarps bins below nbins - w * seg (warp 0 the largest keys) and reads it in
+    // rows of 32 consecutive bins, largest first: lane l of row i holds bin hi - 1 - 32 i - l.
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int seg = nbins / nwarps, rows = seg / 32;  // nbins is a multiple of 32 * nwarps (32768 / 1024 threads, 256 / 256)
+    const int hi = nbins - warp * seg;
     uint32_t mine = 0;
-    for (int b = hi - 1; b >= hi - per; --b) mine += h[b];
-    s_part[threadIdx.x] = mine;
+    for (int i = 0; i < rows; ++i) mine += h[hi - 1 - 32 * i - lane];
+#pragma unroll
+    for (int o = 16; o; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+    if (lane == 0) s_tot[warp] = mine;
     if (threadIdx.x == 0) { s_found_bin = 0xFFFFFFFFu; s_found_above = 0; }
     __syncthreads();
-    // exclusive prefix over threads (counts of strictly larger bins), simple Hillis-Steele in shared memory
-    uint32_t incl = mine;
-    for (int off = 1; off < blockDim.x; off <<= 1) {
-        uint32_t add = threadIdx.x >= off ? s_part[threadIdx.x - off] : 0;
-        __syncthreads();
-        incl += add;
-        s_part[threadIdx.x] = incl;
-        __syncthreads();
-    }
-    uint32_t above = incl - mine;
+    uint32_t above = 0;  // keys in the segments of larger keys
+    for (int w = 0; w < warp; ++w) above += s_tot[w];
     if (st.k_rem > 0 && above < st.k_rem && st.k_rem <= above + mine) {
-        for (int b = hi - 1; b >= hi - per; --b) {
+        // the k-th key lies in this warp's segment: walk its rows with a warp scan (the condition is warp-uniform)
+        for (int i = 0; i < rows; ++i) {
+            const int b = hi - 1 - 32 * i - lane;
             const uint32_t c = h[b];
-            if (st.k_rem <= above + c) { s_found_bin = (uint32_t)b; s_found_above = above; break; }
-            above += c;
+            uint32_t incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const uint32_t before = above + incl - c;  // keys larger than bin b
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, before < st.k_rem && st.k_rem <= before + c);
+            if (hit) {
+                if (lane == __ffs((int)hit) - 1) { s_found_bin = (uint32_t)b; s_found_above = before; }
+                break;
+            }
+            above += __shfl_sync(0xFFFFFFFFu, incl, 31);
         }
     }
     __syncthreads();
-    for (int b = hi - 1; b >= hi - per; --b) h[b] = 0;
+    for (int i = 0; i < rows; ++i) h[hi - 1 - 32 * i - lane] = 0;
     if (threadIdx.x == 0) {
         if (st.k_rem == 0 || s_found_bin == 0xFFFFFFFFu) {
             // nothing (left) to take: a threshold above every key
