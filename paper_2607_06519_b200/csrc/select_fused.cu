@@ -3,10 +3,12 @@
 //
 // Persistent thread blocks take 32 KiB chunks of the unit-tensors in ticket order (a global counter, so every chunk
 // with a lower ticket has been started by a block that is resident: the look-back below cannot wait on work that
-// has no SM).  Tickets run over the unit-tensors first (ticket t = chunk t / n of unit-tensor t % n): the blocks that
-// are resident at one time then work on different unit-tensors, and a look-back finds a finished record a few
-// chunks back instead of walking through hundreds of chunks that are all in flight.  A chunk is copied into shared memory by one bulk TMA copy while the previous chunk is processed (two
-// buffers, one mbarrier each).  Per chunk:
+// has no SM).  Six blocks share an SM: while one waits for its copy or at a barrier, the others compute, which
+// measured faster than three blocks that each prefetch their next chunk into a second buffer.  Tickets run over
+// the unit-tensors first (ticket t = chunk t / n of unit-tensor t % n): the blocks that are resident at one time
+// then work on different unit-tensors, and a look-back finds a finished record a few chunks back instead of
+// walking through hundreds of chunks that are all in flight.  A chunk is copied into shared memory by one bulk TMA
+// copy (mbarrier transaction count).  Per chunk:
 //   A  every thread compares its 16-byte vectors with the threshold (bf16: on 16-bit pairs inside 32-bit registers) and
 //      writes one keep byte and one tie byte per eight elements into two bit maps; K tensors also get their copy with
 //      the kept coefficients zeroed (the second operand of the probe);
@@ -37,13 +39,13 @@ constexpr int kFusedThreads = 256;
 constexpr uint32_t kSpinCap = 1u << 22;         // polls of a look-back before it gives up
 
 // shared memory (bytes)
-constexpr int oBuf = 0;                               // 2 x 32 KiB chunk buffers
-constexpr int oKeep = 2 * kChunkBytes;                // keep map
-constexpr int oTie = oKeep + kMaxChunkWords * 4;      // tie map
-constexpr int oPre = oTie + kMaxChunkWords * 4;       // list position of every word's first entry
+constexpr int oBuf = 0;                               // the chunk
+constexpr int oKeep = kChunkBytes;                    // keep map
+constexpr int oTie = oKeep + kMaxChunkWords * 4;      // tie map; from step C on the list position of every word's first entry
+constexpr int oPre = oTie;                            // (a thread holds its tie words in registers before it writes their positions)
 constexpr int oWarp = oPre + (kMaxChunkWords + 8) * 4;  // per-warp sums
-constexpr int oMisc = oWarp + 128;                    // tickets [2], before_gt, before_eq, abort flag
-constexpr int oBar = oMisc + 64;                      // two mbarriers
+constexpr int oMisc = oWarp + 128;                    // ticket, (unused), before_gt, before_eq, abort flag
+constexpr int oBar = oMisc + 64;                      // the copy's mbarrier
 constexpr int kFusedSmem = oBar + 16;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -113,16 +115,16 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_kernel(SelectArgs 
     volatile uint32_t* const abort_flag = misc + 4;
     const uint32_t bar0 = smem_u32(smem + oBar);
 
-    // one thread takes a ticket and starts the copy of that chunk into buffer `b`
-    auto fetch = [&](int b) {
+    // one thread takes a ticket and starts the copy of that chunk
+    auto fetch = [&]() {
         const uint32_t t = atomicAdd(ticket, 1u);
-        misc[b] = t;
+        misc[0] = t;
         if (t < (uint32_t)nchunks) {
             const int ut = a.ut_begin + (int)(t % (uint32_t)a.ut_count), ck = (int)(t / (uint32_t)a.ut_count);
             const int64_t e0 = (int64_t)ck * kChunkElems;
             const uint32_t bytes = (uint32_t)min((int64_t)kChunkElems, (int64_t)a.T * a.d - e0) * (uint32_t)sizeof(T);
             const T* src = reinterpret_cast<const T*>(a.z1) + (int64_t)ut * a.unit_stride + e0;
-            const uint32_t bar = bar0 + 8 * b, dst = smem_u32(smem + oBuf + b * kChunkBytes);
+            const uint32_t bar = bar0, dst = smem_u32(smem + oBuf);
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                          "l"(src), "r"(bytes), "r"(bar)
@@ -131,23 +133,20 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_kernel(SelectArgs 
     };
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         *abort_flag = 0;
-        fetch(0);
+        fetch();
     }
     __syncthreads();
 
     for (uint32_t it = 0;; ++it) {
-        const int cur = (int)(it & 1u);
-        const uint32_t tk = misc[cur];
+        const uint32_t tk = misc[0];
         if (tk >= (uint32_t)nchunks) break;
-        if (tid == 0) fetch(cur ^ 1);  // (that buffer's last readers passed the barrier that ends the previous round)
         const int ut = a.ut_begin + (int)(tk % (uint32_t)a.ut_count), ck = (int)(tk / (uint32_t)a.ut_count);
         const uint32_t tau = a.sel[ut].tau, need = a.sel[ut].need;
         const int64_t e0 = (int64_t)ck * kChunkElems;
         const int n_e = (int)min((int64_t)kChunkElems, (int64_t)a.T * a.d - e0);  // a multiple of 8
-        const uint8_t* const buf = smem + oBuf + cur * kChunkBytes;
+        const uint8_t* const buf = smem + oBuf;
         // (only bf16 storage has the copy without the kept entries: it is the tensor-core probe's operand)
         __nv_bfloat16* const drop = (BF && a.z1drop && !(ut & 1))
                                         ? reinterpret_cast<__nv_bfloat16*>(a.z1drop) + (int64_t)(ut >> 1) * a.unit_stride + e0
@@ -157,7 +156,7 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_kernel(SelectArgs 
         const uint32_t add_gt = none ? 0u : (0x7FFFu - (tau >> 16)) * 0x00010001u;
         const uint32_t add_ge = none ? 0u : (0x8000u - (tau >> 16)) * 0x00010001u;
 
-        mbar_wait_bounded(bar0 + 8 * cur, (it >> 1) & 1u, abort_flag, a.status);
+        mbar_wait_bounded(bar0, it & 1u, abort_flag, a.status);
 
         // ---- A: keep and tie bytes, the dropped-coefficient copy ----
 #pragma unroll 4
@@ -304,7 +303,9 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_kernel(SelectArgs 
                 }
             }
         }
-        __syncthreads();  // the buffer and the maps are free again
+        __syncthreads();  // the buffer and the maps are free again: the next ticket and its copy
+        if (tid == 0) fetch();
+        __syncthreads();
     }
 }
 
@@ -332,7 +333,7 @@ cudaError_t launch_select_fused(const SelectArgs& a, int dtype, cudaStream_t st)
     int dev = 0, sms = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    const int grid = (int)std::min<int64_t>(nchunks, (int64_t)sms * 3);  // three blocks of 70 KiB per SM
+    const int grid = (int)std::min<int64_t>(nchunks, (int64_t)sms * 6);  // six blocks of 37 KiB per SM
     if (dtype == FDKV_BF16)
         select_fused_kernel<__nv_bfloat16><<<grid, kFusedThreads, kFusedSmem, st>>>(a, chunks_per_ut, (int)nchunks, ticket, records);
     else
