@@ -55,9 +55,9 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.kcap = (int64_t)align_up((size_t)(s.kmax + kListPad), 64);
     s.ntiles_max = (s.Tmax + kResTile - 1) / kResTile;
     // per-unit partial-sum slots of the probe: one per 64-token tile (portable kernel) or one per work item of the
-    // tensor-core kernel (layers x 256-row blocks x key splits of at least 8 tiles), whichever is more
+    // tensor-core kernel (layers x 128-row blocks x key splits of at least 8 tiles), whichever is more
     s.nptiles_max = std::max((s.Tmax + kProbeTile - 1) / kProbeTile,
-                             B * ((G * kMaxW + 255) / 256) * (((s.Tmax - 1) / kProbeBoxRows + 1 + 7) / 8));
+                             B * ((G * kMaxW + 127) / 128) * (((s.Tmax - 1) / kProbeBoxRows + 1 + 7) / 8));
     s.tail_rows = (s.max_tail + kRowPad - 1) / kRowPad * kRowPad;
     if (c.residual_rule != FDKV_RESIDUAL_ENTRIES && c.residual_rule != FDKV_RESIDUAL_TOKENS) return false;
     s.tok_rule = c.residual_rule == FDKV_RESIDUAL_TOKENS;

@@ -19,7 +19,7 @@ constexpr int kMaxSplits = 160;      // split-K partial slots per (sequence, que
 constexpr int kMaxW = 128;           // probe queries
 constexpr int kListPad = 32;         // slack entries after each residual list (aligned over-reads stay in bounds)
 constexpr int kMaxGroup = 8;
-constexpr int kProbeBoxRows = 128;   // key tokens per tile of the tensor-core probe (rows of its TMA boxes)
+constexpr int kProbeBoxRows = 256;   // key tokens per tile of the tensor-core probe (rows of its TMA boxes)
 constexpr int kFastMaxUnits = 1024;   // (sequences x KV heads) one launch of the bf16 / head_dim 128 decode kernel plans for
 constexpr int kProbeTile = 64;       // tokens per probe CTA (generic kernel)
 constexpr int kRowPad = 128;         // packed row blocks and tails are padded (zero rows) to this many tokens

@@ -4,16 +4,17 @@
 // needs sum_{rows, keys j <= pos(row)} (Q_row . R_j)^2 over the 2*G*W probe rows (2 layers x G group heads x W
 // probe queries).  That is a dense [rows x 128] x [128 x T] contraction whose result is squared, masked causally
 // and summed without ever leaving the SM:
-//   * work item = (unit, layer of the pair, block of 256 probe rows, candidate, range of 128-token key tiles);
+//   * work item = (unit, layer of the pair, block of 128 probe rows, candidate, range of 256-token key tiles);
 //     one CTA per item, 6 warps: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner), warps 2-5 = epilogue;
-//   * A (the item's 256 Q rows, two M tiles) is written once into shared memory by the epilogue threads, in the
-//     128-byte-swizzled K-major layout a TMA copy would give it; B tiles (128 tokens x 128 channels, same layout)
-//     stream through a 5-stage TMA ring;
-//   * per key tile 16 tcgen05.mma (M = 128, N = 128, K = 16, kind::f16, both operands from shared memory,
-//     bf16 x bf16 -> f32) fill one of two alternating sets of two 128 x 128 f32 accumulators: all 512 columns of
-//     tensor memory.  The hand-over of an accumulator set (commit -> epilogue -> release -> next MMA) is a round trip of
-//     about a microsecond; with a single set it was paid on every tile and cost as much as the arithmetic, which is
-//     why A lives in shared memory: the 128 columns it took in tensor memory buy the second set;
+//   * A (the item's 128 Q rows) is written once into shared memory by the epilogue threads, in the
+//     128-byte-swizzled K-major layout a TMA copy would give it; B tiles (256 tokens x 128 channels, same layout)
+//     stream through a 3-stage TMA ring;
+//   * per key tile 8 tcgen05.mma (M = 128, N = 256, K = 16, kind::f16, both operands from shared memory,
+//     bf16 x bf16 -> f32) fill one of two alternating 128 x 256 f32 accumulators: all 512 columns of tensor memory.
+//     The hand-over of an accumulator (commit -> epilogue -> release -> next MMA) is a round trip of about a
+//     microsecond; with a single set it was paid on every tile and cost as much as the arithmetic, which is why A
+//     lives in shared memory: the columns it took in tensor memory buy the second set.  (Two M tiles against
+//     128-token key tiles, the same bytes per flop, measured 4 % slower.);
 //   * epilogue: tcgen05.ld (32 lanes x 32 columns per instruction), square, mask keys after the row's probe
 //     position, accumulate; the set is released as soon as its last columns are in registers; one float64 sum per
 //     item, summed across items in a fixed order by the finalize kernel.
@@ -31,19 +32,20 @@ namespace fdkv {
 namespace {
 
 constexpr int kBN = kProbeBoxRows;             // key tokens per tile (N of the MMA)
-constexpr int kBStages = 5;
+constexpr int kMT = 256 / kBN;                 // M tiles (128 Q rows each) per work item: 2 at N = 128, 1 at N = 256
+constexpr int kBStages = kBN == 128 ? 5 : 3;
 constexpr int kAccSets = 2;
-constexpr int kBHalf = kBN * 128;              // one 64-channel half of a B tile: 16 KiB
-constexpr int kBStageBytes = 2 * kBHalf;       // 32 KiB
+constexpr int kBHalf = kBN * 128;              // one 64-channel half of a B tile: 32 KiB
+constexpr int kBStageBytes = 2 * kBHalf;       // 64 KiB
 constexpr int kHdr = 1024;
 constexpr int kAHalf = 128 * 128;              // one 64-channel half of an A tile (128 Q rows): 16 KiB
-constexpr int kABytes = 2 * 2 * kAHalf;        // two M tiles: 64 KiB
-constexpr int kProbeSmem = kHdr + kABytes + kBStages * kBStageBytes;  // 225 KiB
+constexpr int kABytes = kMT * 2 * kAHalf;      // the item's M tiles
+constexpr int kProbeSmem = kHdr + kABytes + kBStages * kBStageBytes;  // 225 KiB in either form
 constexpr int kPThreads = 6 * 32;
-// Tensor memory (512 columns): two alternating sets of two 128 x 128 f32 accumulators (one per M tile).
+// Tensor memory (512 columns): two alternating sets of kMT 128 x kBN f32 accumulators (one per M tile).
 constexpr int kTmemCols = 512;
-constexpr int kAccSet = 2 * kBN;
-static_assert(kAccSets * kAccSet <= kTmemCols && kBN == 128, "tensor memory budget");
+constexpr int kAccSet = kMT * kBN;
+static_assert(kAccSets * kAccSet <= kTmemCols && (kBN == 128 || kBN == 256), "tensor memory budget");
 // header: full[8] @0, empty[8] @64, tfull[2] @128, tempty[2] @144, tmem slot @160, abort @164, reduce @192 (4 doubles)
 constexpr int oFull = 0, oEmpty = 64, oTFull = 128, oTEmpty = 144, oSlot = 160, oAbort = 164, oRed = 192;
 
@@ -151,8 +153,8 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         const int rl = (warp & 3) * 32 + lane;
         const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q_layers_dev[a.B * pair + layer]);
 #pragma unroll 1
-        for (int mt = 0; mt < 2; ++mt) {
-            const int r = mblock * 256 + mt * 128 + rl;
+        for (int mt = 0; mt < kMT; ++mt) {
+            const int r = mblock * (128 * kMT) + mt * 128 + rl;
             uint8_t* const arow = smem + kHdr + mt * 2 * kAHalf + rl * 128;
             const uint4* src = reinterpret_cast<const uint4*>(q + ((int64_t)(r % a.W) * a.Hq + h * a.G + r / a.W) * 128);
 #pragma unroll
@@ -200,7 +202,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {  // 8 steps of 16 channels: 32 bytes inside the swizzle atom of either operand
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {  // the two M tiles alternate: consecutive MMAs never wait for each other's accumulator
+                    for (int mt = 0; mt < kMT; ++mt) {  // the M tiles alternate: consecutive MMAs never wait for each other's accumulator
                         const uint64_t db = db_stage + (uint64_t)(((k >> 2) * kBHalf + (k & 3) * 32) >> 4);
                         const uint64_t da = da_all + (uint64_t)((mt * 2 * kAHalf + (k >> 2) * kAHalf + (k & 3) * 32) >> 4);
                         if (k == 0) umma_ss<0>(d0 + mt * kBN, da, db);
@@ -215,10 +217,10 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
         // ================= epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 =================
         const int lq = warp & 3;
         const int rl = lq * 32 + lane;  // row within a 128-row M tile == TMEM lane
-        int pos_row[2];
+        int pos_row[kMT];
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-            const int r = mblock * 256 + mt * 128 + rl;
+        for (int mt = 0; mt < kMT; ++mt) {
+            const int r = mblock * (128 * kMT) + mt * 128 + rl;
             pos_row[mt] = r < rows_layer ? a.pos[r % a.W] : -1;  // padding rows never count
         }
         double total = 0.0;
@@ -231,15 +233,15 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_z1, const __grid_consta
             if (!*abort_flag) {
                 const bool all_visible = t0 + kBN - 1 <= pl.pos_min;  // every key of the tile precedes every probe position
 #pragma unroll
-                for (int round = 0; round < 4; ++round) {  // 64 accumulator columns of this lane per round, two loads in flight
-                    const int mt = round >> 1, c0 = (round & 1) * 64;
+                for (int round = 0; round < kAccSet / 64; ++round) {  // 64 accumulator columns of this lane per round, two loads in flight
+                    const int mt = round / (kBN / 64), c0 = (round % (kBN / 64)) * 64;
                     uint32_t r0[32], r1[32];
                     const uint32_t ta = tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(as * kAccSet + mt * kBN + c0);
                     const int tc = t0 + c0;
                     tmem_ld32(ta, r0);
                     tmem_ld32(ta + 32, r1);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (round == 3) {  // the set's last columns are in registers: hand it back before the arithmetic
+                    if (round == kAccSet / 64 - 1) {  // the set's last columns are in registers: hand it back before the arithmetic
                         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                         __syncwarp();
                         if (lane == 0) mb_arrive(sm0 + oTEmpty + 8 * as);
@@ -301,7 +303,7 @@ cudaError_t launch_probe_tc(const ProbeArgs& a, int dtype, cudaStream_t st, bool
     pl.pos_min = a.pos_host[0];
     pl.pos_max = a.pos_host[a.W - 1];
     pl.ntiles = pl.pos_max / kBN + 1;  // keys after the last probe position never count
-    pl.mblocks = (a.G * a.W + 255) / 256;
+    pl.mblocks = (a.G * a.W + 128 * kMT - 1) / (128 * kMT);
     const int base_items = a.unit_count * a.B * pl.mblocks * 2;
     // split the key range so that the grid fills the machine several times over, but keep >= 8 tiles per item
     int nsplits = std::max(1, std::min((4 * sm_count + base_items - 1) / base_items, (pl.ntiles + 7) / 8));
