@@ -313,11 +313,12 @@ __global__ void __launch_bounds__(kFusedThreads) select_fused_kernel(SelectArgs 
 
 cudaError_t launch_select_fused(const SelectArgs& a, int dtype, cudaStream_t st) {
     static PerDevice once;
+    int sms = 0;
     cudaError_t e = once.ensure([&]() {
         cudaError_t e1 = cudaFuncSetAttribute(select_fused_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem);
         if (e1 != cudaSuccess) return e1;
         return cudaFuncSetAttribute(select_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem);
-    });
+    }, &sms);
     if (e != cudaSuccess) return e;
     const int64_t n = (int64_t)a.T * a.d;
     const int chunk_elems = kChunkBytes / (dtype == FDKV_BF16 ? 2 : 4);
@@ -330,9 +331,6 @@ cudaError_t launch_select_fused(const SelectArgs& a, int dtype, cudaStream_t st)
     uint32_t* ticket = a.lb_ticket;
     if ((e = cudaMemsetAsync(records, 0, (size_t)nchunks * 8, st)) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(ticket, 0, 4, st)) != cudaSuccess) return e;
-    int dev = 0, sms = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const int grid = (int)std::min<int64_t>(nchunks, (int64_t)sms * 6);  // six blocks of 37 KiB per SM
     if (dtype == FDKV_BF16)
         select_fused_kernel<__nv_bfloat16><<<grid, kFusedThreads, kFusedSmem, st>>>(a, chunks_per_ut, (int)nchunks, ticket, records);
