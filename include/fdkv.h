@@ -201,6 +201,10 @@ fdkv_status fdkv_commit(fdkv_ctx* ctx, int32_t seq, void* stream);
  * (the kernels start early under programmatic dependent launch, but wait before their first read of caller data),
  * so the caller's projection kernels may be enqueued directly ahead of this call.  The tail lengths are tracked on
  * the host: a call that would exceed max_tail returns FDKV_ERR_STATE before anything is enqueued.
+ * CUDA graphs: the work distribution and the tail lengths are computed on the host and travel in the launch
+ * parameters, so a captured call replays exactly the state it was captured in.  Calls on layers without generated
+ * tokens and without k_new may be captured and replayed (the benchmark does); a call that appends, or that follows
+ * appends made outside the graph, must be issued on the stream.
  */
 fdkv_status fdkv_decode_attn(fdkv_ctx* ctx, int32_t layer, int32_t batch, const void* q, const void* k_new,
                              const void* v_new, void* out, int32_t out_dtype, void* stream);
