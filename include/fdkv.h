@@ -111,8 +111,9 @@ typedef enum { FDKV_ROWS_STORAGE = 0, FDKV_ROWS_E4M3 = 1 } fdkv_row_format;
  *   probe_pos[q] >= t of | Q . (c * Z1K[t,:]) |; the k_tok = floor(T * keep_num / keep_den) tokens with the
  *   largest score (ties: lowest t) keep ALL head_dim high-frequency coefficients of K and of V.  The scores
  *   need the probe queries, so the set is chosen inside fdkv_probe (which is then mandatory before commit, even
- *   when modes are overridden); Omega(residual) counts 2*k_tok*d*e + 4*k_tok bytes.  bf16, head_dim 128 only; either
- *   block size (see the note on block size 4 above for the score and the stored rows there).
+ *   when modes are overridden); Omega(residual) counts 2*k_tok*d*e + 4*k_tok bytes.  Either storage type, head
+ *   dimension and block size (see the note on block size 4 above for the score and the stored rows there); bf16 with
+ *   head_dim 128 runs the tensor-core kernels, the rest the float32 score and probe kernels and the portable decode kernel.
  */
 typedef enum { FDKV_RESIDUAL_ENTRIES = 0, FDKV_RESIDUAL_TOKENS = 1 } fdkv_residual_rule;
 

@@ -61,7 +61,6 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.tail_rows = (s.max_tail + kRowPad - 1) / kRowPad * kRowPad;
     if (c.residual_rule != FDKV_RESIDUAL_ENTRIES && c.residual_rule != FDKV_RESIDUAL_TOKENS) return false;
     s.tok_rule = c.residual_rule == FDKV_RESIDUAL_TOKENS;
-    if (s.tok_rule && !(c.dtype == FDKV_BF16 && c.head_dim == 128)) return false;  // tensor-core kernels only
     s.ktok_max = (int64_t)s.Tmax * s.keep_num / s.keep_den;
     s.ktok_cap = (int64_t)align_up((size_t)(s.ktok_max + 32), 64);
     s.NU = s.P * s.Hkv;
@@ -217,14 +216,15 @@ fdkv_status fdkv_create(const fdkv_config* cfg, void* arena, size_t arena_bytes,
     if (s.dtype == FDKV_BF16 && s.d == 128) c->has_tmap = make_arena_tensor_map(c->arena, arena_bytes, c->tmap);
     c->packed_lists = c->has_tmap && s.max_batch * s.Hkv <= kFastMaxUnits;
     if (s.rows_f8 && !(c->packed_lists && make_rows_tensor_map_u8(c->arena, arena_bytes, kRowPad, c->tmap_u8))) { delete c; return FDKV_ERR_UNSUPPORTED; }
-    if (s.tok_rule) {
-        const bool ok = c->packed_lists && make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.NB * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
-        if (!ok) { delete c; return FDKV_ERR_UNSUPPORTED; }
-    }
+    // token rule: the tensor-core score kernel and the packed decode kernel serve bf16 / head_dim 128; everything else
+    // takes the float32 score kernel, the float32 probe kernel (which masks the selected rows itself) and the portable decode kernel
+    if (s.tok_rule && c->packed_lists)
+        c->tok_tc = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.NB * s.Tmax * s.d * s.esize, 128, c->tmap_z1_128);
+    if (s.tok_rule && s.dtype == FDKV_BF16 && s.d == 128 && !c->tok_tc) { delete c; return FDKV_ERR_UNSUPPORTED; }
     if (s.dtype == FDKV_BF16 && s.d == 128)
         c->has_probe_tmaps = make_rows_tensor_map(c->work + c->ws.z1, (size_t)s.NT * s.NB * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_z1) &&
                              make_rows_tensor_map(c->work + c->ws.z1drop, (size_t)s.NU * s.NB * s.Tmax * s.d * s.esize, kProbeBoxRows, c->tmap_drop);
-    if (s.tok_rule && !c->has_probe_tmaps) { delete c; return FDKV_ERR_UNSUPPORTED; }
+    if (c->tok_tc && !c->has_probe_tmaps) { delete c; return FDKV_ERR_UNSUPPORTED; }
     *out = c;
     return FDKV_OK;
 }
@@ -401,6 +401,7 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
     a.z1 = c->work + c->ws.z1;
     a.idx = wsp<int32_t>(c, c->ws.idx);
     a.tile_off = wsp<int32_t>(c, c->ws.tile_off);
+    a.tok_flag = (s.tok_rule && !c->tok_tc) ? wsp<uint8_t>(c, c->ws.tok_flag) : nullptr;
     a.q_layers_dev = qptr_dev;
     a.pos = pos_dev;
     a.part = wsp<double>(c, c->ws.probe_part);
@@ -426,7 +427,7 @@ fdkv_status fdkv_probe(fdkv_ctx* c, int32_t seq, int32_t pb, int32_t pe, const v
         t.list = wsp<int32_t>(c, c->ws.tok_list); t.off = wsp<int32_t>(c, c->ws.tok_off);
         t.tmap_z1_128 = c->tmap_z1_128;
         t.status = wsp<int32_t>(c, c->ws.status);
-        CU(launch_token_select(t, st));
+        CU(launch_token_select(t, s.dtype, s.d, c->tok_tc, st));
         for (int p = pb; p < pe; ++p) c->pair_scored[p] = 1;
     }
     CU(launch_probe(a, s.dtype, st));
@@ -616,7 +617,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                     for (int j = 0; j < s.NB; ++j) {
                         rows_l[j] = take(trow_b);
                         CU(launch_token_gather(c->work + c->ws.z1 + (ut * s.NB + j) * unit_stride_b, wsp<int32_t>(c, c->ws.tok_list) + (size_t)u * s.ktok_cap, k_tok,
-                                               rows_l[j], s.B == 4 ? 1 : 0, st));
+                                               rows_l[j], s.d * s.esize, (s.B == 4 && c->packed_lists) ? 1 : 0, st));
                     }
                     for (int l = 0; l < s.B; ++l) {
                         UnitDesc* d = dl[l];

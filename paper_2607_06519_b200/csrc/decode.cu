@@ -125,7 +125,26 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
                 if (lane == tt) s[g] = p;
             }
         }
-        if (with_res) {
+        if (with_res && u.res_kind == 1) {
+            // token rule: the tile's selected tokens carry whole high-frequency rows (k_idx = ascending token list, k_off =
+            // tokens kept before every 16-token slice, k_val / v_val = their rows, densely packed)
+            const T* rows = reinterpret_cast<const T*>(u.k_val);
+            const int j1 = u.k_off[min(nres, (jt + 1) * kSub)];
+            for (int j = u.k_off[jt * kSub]; j < j1; ++j) {
+                const int tt = u.k_idx[j] - jt * kGTile;
+                float kf[EPL];
+                load_row<T, EPL>(rows + (int64_t)j * D, lane, kf);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float p = 0.f;
+#pragma unroll
+                    for (int i = 0; i < EPL; ++i) p = fmaf(q[g][i], kf[i], p);
+#pragma unroll
+                    for (int o = 16; o; o >>= 1) p += __shfl_xor_sync(0xFFFFFFFFu, p, o);
+                    if (lane == tt) s[g] = fmaf(u.sign, p, s[g]);
+                }
+            }
+        } else if (with_res) {
             // sparse correction in the logit domain: q . z1 over this tile's kept K entries
 #pragma unroll
             for (int g = 0; g < G; ++g) s_corr[warp][g][lane] = 0.f;
@@ -172,7 +191,21 @@ __global__ void __launch_bounds__(kWarps * 32) decode_generic_kernel(DecodeArgs 
                 for (int i = 0; i < EPL; ++i) acc[g][i] = fmaf(pg, vf[i], acc[g][i]);
             }
         }
-        if (with_res) {
+        if (with_res && u.res_kind == 1) {
+            const T* rows = reinterpret_cast<const T*>(u.v_val);
+            const int j1 = u.k_off[min(nres, (jt + 1) * kSub)];
+            for (int j = u.k_off[jt * kSub]; j < j1; ++j) {
+                const int tt = u.k_idx[j] - jt * kGTile;
+                float vf[EPL];
+                load_row<T, EPL>(rows + (int64_t)j * D, lane, vf);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const float pg = u.sign * __shfl_sync(0xFFFFFFFFu, p[g], tt);
+#pragma unroll
+                    for (int i = 0; i < EPL; ++i) acc[g][i] = fmaf(pg, vf[i], acc[g][i]);
+                }
+            }
+        } else if (with_res) {
 #pragma unroll
             for (int g = 0; g < G; ++g) s_p[warp][g][lane] = p[g];
             __syncwarp();

@@ -122,6 +122,7 @@ struct fdkv_ctx {
     alignas(64) unsigned char tmap_z1[128], tmap_drop[128];  // probe operands (bf16, head_dim 128 only)
     bool has_probe_tmaps = false;
     alignas(64) unsigned char tmap_z1_128[128];  // staged Z1 with 128-token boxes (token-score kernel)
+    bool tok_tc = false;                         // token rule served by the tensor-core kernels (bf16, head_dim 128)
     std::vector<uint8_t> pair_scored;            // token rule: the probe has chosen this pair's token sets
     bool packed_lists = false;              // decode runs the bf16 / head_dim 128 kernel on packed residual entries
     alignas(64) unsigned char tmap_u8[128]; // CUtensorMap of the arena as 128-byte rows (8-bit row streams)
@@ -202,6 +203,7 @@ struct ProbeArgs {
     const void* z1;  // staged Z1 (unit-tensor ut = unit*2 for K)
     const int32_t* idx;
     const int32_t* tile_off;
+    const uint8_t* tok_flag;          // token rule, float32 probe kernel: [NU][Tmax] flags of the selected tokens (else null)
     const void* const* q_layers_dev;  // device array [L] of pointers
     const int32_t* pos;
     double* part;    // [NU][nptiles_max][2]
@@ -307,8 +309,9 @@ struct TokenArgs {
     const void* tmap_z1_128;
     int32_t* status;
 };
-cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st);
-cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, int twice, cudaStream_t st);
+// tensor_core: bf16 / head_dim 128 contexts (tcgen05 score kernel + the dropped-row copy); otherwise the float32 score kernel
+cudaError_t launch_token_select(const TokenArgs& a, int dtype, int d, bool tensor_core, cudaStream_t st);
+cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, int row_bytes, int twice, cudaStream_t st);
 
 // Function attributes (the opt-in to large dynamic shared memory) and the SM count belong to a device, not to the
 // process: every launcher keeps one of these and runs its set-up the first time it meets the current device.

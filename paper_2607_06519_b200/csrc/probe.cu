@@ -48,7 +48,12 @@ __global__ void __launch_bounds__(256) probe_tile_kernel(ProbeArgs a) {
             drop[t * ld + c] = v;
         }
         __syncthreads();
-        {
+        if (a.tok_flag) {
+            // token rule: the residual candidate keeps whole rows -- the selected tokens drop nothing
+            const uint8_t* flag = a.tok_flag + (int64_t)unit * a.Tmax + t0;
+            for (int i = threadIdx.x; i < nt * d; i += blockDim.x)
+                if (flag[i / d]) drop[(i / d) * ld + (i % d)] = 0.f;
+        } else {
             const int32_t* off = a.tile_off + (int64_t)ut * (a.ntiles_max + 1);
             const int ntiles = (a.T + kResTile - 1) / kResTile;
             const int j0 = t0 / kResTile, j1 = min(ntiles, (t0 + kProbeTile) / kResTile);

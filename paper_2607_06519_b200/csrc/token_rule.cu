@@ -1,4 +1,6 @@
-// Token-granular sparse residual (the paper's rule, Method between Eq. 2 and Eq. 3; bf16, head_dim 128).
+// Token-granular sparse residual (the paper's rule, Method between Eq. 2 and Eq. 3).  The tensor-core kernels below
+// serve bf16 storage with head_dim 128; other storage types and head dimensions take token_score_tile_kernel, a plain
+// float32 product, and the same selection.
 //
 //   s_t = max over (layer of the depth block, group query head, probe query q with pos[q] >= t) | Q_l . (K_l[t,:] - Khat_l^shared[t,:]) |
 //       = | Q_l . (+-c Z1K[t,:]) | for a pair, | Q_l . dev_l[t,:] | for a block of four (dev_l = layer l's deviation from the block mean);
@@ -342,11 +344,13 @@ __global__ void __launch_bounds__(256) token_drop_kernel(TokenArgs a) {
     }
 }
 
-// out[j][:] = z1[list[j]][:], optionally doubled (exact in bf16): a block of four scales its rows by 1/2 at decode time and
-// its deviations by 1, so their stored rows carry the factor 2
-__global__ void __launch_bounds__(256) token_gather_kernel(const uint4* z1, const int32_t* list, int64_t k_tok, uint4* out, int twice) {
-    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < k_tok * 16; v += (int64_t)gridDim.x * blockDim.x) {
-        uint4 x = z1[(int64_t)list[v >> 4] * 16 + (v & 15)];
+// out[j][:] = z1[list[j]][:] (rows of row_u4 16-byte vectors), optionally doubled (bf16 rows of the tensor-core decode
+// kernel only; exact): a block of four scales its rows by 1/2 at decode time and its deviations by 1, so their stored
+// rows carry the factor 2
+__global__ void __launch_bounds__(256) token_gather_kernel(const uint4* z1, const int32_t* list, int64_t k_tok, uint4* out, int row_u4,
+                                                           int twice) {
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < k_tok * row_u4; v += (int64_t)gridDim.x * blockDim.x) {
+        uint4 x = z1[(int64_t)list[v / row_u4] * row_u4 + (v % row_u4)];
         if (twice) {
             __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&x);
 #pragma unroll
@@ -356,16 +360,101 @@ __global__ void __launch_bounds__(256) token_gather_kernel(const uint4* z1, cons
     }
 }
 
+// ---- storage types and head dimensions without the tensor-core kernel: the same score as a float32 product ----
+template <typename T>
+__device__ __forceinline__ float to_f32(T x);
+template <>
+__device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+constexpr int kSTile = 64;   // tokens per thread block
+constexpr int kSRows = 16;   // probe rows staged per round
+// grid (64-token tiles, units), 256 threads: thread (token j, row group rg) takes the maximum of |q_r . z[t]| over the
+// rows r of its group whose probe position sees token t; the groups and the layers merge by atomicMax on the bit
+// patterns of the non-negative floats.
+template <typename T>
+__global__ void __launch_bounds__(256) token_score_tile_kernel(TokenArgs a, int d) {
+    extern __shared__ float ssm[];
+    const int ld = d + 1;
+    float* zs = ssm;                 // [64][d + 1]
+    float* qs = zs + kSTile * ld;    // [16][d]
+    const int unit = a.unit_begin + blockIdx.y;
+    const int t0 = blockIdx.x * kSTile;
+    const int nt = min(kSTile, a.T - t0);
+    const int h = unit % a.Hkv, pair = unit / a.Hkv;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int j = (warp & 1) * 32 + lane, rg = warp >> 1;
+    const int n_ops = a.B == 4 ? 4 : 1;
+    const int M = (a.B == 4 ? 1 : 2) * a.G * a.W;  // probe rows per operand
+    float best = 0.f;
+    for (int op = 0; op < n_ops; ++op) {
+        const T* z1 = reinterpret_cast<const T*>(a.z1) + ((int64_t)unit * 2 * n_ops + op) * a.unit_stride + (int64_t)t0 * d;
+        for (int i = threadIdx.x; i < kSTile * d; i += blockDim.x) {
+            const int t = i / d, c = i % d;
+            zs[t * ld + c] = t < nt ? to_f32<T>(z1[i]) : 0.f;
+        }
+        __syncthreads();
+        for (int rb = 0; rb < M; rb += kSRows) {
+            for (int i = threadIdx.x; i < kSRows * d; i += blockDim.x) {
+                const int r = rb + i / d, c = i % d;
+                float v = 0.f;
+                if (r < M) {
+                    const int layer = a.B == 4 ? op : r / (a.G * a.W), g = (r / a.W) % a.G, qi = r % a.W;
+                    const T* q = reinterpret_cast<const T*>(a.q_layers_dev[a.B * pair + layer]);
+                    v = to_f32<T>(q[((int64_t)qi * a.Hq + h * a.G + g) * d + c]);
+                }
+                qs[i] = v;
+            }
+            __syncthreads();
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            const float* zr = zs + j * ld;
+            const float* qr = qs + rg * 4 * d;
+            for (int c = 0; c < d; ++c) {
+                const float zv = zr[c];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[i] = fmaf(qr[i * d + c], zv, acc[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = rb + rg * 4 + i;
+                if (r < M && j < nt && t0 + j <= a.pos[r % a.W]) best = fmaxf(best, fabsf(acc[i]));
+            }
+            __syncthreads();
+        }
+    }
+    // the score carries the factor of Eq. 1's inverse (c for a pair; a block of four's deviations are in layer space already)
+    if (j < nt) atomicMax(a.score + (int64_t)unit * a.Tmax + t0 + j, __float_as_uint(best * (a.B == 4 ? 1.f : __uint_as_float(0x3F3504F3u))));
+}
+
 }  // namespace
 
-cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st) {
+cudaError_t launch_token_select(const TokenArgs& a, int dtype, int d, bool tensor_core, cudaStream_t st) {
     if (a.unit_count <= 0) return cudaSuccess;
     static PerDevice once;
     int sm_count = 0;
-    cudaError_t e0 = once.ensure([&]() { return cudaFuncSetAttribute(token_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmem); }, &sm_count);
+    const size_t tile_smem = (size_t)(kSTile * (d + 1) + kSRows * d) * sizeof(float);
+    cudaError_t e0 = once.ensure([&]() {
+        cudaError_t e1 = cudaFuncSetAttribute(token_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmem);
+        if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(token_score_tile_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+        if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(token_score_tile_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+        return e1;
+    }, &sm_count);
     if (e0 != cudaSuccess) return e0;
     cudaError_t e = cudaMemsetAsync(a.score + (int64_t)a.unit_begin * a.Tmax, 0, (size_t)a.unit_count * a.Tmax * 4, st);
     if (e != cudaSuccess) return e;
+    if (!tensor_core) {
+        // tokens after the last probe position are seen by nobody: score 0
+        const int ntiles = std::min(a.T - 1, a.pos_host[a.W - 1]) / kSTile + 1;
+        if (dtype == FDKV_BF16)
+            token_score_tile_kernel<__nv_bfloat16><<<dim3(ntiles, a.unit_count), 256, tile_smem, st>>>(a, d);
+        else
+            token_score_tile_kernel<float><<<dim3(ntiles, a.unit_count), 256, tile_smem, st>>>(a, d);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        token_select_kernel<<<a.unit_count, 1024, 0, st>>>(a);
+        count_launch(2);
+        return cudaGetLastError();  // (the float32 probe kernel masks the selected rows itself: no dropped copy)
+    }
     ScorePlan pl;
     pl.pos_min = a.pos_host[0];
     pl.ntiles = a.pos_host[a.W - 1] / kTM + 1;  // tokens after the last probe position are seen by nobody: score 0
@@ -386,10 +475,11 @@ cudaError_t launch_token_select(const TokenArgs& a, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, int twice, cudaStream_t st) {
+cudaError_t launch_token_gather(const void* z1, const int32_t* list, int64_t k_tok, void* out, int row_bytes, int twice, cudaStream_t st) {
     if (k_tok <= 0) return cudaSuccess;
-    const int blocks = (int)std::min<int64_t>(256, (k_tok * 16 + 255) / 256);
-    token_gather_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(z1), list, k_tok, reinterpret_cast<uint4*>(out), twice);
+    const int row_u4 = row_bytes / 16;
+    const int blocks = (int)std::min<int64_t>(256, (k_tok * row_u4 + 255) / 256);
+    token_gather_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(z1), list, k_tok, reinterpret_cast<uint4*>(out), row_u4, twice);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -134,7 +134,7 @@ def test_unsupported_combinations_and_reset_reuse():
 
     base = dict(n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=128, max_batch=1, max_prefill=512, max_tail=4, dtype=B.BF16,
                 keep_num=1, keep_den=16)
-    for bad in (dict(block_size=3), dict(residual_rule=1, head_dim=64), dict(row_format=1, head_dim=64),
+    for bad in (dict(block_size=3), dict(residual_rule=2), dict(row_format=1, head_dim=64),
                 dict(row_format=1, dtype=B.F32), dict(row_format=1, max_fold=16), dict(row_format=1, n_q_heads=16),
                 dict(row_format=2), dict(max_fold=-1), dict(n_layers=6, block_size=4)):
         cfg = dict(base)
