@@ -78,7 +78,7 @@ typedef struct {
  *       code = e4m3(R[t][c] / scale_c)   (float32 division, round to nearest even, saturating);
  *       attention sees decode(code) * scale_c.
  *   Sparse residual values and the generated-token tails keep the storage type.  Halves the bytes a decode call
- *   streams.  bf16 storage, head_dim 128, either block size, entry residual rule, group size <= 4; fdkv_fold_tail is
+ *   streams.  bf16 storage, head_dim 128, either block size, either residual rule, group size <= 4; fdkv_fold_tail is
  *   unavailable.  Compression and the probe are unchanged (they see the unquantised coefficients).
  */
 typedef enum { FDKV_ROWS_STORAGE = 0, FDKV_ROWS_E4M3 = 1 } fdkv_row_format;

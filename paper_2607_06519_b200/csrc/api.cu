@@ -48,8 +48,7 @@ bool make_shape(const fdkv_config& c, Shape& s) {
     s.max_fold = c.max_fold;
     if (c.row_format != FDKV_ROWS_STORAGE && c.row_format != FDKV_ROWS_E4M3) return false;
     s.rows_f8 = c.row_format == FDKV_ROWS_E4M3;
-    if (s.rows_f8 && !(c.dtype == FDKV_BF16 && c.head_dim == 128 && G <= 4 && c.residual_rule == FDKV_RESIDUAL_ENTRIES && c.max_fold == 0))
-        return false;
+    if (s.rows_f8 && !(c.dtype == FDKV_BF16 && c.head_dim == 128 && G <= 4 && c.max_fold == 0)) return false;
     s.kfold_max = (int64_t)s.max_fold * s.d * s.keep_num / s.keep_den;
     s.kmax = (int64_t)s.Tmax * s.d * s.keep_num / s.keep_den;
     s.kcap = (int64_t)align_up((size_t)(s.kmax + kListPad), 64);
@@ -619,6 +618,9 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
                         CU(launch_token_gather(c->work + c->ws.z1 + (ut * s.NB + j) * unit_stride_b, wsp<int32_t>(c, c->ws.tok_list) + (size_t)u * s.ktok_cap, k_tok,
                                                rows_l[j], s.d * s.esize, (s.B == 4 && c->packed_lists) ? 1 : 0, st));
                     }
+                    if (s.rows_f8)  // 8-bit rows: the kept rows become f16(value / scale[channel]) in the fragment order of the 8-bit tiles
+                        for (int j = 0; j < s.NB; ++j)
+                            rjobs.push_back(RepackJob{reinterpret_cast<uint32_t*>(rows_l[j]), reinterpret_cast<const uint32_t*>(rows_l[j]), k_tok, sc8, is_v, 1});
                     for (int l = 0; l < s.B; ++l) {
                         UnitDesc* d = dl[l];
                         d->res_kind = 1;
@@ -674,7 +676,7 @@ fdkv_status fdkv_commit(fdkv_ctx* c, int32_t seq, void* stream) {
         CU(launch_quantise_jobs(qd, (int)qjobs.size(), T, st));
         if (!rjobs.empty()) {
             CU(cudaMemcpyAsync(rd, rjobs.data(), rjobs.size() * sizeof(RepackJob), cudaMemcpyHostToDevice, st));
-            CU(launch_repack_jobs(rd, (int)rjobs.size(), k, st));
+            CU(launch_repack_jobs(rd, (int)rjobs.size(), s.tok_rule ? k_tok * 32 : k, st));
         }
     }
     const size_t seq_desc = (size_t)s.L * s.Hkv;

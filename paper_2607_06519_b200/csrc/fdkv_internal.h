@@ -264,12 +264,13 @@ struct QuantJob {
 };
 // One residual list of a unit whose rows are 8-bit: value -> f16(value / scale[channel]), position permuted inside its
 // 16-channel group to the order the kernel's converted fragments use (K and V differ).
+// (rows = 1: dst == src are n densely packed 128-channel bf16 rows of the token rule, converted in place.)
 struct RepackJob {
     uint32_t* dst;
     const uint32_t* src;
     int64_t n;
     const float* scale;
-    int32_t is_v, pad_;
+    int32_t is_v, rows;
 };
 // One copy of the commit step: dst[0, bytes) = consecutive rows of row_bytes taken every src_pitch bytes from src
 // (row_bytes == src_pitch: a plain copy).  Pointers 16-byte aligned, row_bytes and src_pitch multiples of 16, bytes a

@@ -91,6 +91,24 @@ __device__ __forceinline__ int slot_v(int c) { return (c >> 1) + 8 * (c & 1); }
 __global__ void __launch_bounds__(256) repack_entries_f8_kernel(const RepackJob* jobs) {
     const RepackJob jb = jobs[blockIdx.y];
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (jb.rows) {
+        // token rule: one warp per kept row, a lane per four channels; the whole row is read before any of it is written
+        const int64_t row = i >> 5;
+        if (row >= jb.n) return;  // (warp-uniform)
+        const int lane = threadIdx.x & 31;
+        uint16_t* const r16 = reinterpret_cast<uint16_t*>(jb.dst) + row * kD;
+        const uint2 in = *reinterpret_cast<const uint2*>(r16 + 4 * lane);
+        const uint32_t w2[2] = {in.x, in.y};
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int ch = 4 * lane + j;
+            const float v = __uint_as_float((j & 1) ? (w2[j >> 1] & 0xFFFF0000u) : (w2[j >> 1] << 16));
+            const int cs = (ch & ~15) + (jb.is_v ? slot_v(ch & 15) : slot_k(ch & 15));
+            r16[cs] = __half_as_ushort(__float2half_rn(__fdiv_rn(v, jb.scale[ch])));
+        }
+        return;
+    }
     if (i >= jb.n) return;
     const uint32_t w = jb.src[i];
     // undo the pair-path offset: byte offset / 2 = half << 10 | row << 6 | (chunk ^ row) << 3 | ch & 7

@@ -60,6 +60,49 @@ def test_rows_e4m3_parity(T, Hq, Hkv, keep, n_steps):
     pf.ctx.close()
 
 
+@pytest.mark.parametrize("T,keep,tail", [(1300 + 37, (1, 16), 2), (300, (1, 8), 0)])
+def test_rows_e4m3_with_token_rule(T, keep, tail):
+    """8-bit rows combined with the token rule: the kept tokens' high-frequency rows stay 16-bit (rescaled by the rows'
+    channel scales for the 8-bit tiles' products); attention on the GPU's own token set against the oracle."""
+    from paper_2607_06519_b200 import runner
+
+    Hq, Hkv = 8, 2
+    w = synth.Workload(name="f8tok", n_layers=4, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=128, batch=1, T=T, dtype="bf16",
+                       keep_num=keep[0], keep_den=keep[1], n_needles=4, W=8, seed=57, n_steps=max(tail, 1), row_format=1,
+                       residual_rule=1)
+    pf = runner.Prefilled(w, max_tail=max(tail, 1))
+    pf.compress(0)
+    pf.probe(0, 1.0)
+    units = {}
+    for p in range(2):
+        for h in range(Hkv):
+            u = _unit8(w, p, h)
+            tok, _ = pf.ctx.get_token_set(0, p, h, w.T)
+            u.use_tokens(tok.cpu().numpy())
+            units[(p, h)] = u
+    modes = np.array([[1, (p + 1) % 3] for p in range(2)], dtype=np.int32)
+    pf.ctx.set_modes(0, modes)
+    pf.commit(0)
+    G = w.group
+    worst = 0.0
+    for step in range(max(tail, 1)):
+        for layer in range(4):
+            q = pf.decode_q(layer, step)
+            kn = vn = None
+            if tail:
+                kn, vn = pf.new_rows(layer, step)
+                for h in range(Hkv):
+                    units[(layer // 2, h)].append(layer & 1, f32(kn)[0, h], f32(vn)[0, h])
+            out = f32(pf.ctx.decode_attn(layer, q, kn, vn, out_dtype=0))[0]
+            torch.cuda.synchronize()
+            for h in range(Hkv):
+                ref = units[(layer // 2, h)].attend(int(modes[layer // 2][h]), layer & 1, f32(q)[0][h * G:(h + 1) * G])
+                worst = max(worst, float(vector_errors(out[h * G:(h + 1) * G], ref).max()))
+    assert worst <= TOL["bf16"], worst
+    assert pf.ctx.device_status() == 0
+    pf.ctx.close()
+
+
 def test_rows_e4m3_benchmark_workload_sampled():
     """decode32k_fp8 (the 32k workload with 8-bit rows, quota mode mix) through the calls bench.py times: sampled units'
     codes and scales bit-exact, one decode step of all layers within tolerance on those units."""
